@@ -1,0 +1,217 @@
+/*
+ * splitlora.h -- C ABI of the B200 (sm_100a) split-LoRA round library.
+ *
+ * One training round t of SplitLoRA (arxiv 2407.00952, Algorithm 1) on a GPT-style pre-LN decoder
+ * cut after block `cut`:
+ *   splitlora_client_fwd   step a1/a2, Eq. 2 : K clients run blocks 1..cut, each with its own adapters
+ *   splitlora_server_step  step a3/a4, Eq. 3-5: server forward + loss + backward + server update
+ *   splitlora_client_bwd   step a5, Eq. 6-7  : activation gradients back through the client blocks + update
+ *   splitlora_aggregate    stage b, Eq. 8-9  : data-size-weighted average of the client A and B matrices
+ *   splitlora_round        one iteration of Algorithm 1 (the four calls above; aggregation every I rounds)
+ *
+ * General rules
+ *   - Every function returns 0 (SPLITLORA_OK) or a negative error code; nothing throws, exits or
+ *     falls back to the CPU.  splitlora_last_error() gives a text for the last failure of a context.
+ *   - Unless a parameter is marked HOST it is a DEVICE pointer, 16-byte aligned, contiguous,
+ *     row-major, owned by the caller and only borrowed (frozen weights and the workspace for the
+ *     life of the context, everything else for the duration of the call).
+ *   - Work is enqueued on the CUDA stream given at creation; calls return without synchronising
+ *     unless they write to a HOST pointer (loss_out).
+ *   - The library never allocates device memory in the calls below: all of its state lives in the
+ *     caller-provided workspace (splitlora_workspace_bytes / splitlora_bind_workspace).
+ *   - Conventions: a linear layer stores W as [out, in]; a LoRA adapter is A [r, in], B [out, r]
+ *     and the adapted layer computes  y = x W^T + bias + (alpha/r) (x A^T) B^T   (Sec. II-C).
+ *     Activations are [K, b, T, d] = [clients, sequences per client, positions, width].
+ */
+#ifndef SPLITLORA_H_
+#define SPLITLORA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPLITLORA_OK              0
+#define SPLITLORA_ERR_ARG        -1   /* null pointer, out-of-range or inconsistent argument        */
+#define SPLITLORA_ERR_ALIGN      -2   /* a device pointer is not 16-byte aligned                    */
+#define SPLITLORA_ERR_STATE      -3   /* call order (e.g. client_bwd without client_fwd, unbound weights) */
+#define SPLITLORA_ERR_ARCH       -4   /* the current device is not compute capability 10.x          */
+#define SPLITLORA_ERR_WORKSPACE  -5   /* workspace missing or too small                             */
+#define SPLITLORA_ERR_COUNTS     -6   /* a negative sample count, or all counts zero                */
+#define SPLITLORA_ERR_TIMEOUT    -7   /* a bounded wait inside a kernel expired (see device_status) */
+#define SPLITLORA_ERR_CUDA       -8   /* a CUDA call failed; text in splitlora_last_error           */
+#define SPLITLORA_ERR_UNSUPPORTED -9  /* a valid request that this build does not implement         */
+
+#define SPLITLORA_DTYPE_FP32 0        /* everything fp32 (plain FMA arithmetic, no tensor cores)    */
+#define SPLITLORA_DTYPE_BF16 1        /* bf16 activations + frozen tensors, fp32 accumulation, fp32 adapters */
+
+#define SPLITLORA_OPT_SGD   0         /* Eq. 4-7 literally: P <- P - gamma G                        */
+#define SPLITLORA_OPT_ADAMW 1         /* AdamW with bias correction and decoupled weight decay      */
+
+#define SPLITLORA_TARGET_Q 1u         /* bits of lora_targets: which slices of the fused qkv        */
+#define SPLITLORA_TARGET_K 2u         /* projection carry an adapter                                */
+#define SPLITLORA_TARGET_V 4u
+
+#define SPLITLORA_SIDE_CLIENT 0
+#define SPLITLORA_SIDE_SERVER 1
+
+typedef struct splitlora_ctx splitlora_ctx;   /* opaque */
+
+/* Inputs of Algorithm 1 (b, I, gamma_c, gamma_s, N) plus the model shape.  Plain data. */
+typedef struct {
+  int32_t n_layer;           /* blocks in the whole model                                   */
+  int32_t cut;               /* blocks 0..cut-1 run on the clients; 1 <= cut < n_layer      */
+  int32_t d_model, n_head, d_ff, vocab, max_seq;
+  int32_t lora_r;            /* rank r, 1..64                                               */
+  float   lora_alpha;        /* scaling alpha; the update is scaled by alpha / r            */
+  uint32_t lora_targets;     /* SPLITLORA_TARGET_* bits                                     */
+  int32_t n_clients;         /* K (the paper's N)                                           */
+  int32_t batch_per_client;  /* b                                                           */
+  int32_t seq;               /* T <= max_seq                                                */
+  int32_t dtype;             /* SPLITLORA_DTYPE_*                                           */
+  int32_t optimizer;         /* SPLITLORA_OPT_*                                             */
+  float   lr_client, lr_server;          /* gamma_c, gamma_s                                */
+  float   beta1, beta2, adam_eps, weight_decay;
+  int32_t agg_interval;      /* I: aggregate when round_index % I == 0, round_index from 1  */
+  float   norm_eps;
+  int32_t gelu_tanh;         /* 1: tanh form of GELU (GPT-2), 0: erf form                   */
+  int32_t use_tensor_cores;  /* bf16 only: 1 = tcgen05 GEMMs + tensor-core attention (default),
+                                0 = plain FMA kernels (a second opinion for debugging)      */
+} splitlora_config;
+
+/* ---- context ------------------------------------------------------------------------------ */
+
+/* Validates cfg (HOST), checks the device, records `cuda_stream` (a cudaStream_t, may be NULL for
+ * the default stream).  *out is owned by the caller until splitlora_destroy. */
+int splitlora_create(const splitlora_config* cfg, void* cuda_stream, splitlora_ctx** out);
+int splitlora_destroy(splitlora_ctx* ctx);
+
+/* Bytes of device memory the context needs for saved activations, adapters, optimizer state,
+ * transposed frozen copies and scratch.  bytes is HOST. */
+int splitlora_workspace_bytes(const splitlora_config* cfg, size_t* bytes);
+/* Gives the context its workspace (256-byte aligned).  Initialises adapters to zero, optimizer
+ * state to zero, round counter to 0. */
+int splitlora_bind_workspace(splitlora_ctx* ctx, void* dev, size_t bytes);
+
+/* Frozen tensors of W_c and W_s, in the context dtype.  Names (l = block index from 0):
+ *   "wte" [vocab, d]   "wpe" [max_seq, d]   "lnf.g" [d]   "lnf.b" [d]
+ *   "h.<l>.ln1.g" "h.<l>.ln1.b" [d]          "h.<l>.attn.qkv.w" [3d, d]  "h.<l>.attn.qkv.b" [3d]
+ *   "h.<l>.attn.proj.w" [d, d] "h.<l>.attn.proj.b" [d]   "h.<l>.ln2.g" "h.<l>.ln2.b" [d]
+ *   "h.<l>.mlp.fc1.w" [d_ff, d] "h.<l>.mlp.fc1.b" [d_ff] "h.<l>.mlp.fc2.w" [d, d_ff] "h.<l>.mlp.fc2.b" [d]
+ * The LM head is tied to "wte".  Tensors are borrowed and never written.  `bytes` must equal the
+ * size implied by the shape.  Requires a bound workspace (transposed copies for the backward
+ * products are made at bind time, on the context stream). */
+int splitlora_bind_frozen(splitlora_ctx* ctx, const char* name, const void* dev, size_t bytes);
+
+/* Adapter access (fp32).  side: SPLITLORA_SIDE_*; client: 0..K-1 (ignored for the server);
+ * layer: block index (0..cut-1 for clients, cut..n_layer-1 for the server); target: one
+ * SPLITLORA_TARGET_* bit.  A [r, d], B [d, r] device buffers; copied in / out on the stream.
+ * Either pointer may be NULL to skip that matrix. */
+int splitlora_set_adapter(splitlora_ctx* ctx, int side, int client, int layer, uint32_t target,
+                          const float* A, const float* B);
+int splitlora_get_adapter(splitlora_ctx* ctx, int side, int client, int layer, uint32_t target,
+                          float* A, float* B);
+/* Gradients G_A, G_B of the last backward pass (Eq. 4-7), same addressing. */
+int splitlora_get_adapter_grad(splitlora_ctx* ctx, int side, int client, int layer, uint32_t target,
+                               float* dA, float* dB);
+/* AdamW first/second moments, same addressing; for checkpoint / resume. */
+int splitlora_get_opt_state(splitlora_ctx* ctx, int side, int client, int layer, uint32_t target,
+                            float* mA, float* vA, float* mB, float* vB);
+int splitlora_set_opt_state(splitlora_ctx* ctx, int side, int client, int layer, uint32_t target,
+                            const float* mA, const float* vA, const float* mB, const float* vB);
+/* Round counter t and optimizer step counters (HOST out / in); for resume. */
+int splitlora_get_counters(splitlora_ctx* ctx, int64_t* round_index, int64_t* server_steps, int64_t* client_steps);
+int splitlora_set_counters(splitlora_ctx* ctx, int64_t round_index, int64_t server_steps, int64_t client_steps);
+
+/* ---- the round (Algorithm 1) -------------------------------------------------------------- */
+
+/* Step a1, Eq. 2.  tokens [K, b, T] int32 in [0, vocab).  Writes the cut-layer activations
+ * s_1..s_K to act_out [K, b, T, d] (context dtype): the hand-off buffer of step a2.  Keeps what
+ * client_bwd needs inside the workspace. */
+int splitlora_client_fwd(splitlora_ctx* ctx, const int32_t* tokens, void* act_out);
+
+/* Step a3/a4, Eq. 3-5.  act_in [K, b, T, d] is treated as the concatenation S^t; labels [K, b, T]
+ * int32, negative = ignored position.  One forward/backward over the concatenated batch with the
+ * single server adapter set, loss = mean cross-entropy over valid positions, server adapters
+ * updated with lr_server.  Writes dL/dS to act_grad_out [K, b, T, d] (context dtype).
+ * loss_out is HOST and may be NULL; when given, the call synchronises the stream. */
+int splitlora_server_step(splitlora_ctx* ctx, const void* act_in, const int32_t* labels,
+                          void* act_grad_out, float* loss_out);
+
+/* Step a5, Eq. 6-7.  Back-propagates act_grad_in [K, b, T, d] through each client's blocks and
+ * updates each client's adapters with lr_client.  Needs the saved state of the preceding
+ * splitlora_client_fwd on this context, else SPLITLORA_ERR_STATE. */
+int splitlora_client_bwd(splitlora_ctx* ctx, const void* act_grad_in);
+
+/* Stage b, Eq. 8-9 and the downlink b3.  sample_counts is HOST int64 [K] (|D_i|), all >= 0 and not
+ * all zero.  Every client A and B becomes sum_i (|D_i|/|D|) P_i, written back to all K clients. */
+int splitlora_aggregate(splitlora_ctx* ctx, const int64_t* sample_counts);
+
+/* One iteration t of Algorithm 1: client_fwd, server_step, client_bwd (through internal hand-off
+ * buffers) and, when t % agg_interval == 0, aggregate.  tokens, labels DEVICE [K, b, T] int32;
+ * sample_counts HOST; loss_out HOST or NULL. */
+int splitlora_round(splitlora_ctx* ctx, const int32_t* tokens, const int32_t* labels,
+                    const int64_t* sample_counts, float* loss_out);
+
+/* Same round with HOST tokens and labels: copies them to the device on the stream first.  This is
+ * the end-to-end call (host in, host loss out). */
+int splitlora_round_host(splitlora_ctx* ctx, const int32_t* tokens_host, const int32_t* labels_host,
+                         const int64_t* sample_counts, float* loss_out);
+
+/* Device loss of the last server_step (fp32 scalar, DEVICE pointer into the workspace). */
+int splitlora_loss_device(splitlora_ctx* ctx, const float** loss_dev);
+
+const char* splitlora_last_error(const splitlora_ctx* ctx);
+/* Reads the device status word (HOST out): 0, or the code left by a bounded wait that expired.
+ * Synchronises the stream. */
+int splitlora_device_status(splitlora_ctx* ctx, int32_t* code);
+/* Number of kernels the context has launched since creation (HOST out). */
+int splitlora_launch_count(const splitlora_ctx* ctx, int64_t* launches);
+/* Per-kernel-class device time: when enabled, each launch is bracketed by CUDA events on the
+ * context stream; splitlora_profile_report copies up to `cap` entries of {name, launches,
+ * milliseconds} into HOST arrays and returns the number of classes in *n. */
+int splitlora_profile_enable(splitlora_ctx* ctx, int on);
+int splitlora_profile_report(splitlora_ctx* ctx, char (*names)[48], int64_t* launches, double* ms,
+                             int cap, int* n);
+
+/* ---- stand-alone operators (kernel-level tests, the LoRA-linear sweep, bandwidth sweeps) ----
+ * All pointers DEVICE; `stream` is a cudaStream_t.  `workspace` is scratch of at least the size
+ * the matching *_workspace_bytes call reports. */
+
+/* Grouped LoRA linear forward (Sec. II-C applied to G adapters over one shared frozen W):
+ *   y[m,:] = x[m,:] W^T + bias + (alpha/r) (x[m,:] A_g^T) B_g^T,  g = m / (M/G)
+ * x [M, in], W [out, in], bias [out] or NULL, y [M, out] in `dtype`; A [G, r, in], B [G, out, r] fp32.
+ * M % G == 0; in bf16 mode M/G % 128 == 0, in % 64 == 0, out % 8 == 0. */
+int splitlora_lora_linear_workspace_bytes(int dtype, int M, int n_in, int n_out, int r, int G, size_t* bytes);
+int splitlora_lora_linear_fwd(int dtype, int use_tensor_cores, const void* x, const void* W, const void* bias,
+                              const float* A, const float* B, float alpha, int M, int n_in, int n_out,
+                              int r, int G, void* y, void* workspace, size_t workspace_bytes, void* stream);
+/* Backward of the same layer (the G_A, G_B of Eq. 4-7 and the gradient passed on; W is frozen, no dW):
+ *   dx = dy W + (alpha/r)(dy B_g) A_g ;  dA_g = (alpha/r)(dy_g B_g)^T x_g ;  dB_g = (alpha/r) dy_g^T (x_g A_g^T)
+ * dy [M, out], dx [M, in] in `dtype`; dA [G, r, in], dB [G, out, r] fp32.  Wt is W transposed,
+ * [in, out], in `dtype` (the caller keeps it; W is frozen so it is built once). */
+int splitlora_lora_linear_bwd(int dtype, int use_tensor_cores, const void* x, const void* Wt, const void* dy,
+                              const float* A, const float* B, float alpha, int M, int n_in, int n_out,
+                              int r, int G, void* dx, float* dA, float* dB,
+                              void* workspace, size_t workspace_bytes, void* stream);
+/* out [cols, rows] = in [rows, cols]^T in `dtype` (for building Wt). */
+int splitlora_transpose(int dtype, const void* in, int rows, int cols, void* out, void* stream);
+
+/* Eq. 8-9 on raw buffers: params [K, P] fp32; weights HOST double [K] (already |D_i|/|D|);
+ * every row is overwritten with sum_i w_i params[i, :].  P % 4 == 0. */
+int splitlora_aggregate_buffers(float* params, int K, int64_t P, const double* weights, void* stream);
+
+/* Causal multi-head attention on a fused qkv buffer [nseq*T, 3d] -> o [nseq*T, d], lse [nseq, H, T] fp32
+ * (natural-log sum of exp of the scaled scores), and its backward -> dqkv [nseq*T, 3d]. */
+int splitlora_attention_fwd(int dtype, int use_tensor_cores, const void* qkv, int nseq, int T, int n_head,
+                            int d_model, void* o, float* lse, void* stream);
+int splitlora_attention_bwd(int dtype, int use_tensor_cores, const void* qkv, const void* o, const float* lse,
+                            const void* d_o, int nseq, int T, int n_head, int d_model, void* dqkv,
+                            float* scratch_rowdot /* [nseq*T*H] */, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPLITLORA_H_ */

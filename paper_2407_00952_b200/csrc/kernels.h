@@ -1,0 +1,118 @@
+// Internal launchers of the split-LoRA kernels.  Host-callable, stream-ordered, no allocation.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace sl {
+
+enum { DT_F32 = 0, DT_BF16 = 1 };
+static inline size_t dtype_size(int dt) { return dt == DT_BF16 ? 2 : 4; }
+
+// Epilogues of the linear-layer kernels.
+enum Epilogue {
+  EPI_BIAS = 0,          // Y = acc + bias
+  EPI_BIAS_GELU = 1,     // Z = acc + bias ; Y = gelu(Z)
+  EPI_BIAS_RESID = 2,    // Y = acc + bias + R
+  EPI_MUL_GELUGRAD = 3   // Y = acc * gelu'(R)           (R holds the saved pre-activation)
+};
+
+// Width of one block of the rank-r extension of the contraction (elements).
+static const int EXT_BLOCK = 64;
+
+// Y[M,N] = epilogue( X[M,K] W[N,K]^T + Xe[M,Ke] We[N,Ke]^T )
+// Rows are split into groups of rows_per_group consecutive rows (0: one group).  A grouped operand
+// holds one [N, .] matrix per group, stacked along rows.  The extension term is how the rank-r LoRA
+// path enters: Xe is the down-projected activation, We the (scaled) up-projection of the row's group.
+struct GemmArgs {
+  int dtype = DT_BF16;
+  const void* X = nullptr; int64_t ldx = 0;
+  const void* W = nullptr; int64_t ldw = 0;
+  void* Y = nullptr;       int64_t ldy = 0;
+  int M = 0, N = 0, K = 0;
+  int w_rows = 0;           // number of valid rows of W (rows >= w_rows read as zero); 0 means N
+  int rows_per_group = 0;
+  int w_grouped = 0;        // W is [G*N, K]
+  const void* bias = nullptr;
+  int epi = EPI_BIAS;
+  const void* R = nullptr; int64_t ldr = 0;
+  void* Z = nullptr;       int64_t ldz = 0;
+  int gelu_tanh = 1;
+  const void* Xe = nullptr; int64_t ldxe = 0;
+  const void* We = nullptr; int64_t ldwe = 0;
+  int Ke = 0;               // 0: no extension; else a multiple of 16
+  int we_grouped = 0;       // We is [G*N, Ke]
+};
+
+// Plain-FMA tiled kernel, any shape, fp32 or bf16 storage with fp32 accumulation.
+cudaError_t gemm_simt(const GemmArgs& a, cudaStream_t st);
+// tcgen05 / TMEM / TMA kernel (bf16 only).  Shape rules: M % 128 == 0, K % 64 == 0, N % 8 == 0,
+// rows_per_group % 128 == 0, leading dimensions multiples of 8 elements, 16-byte aligned bases.
+// status: device word that receives a non-zero code if a bounded wait expires.
+bool gemm_tc_supported(const GemmArgs& a);
+cudaError_t gemm_tc(const GemmArgs& a, int* status, cudaStream_t st);
+int gemm_tc_init();   // resolves the driver entry point for tensor-map encoding; 0 on success
+
+cudaError_t embed(int dt, const int32_t* tokens, const void* wte, const void* wpe, void* out,
+                  int M, int T, int d, int vocab, cudaStream_t st);
+cudaError_t layernorm_fwd(int dt, const void* x, const void* g, const void* b, void* y, float* mean,
+                          float* rstd, int M, int d, float eps, cudaStream_t st);
+// dx = resid + dLN(dy)  (resid may be null); gradient w.r.t. the input only.
+cudaError_t layernorm_bwd(int dt, const void* dy, const void* x, const void* g, const float* mean,
+                          const float* rstd, const void* resid, void* dx, int M, int d, cudaStream_t st);
+
+// Cross-entropy over logits [M, ld] (V valid columns): writes per-row losses, then overwrites the
+// logits with d loss / d logits (zero in the pad columns) and reduces the mean loss.
+cudaError_t cross_entropy(int dt, void* logits, int64_t ld, const int32_t* labels, int M, int V,
+                          float* row_loss, int* n_valid, float* loss, cudaStream_t st);
+
+// Attention, fused qkv layout [nseq*T, 3d]; heads are contiguous slices of width d/H.
+cudaError_t attention_fwd_simt(int dt, const void* qkv, int nseq, int T, int H, int d, void* o, float* lse,
+                               cudaStream_t st);
+cudaError_t attention_bwd_simt(int dt, const void* qkv, const void* o, const float* lse, const void* d_o,
+                               int nseq, int T, int H, int d, void* dqkv, float* rowdot, cudaStream_t st);
+bool attention_tc_supported(int dt, int T, int H, int d);
+cudaError_t attention_fwd_tc(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, cudaStream_t st);
+cudaError_t attention_bwd_tc(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq,
+                             int T, int H, int d, void* dqkv, float* rowdot, cudaStream_t st);
+
+// out[g][j][c] = scale * sum_{m in group g} Wt[m, wcol0 + j] * Z[m, zcol0 + c],  j < R, c < C.
+// Stored at out + g*out_group_stride with element (j, c) at j*out_sj + c*out_sc.
+// partial: scratch of at least lora_grad_scratch_floats(...) floats.
+size_t lora_grad_scratch_floats(int M, int rows_per_group, int R, int C);
+cudaError_t lora_grad(int dt, const void* Z, int64_t ldz, int zcol0, int C, const void* Wt, int64_t ldwt,
+                      int wcol0, int R, int M, int rows_per_group, float scale, float* out,
+                      int64_t out_group_stride, int64_t out_sj, int64_t out_sc, float* partial,
+                      cudaStream_t st);
+
+struct OptArgs {
+  int optimizer; float lr, beta1, beta2, eps, wd; float bc1, bc2;   // bc = 1 - beta^step
+};
+cudaError_t optimizer_step(float* p, const float* g, float* m, float* v, int64_t n, const OptArgs& o,
+                           cudaStream_t st);
+
+// Eq. 8-9 and the write-back: every row of params [K, P] becomes sum_i w[i] params[i, :].
+static const int AGG_MAX_CLIENTS = 64;
+cudaError_t aggregate(float* params, int K, int64_t P, const float* w_host, cudaStream_t st);
+
+// Compute copies of the adapters of one layer (G groups), built from fp32 masters.
+// Target t of group g has A_t [r, d_in] at A + g*a_gs + t*a_ts and B_t [d_out, r] at B + g*b_gs + t*b_ts.
+// With col = t*rp + j the copies are
+//   Acat  [G][ext, d_in]  : Acat[col, c]  = A_t[j, c]          AcatT [G][d_in, ext] : its transpose
+//   Bext  [G][n_out, ext] : Bext[slice_off[t] + c, col] = scale * B_t[c, j]
+//   BextT [G][ext, n_out] : its transpose
+// Only live entries are written; the padding must have been zeroed once.
+struct AdapterCopyArgs {
+  int dtype;
+  const float* A; int64_t a_gs, a_ts;
+  const float* B; int64_t b_gs, b_ts;
+  int G, n_targets, r, rp, d_in, d_out, n_out, ext;
+  int slice_off[4];
+  float scale;
+  void *Acat, *AcatT, *Bext, *BextT;   // any of them may be null (skipped)
+};
+cudaError_t refresh_adapter_copies(const AdapterCopyArgs& a, cudaStream_t st);
+
+cudaError_t transpose(int dt, const void* in, int rows, int cols, void* out, int64_t ldo, cudaStream_t st);
+
+}  // namespace sl

@@ -1,0 +1,770 @@
+// Split-model runtime and C ABI: context, workspace plan, the per-step kernel schedules of
+// Algorithm 1 (client forward, server step, client backward, aggregation) and the stand-alone
+// operator entry points.  Host code only; every device operation is a launcher from kernels.h.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <vector>
+
+#include "../../include/splitlora.h"
+#include "kernels.h"
+
+using namespace sl;
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct FrozenLayer {
+  const void *ln1g = nullptr, *ln1b = nullptr, *qkvw = nullptr, *qkvb = nullptr, *projw = nullptr,
+             *projb = nullptr, *ln2g = nullptr, *ln2b = nullptr, *fc1w = nullptr, *fc1b = nullptr,
+             *fc2w = nullptr, *fc2b = nullptr;
+  void *qkvwT = nullptr, *projwT = nullptr, *fc1wT = nullptr, *fc2wT = nullptr;   // [in, out] copies
+};
+
+// What one block keeps from its forward pass for its backward pass.
+struct LayerBuf {
+  void *u = nullptr, *hcat = nullptr, *qkv = nullptr, *o = nullptr, *x_mid = nullptr, *z = nullptr,
+       *x_out = nullptr;
+  float *mean1 = nullptr, *rstd1 = nullptr, *mean2 = nullptr, *rstd2 = nullptr, *lse = nullptr;
+  const void* x_in = nullptr;
+  // adapter compute copies of this layer (all groups stacked)
+  void *Acat = nullptr, *AcatT = nullptr, *Bext = nullptr, *BextT = nullptr;
+};
+
+struct ProfRec { int cls; cudaEvent_t a, b; };
+
+// Arena cursor: with base == nullptr it only measures.
+struct Arena {
+  char* base; size_t off = 0;
+  explicit Arena(char* b) : base(b) {}
+  void* take(size_t bytes) {
+    off = align_up(off, 256);
+    void* p = base ? base + off : nullptr;
+    off += bytes;
+    return p;
+  }
+};
+
+}  // namespace
+
+struct splitlora_ctx {
+  splitlora_config cfg;
+  cudaStream_t st = nullptr;
+  std::string err;
+  int dt = 0; size_t es = 4;
+  int M = 0, nseq = 0, d = 0, F = 0, V = 0, Vpad = 0, L = 0, cut = 0, K = 0, rows_per_client = 0;
+  int r = 0, rp = 0, ext = 0, ke = 0, n_targets = 0;
+  int slice_idx[4] = {0, 0, 0, 0};
+  uint32_t target_bit[4] = {0, 0, 0, 0};
+  float scale = 1.f;
+  bool tc = false;
+  // frozen
+  const void *wte = nullptr, *wpe = nullptr, *lnfg = nullptr, *lnfb = nullptr;
+  void* wteT = nullptr;
+  std::vector<FrozenLayer> fl;
+  int n_bound = 0;
+  // workspace
+  char* ws = nullptr; size_t ws_bytes = 0;
+  std::vector<LayerBuf> lb;
+  int64_t per_layer = 0, Pc = 0, Ps = 0;     // floats per layer, per client set, server set
+  float *cp = nullptr, *cg = nullptr, *cm = nullptr, *cv = nullptr;   // client params/grads/moments [K, Pc]
+  float *sp = nullptr, *sg = nullptr, *sm = nullptr, *sv = nullptr;   // server [Ps]
+  void *emb = nullptr, *u2 = nullptr, *act = nullptr, *xf = nullptr, *logits = nullptr;
+  float *meanf = nullptr, *rstdf = nullptr, *row_loss = nullptr, *rowdot = nullptr, *loss_dev = nullptr,
+        *grad_scratch = nullptr;
+  int *n_valid = nullptr, *status = nullptr;
+  void *g_a = nullptr, *g_b = nullptr, *g_dz = nullptr, *g_du2 = nullptr, *g_dxmid = nullptr, *g_do = nullptr,
+       *g_dqkv = nullptr, *g_dhcat = nullptr, *g_du = nullptr;
+  void *S = nullptr, *dS = nullptr;
+  int32_t *tok_dev = nullptr, *lab_dev = nullptr;
+  // state
+  bool client_copies_dirty = true, server_copies_dirty = true;
+  bool have_client_fwd = false;
+  int64_t round_index = 0, server_steps = 0, client_steps = 0;
+  int64_t launches = 0;
+  // profiling
+  bool prof_on = false;
+  std::vector<std::string> prof_names;
+  std::map<std::string, int> prof_ids;
+  std::vector<ProfRec> prof_recs;
+  std::vector<cudaEvent_t> event_pool;
+};
+
+namespace {
+
+int fail(splitlora_ctx* c, int code, const std::string& msg) {
+  if (c) c->err = msg;
+  return code;
+}
+
+#define CK(ctx, expr)                                                                         \
+  do {                                                                                        \
+    cudaError_t e__ = (expr);                                                                 \
+    if (e__ != cudaSuccess)                                                                   \
+      return fail(ctx, SPLITLORA_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); \
+  } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int validate(const splitlora_config* c, std::string* why) {
+  auto bad = [&](const char* m) { *why = m; return SPLITLORA_ERR_ARG; };
+  if (!c) return bad("null config");
+  if (c->n_layer < 2 || c->cut < 1 || c->cut >= c->n_layer) return bad("need 1 <= cut < n_layer");
+  if (c->d_model < 8 || c->n_head < 1 || c->d_model % c->n_head != 0) return bad("d_model must be a multiple of n_head");
+  if (c->d_model % 8 != 0 || c->d_ff % 8 != 0) return bad("d_model and d_ff must be multiples of 8");
+  if (c->d_model / c->n_head > 128) return bad("head width above 128");
+  if (c->vocab < 2 || c->max_seq < 1 || c->seq < 1 || c->seq > c->max_seq) return bad("bad vocab / seq");
+  if (c->lora_r < 1 || c->lora_r > 64) return bad("lora_r must be in 1..64");
+  if ((c->lora_targets & 7u) == 0 || (c->lora_targets & ~7u)) return bad("lora_targets must name q, k and/or v");
+  if (c->n_clients < 1 || c->n_clients > AGG_MAX_CLIENTS) return bad("n_clients must be in 1..64");
+  if (c->batch_per_client < 1) return bad("batch_per_client must be positive");
+  if (((int64_t)c->batch_per_client * c->seq) % 256 != 0 && c->n_clients > 1)
+    return bad("batch_per_client * seq must be a multiple of 256 (client segments align with kernel tiles)");
+  if (c->dtype != SPLITLORA_DTYPE_FP32 && c->dtype != SPLITLORA_DTYPE_BF16) return bad("bad dtype");
+  if (c->optimizer != SPLITLORA_OPT_SGD && c->optimizer != SPLITLORA_OPT_ADAMW) return bad("bad optimizer");
+  if (c->agg_interval < 1) return bad("agg_interval must be >= 1");
+  if (!(c->norm_eps > 0.f)) return bad("norm_eps must be positive");
+  return SPLITLORA_OK;
+}
+
+void derive(splitlora_ctx* c) {
+  const splitlora_config& g = c->cfg;
+  c->dt = g.dtype; c->es = dtype_size(g.dtype);
+  c->L = g.n_layer; c->cut = g.cut; c->K = g.n_clients;
+  c->d = g.d_model; c->F = g.d_ff; c->V = g.vocab;
+  c->Vpad = (int)align_up((size_t)g.vocab, 64);
+  c->nseq = g.n_clients * g.batch_per_client;
+  c->rows_per_client = g.batch_per_client * g.seq;
+  c->M = c->nseq * g.seq;
+  c->r = g.lora_r; c->rp = (int)align_up((size_t)g.lora_r, 16);
+  c->n_targets = 0;
+  for (int s = 0; s < 3; ++s)
+    if (g.lora_targets & (1u << s)) { c->slice_idx[c->n_targets] = s; c->target_bit[c->n_targets] = 1u << s; c->n_targets++; }
+  c->ke = c->n_targets * c->rp;
+  c->ext = (int)align_up((size_t)c->ke, EXT_BLOCK);
+  c->scale = g.lora_alpha / (float)g.lora_r;
+  c->per_layer = (int64_t)c->n_targets * 2 * c->r * c->d;
+  c->Pc = c->per_layer * c->cut;
+  c->Ps = c->per_layer * (c->L - c->cut);
+  c->tc = (g.dtype == SPLITLORA_DTYPE_BF16) && g.use_tensor_cores != 0;
+}
+
+// Lays out the workspace.  With ws == nullptr only the size is computed.
+size_t plan(splitlora_ctx* c, char* ws) {
+  Arena a(ws);
+  const size_t es = c->es;
+  const size_t M = c->M, d = c->d, F = c->F, ext = c->ext;
+  c->status = (int*)a.take(256);
+  c->loss_dev = (float*)a.take(256);
+  c->n_valid = (int*)a.take(256);
+  // adapters: masters, gradients, moments
+  c->cp = (float*)a.take((size_t)c->K * c->Pc * 4); c->cg = (float*)a.take((size_t)c->K * c->Pc * 4);
+  c->cm = (float*)a.take((size_t)c->K * c->Pc * 4); c->cv = (float*)a.take((size_t)c->K * c->Pc * 4);
+  c->sp = (float*)a.take((size_t)c->Ps * 4); c->sg = (float*)a.take((size_t)c->Ps * 4);
+  c->sm = (float*)a.take((size_t)c->Ps * 4); c->sv = (float*)a.take((size_t)c->Ps * 4);
+  c->fl.resize(c->L);
+  c->lb.resize(c->L);
+  for (int l = 0; l < c->L; ++l) {
+    FrozenLayer& f = c->fl[l];
+    f.qkvwT = a.take(3 * d * d * es); f.projwT = a.take(d * d * es);
+    f.fc1wT = a.take(F * d * es); f.fc2wT = a.take(d * F * es);
+    LayerBuf& b = c->lb[l];
+    const size_t G = l < c->cut ? c->K : 1;
+    b.Acat = a.take(G * ext * d * es); b.AcatT = a.take(G * d * ext * es);
+    b.Bext = a.take(G * 3 * d * ext * es); b.BextT = a.take(G * ext * 3 * d * es);
+    b.u = a.take(M * d * es); b.hcat = a.take(M * ext * es); b.qkv = a.take(M * 3 * d * es);
+    b.o = a.take(M * d * es); b.x_mid = a.take(M * d * es); b.z = a.take(M * F * es);
+    b.x_out = a.take(M * d * es);
+    b.mean1 = (float*)a.take(M * 4); b.rstd1 = (float*)a.take(M * 4);
+    b.mean2 = (float*)a.take(M * 4); b.rstd2 = (float*)a.take(M * 4);
+    b.lse = (float*)a.take((size_t)c->nseq * c->cfg.n_head * c->cfg.seq * 4);
+  }
+  c->wteT = a.take(d * (size_t)c->Vpad * es);
+  c->emb = a.take(M * d * es); c->u2 = a.take(M * d * es); c->act = a.take(M * F * es);
+  c->xf = a.take(M * d * es); c->logits = a.take(M * (size_t)c->Vpad * es);
+  c->meanf = (float*)a.take(M * 4); c->rstdf = (float*)a.take(M * 4); c->row_loss = (float*)a.take(M * 4);
+  c->rowdot = (float*)a.take((size_t)c->nseq * c->cfg.n_head * c->cfg.seq * 4);
+  c->grad_scratch = (float*)a.take(lora_grad_scratch_floats(c->M, c->rows_per_client, c->r, c->d) * 4);
+  c->g_a = a.take(M * d * es); c->g_b = a.take(M * d * es); c->g_dz = a.take(M * F * es);
+  c->g_du2 = a.take(M * d * es); c->g_dxmid = a.take(M * d * es); c->g_do = a.take(M * d * es);
+  c->g_dqkv = a.take(M * 3 * d * es); c->g_dhcat = a.take(M * ext * es); c->g_du = a.take(M * d * es);
+  c->S = a.take(M * d * es); c->dS = a.take(M * d * es);
+  c->tok_dev = (int32_t*)a.take(M * 4); c->lab_dev = (int32_t*)a.take(M * 4);
+  return align_up(a.off, 256);
+}
+
+// ---- profiling -----------------------------------------------------------------------------
+struct Scope {
+  splitlora_ctx* c; int cls = -1; cudaEvent_t a = nullptr, b = nullptr;
+  Scope(splitlora_ctx* ctx, const char* name, int kernels) : c(ctx) {
+    c->launches += kernels;
+    if (!c->prof_on) return;
+    auto it = c->prof_ids.find(name);
+    if (it == c->prof_ids.end()) {
+      cls = (int)c->prof_names.size();
+      c->prof_names.push_back(name); c->prof_ids[name] = cls;
+    } else cls = it->second;
+    auto get = [&]() {
+      cudaEvent_t e;
+      if (!c->event_pool.empty()) { e = c->event_pool.back(); c->event_pool.pop_back(); }
+      else cudaEventCreate(&e);
+      return e;
+    };
+    a = get(); b = get();
+    cudaEventRecord(a, c->st);
+  }
+  ~Scope() {
+    if (cls < 0) return;
+    cudaEventRecord(b, c->st);
+    c->prof_recs.push_back({cls, a, b});
+  }
+};
+
+cudaError_t linear(splitlora_ctx* c, const char* name, const GemmArgs& a) {
+  Scope s(c, name, 1);
+  if (c->tc && gemm_tc_supported(a)) return gemm_tc(a, c->status, c->st);
+  return gemm_simt(a, c->st);
+}
+
+GemmArgs base_args(splitlora_ctx* c, const void* X, int64_t ldx, const void* W, int64_t ldw, void* Y, int64_t ldy,
+                   int M, int N, int K) {
+  GemmArgs a;
+  a.dtype = c->dt; a.X = X; a.ldx = ldx; a.W = W; a.ldw = ldw; a.Y = Y; a.ldy = ldy; a.M = M; a.N = N; a.K = K;
+  a.gelu_tanh = c->cfg.gelu_tanh;
+  return a;
+}
+
+bool all_frozen_bound(const splitlora_ctx* c) { return c->n_bound == 4 + 12 * c->L; }
+
+cudaError_t refresh_side(splitlora_ctx* c, bool client) {
+  AdapterCopyArgs a;
+  a.dtype = c->dt;
+  a.a_gs = a.b_gs = client ? c->Pc : 0;
+  a.a_ts = a.b_ts = (int64_t)2 * c->r * c->d;
+  a.n_targets = c->n_targets; a.r = c->r; a.rp = c->rp; a.d_in = c->d; a.d_out = c->d; a.n_out = 3 * c->d;
+  a.ext = c->ext;
+  for (int t = 0; t < 4; ++t) a.slice_off[t] = c->slice_idx[t] * c->d;
+  a.scale = c->scale;
+  a.G = client ? c->K : 1;
+  const int l0 = client ? 0 : c->cut, l1 = client ? c->cut : c->L;
+  for (int l = l0; l < l1; ++l) {
+    a.A = (client ? c->cp : c->sp) + (size_t)(l - l0) * c->per_layer;
+    a.B = a.A + (size_t)c->r * c->d;
+    a.Acat = c->lb[l].Acat; a.AcatT = c->lb[l].AcatT; a.Bext = c->lb[l].Bext; a.BextT = c->lb[l].BextT;
+    Scope s(c, "adapter_copies", 1);
+    cudaError_t e = refresh_adapter_copies(a, c->st);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+// ---- one block -----------------------------------------------------------------------------
+cudaError_t block_forward(splitlora_ctx* c, int l, const void* x_in, void* x_out) {
+  const bool client = l < c->cut;
+  const int M = c->M, d = c->d, F = c->F, ext = c->ext;
+  const int rpg = client ? c->rows_per_client : 0;
+  const bool grouped = client && c->K > 1;
+  const FrozenLayer& f = c->fl[l];
+  LayerBuf& b = c->lb[l];
+  b.x_in = x_in;
+  cudaError_t e;
+  { Scope s(c, "layernorm_fwd", 1);
+    if ((e = layernorm_fwd(c->dt, x_in, f.ln1g, f.ln1b, b.u, b.mean1, b.rstd1, M, d, c->cfg.norm_eps, c->st))) return e; }
+  {  // h = u A_g^T for every target of the layer, one padded block of `ext` columns
+    GemmArgs a = base_args(c, b.u, d, b.Acat, d, b.hcat, ext, M, ext, d);
+    a.rows_per_group = rpg; a.w_grouped = grouped;
+    if ((e = linear(c, "lora_down_fwd", a))) return e;
+  }
+  {  // qkv = u Wqkv^T + b + hcat Bext_g^T   (the LoRA linear of Sec. II-C, grouped by client)
+    GemmArgs a = base_args(c, b.u, d, f.qkvw, d, b.qkv, 3 * d, M, 3 * d, d);
+    a.bias = f.qkvb; a.rows_per_group = rpg;
+    a.Xe = b.hcat; a.ldxe = ext; a.We = b.Bext; a.ldwe = ext; a.Ke = c->ke; a.we_grouped = grouped;
+    if ((e = linear(c, "lora_linear_fwd", a))) return e;
+  }
+  { Scope s(c, "attention_fwd", 1);
+    if (c->tc && attention_tc_supported(c->dt, c->cfg.seq, c->cfg.n_head, d))
+      e = attention_fwd_tc(b.qkv, c->nseq, c->cfg.seq, c->cfg.n_head, d, b.o, b.lse, c->st);
+    else
+      e = attention_fwd_simt(c->dt, b.qkv, c->nseq, c->cfg.seq, c->cfg.n_head, d, b.o, b.lse, c->st);
+    if (e) return e; }
+  { GemmArgs a = base_args(c, b.o, d, f.projw, d, b.x_mid, d, M, d, d);
+    a.bias = f.projb; a.epi = EPI_BIAS_RESID; a.R = x_in; a.ldr = d;
+    if ((e = linear(c, "linear_fwd", a))) return e; }
+  { Scope s(c, "layernorm_fwd", 1);
+    if ((e = layernorm_fwd(c->dt, b.x_mid, f.ln2g, f.ln2b, c->u2, b.mean2, b.rstd2, M, d, c->cfg.norm_eps, c->st))) return e; }
+  { GemmArgs a = base_args(c, c->u2, d, f.fc1w, d, c->act, F, M, F, d);
+    a.bias = f.fc1b; a.epi = EPI_BIAS_GELU; a.Z = b.z; a.ldz = F;
+    if ((e = linear(c, "linear_fwd", a))) return e; }
+  { GemmArgs a = base_args(c, c->act, F, f.fc2w, F, x_out, d, M, d, F);
+    a.bias = f.fc2b; a.epi = EPI_BIAS_RESID; a.R = b.x_mid; a.ldr = d;
+    if ((e = linear(c, "linear_fwd", a))) return e; }
+  return cudaSuccess;
+}
+
+// dy: gradient w.r.t. the block output.  dx: gradient w.r.t. the block input, or nullptr when it is
+// not needed (first client block: the embedding below it is frozen).
+cudaError_t block_backward(splitlora_ctx* c, int l, const void* dy, void* dx) {
+  const bool client = l < c->cut;
+  const int M = c->M, d = c->d, F = c->F, ext = c->ext;
+  const int rpg = client ? c->rows_per_client : 0;
+  const bool grouped = client && c->K > 1;
+  const FrozenLayer& f = c->fl[l];
+  LayerBuf& b = c->lb[l];
+  cudaError_t e;
+  { GemmArgs a = base_args(c, dy, d, f.fc2wT, d, c->g_dz, F, M, F, d);
+    a.epi = EPI_MUL_GELUGRAD; a.R = b.z; a.ldr = F;
+    if ((e = linear(c, "linear_bwd", a))) return e; }
+  { GemmArgs a = base_args(c, c->g_dz, F, f.fc1wT, F, c->g_du2, d, M, d, F);
+    if ((e = linear(c, "linear_bwd", a))) return e; }
+  { Scope s(c, "layernorm_bwd", 1);
+    if ((e = layernorm_bwd(c->dt, c->g_du2, b.x_mid, f.ln2g, b.mean2, b.rstd2, dy, c->g_dxmid, M, d, c->st))) return e; }
+  { GemmArgs a = base_args(c, c->g_dxmid, d, f.projwT, d, c->g_do, d, M, d, d);
+    if ((e = linear(c, "linear_bwd", a))) return e; }
+  { Scope s(c, "attention_bwd", 3);
+    if (c->tc && attention_tc_supported(c->dt, c->cfg.seq, c->cfg.n_head, d))
+      e = attention_bwd_tc(b.qkv, b.o, b.lse, c->g_do, c->nseq, c->cfg.seq, c->cfg.n_head, d, c->g_dqkv, c->rowdot, c->st);
+    else
+      e = attention_bwd_simt(c->dt, b.qkv, b.o, b.lse, c->g_do, c->nseq, c->cfg.seq, c->cfg.n_head, d, c->g_dqkv, c->rowdot, c->st);
+    if (e) return e; }
+  {  // dh = (alpha/r) dqkv B_g for every target (the scale lives in the compute copy)
+    GemmArgs a = base_args(c, c->g_dqkv, 3 * d, b.BextT, 3 * d, c->g_dhcat, ext, M, ext, 3 * d);
+    a.rows_per_group = rpg; a.w_grouped = grouped;
+    if ((e = linear(c, "lora_down_bwd", a))) return e;
+  }
+  // G_A = dh^T u, G_B = (alpha/r) dy^T h, per group (Eq. 4-7)
+  float* gbase = client ? c->cg + (size_t)l * c->per_layer : c->sg + (size_t)(l - c->cut) * c->per_layer;
+  const int64_t gstride = client ? c->Pc : 0;
+  for (int t = 0; t < c->n_targets; ++t) {
+    float* gA = gbase + (size_t)t * 2 * c->r * d;
+    float* gB = gA + (size_t)c->r * d;
+    { Scope s(c, "lora_grad", 2);
+      if ((e = lora_grad(c->dt, b.u, d, 0, d, c->g_dhcat, ext, t * c->rp, c->r, M, rpg, 1.0f, gA, gstride, d, 1,
+                         c->grad_scratch, c->st))) return e; }
+    { Scope s(c, "lora_grad", 2);
+      if ((e = lora_grad(c->dt, c->g_dqkv, 3 * d, c->slice_idx[t] * d, d, b.hcat, ext, t * c->rp, c->r, M, rpg,
+                         c->scale, gB, gstride, 1, c->r, c->grad_scratch, c->st))) return e; }
+  }
+  if (dx) {
+    GemmArgs a = base_args(c, c->g_dqkv, 3 * d, f.qkvwT, 3 * d, c->g_du, d, M, d, 3 * d);
+    a.rows_per_group = rpg;
+    a.Xe = c->g_dhcat; a.ldxe = ext; a.We = b.AcatT; a.ldwe = ext; a.Ke = c->ke; a.we_grouped = grouped;
+    if ((e = linear(c, "lora_linear_bwd", a))) return e;
+    Scope s(c, "layernorm_bwd", 1);
+    if ((e = layernorm_bwd(c->dt, c->g_du, b.x_in, f.ln1g, b.mean1, b.rstd1, c->g_dxmid, dx, M, d, c->st))) return e;
+  }
+  return cudaSuccess;
+}
+
+cudaError_t run_optimizer(splitlora_ctx* c, bool client) {
+  OptArgs o;
+  o.optimizer = c->cfg.optimizer; o.lr = client ? c->cfg.lr_client : c->cfg.lr_server;
+  o.beta1 = c->cfg.beta1; o.beta2 = c->cfg.beta2; o.eps = c->cfg.adam_eps; o.wd = c->cfg.weight_decay;
+  int64_t step = client ? ++c->client_steps : ++c->server_steps;
+  o.bc1 = (float)(1.0 - std::pow((double)c->cfg.beta1, (double)step));
+  o.bc2 = (float)(1.0 - std::pow((double)c->cfg.beta2, (double)step));
+  Scope s(c, "optimizer", 1);
+  if (client) return optimizer_step(c->cp, c->cg, c->cm, c->cv, (int64_t)c->K * c->Pc, o, c->st);
+  return optimizer_step(c->sp, c->sg, c->sm, c->sv, c->Ps, o, c->st);
+}
+
+int check_ready(splitlora_ctx* c) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
+  if (!all_frozen_bound(c)) return fail(c, SPLITLORA_ERR_STATE, "not every frozen tensor is bound");
+  return SPLITLORA_OK;
+}
+
+float* adapter_ptr(splitlora_ctx* c, float* client_base, float* server_base, int side, int client, int layer,
+                   uint32_t target, int* rc) {
+  *rc = SPLITLORA_OK;
+  int t = -1;
+  for (int i = 0; i < c->n_targets; ++i) if (c->target_bit[i] == target) t = i;
+  if (t < 0) { *rc = fail(c, SPLITLORA_ERR_ARG, "target is not an adapted slice"); return nullptr; }
+  if (side == SPLITLORA_SIDE_CLIENT) {
+    if (client < 0 || client >= c->K || layer < 0 || layer >= c->cut) { *rc = fail(c, SPLITLORA_ERR_ARG, "client/layer out of range"); return nullptr; }
+    return client_base + (size_t)client * c->Pc + (size_t)layer * c->per_layer + (size_t)t * 2 * c->r * c->d;
+  }
+  if (side == SPLITLORA_SIDE_SERVER) {
+    if (layer < c->cut || layer >= c->L) { *rc = fail(c, SPLITLORA_ERR_ARG, "layer out of range"); return nullptr; }
+    return server_base + (size_t)(layer - c->cut) * c->per_layer + (size_t)t * 2 * c->r * c->d;
+  }
+  *rc = fail(c, SPLITLORA_ERR_ARG, "bad side");
+  return nullptr;
+}
+
+}  // namespace
+
+// =============================================================================================
+// C ABI
+// =============================================================================================
+extern "C" {
+
+int splitlora_create(const splitlora_config* cfg, void* cuda_stream, splitlora_ctx** out) {
+  if (!out) return SPLITLORA_ERR_ARG;
+  *out = nullptr;
+  std::string why;
+  int rc = validate(cfg, &why);
+  if (rc) return rc;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SPLITLORA_ERR_CUDA;
+  if (prop.major != 10) return SPLITLORA_ERR_ARCH;
+  if (gemm_tc_init() != 0) return SPLITLORA_ERR_CUDA;
+  splitlora_ctx* c = new splitlora_ctx();
+  c->cfg = *cfg;
+  c->st = (cudaStream_t)cuda_stream;
+  derive(c);
+  *out = c;
+  return SPLITLORA_OK;
+}
+
+int splitlora_destroy(splitlora_ctx* c) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  for (auto& r : c->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  for (auto& e : c->event_pool) cudaEventDestroy(e);
+  delete c;
+  return SPLITLORA_OK;
+}
+
+int splitlora_workspace_bytes(const splitlora_config* cfg, size_t* bytes) {
+  if (!bytes) return SPLITLORA_ERR_ARG;
+  std::string why;
+  int rc = validate(cfg, &why);
+  if (rc) return rc;
+  splitlora_ctx tmp;
+  tmp.cfg = *cfg;
+  derive(&tmp);
+  *bytes = plan(&tmp, nullptr);
+  return SPLITLORA_OK;
+}
+
+int splitlora_bind_workspace(splitlora_ctx* c, void* dev, size_t bytes) {
+  if (!c || !dev) return SPLITLORA_ERR_ARG;
+  if (reinterpret_cast<uintptr_t>(dev) & 255u) return fail(c, SPLITLORA_ERR_ALIGN, "workspace must be 256-byte aligned");
+  size_t need = plan(c, nullptr);
+  if (bytes < need) return fail(c, SPLITLORA_ERR_WORKSPACE, "workspace too small");
+  plan(c, (char*)dev);
+  c->ws = (char*)dev; c->ws_bytes = bytes;
+  c->n_bound = 0;
+  // zero: status, adapters, gradients, moments, and the padded compute copies
+  CK(c, cudaMemsetAsync(c->status, 0, 256 * 3, c->st));
+  for (float* p : {c->cp, c->cg, c->cm, c->cv}) CK(c, cudaMemsetAsync(p, 0, (size_t)c->K * c->Pc * 4, c->st));
+  for (float* p : {c->sp, c->sg, c->sm, c->sv}) CK(c, cudaMemsetAsync(p, 0, (size_t)c->Ps * 4, c->st));
+  for (int l = 0; l < c->L; ++l) {
+    const size_t G = l < c->cut ? c->K : 1;
+    const size_t es = c->es, d = c->d, ext = c->ext;
+    CK(c, cudaMemsetAsync(c->lb[l].Acat, 0, G * ext * d * es, c->st));
+    CK(c, cudaMemsetAsync(c->lb[l].AcatT, 0, G * ext * d * es, c->st));
+    CK(c, cudaMemsetAsync(c->lb[l].Bext, 0, G * 3 * d * ext * es, c->st));
+    CK(c, cudaMemsetAsync(c->lb[l].BextT, 0, G * 3 * d * ext * es, c->st));
+  }
+  CK(c, cudaMemsetAsync(c->wteT, 0, (size_t)c->d * c->Vpad * c->es, c->st));
+  c->client_copies_dirty = c->server_copies_dirty = true;
+  c->have_client_fwd = false;
+  c->round_index = c->server_steps = c->client_steps = 0;
+  return SPLITLORA_OK;
+}
+
+int splitlora_bind_frozen(splitlora_ctx* c, const char* name, const void* dev, size_t bytes) {
+  if (!c || !name || !dev) return SPLITLORA_ERR_ARG;
+  if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "bind the workspace first");
+  if (!aligned16(dev)) return fail(c, SPLITLORA_ERR_ALIGN, std::string(name) + " is not 16-byte aligned");
+  const size_t es = c->es, d = c->d, F = c->F;
+  auto expect = [&](size_t elems) { return bytes == elems * es; };
+  auto bad_size = [&]() { return fail(c, SPLITLORA_ERR_ARG, std::string("wrong byte size for ") + name); };
+  auto set = [&](const void** slot) { if (!*slot) c->n_bound++; *slot = dev; };
+  std::string n(name);
+  if (n == "wte") {
+    if (!expect((size_t)c->V * d)) return bad_size();
+    set(&c->wte);
+    Scope s(c, "transpose", 1);
+    CK(c, transpose(c->dt, dev, c->V, c->d, c->wteT, c->Vpad, c->st));
+    return SPLITLORA_OK;
+  }
+  if (n == "wpe") { if (!expect((size_t)c->cfg.max_seq * d)) return bad_size(); set(&c->wpe); return SPLITLORA_OK; }
+  if (n == "lnf.g") { if (!expect(d)) return bad_size(); set(&c->lnfg); return SPLITLORA_OK; }
+  if (n == "lnf.b") { if (!expect(d)) return bad_size(); set(&c->lnfb); return SPLITLORA_OK; }
+  int l = -1; char rest[64];
+  if (sscanf(name, "h.%d.%63s", &l, rest) != 2 || l < 0 || l >= c->L) return fail(c, SPLITLORA_ERR_ARG, std::string("unknown tensor ") + name);
+  FrozenLayer& f = c->fl[l];
+  std::string r(rest);
+  struct Ent { const char* nm; const void** slot; size_t elems; void* tr; int rows, cols; };
+  Ent ents[] = {
+      {"ln1.g", &f.ln1g, d, nullptr, 0, 0}, {"ln1.b", &f.ln1b, d, nullptr, 0, 0},
+      {"attn.qkv.w", &f.qkvw, 3 * d * d, f.qkvwT, 3 * c->d, c->d}, {"attn.qkv.b", &f.qkvb, 3 * d, nullptr, 0, 0},
+      {"attn.proj.w", &f.projw, d * d, f.projwT, c->d, c->d}, {"attn.proj.b", &f.projb, d, nullptr, 0, 0},
+      {"ln2.g", &f.ln2g, d, nullptr, 0, 0}, {"ln2.b", &f.ln2b, d, nullptr, 0, 0},
+      {"mlp.fc1.w", &f.fc1w, F * d, f.fc1wT, c->F, c->d}, {"mlp.fc1.b", &f.fc1b, F, nullptr, 0, 0},
+      {"mlp.fc2.w", &f.fc2w, d * F, f.fc2wT, c->d, c->F}, {"mlp.fc2.b", &f.fc2b, d, nullptr, 0, 0}};
+  for (auto& e : ents) {
+    if (r == e.nm) {
+      if (!expect(e.elems)) return bad_size();
+      set(e.slot);
+      if (e.tr) {
+        Scope s(c, "transpose", 1);
+        CK(c, transpose(c->dt, dev, e.rows, e.cols, e.tr, e.rows, c->st));
+      }
+      return SPLITLORA_OK;
+    }
+  }
+  return fail(c, SPLITLORA_ERR_ARG, std::string("unknown tensor ") + name);
+}
+
+int splitlora_set_adapter(splitlora_ctx* c, int side, int client, int layer, uint32_t target, const float* A,
+                          const float* B) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
+  int rc;
+  float* p = adapter_ptr(c, c->cp, c->sp, side, client, layer, target, &rc);
+  if (!p) return rc;
+  const size_t n = (size_t)c->r * c->d * 4;
+  if (A) CK(c, cudaMemcpyAsync(p, A, n, cudaMemcpyDeviceToDevice, c->st));
+  if (B) CK(c, cudaMemcpyAsync(p + (size_t)c->r * c->d, B, n, cudaMemcpyDeviceToDevice, c->st));
+  (side == SPLITLORA_SIDE_CLIENT ? c->client_copies_dirty : c->server_copies_dirty) = true;
+  return SPLITLORA_OK;
+}
+
+static int get_pair(splitlora_ctx* c, float* cb, float* sb, int side, int client, int layer, uint32_t target,
+                    float* A, float* B) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
+  int rc;
+  float* p = adapter_ptr(c, cb, sb, side, client, layer, target, &rc);
+  if (!p) return rc;
+  const size_t n = (size_t)c->r * c->d * 4;
+  if (A) CK(c, cudaMemcpyAsync(A, p, n, cudaMemcpyDeviceToDevice, c->st));
+  if (B) CK(c, cudaMemcpyAsync(B, p + (size_t)c->r * c->d, n, cudaMemcpyDeviceToDevice, c->st));
+  return SPLITLORA_OK;
+}
+
+int splitlora_get_adapter(splitlora_ctx* c, int side, int client, int layer, uint32_t target, float* A, float* B) {
+  return get_pair(c, c ? c->cp : nullptr, c ? c->sp : nullptr, side, client, layer, target, A, B);
+}
+int splitlora_get_adapter_grad(splitlora_ctx* c, int side, int client, int layer, uint32_t target, float* dA, float* dB) {
+  return get_pair(c, c ? c->cg : nullptr, c ? c->sg : nullptr, side, client, layer, target, dA, dB);
+}
+int splitlora_get_opt_state(splitlora_ctx* c, int side, int client, int layer, uint32_t target, float* mA, float* vA,
+                            float* mB, float* vB) {
+  int rc = get_pair(c, c ? c->cm : nullptr, c ? c->sm : nullptr, side, client, layer, target, mA, mB);
+  if (rc) return rc;
+  return get_pair(c, c->cv, c->sv, side, client, layer, target, vA, vB);
+}
+int splitlora_set_opt_state(splitlora_ctx* c, int side, int client, int layer, uint32_t target, const float* mA,
+                            const float* vA, const float* mB, const float* vB) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
+  int rc;
+  float* pm = adapter_ptr(c, c->cm, c->sm, side, client, layer, target, &rc);
+  if (!pm) return rc;
+  float* pv = adapter_ptr(c, c->cv, c->sv, side, client, layer, target, &rc);
+  const size_t n = (size_t)c->r * c->d * 4, o = (size_t)c->r * c->d;
+  if (mA) CK(c, cudaMemcpyAsync(pm, mA, n, cudaMemcpyDeviceToDevice, c->st));
+  if (mB) CK(c, cudaMemcpyAsync(pm + o, mB, n, cudaMemcpyDeviceToDevice, c->st));
+  if (vA) CK(c, cudaMemcpyAsync(pv, vA, n, cudaMemcpyDeviceToDevice, c->st));
+  if (vB) CK(c, cudaMemcpyAsync(pv + o, vB, n, cudaMemcpyDeviceToDevice, c->st));
+  return SPLITLORA_OK;
+}
+int splitlora_get_counters(splitlora_ctx* c, int64_t* round_index, int64_t* server_steps, int64_t* client_steps) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  if (round_index) *round_index = c->round_index;
+  if (server_steps) *server_steps = c->server_steps;
+  if (client_steps) *client_steps = c->client_steps;
+  return SPLITLORA_OK;
+}
+int splitlora_set_counters(splitlora_ctx* c, int64_t round_index, int64_t server_steps, int64_t client_steps) {
+  if (!c || round_index < 0 || server_steps < 0 || client_steps < 0) return SPLITLORA_ERR_ARG;
+  c->round_index = round_index; c->server_steps = server_steps; c->client_steps = client_steps;
+  return SPLITLORA_OK;
+}
+
+// ---- Algorithm 1 ---------------------------------------------------------------------------
+
+int splitlora_client_fwd(splitlora_ctx* c, const int32_t* tokens, void* act_out) {
+  int rc = check_ready(c);
+  if (rc) return rc;
+  if (!tokens || !act_out) return fail(c, SPLITLORA_ERR_ARG, "null pointer");
+  if (!aligned16(tokens) || !aligned16(act_out)) return fail(c, SPLITLORA_ERR_ALIGN, "tokens / act_out not 16-byte aligned");
+  if (c->client_copies_dirty) { CK(c, refresh_side(c, true)); c->client_copies_dirty = false; }
+  { Scope s(c, "embed", 1);
+    CK(c, embed(c->dt, tokens, c->wte, c->wpe, c->emb, c->M, c->cfg.seq, c->d, c->V, c->st)); }
+  const void* x = c->emb;
+  for (int l = 0; l < c->cut; ++l) {
+    void* out = (l == c->cut - 1) ? act_out : c->lb[l].x_out;
+    CK(c, block_forward(c, l, x, out));
+    x = out;
+  }
+  c->have_client_fwd = true;
+  return SPLITLORA_OK;
+}
+
+int splitlora_server_step(splitlora_ctx* c, const void* act_in, const int32_t* labels, void* act_grad_out,
+                          float* loss_out) {
+  int rc = check_ready(c);
+  if (rc) return rc;
+  if (!act_in || !labels || !act_grad_out) return fail(c, SPLITLORA_ERR_ARG, "null pointer");
+  if (!aligned16(act_in) || !aligned16(labels) || !aligned16(act_grad_out)) return fail(c, SPLITLORA_ERR_ALIGN, "buffer not 16-byte aligned");
+  if (c->server_copies_dirty) { CK(c, refresh_side(c, false)); c->server_copies_dirty = false; }
+  const int M = c->M, d = c->d;
+  // forward over the concatenated batch S^t (Eq. 3)
+  const void* x = act_in;
+  for (int l = c->cut; l < c->L; ++l) {
+    CK(c, block_forward(c, l, x, c->lb[l].x_out));
+    x = c->lb[l].x_out;
+  }
+  { Scope s(c, "layernorm_fwd", 1);
+    CK(c, layernorm_fwd(c->dt, x, c->lnfg, c->lnfb, c->xf, c->meanf, c->rstdf, M, d, c->cfg.norm_eps, c->st)); }
+  { GemmArgs a = base_args(c, c->xf, d, c->wte, d, c->logits, c->Vpad, M, c->Vpad, d);
+    a.w_rows = c->V;
+    CK(c, linear(c, "head_fwd", a)); }
+  { Scope s(c, "cross_entropy", 3);
+    CK(c, cross_entropy(c->dt, c->logits, c->Vpad, labels, M, c->V, c->row_loss, c->n_valid, c->loss_dev, c->st)); }
+  // backward: head, final norm, blocks L-1 .. cut
+  { GemmArgs a = base_args(c, c->logits, c->Vpad, c->wteT, c->Vpad, c->g_a, d, M, d, c->Vpad);
+    CK(c, linear(c, "head_bwd", a)); }
+  void* cur = c->g_b;
+  { Scope s(c, "layernorm_bwd", 1);
+    CK(c, layernorm_bwd(c->dt, c->g_a, x, c->lnfg, c->meanf, c->rstdf, nullptr, cur, M, d, c->st)); }
+  void* other = c->g_a;
+  for (int l = c->L - 1; l >= c->cut; --l) {
+    void* dst = (l == c->cut) ? act_grad_out : other;
+    CK(c, block_backward(c, l, cur, dst));
+    other = cur; cur = dst;
+  }
+  // Eq. 4-5: server update
+  CK(c, run_optimizer(c, false));
+  c->server_copies_dirty = true;
+  if (loss_out) {
+    CK(c, cudaMemcpyAsync(loss_out, c->loss_dev, 4, cudaMemcpyDeviceToHost, c->st));
+    CK(c, cudaStreamSynchronize(c->st));
+    int code = 0;
+    CK(c, cudaMemcpy(&code, c->status, 4, cudaMemcpyDeviceToHost));
+    if (code) return fail(c, SPLITLORA_ERR_TIMEOUT, "a bounded device wait expired (code " + std::to_string(code) + ")");
+  }
+  return SPLITLORA_OK;
+}
+
+int splitlora_client_bwd(splitlora_ctx* c, const void* act_grad_in) {
+  int rc = check_ready(c);
+  if (rc) return rc;
+  if (!act_grad_in) return fail(c, SPLITLORA_ERR_ARG, "null pointer");
+  if (!aligned16(act_grad_in)) return fail(c, SPLITLORA_ERR_ALIGN, "act_grad_in not 16-byte aligned");
+  if (!c->have_client_fwd) return fail(c, SPLITLORA_ERR_STATE, "client_bwd needs a preceding client_fwd");
+  const void* cur = act_grad_in;
+  void* bufs[2] = {c->g_a, c->g_b};
+  int which = 0;
+  for (int l = c->cut - 1; l >= 0; --l) {
+    void* dst = (l == 0) ? nullptr : bufs[which];
+    CK(c, block_backward(c, l, cur, dst));
+    cur = dst; which ^= 1;
+  }
+  CK(c, run_optimizer(c, true));   // Eq. 6-7, all K clients in one launch
+  c->client_copies_dirty = true;
+  c->have_client_fwd = false;
+  return SPLITLORA_OK;
+}
+
+int splitlora_aggregate(splitlora_ctx* c, const int64_t* counts) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
+  if (!counts) return fail(c, SPLITLORA_ERR_ARG, "null counts");
+  double total = 0.0;
+  for (int i = 0; i < c->K; ++i) {
+    if (counts[i] < 0) return fail(c, SPLITLORA_ERR_COUNTS, "negative sample count");
+    total += (double)counts[i];
+  }
+  if (!(total > 0.0)) return fail(c, SPLITLORA_ERR_COUNTS, "all sample counts are zero");
+  float w[AGG_MAX_CLIENTS];
+  for (int i = 0; i < c->K; ++i) w[i] = (float)((double)counts[i] / total);
+  { Scope s(c, "aggregate", 1);
+    CK(c, aggregate(c->cp, c->K, c->Pc, w, c->st)); }
+  c->client_copies_dirty = true;
+  return SPLITLORA_OK;
+}
+
+int splitlora_round(splitlora_ctx* c, const int32_t* tokens, const int32_t* labels, const int64_t* counts,
+                    float* loss_out) {
+  int rc = check_ready(c);
+  if (rc) return rc;
+  if (!counts) return fail(c, SPLITLORA_ERR_ARG, "null counts");
+  if ((rc = splitlora_client_fwd(c, tokens, c->S))) return rc;
+  if ((rc = splitlora_server_step(c, c->S, labels, c->dS, nullptr))) return rc;
+  if ((rc = splitlora_client_bwd(c, c->dS))) return rc;
+  c->round_index++;
+  if (c->round_index % c->cfg.agg_interval == 0)
+    if ((rc = splitlora_aggregate(c, counts))) return rc;
+  if (loss_out) {
+    CK(c, cudaMemcpyAsync(loss_out, c->loss_dev, 4, cudaMemcpyDeviceToHost, c->st));
+    CK(c, cudaStreamSynchronize(c->st));
+    int code = 0;
+    CK(c, cudaMemcpy(&code, c->status, 4, cudaMemcpyDeviceToHost));
+    if (code) return fail(c, SPLITLORA_ERR_TIMEOUT, "a bounded device wait expired (code " + std::to_string(code) + ")");
+  }
+  return SPLITLORA_OK;
+}
+
+int splitlora_round_host(splitlora_ctx* c, const int32_t* tokens_host, const int32_t* labels_host,
+                         const int64_t* counts, float* loss_out) {
+  int rc = check_ready(c);
+  if (rc) return rc;
+  if (!tokens_host || !labels_host) return fail(c, SPLITLORA_ERR_ARG, "null pointer");
+  CK(c, cudaMemcpyAsync(c->tok_dev, tokens_host, (size_t)c->M * 4, cudaMemcpyHostToDevice, c->st));
+  CK(c, cudaMemcpyAsync(c->lab_dev, labels_host, (size_t)c->M * 4, cudaMemcpyHostToDevice, c->st));
+  return splitlora_round(c, c->tok_dev, c->lab_dev, counts, loss_out);
+}
+
+int splitlora_loss_device(splitlora_ctx* c, const float** loss_dev) {
+  if (!c || !loss_dev) return SPLITLORA_ERR_ARG;
+  if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
+  *loss_dev = c->loss_dev;
+  return SPLITLORA_OK;
+}
+
+const char* splitlora_last_error(const splitlora_ctx* c) { return c ? c->err.c_str() : "null context"; }
+
+int splitlora_device_status(splitlora_ctx* c, int32_t* code) {
+  if (!c || !code) return SPLITLORA_ERR_ARG;
+  if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
+  CK(c, cudaStreamSynchronize(c->st));
+  CK(c, cudaMemcpy(code, c->status, 4, cudaMemcpyDeviceToHost));
+  return SPLITLORA_OK;
+}
+
+int splitlora_launch_count(const splitlora_ctx* c, int64_t* launches) {
+  if (!c || !launches) return SPLITLORA_ERR_ARG;
+  *launches = c->launches;
+  return SPLITLORA_OK;
+}
+
+int splitlora_profile_enable(splitlora_ctx* c, int on) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  c->prof_on = on != 0;
+  return SPLITLORA_OK;
+}
+
+int splitlora_profile_report(splitlora_ctx* c, char (*names)[48], int64_t* launches, double* ms, int cap, int* n) {
+  if (!c || !n) return SPLITLORA_ERR_ARG;
+  CK(c, cudaStreamSynchronize(c->st));
+  std::vector<double> tot(c->prof_names.size(), 0.0);
+  std::vector<int64_t> cnt(c->prof_names.size(), 0);
+  for (auto& r : c->prof_recs) {
+    float t = 0.f;
+    CK(c, cudaEventElapsedTime(&t, r.a, r.b));
+    tot[r.cls] += t; cnt[r.cls] += 1;
+    c->event_pool.push_back(r.a); c->event_pool.push_back(r.b);
+  }
+  c->prof_recs.clear();
+  *n = (int)c->prof_names.size();
+  for (int i = 0; i < *n && i < cap; ++i) {
+    if (names) { std::strncpy(names[i], c->prof_names[i].c_str(), 47); names[i][47] = 0; }
+    if (launches) launches[i] = cnt[i];
+    if (ms) ms[i] = tot[i];
+  }
+  return SPLITLORA_OK;
+}
+
+}  // extern "C"
