@@ -293,7 +293,8 @@ def block_bwd(cfg: OracleConfig, params, l: int, adapters, dy, cache):
 def embed(cfg: OracleConfig, params, tokens):
     """x0[b, t, :] = wte[tokens[b, t], :] + wpe[t, :]  (input side of the client sub-model)."""
     nseq, T = tokens.shape
-    return params["wte"][tokens] + params["wpe"][:T][None, :, :]
+    # stored values (fp32 or bf16-exact) are widened to fp64 before the first addition
+    return params["wte"][tokens].astype(F64) + params["wpe"][:T][None, :, :].astype(F64)
 
 
 def client_fwd(cfg: OracleConfig, params, client_adapters: Sequence[dict], tokens):
