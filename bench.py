@@ -1,0 +1,304 @@
+#!/usr/bin/env python
+"""Benchmark of the split-LoRA round: training tokens/s on the GPT-2-medium-shaped workload.
+
+  python bench.py --gpus 1 --steps 10 --warmup 3            # the CUDA library
+  python bench.py --impl reference --steps 2 --warmup 1     # the CPU oracle on a bounded sample
+
+A step is one full round of Algorithm 1 (client forward, server step, client backward and the
+weighted aggregation) over one batch of synthetic tokens.  Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2407_00952_b200 import synth  # noqa: E402
+
+METRIC = "split-LoRA training tokens/sec"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    """Measured roofline denominators; falls back to an earlier measurement on the same pool."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], tflops_burst=p["bf16_tflops"], tflops_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+def workload_description(w):
+    return {"workload": f"cfg{w.index} {w.name}: L={w.n_layer} cut={w.cut} d={w.d_model} H={w.n_head} F={w.d_ff} "
+                        f"V={w.vocab} T={w.seq} r={w.lora_r} alpha={w.lora_alpha:g} targets={''.join(w.targets)} "
+                        f"K={w.n_clients} b={w.batch_per_client} I={w.agg_interval} AdamW",
+            "tokens_per_step": w.tokens_per_round,
+            "l2": "inputs larger than L2 (the activations of one step exceed 126 MB many times over)"}
+
+
+def gemm_flops_per_round(w):
+    """Algorithmic FLOPs of the tensor-core linear layers per round, by launch class (no dW)."""
+    M, d, F, V, L = w.tokens_per_round, w.d_model, w.d_ff, w.vocab, w.n_layer
+    nt, r = len(w.targets), w.lora_r
+    return {
+        "lora_linear_fwd": L * (2.0 * M * d * 3 * d + 2.0 * M * r * d * nt),
+        "linear_fwd": L * (2.0 * M * d * d + 4.0 * M * d * F),
+        "linear_bwd": L * (2.0 * M * d * d + 4.0 * M * d * F),
+        "lora_linear_bwd": (L - 1) * (2.0 * M * 3 * d * d + 2.0 * M * r * d * nt),
+        "head_fwd": 2.0 * M * d * V,
+        "head_bwd": 2.0 * M * d * V,
+    }
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("uuid,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.uuid = uuid
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        self.proc.wait()
+        self.tmp.flush()
+        rows = [l.strip().split(", ") for l in open(self.tmp.name) if l.strip()]
+        os.unlink(self.tmp.name)
+        rows = [r for r in rows if len(r) >= 9]
+        mine = [r for r in rows if self.uuid and self.uuid in r[0]] or rows
+        if not mine:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = sorted(float(r[1]) for r in mine)
+        reasons = set()
+        for r in mine:
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if v.strip().lower() == "active":
+                    reasons.add(name)
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(mine[0][2]), "samples": len(mine),
+                "power_w_max": max(float(r[3]) for r in mine), "reasons": sorted(reasons)}
+
+
+def oracle_sample_workload(w):
+    """The bounded sample the CPU oracle is timed on: same model, 2 clients x 1 sequence."""
+    return synth.scaled(w, n_clients=min(2, w.n_clients), batch_per_client=1, counts=None)
+
+
+def time_oracle_rounds(w, steps, warmup):
+    """Times oracle rounds (as the oracle stands) on the host cores."""
+    from oracle import splitlora_oracle as O
+    ws = oracle_sample_workload(w)
+    frozen = synth.make_frozen(ws)          # fp32 arrays holding bf16-exact values; widened on use
+    cads = [synth.make_adapters(ws, range(ws.cut)) for _ in range(ws.n_clients)]
+    sads = synth.make_adapters(ws, range(ws.cut, ws.n_layer))
+    to64 = lambda a: {k: {"A": v["A"].astype(np.float64), "B": v["B"].astype(np.float64)} for k, v in a.items()}
+    st = O.OracleState(client_adapters=[to64(a) for a in cads], server_adapters=to64(sads))
+    cfg = O.OracleConfig(n_layer=ws.n_layer, cut=ws.cut, d_model=ws.d_model, n_head=ws.n_head, d_ff=ws.d_ff,
+                         vocab=ws.vocab, max_seq=ws.max_seq, lora_r=ws.lora_r, lora_alpha=ws.lora_alpha,
+                         targets=ws.targets, n_clients=ws.n_clients, batch_per_client=ws.batch_per_client, seq=ws.seq,
+                         bf16_handoff=(ws.dtype == "bf16"), optimizer="adamw", lr_client=ws.lr, lr_server=ws.lr,
+                         agg_interval=ws.agg_interval)
+    counts = synth.make_counts(ws)
+    times = []
+    for s in range(warmup + steps):
+        tokens, labels = synth.make_tokens(ws, round_index=s)
+        t0 = time.perf_counter()
+        O.split_round(cfg, frozen, st, tokens, labels, counts)
+        dt = time.perf_counter() - t0
+        if s >= warmup:
+            times.append(dt)
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    sec = float(np.mean(times))
+    return ws.tokens_per_round / sec, sec, threads, ws
+
+
+def sample_text(ws, sec=None):
+    s = (f"one oracle round (numpy fp64) of the same model on {ws.n_clients} clients x {ws.batch_per_client} "
+         f"sequence x {ws.seq} tokens = {ws.tokens_per_round} tokens")
+    return s + (f" ({sec:.1f} s)" if sec is not None else "")
+
+
+def run_reference(args, w):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    tps, sec, threads, ws = time_oracle_rounds(w, args.steps, args.warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": workload_description(w),
+            "cpu_baseline": {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample_text(ws)},
+            "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def run_gpu(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2407_00952_b200 import runner
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    frozen = synth.make_frozen(w)
+    cads = [synth.make_adapters(w, range(w.cut)) for _ in range(w.n_clients)]
+    sads = synth.make_adapters(w, range(w.cut, w.n_layer))
+    eng = runner.make_engine(w, frozen, cads, sads, optimizer="adamw")
+    del frozen
+    counts = synth.make_counts(w)
+    nbatch = 4
+    host_tok, host_lab, dev_tok, dev_lab = [], [], [], []
+    for s in range(nbatch):
+        t, l = synth.make_tokens(w, round_index=1000 * rank + s)
+        host_tok.append(torch.from_numpy(t).pin_memory())
+        host_lab.append(torch.from_numpy(l).pin_memory())
+        dev_tok.append(host_tok[-1].cuda())
+        dev_lab.append(host_lab[-1].cuda())
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident inputs: the headline value ----
+    for s in range(args.warmup):
+        eng.round(dev_tok[s % nbatch], dev_lab[s % nbatch], counts, want_loss=False)
+    barrier()
+    try:
+        uuid = str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        uuid = None
+    sampler = ClockSampler(uuid)
+    sampler.start()
+    eng.profile_enable(True)
+    eng.profile_report()                         # drop anything recorded before
+    launches0 = eng.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for s in range(args.steps):
+        eng.round(dev_tok[s % nbatch], dev_lab[s % nbatch], counts, want_loss=False)
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = eng.launch_count() - launches0
+    prof = eng.profile_report()
+    eng.profile_enable(False)
+    clocks = sampler.stop()
+    status = eng.device_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status}: a bounded wait expired")
+
+    # ---- end to end: host tokens in, host loss out, every step ----
+    for s in range(2):
+        eng.round_host(host_tok[s % nbatch], host_lab[s % nbatch], counts, want_loss=True)
+    barrier()
+    e0.record(stream)
+    losses = []
+    for s in range(args.steps):
+        losses.append(eng.round_host(host_tok[s % nbatch], host_lab[s % nbatch], counts, want_loss=True))
+    e1.record(stream)
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    tokens_total = w.tokens_per_round * args.steps * world
+    value = tokens_total / (ms * 1e-3)
+    e2e_value = tokens_total / (ms_e2e * 1e-3)
+    peaks = load_peaks()
+    fl = gemm_flops_per_round(w)
+    t_ms = sum(prof[k][1] for k in fl if k in prof)
+    n_launch = sum(prof[k][0] for k in fl if k in prof)
+    flops = sum(fl[k] for k in fl if k in prof) * args.steps
+    achieved = flops / (t_ms * 1e-3) / 1e12 if t_ms > 0 else 0.0
+    peak = peaks["tflops_sustained"]
+    by_class = {k: {"launches": prof[k][0], "ms_total": round(prof[k][1], 3),
+                    "tflops": round(fl[k] * args.steps / (prof[k][1] * 1e-3) / 1e12, 1)}
+                for k in fl if k in prof and prof[k][1] > 0}
+    roofline = {"bound": "tensor",
+                "kernel": "gemm_tc_kernel (tcgen05 linear layers incl. the LoRA-fused projections; skinny rank-r "
+                          "down-projections excluded)",
+                "achieved": round(achieved, 1), "peak": peak, "unit": "TFLOP/s",
+                "frac": round(achieved / peak, 4) if peak else None,
+                "peak_source": f"{peaks['source']} sustained bf16 (kernel timed inside a long step)",
+                "traffic": None, "launches": n_launch, "avg_launch_us": round(t_ms * 1e3 / max(1, n_launch), 2),
+                "by_class": by_class, "share_of_step": round(t_ms / ms, 4)}
+    breakdown = {k: {"launches": v[0], "ms_per_step": round(v[1] / args.steps, 3)}
+                 for k, v in sorted(prof.items(), key=lambda kv: -kv[1][1])}
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        tps, sec, threads, ws = time_oracle_rounds(w, 1, 0)
+        cpu = {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample_text(ws, sec)}
+
+    M = w.tokens_per_round
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": dict(workload_description(w), parallelism="1 GPU" if world == 1 else f"{world} independent replicas"),
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 2 * M * 4, "d2h_bytes_per_step": 4,
+                    "ms_per_step": ms_e2e / args.steps, "last_loss": losses[-1]},
+            "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu, "kernel_breakdown": breakdown}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=3, help="workload index (3 = GPT-2-medium-shaped, the headline)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "ours":
+        args.warmup = max(args.warmup, 3)
+    w = synth.WORKLOADS[args.config]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_gpu(args, w)
+
+
+if __name__ == "__main__":
+    main()
