@@ -258,99 +258,6 @@ cudaError_t cross_entropy(int dt, void* logits, int64_t ld, const int32_t* label
 }
 
 // ------------------------------------------------------------------------------------------
-// adapter gradients: out[g][j][c] = scale * sum_{m in g} Wt[m, wcol0 + j] * Z[m, zcol0 + c]
-// Column-parallel: a thread owns one 16-byte vector of columns and RJ weight columns; rows of a
-// group are split into chunks of LG_ROWS, partial sums go to scratch and are summed in chunk order.
-// ------------------------------------------------------------------------------------------
-static const int LG_ROWS = 256;
-static const int LG_RJ = 4;
-
-template <typename T>
-__global__ void lora_grad_partial_kernel(const T* __restrict__ Z, int64_t ldz, int zcol0, int C,
-                                         const T* __restrict__ Wt, int64_t ldwt, int wcol0, int R, int M,
-                                         float* __restrict__ partial) {
-  constexpr int N = Vec16<T>::N;
-  int cv = blockIdx.x * blockDim.x + threadIdx.x;      // vector column index
-  int c = cv * N;
-  int chunk = blockIdx.y;
-  int j0 = blockIdx.z * LG_RJ;
-  int m0 = chunk * LG_ROWS;
-  int m1 = min(m0 + LG_ROWS, M);
-  if (c >= C) return;
-  float acc[LG_RJ][N];
-#pragma unroll
-  for (int j = 0; j < LG_RJ; ++j)
-#pragma unroll
-    for (int i = 0; i < N; ++i) acc[j][i] = 0.f;
-  for (int m = m0; m < m1; ++m) {
-    Vec16<T> v; v.load(Z + (size_t)m * ldz + zcol0 + c);
-    float w[LG_RJ];
-#pragma unroll
-    for (int j = 0; j < LG_RJ; ++j) w[j] = (j0 + j < R) ? to_f<T>(Wt[(size_t)m * ldwt + wcol0 + j0 + j]) : 0.f;
-#pragma unroll
-    for (int i = 0; i < N; ++i) {
-      float zv = v.get(i);
-#pragma unroll
-      for (int j = 0; j < LG_RJ; ++j) acc[j][i] = fmaf(w[j], zv, acc[j][i]);
-    }
-  }
-  // partial layout: [chunk][R][C]
-#pragma unroll
-  for (int j = 0; j < LG_RJ; ++j) {
-    if (j0 + j < R) {
-      float* p = partial + ((size_t)chunk * R + (j0 + j)) * C + c;
-#pragma unroll
-      for (int i = 0; i < N; ++i) p[i] = acc[j][i];
-    }
-  }
-}
-
-__global__ void lora_grad_reduce_kernel(const float* __restrict__ partial, int R, int C, int chunks_per_group,
-                                        float scale, float* __restrict__ out, int64_t out_group_stride,
-                                        int64_t out_sj, int64_t out_sc) {
-  int idx = blockIdx.x * blockDim.x + threadIdx.x;   // over R*C
-  int g = blockIdx.y;
-  if (idx >= R * C) return;
-  int j = idx / C, c = idx % C;
-  float s = 0.f;
-  for (int k = 0; k < chunks_per_group; ++k)
-    s += partial[((size_t)(g * chunks_per_group + k) * R + j) * C + c];
-  out[(size_t)g * out_group_stride + (size_t)j * out_sj + (size_t)c * out_sc] = scale * s;
-}
-
-size_t lora_grad_scratch_floats(int M, int rows_per_group, int R, int C) {
-  (void)rows_per_group;
-  size_t chunks = (size_t)(M + LG_ROWS - 1) / LG_ROWS;
-  return chunks * (size_t)R * (size_t)C;
-}
-
-cudaError_t lora_grad(int dt, const void* Z, int64_t ldz, int zcol0, int C, const void* Wt, int64_t ldwt,
-                      int wcol0, int R, int M, int rows_per_group, float scale, float* out,
-                      int64_t out_group_stride, int64_t out_sj, int64_t out_sc, float* partial,
-                      cudaStream_t st) {
-  const int rpg = rows_per_group > 0 ? rows_per_group : M;
-  const int n = dt == DT_BF16 ? 8 : 4;
-  const int chunks = (M + LG_ROWS - 1) / LG_ROWS;
-  int chunks_per_group, groups;
-  if (rpg >= M) { groups = 1; chunks_per_group = chunks; }
-  else {
-    // row chunks must not straddle groups
-    if (rpg % LG_ROWS != 0 || M % rpg != 0) return cudaErrorInvalidValue;
-    groups = M / rpg; chunks_per_group = rpg / LG_ROWS;
-  }
-  if (C % n != 0) return cudaErrorInvalidValue;
-  int cvec = C / n;
-  dim3 grid((cvec + 127) / 128, chunks, (R + LG_RJ - 1) / LG_RJ);
-  if (dt == DT_BF16)
-    lora_grad_partial_kernel<bf16><<<grid, 128, 0, st>>>((const bf16*)Z, ldz, zcol0, C, (const bf16*)Wt, ldwt, wcol0, R, M, partial);
-  else
-    lora_grad_partial_kernel<float><<<grid, 128, 0, st>>>((const float*)Z, ldz, zcol0, C, (const float*)Wt, ldwt, wcol0, R, M, partial);
-  dim3 g2((R * C + 255) / 256, groups);
-  lora_grad_reduce_kernel<<<g2, 256, 0, st>>>(partial, R, C, chunks_per_group, scale, out, out_group_stride, out_sj, out_sc);
-  return cudaGetLastError();
-}
-
-// ------------------------------------------------------------------------------------------
 // optimizer on adapter parameters only (Eq. 4-7; AdamW as configured)
 // ------------------------------------------------------------------------------------------
 __global__ void optimizer_kernel(float* __restrict__ p, const float* __restrict__ g, float* __restrict__ m,

@@ -9,8 +9,9 @@
 // through a second pair of tensor maps whose rows are selected by the row group (client) of the
 // tile, so K clients with their own adapters share one pass over the frozen W.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = tensor-memory owner + MMA issuer,
-// warps 2..5 = epilogue (each owns the 32 accumulator lanes its warp id modulo 4 selects).
+// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = tensor-memory owner + MMA issuer,
+// warps 2..9 = epilogue (a warp reads the 32 accumulator lanes its warp id modulo 4 selects; the
+// two warps of a lane quarter take one half of the tile's columns each).
 // Every wait on an mbarrier is bounded: when it expires the kernel records a code in `status`,
 // stops issuing work, waits briefly for copies in flight, frees its tensor memory and returns.
 #include <cuda.h>
@@ -24,7 +25,7 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;            // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;
 constexpr int GROUP_M = 16;       // output tiles are walked in bands of GROUP_M tile rows
 constexpr unsigned long long WAIT_LIMIT_NS = 4000000000ull;
 
@@ -187,7 +188,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -274,6 +275,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
   } else {
     // ---------------- epilogue ----------------
     const int q = warp & 3;                     // lanes [32q, 32q+32) of tensor memory
+    const int half = (warp - 2) >> 2;           // two warps share a lane quarter and split the columns
+    const int c_begin = half * (BN / 2), c_end = c_begin + BN / 2;
     int as = 0; uint32_t aphase = 0;
     const bool tanh_form = p.gelu_tanh != 0;
     bool ok = true;
@@ -285,7 +288,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN);
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
+      for (int c = c_begin; c < c_end; c += 32) {
         const int n = n0 + c;
         if (n >= p.N) break;                    // warp-uniform
         float v[32];

@@ -76,14 +76,16 @@ cudaError_t attention_fwd_tc(const void* qkv, int nseq, int T, int H, int d, voi
 cudaError_t attention_bwd_tc(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq,
                              int T, int H, int d, void* dqkv, float* rowdot, cudaStream_t st);
 
-// out[g][j][c] = scale * sum_{m in group g} Wt[m, wcol0 + j] * Z[m, zcol0 + c],  j < R, c < C.
-// Stored at out + g*out_group_stride with element (j, c) at j*out_sj + c*out_sc.
-// partial: scratch of at least lora_grad_scratch_floats(...) floats.
-size_t lora_grad_scratch_floats(int M, int rows_per_group, int R, int C);
+// Adapter gradients: for nt targets of rank r (weight columns wcol0 + t*rp + jj of Wt),
+//   out[g][t][jj][c] = scale * sum_{m in group g} Wt[m, wcol0 + t*rp + jj] * Z[m, zcol0 + c],  c < C,
+// stored at out + g*out_group_stride + t*out_target_stride + jj*out_sj + c*out_sc.
+// rows_per_group (0: one group) must be a multiple of 128.  partial: scratch of at least
+// lora_grad_scratch_floats(M, nt*r, C) floats.
+size_t lora_grad_scratch_floats(int M, int R, int C);
 cudaError_t lora_grad(int dt, const void* Z, int64_t ldz, int zcol0, int C, const void* Wt, int64_t ldwt,
-                      int wcol0, int R, int M, int rows_per_group, float scale, float* out,
-                      int64_t out_group_stride, int64_t out_sj, int64_t out_sc, float* partial,
-                      cudaStream_t st);
+                      int wcol0, int r, int rp, int nt, int M, int rows_per_group, float scale, float* out,
+                      int64_t out_group_stride, int64_t out_target_stride, int64_t out_sj, int64_t out_sc,
+                      float* partial, cudaStream_t st);
 
 struct OptArgs {
   int optimizer; float lr, beta1, beta2, eps, wd; float bc1, bc2;   // bc = 1 - beta^step

@@ -1,0 +1,145 @@
+// Adapter gradients G_A, G_B (Eq. 4-7): skinny reductions over the tokens of each group,
+//   out[g][t][jj][c] = scale * sum_{m in group g} Wt[m, wcol0 + t*rp + jj] * Z[m, zcol0 + c]
+// for nt targets of rank r (R = nt*r weight columns) and C feature columns.  HBM-bound: Z is read
+// once per RJ weight columns.  A block is 128 column threads (one 16-byte vector each) x 4 row
+// lanes over a chunk of LG_ROWS rows; the row lanes are summed through shared memory, chunk
+// partials go to scratch and a second kernel adds them in chunk order (no float atomics, so the
+// result does not depend on scheduling).
+#include "common.cuh"
+#include "kernels.h"
+
+namespace sl {
+namespace {
+
+constexpr int LG_ROWS = 128;   // rows per chunk; group sizes must be multiples of it
+constexpr int LG_CT = 128;     // column threads per block
+constexpr int LG_RL = 4;       // row lanes per block
+
+template <typename T, int RJ>
+__global__ void __launch_bounds__(LG_CT * LG_RL)
+lora_grad_partial_kernel(const T* __restrict__ Z, int64_t ldz, int zcol0, int C, const T* __restrict__ Wt,
+                         int64_t ldwt, int wcol0, int r, int rp, int R, int M, float* __restrict__ partial) {
+  constexpr int N = Vec16<T>::N;
+  __shared__ float red[RJ * N][LG_CT];
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  const int c = (blockIdx.x * LG_CT + tx) * N;
+  const int chunk = blockIdx.y;
+  const int j0 = blockIdx.z * RJ;
+  const int m0 = chunk * LG_ROWS;
+  const int m1 = min(m0 + LG_ROWS, M);
+  const bool active = c < C;
+  int wc[RJ];
+#pragma unroll
+  for (int j = 0; j < RJ; ++j) {
+    int jj = j0 + j;
+    wc[j] = jj < R ? wcol0 + (jj / r) * rp + (jj % r) : -1;
+  }
+  float acc[RJ][N];
+#pragma unroll
+  for (int j = 0; j < RJ; ++j)
+#pragma unroll
+    for (int i = 0; i < N; ++i) acc[j][i] = 0.f;
+  if (active) {
+#pragma unroll 4
+    for (int m = m0 + ty; m < m1; m += LG_RL) {
+      Vec16<T> v; v.load(Z + (size_t)m * ldz + zcol0 + c);
+      float w[RJ];
+#pragma unroll
+      for (int j = 0; j < RJ; ++j) w[j] = wc[j] >= 0 ? to_f<T>(Wt[(size_t)m * ldwt + wc[j]]) : 0.f;
+#pragma unroll
+      for (int i = 0; i < N; ++i) {
+        float zv = v.get(i);
+#pragma unroll
+        for (int j = 0; j < RJ; ++j) acc[j][i] = fmaf(w[j], zv, acc[j][i]);
+      }
+    }
+  }
+  // add row lanes 1..3 into lane 0, one lane at a time (fixed order)
+  for (int lane = 1; lane < LG_RL; ++lane) {
+    if (ty == lane) {
+#pragma unroll
+      for (int j = 0; j < RJ; ++j)
+#pragma unroll
+        for (int i = 0; i < N; ++i) red[j * N + i][tx] = acc[j][i];
+    }
+    __syncthreads();
+    if (ty == 0) {
+#pragma unroll
+      for (int j = 0; j < RJ; ++j)
+#pragma unroll
+        for (int i = 0; i < N; ++i) acc[j][i] += red[j * N + i][tx];
+    }
+    __syncthreads();
+  }
+  if (ty == 0 && active) {
+    // partial layout: [chunk][R][C]
+#pragma unroll
+    for (int j = 0; j < RJ; ++j) {
+      if (j0 + j < R) {
+        float* p = partial + ((size_t)chunk * R + (j0 + j)) * C + c;
+#pragma unroll
+        for (int i = 0; i < N; i += 4)
+          *reinterpret_cast<float4*>(p + i) = make_float4(acc[j][i], acc[j][i + 1], acc[j][i + 2], acc[j][i + 3]);
+      }
+    }
+  }
+}
+
+__global__ void lora_grad_reduce_kernel(const float* __restrict__ partial, int r, int R, int C, int chunks_per_group,
+                                        float scale, float* __restrict__ out, int64_t out_group_stride,
+                                        int64_t out_target_stride, int64_t out_sj, int64_t out_sc) {
+  int idx = blockIdx.x * blockDim.x + threadIdx.x;   // over R*C
+  int g = blockIdx.y;
+  if (idx >= R * C) return;
+  int j = idx / C, c = idx % C;
+  float s = 0.f;
+  for (int k = 0; k < chunks_per_group; ++k)
+    s += partial[((size_t)(g * chunks_per_group + k) * R + j) * C + c];
+  out[(size_t)g * out_group_stride + (size_t)(j / r) * out_target_stride + (size_t)(j % r) * out_sj +
+      (size_t)c * out_sc] = scale * s;
+}
+
+template <typename T>
+void launch_partial(dim3 grid, cudaStream_t st, int RJ, const void* Z, int64_t ldz, int zcol0, int C, const void* Wt,
+                    int64_t ldwt, int wcol0, int r, int rp, int R, int M, float* partial) {
+  dim3 block(LG_CT, LG_RL);
+  if (RJ == 8)
+    lora_grad_partial_kernel<T, 8><<<grid, block, 0, st>>>((const T*)Z, ldz, zcol0, C, (const T*)Wt, ldwt, wcol0, r, rp, R, M, partial);
+  else
+    lora_grad_partial_kernel<T, 4><<<grid, block, 0, st>>>((const T*)Z, ldz, zcol0, C, (const T*)Wt, ldwt, wcol0, r, rp, R, M, partial);
+}
+
+}  // namespace
+
+size_t lora_grad_scratch_floats(int M, int R, int C) {
+  size_t chunks = (size_t)(M + LG_ROWS - 1) / LG_ROWS;
+  return chunks * (size_t)R * (size_t)C;
+}
+
+cudaError_t lora_grad(int dt, const void* Z, int64_t ldz, int zcol0, int C, const void* Wt, int64_t ldwt, int wcol0,
+                      int r, int rp, int nt, int M, int rows_per_group, float scale, float* out,
+                      int64_t out_group_stride, int64_t out_target_stride, int64_t out_sj, int64_t out_sc,
+                      float* partial, cudaStream_t st) {
+  const int R = nt * r;
+  const int rpg = rows_per_group > 0 ? rows_per_group : M;
+  const int n = dt == DT_BF16 ? 8 : 4;
+  const int chunks = (M + LG_ROWS - 1) / LG_ROWS;
+  int chunks_per_group, groups;
+  if (rpg >= M) { groups = 1; chunks_per_group = chunks; }
+  else {
+    if (rpg % LG_ROWS != 0 || M % rpg != 0) return cudaErrorInvalidValue;   // chunks must not straddle groups
+    groups = M / rpg; chunks_per_group = rpg / LG_ROWS;
+  }
+  if (C % n != 0 || R < 1) return cudaErrorInvalidValue;
+  const int RJ = (dt == DT_BF16) ? (R > 4 ? 8 : 4) : 4;     // fp32 vectors are 4 wide: keep registers in check
+  const int cvec = C / n;
+  dim3 grid((cvec + LG_CT - 1) / LG_CT, chunks, (R + RJ - 1) / RJ);
+  if (dt == DT_BF16) launch_partial<bf16>(grid, st, RJ, Z, ldz, zcol0, C, Wt, ldwt, wcol0, r, rp, R, M, partial);
+  else launch_partial<float>(grid, st, RJ, Z, ldz, zcol0, C, Wt, ldwt, wcol0, r, rp, R, M, partial);
+  dim3 g2((R * C + 255) / 256, groups);
+  lora_grad_reduce_kernel<<<g2, 256, 0, st>>>(partial, r, R, C, chunks_per_group, scale, out, out_group_stride,
+                                              out_target_stride, out_sj, out_sc);
+  return cudaGetLastError();
+}
+
+}  // namespace sl

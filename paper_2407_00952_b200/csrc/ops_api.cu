@@ -31,7 +31,7 @@ LinearPlan plan_linear(int dtype, int M, int n_in, int n_out, int r, int G) {
   p.off_bextT = take((size_t)G * p.ext * n_out * es);
   p.off_h = take((size_t)M * p.ext * es);
   p.off_dh = take((size_t)M * p.ext * es);
-  size_t sc = lora_grad_scratch_floats(M, M / G, r, n_in > n_out ? n_in : n_out);
+  size_t sc = lora_grad_scratch_floats(M, r, n_in > n_out ? n_in : n_out);
   p.off_scratch = take(sc * 4);
   p.total = align_up(off, 256);
   return p;
@@ -41,7 +41,7 @@ int check_linear(int dtype, int M, int n_in, int n_out, int r, int G) {
   if (dtype != DT_F32 && dtype != DT_BF16) return SPLITLORA_ERR_ARG;
   if (M < 1 || n_in < 8 || n_out < 8 || r < 1 || r > 64 || G < 1 || M % G != 0) return SPLITLORA_ERR_ARG;
   if (n_in % 8 != 0 || n_out % 8 != 0) return SPLITLORA_ERR_ARG;
-  if (G > 1 && (M / G) % 256 != 0) return SPLITLORA_ERR_ARG;
+  if (G > 1 && (M / G) % 128 != 0) return SPLITLORA_ERR_ARG;
   return SPLITLORA_OK;
 }
 
@@ -146,9 +146,9 @@ int splitlora_lora_linear_bwd(int dtype, int use_tc, const void* x, const void* 
   a.Xe = ws + p.off_dh; a.ldxe = p.ext; a.We = ws + p.off_acatT; a.ldwe = p.ext; a.Ke = p.rp; a.we_grouped = G > 1;
   if (run_gemm(use_tc, a, status, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
   float* scratch = (float*)(ws + p.off_scratch);
-  if (lora_grad(dtype, x, n_in, 0, n_in, ws + p.off_dh, p.ext, 0, r, M, rpg, 1.0f, dA, (int64_t)r * n_in, n_in, 1,
+  if (lora_grad(dtype, x, n_in, 0, n_in, ws + p.off_dh, p.ext, 0, r, p.rp, 1, M, rpg, 1.0f, dA, (int64_t)r * n_in, 0, n_in, 1,
                 scratch, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
-  if (lora_grad(dtype, dy, n_out, 0, n_out, ws + p.off_h, p.ext, 0, r, M, rpg, s, dB, (int64_t)n_out * r, 1, r,
+  if (lora_grad(dtype, dy, n_out, 0, n_out, ws + p.off_h, p.ext, 0, r, p.rp, 1, M, rpg, s, dB, (int64_t)n_out * r, 0, 1, r,
                 scratch, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
   return SPLITLORA_OK;
 }

@@ -189,7 +189,7 @@ size_t plan(splitlora_ctx* c, char* ws) {
   c->xf = a.take(M * d * es); c->logits = a.take(M * (size_t)c->Vpad * es);
   c->meanf = (float*)a.take(M * 4); c->rstdf = (float*)a.take(M * 4); c->row_loss = (float*)a.take(M * 4);
   c->rowdot = (float*)a.take((size_t)c->nseq * c->cfg.n_head * c->cfg.seq * 4);
-  c->grad_scratch = (float*)a.take(lora_grad_scratch_floats(c->M, c->rows_per_client, c->r, c->d) * 4);
+  c->grad_scratch = (float*)a.take(lora_grad_scratch_floats(c->M, c->n_targets * c->r, c->d) * 4);
   c->g_a = a.take(M * d * es); c->g_b = a.take(M * d * es); c->g_dz = a.take(M * F * es);
   c->g_du2 = a.take(M * d * es); c->g_dxmid = a.take(M * d * es); c->g_do = a.take(M * d * es);
   c->g_dqkv = a.take(M * 3 * d * es); c->g_dhcat = a.take(M * ext * es); c->g_du = a.take(M * d * es);
@@ -339,15 +339,14 @@ cudaError_t block_backward(splitlora_ctx* c, int l, const void* dy, void* dx) {
   // G_A = dh^T u, G_B = (alpha/r) dy^T h, per group (Eq. 4-7)
   float* gbase = client ? c->cg + (size_t)l * c->per_layer : c->sg + (size_t)(l - c->cut) * c->per_layer;
   const int64_t gstride = client ? c->Pc : 0;
+  { Scope s(c, "lora_grad", 2);   // every target's G_A in one pass over u
+    if ((e = lora_grad(c->dt, b.u, d, 0, d, c->g_dhcat, ext, 0, c->r, c->rp, c->n_targets, M, rpg, 1.0f, gbase,
+                       gstride, (int64_t)2 * c->r * d, d, 1, c->grad_scratch, c->st))) return e; }
   for (int t = 0; t < c->n_targets; ++t) {
-    float* gA = gbase + (size_t)t * 2 * c->r * d;
-    float* gB = gA + (size_t)c->r * d;
-    { Scope s(c, "lora_grad", 2);
-      if ((e = lora_grad(c->dt, b.u, d, 0, d, c->g_dhcat, ext, t * c->rp, c->r, M, rpg, 1.0f, gA, gstride, d, 1,
-                         c->grad_scratch, c->st))) return e; }
-    { Scope s(c, "lora_grad", 2);
-      if ((e = lora_grad(c->dt, c->g_dqkv, 3 * d, c->slice_idx[t] * d, d, b.hcat, ext, t * c->rp, c->r, M, rpg,
-                         c->scale, gB, gstride, 1, c->r, c->grad_scratch, c->st))) return e; }
+    float* gB = gbase + (size_t)t * 2 * c->r * d + (size_t)c->r * d;
+    Scope s(c, "lora_grad", 2);
+    if ((e = lora_grad(c->dt, c->g_dqkv, 3 * d, c->slice_idx[t] * d, d, b.hcat, ext, t * c->rp, c->r, c->rp, 1, M,
+                       rpg, c->scale, gB, gstride, 0, 1, c->r, c->grad_scratch, c->st))) return e;
   }
   if (dx) {
     GemmArgs a = base_args(c, c->g_dqkv, 3 * d, f.qkvwT, 3 * d, c->g_du, d, M, d, 3 * d);
