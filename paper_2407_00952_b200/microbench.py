@@ -1,0 +1,146 @@
+"""Operator micro-benchmarks through the C ABI: the grouped LoRA linear layer (forward / backward),
+the Eq. 8-9 aggregation and causal attention.  Prints one JSON line per case.
+
+  python -m paper_2407_00952_b200.microbench linear --M 32768 --n-in 1024 --n-out 3072 --r 4 --G 8
+  python -m paper_2407_00952_b200.microbench linear-sweep [--quick]
+  python -m paper_2407_00952_b200.microbench aggregate-sweep
+  python -m paper_2407_00952_b200.microbench attention --nseq 64 --T 512 --heads 16
+
+Timing: CUDA events on the launching stream, warm-up first; operands are rotated over several
+buffer sets when one set would fit in L2.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import torch
+
+from . import binding as B
+
+L2_BYTES = 126 * 2 ** 20
+
+
+def _peaks():
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return p["hbm_gbs"], p["bf16_tflops"], "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+def _time(fn, iters, warmup=3):
+    for _ in range(warmup):
+        fn(0)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(iters):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def bench_linear(M, n_in, n_out, r, G, iters=20, backward=True, tc=True):
+    hbm, tflops, src = _peaks()
+    set_bytes = 2 * (M * n_in + M * n_out + n_in * n_out)
+    nset = max(1, min(4, -(-2 * L2_BYTES // set_bytes)))
+    g = torch.Generator(device="cuda").manual_seed(1)
+    mk = lambda *s, sc=1.0: (torch.randn(*s, device="cuda", generator=g) * sc).bfloat16()
+    xs = [mk(M, n_in) for _ in range(nset)]
+    dys = [mk(M, n_out, sc=n_out ** -0.5) for _ in range(nset)]
+    ys = [torch.empty(M, n_out, device="cuda", dtype=torch.bfloat16) for _ in range(nset)]
+    W = mk(n_out, n_in, sc=n_in ** -0.5)
+    Wt = B.transpose(W)
+    A = torch.randn(G, r, n_in, device="cuda", generator=g) * n_in ** -0.5
+    Bm = torch.randn(G, n_out, r, device="cuda", generator=g) * r ** -0.5
+    ws = B.lora_linear_workspace(B.DTYPE_BF16, M, n_in, n_out, r, G)
+    fwd = _time(lambda i: B.lora_linear_fwd(xs[i % nset], W, None, A, Bm, 16.0, y=ys[i % nset], workspace=ws,
+                                            use_tensor_cores=tc), iters)
+    flops = 2.0 * M * n_in * n_out + 2.0 * M * r * (n_in + n_out)
+    out = {"op": "lora_linear", "M": M, "n_in": n_in, "n_out": n_out, "r": r, "G": G,
+           "fwd_us": round(fwd * 1e3, 1), "fwd_tflops": round(flops / fwd / 1e9, 1),
+           "fwd_frac_of_bf16_peak": round(flops / fwd / 1e9 / tflops, 3), "peak_source": src + " burst"}
+    if backward:
+        bwd = _time(lambda i: B.lora_linear_bwd(xs[i % nset], Wt, dys[i % nset], A, Bm, 16.0, workspace=ws,
+                                                use_tensor_cores=tc), max(3, iters // 2))
+        # dx product + both rank-r products + the two skinny gradient reductions (no dW: W is frozen)
+        bflops = 2.0 * M * n_in * n_out + 4.0 * M * r * (n_in + n_out)
+        out.update({"bwd_us": round(bwd * 1e3, 1), "bwd_tflops": round(bflops / bwd / 1e9, 1),
+                    "bwd_frac_of_bf16_peak": round(bflops / bwd / 1e9 / tflops, 3)})
+    return out
+
+
+def bench_aggregate(K, P, iters=50):
+    hbm, _, src = _peaks()
+    nset = max(1, min(8, -(-2 * L2_BYTES // (K * P * 4))))
+    bufs = [torch.randn(K, P, device="cuda") for _ in range(nset)]
+    w = [1.0 / K] * K
+    ms = _time(lambda i: B.aggregate_buffers(bufs[i % nset], w), iters)
+    gbs = 2.0 * K * P * 4 / ms / 1e6        # read K copies, write K copies
+    return {"op": "aggregate", "K": K, "P": P, "us": round(ms * 1e3, 2), "GBps": round(gbs, 1),
+            "frac_of_hbm": round(gbs / hbm, 3), "peak_source": src}
+
+
+def bench_attention(nseq, T, heads, iters=10):
+    _, tflops, src = _peaks()
+    d = heads * 64
+    qkv = torch.randn(nseq * T, 3 * d, device="cuda").bfloat16()
+    do = torch.randn(nseq * T, d, device="cuda").bfloat16()
+    o, lse = B.attention_fwd(qkv, nseq, T, heads, True)
+    f = _time(lambda i: B.attention_fwd(qkv, nseq, T, heads, True), iters)
+    b = _time(lambda i: B.attention_bwd(qkv, o, lse, do, nseq, T, heads, True), iters)
+    fl = 2.0 * nseq * heads * T * T * 64            # causal: half of 4 T^2 dh
+    return {"op": "attention", "nseq": nseq, "T": T, "heads": heads, "fwd_us": round(f * 1e3, 1),
+            "fwd_tflops": round(fl / f / 1e9, 1), "bwd_us": round(b * 1e3, 1),
+            "bwd_tflops_algorithmic": round(2.5 * fl / b / 1e9, 1), "peak_source": src}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("what", choices=["linear", "linear-sweep", "aggregate", "aggregate-sweep", "attention"])
+    ap.add_argument("--M", type=int, default=32768)
+    ap.add_argument("--n-in", type=int, default=1024)
+    ap.add_argument("--n-out", type=int, default=3072)
+    ap.add_argument("--r", type=int, default=4)
+    ap.add_argument("--G", type=int, default=8)
+    ap.add_argument("--K", type=int, default=8)
+    ap.add_argument("--P", type=int, default=98304)
+    ap.add_argument("--nseq", type=int, default=64)
+    ap.add_argument("--T", type=int, default=512)
+    ap.add_argument("--heads", type=int, default=16)
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--no-backward", action="store_true")
+    ap.add_argument("--quick", action="store_true")
+    a = ap.parse_args()
+    if a.what == "linear":
+        print(json.dumps(bench_linear(a.M, a.n_in, a.n_out, a.r, a.G, a.iters, not a.no_backward)))
+    elif a.what == "linear-sweep":
+        Ms = [4096, 16384, 65536]
+        ins = [768, 1024, 4096]
+        outs = [768, 3072, 4096, 11008]
+        rs = [4, 8, 16, 64]
+        Gs = [1, 4, 8, 16]
+        if a.quick:
+            Ms, rs, Gs = [16384], [4, 64], [1, 8]
+        for M in Ms:
+            for n_in in ins:
+                for n_out in outs:
+                    for r in rs:
+                        for G in Gs:
+                            print(json.dumps(bench_linear(M, n_in, n_out, r, G, 10)), flush=True)
+    elif a.what == "aggregate":
+        print(json.dumps(bench_aggregate(a.K, a.P, a.iters)))
+    elif a.what == "aggregate-sweep":
+        for K in (2, 8, 32):
+            for lg in range(17, 27 if K == 32 else 29, 2):
+                print(json.dumps(bench_aggregate(K, 1 << lg)), flush=True)
+        print(json.dumps(dict(bench_aggregate(8, 98304), note="GPT-2-medium-shaped client adapter set")))
+    else:
+        print(json.dumps(bench_attention(a.nseq, a.T, a.heads, a.iters)))
+
+
+if __name__ == "__main__":
+    main()
