@@ -211,6 +211,29 @@ int splitlora_attention_bwd(int dtype, int use_tensor_cores, const void* qkv, co
                             const void* d_o, int nseq, int T, int n_head, int d_model, void* dqkv,
                             float* scratch_rowdot /* [nseq*T*H] */, void* stream);
 
+/* Attention backward without caller scratch and without any allocation.  (The paper has no
+ * counterpart; this serves callers that may not allocate device memory: code running under a
+ * fixed memory budget handed out at start-up, or plug-ins inside a host application that owns the
+ * allocator and forbids cudaMalloc after initialisation.)
+ *
+ * Same inputs, outputs and arithmetic as splitlora_attention_bwd, but the per-row scratch
+ * (one float per sequence x head x position) lives in a fixed array inside the library: every
+ * device that loads the library holds SPLITLORA_STATIC_ATTENTION_ROWS floats (4 MiB) until the
+ * process exits.  Limits and rules:
+ *   - nseq * T * n_head must not exceed SPLITLORA_STATIC_ATTENTION_ROWS, else the call returns
+ *     SPLITLORA_ERR_TOO_LARGE and launches nothing;
+ *   - the first call on a device looks up the array's device address (a cheap runtime query, no
+ *     allocation); make that first call outside any stream capture;
+ *   - all calls on a device share the one array, which keeps the previous call's contents; the
+ *     call overwrites every element it later reads, so nothing needs clearing, but two calls that
+ *     may overlap on the GPU (different streams) race on it: serialise them;
+ *   - the call itself calls no cudaMalloc / cudaFree and no allocating library routine. */
+#define SPLITLORA_STATIC_ATTENTION_ROWS (1 << 20)
+#define SPLITLORA_ERR_TOO_LARGE -10   /* the problem does not fit a fixed-size internal buffer */
+int splitlora_attention_bwd_static(int dtype, int use_tensor_cores, const void* qkv, const void* o,
+                                   const float* lse, const void* d_o, int nseq, int T, int n_head,
+                                   int d_model, void* dqkv, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

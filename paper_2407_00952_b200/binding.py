@@ -27,6 +27,7 @@ EXPORTS = [
     "splitlora_device_status", "splitlora_launch_count", "splitlora_profile_enable", "splitlora_profile_report",
     "splitlora_lora_linear_workspace_bytes", "splitlora_lora_linear_fwd", "splitlora_lora_linear_bwd",
     "splitlora_transpose", "splitlora_aggregate_buffers", "splitlora_attention_fwd", "splitlora_attention_bwd",
+    "splitlora_attention_bwd_static",
 ]
 
 
@@ -310,4 +311,22 @@ def attention_bwd(qkv, o, lse, d_o, nseq, T, n_head, use_tensor_cores=True):
     rowdot = torch.empty(nseq * n_head * T, dtype=torch.float32, device="cuda")
     _rc(lib.splitlora_attention_bwd(_dt(qkv), 1 if use_tensor_cores else 0, _ptr(qkv), _ptr(o), _ptr(lse), _ptr(d_o),
                                     nseq, T, n_head, d, _ptr(dqkv), _ptr(rowdot), _stream_ptr()), "attention_bwd")
+    return dqkv
+
+
+STATIC_ATTENTION_ROWS = 1 << 20
+ERR_TOO_LARGE = -10
+
+
+def attention_bwd_static(qkv, o, lse, d_o, nseq, T, n_head, use_tensor_cores=True, dqkv=None):
+    """Attention backward through splitlora_attention_bwd_static: the library's built-in scratch is
+    used, so the call allocates nothing as long as the caller passes `dqkv`.  Raises SplitLoraError
+    (code ERR_TOO_LARGE) when nseq * T * n_head exceeds STATIC_ATTENTION_ROWS."""
+    lib = load()
+    d = qkv.shape[1] // 3
+    if dqkv is None:
+        dqkv = torch.empty_like(qkv)
+    _rc(lib.splitlora_attention_bwd_static(_dt(qkv), 1 if use_tensor_cores else 0, _ptr(qkv), _ptr(o), _ptr(lse),
+                                           _ptr(d_o), nseq, T, n_head, d, _ptr(dqkv), _stream_ptr()),
+        "attention_bwd_static")
     return dqkv
