@@ -1,0 +1,282 @@
+// Device-side building blocks shared by the tcgen05 linear-layer kernels: mbarrier / TMA / tcgen05
+// PTX wrappers, shared-memory operand descriptors and the epilogue of one 32-column chunk.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace sl {
+namespace tc {
+
+constexpr int BM = 128;           // accumulator rows per CTA (the 128 lanes of tensor memory)
+constexpr int BK = 64;            // 64 bf16 = 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;
+constexpr int GROUP_M = 16;       // output tiles are walked in bands of GROUP_M tile rows
+constexpr unsigned long long WAIT_LIMIT_NS = 4000000000ull;
+
+struct TcParams {
+  int M, N, K;                    // K counts the main contraction only
+  int num_kb;                     // K / 64
+  int ext_blocks;                 // blocks of 64 in the rank-r extension
+  int ext_last_mmas;              // MMAs (of 16) in the last extension block
+  int rows_per_group;             // 0: one group
+  int w_group_rows;               // rows between groups in W (0: shared)
+  int we_group_rows;              // rows between groups in We
+  int tiles_m, tiles_n;
+  int epi, gelu_tanh;
+  const bf16* bias;
+  const bf16* R; long long ldr;
+  bf16* Y; long long ldy;
+  bf16* Z; long long ldz;
+  int* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// arrive on a barrier given by a shared::cluster address (own CTA or the peer of a CTA pair)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false when the limit expired or another role of this CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+  if (mbar_try(bar, parity)) return true;
+  unsigned long long t0 = global_ns();
+  uint32_t spins = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++spins & 1023u) == 0) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1;
+        atomicCAS(status, 0, code);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+// Load issued inside a CTA pair: the completion may be signalled on the partner's barrier
+// (bar is a shared::cluster address).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// Commit of a CTA pair's products; arrives on the barrier at this offset in every CTA of `mask`.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float tanh_fast(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float gelu_tc(float z, bool tanh_form) {
+  if (tanh_form) {
+    float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);
+    return 0.5f * z * (1.0f + tanh_fast(u));
+  }
+  return gelu_f(z, false);
+}
+__device__ __forceinline__ float gelu_grad_tc(float z, bool tanh_form) {
+  if (tanh_form) {
+    float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);
+    float t = tanh_fast(u);
+    float du = 0.7978845608028654f * (1.0f + 0.134145f * z * z);
+    return 0.5f * (1.0f + t) + 0.5f * z * (1.0f - t * t) * du;
+  }
+  return gelu_grad_f(z, false);
+}
+
+// Shared-memory operand descriptor: K-major tile whose rows are 128 bytes, 128-byte swizzle,
+// groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);      // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                        // leading byte offset (unused for this layout)
+  d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                        // 128-byte swizzle
+  return d;
+}
+
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// Output-tile walk: bands of GROUP_M tile rows, rows fastest inside a band.
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
+  const int band_tiles = GROUP_M * tiles_n;
+  int band = tile / band_tiles, in = tile % band_tiles;
+  int m_first = band * GROUP_M;
+  int rows = min(GROUP_M, tiles_m - m_first);
+  tm = m_first + in % rows;
+  tn = in / rows;
+}
+
+// Bytes of shared memory the epilogue warps use to stage output chunks: 8 warps x 2 buffers x
+// (32 rows x 64 bytes).
+constexpr int EPI_STAGE_BYTES = 8 * 2 * 2048;
+
+// One 32-row x 32-column bf16 chunk: registers -> shared (64-byte swizzle, conflict-free 16-byte
+// stores) -> global through a TMA store.  Rows of the output are written as full 64-byte segments
+// by the copy engine instead of 32 scattered 16-byte stores per warp instruction, which keeps the
+// L1 data path free for the tensor core's operand reads.  `packed` holds this thread's row
+// (lane = row).  The buffer is reused once the bulk group that read it has finished reading.
+__device__ __forceinline__ void stage_and_store(uint32_t sbuf, const CUtensorMap* map, const uint32_t* packed,
+                                                int lane, int n, int m_warp0) {
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+  __syncwarp();
+  const uint32_t row = sbuf + (uint32_t)lane * 64u;
+  const uint32_t sw = ((uint32_t)lane >> 1) & 3u;
+#pragma unroll
+  for (uint32_t j = 0; j < 4; ++j) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + ((j ^ sw) << 4)), "r"(packed[4 * j]),
+                 "r"(packed[4 * j + 1]), "r"(packed[4 * j + 2]), "r"(packed[4 * j + 3]) : "memory");
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncwarp();
+  if (lane == 0) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(sbuf), "r"(n), "r"(m_warp0) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  }
+}
+__device__ __forceinline__ void epilogue_drain(int lane) {
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  __syncwarp();
+}
+
+// Epilogue of 32 accumulator columns [n, n+32) of row m (= m_warp0 + lane): bias, activation /
+// residual, bf16 output through the staging buffers `stage` (this warp's two 2 KB buffers).
+__device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, int m, int n, bool tanh_form,
+                                               uint32_t stage, int& buf, const CUtensorMap* mapY,
+                                               const CUtensorMap* mapZ, int m_warp0, int lane) {
+  if (p.bias && p.epi != EPI_MUL_GELUGRAD) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (n + 8 * j < p.N) {
+        uint4 bw = __ldg(reinterpret_cast<const uint4*>(p.bias + n + 8 * j));
+        const bf16* bp = reinterpret_cast<const bf16*>(&bw);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[8 * j + i] += __bfloat162float(bp[i]);
+      }
+    }
+  }
+  uint32_t packed[16];
+  if (p.epi == EPI_BIAS_GELU) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      __nv_bfloat162 z2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+      packed[i] = *reinterpret_cast<uint32_t*>(&z2);
+      v[2 * i] = gelu_tc(__low2float(z2), tanh_form);
+      v[2 * i + 1] = gelu_tc(__high2float(z2), tanh_form);
+    }
+    stage_and_store(stage + (uint32_t)buf * 2048u, mapZ, packed, lane, n, m_warp0);
+    buf ^= 1;
+  } else if (p.epi == EPI_BIAS_RESID || p.epi == EPI_MUL_GELUGRAD) {
+    const bf16* rrow = p.R + (size_t)m * p.ldr + n;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (n + 8 * j < p.N) {
+        uint4 rw = *reinterpret_cast<const uint4*>(rrow + 8 * j);
+        const bf16* rp = reinterpret_cast<const bf16*>(&rw);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float rv = __bfloat162float(rp[i]);
+          if (p.epi == EPI_BIAS_RESID) v[8 * j + i] += rv;
+          else v[8 * j + i] *= gelu_grad_tc(rv, tanh_form);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    __nv_bfloat162 y2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+    packed[i] = *reinterpret_cast<uint32_t*>(&y2);
+  }
+  stage_and_store(stage + (uint32_t)buf * 2048u, mapY, packed, lane, n, m_warp0);
+  buf ^= 1;
+}
+
+}  // namespace tc
+}  // namespace sl
