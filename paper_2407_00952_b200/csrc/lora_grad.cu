@@ -1,10 +1,10 @@
 // Adapter gradients G_A, G_B (Eq. 4-7): skinny reductions over the tokens of each group,
 //   out[g][t][jj][c] = scale * sum_{m in group g} Wt[m, wcol0 + t*rp + jj] * Z[m, zcol0 + c]
 // for nt targets of rank r (R = nt*r weight columns) and C feature columns.  HBM-bound: Z is read
-// once per RJ weight columns.  A block is 128 column threads (one 16-byte vector each) x 4 row
-// lanes over a chunk of LG_ROWS rows; the row lanes are summed through shared memory, chunk
-// partials go to scratch and a second kernel adds them in chunk order (no float atomics, so the
-// result does not depend on scheduling).
+// once per 4 weight columns.  A block is 64 column threads (one 16-byte vector each) x 4 row lanes
+// over a chunk of LG_ROWS rows, four blocks per SM so that enough loads are in flight; the row
+// lanes are summed through shared memory, chunk partials go to scratch and a second kernel adds
+// them in a fixed order (no float atomics, so the result does not depend on scheduling).
 #include "common.cuh"
 #include "kernels.h"
 
@@ -12,11 +12,26 @@ namespace sl {
 namespace {
 
 constexpr int LG_ROWS = 128;   // rows per chunk; group sizes must be multiples of it
-constexpr int LG_CT = 128;     // column threads per block
+constexpr int LG_CT = 64;      // column threads per block
 constexpr int LG_RL = 4;       // row lanes per block
+constexpr int RJ = 4;          // weight columns per block
+constexpr int RED_LANES = 8;   // chunk lanes of the second kernel
 
-template <typename T, int RJ>
-__global__ void __launch_bounds__(LG_CT * LG_RL)
+// four consecutive weights of one row
+template <typename T> __device__ __forceinline__ void load4(const T* p, float* w);
+template <> __device__ __forceinline__ void load4<float>(const float* p, float* w) {
+  float4 v = *reinterpret_cast<const float4*>(p);
+  w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+}
+template <> __device__ __forceinline__ void load4<bf16>(const bf16* p, float* w) {
+  uint2 v = *reinterpret_cast<const uint2*>(p);
+  const bf16* b = reinterpret_cast<const bf16*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) w[i] = __bfloat162float(b[i]);
+}
+
+template <typename T, bool VEC4>
+__global__ void __launch_bounds__(LG_CT * LG_RL, 4)
 lora_grad_partial_kernel(const T* __restrict__ Z, int64_t ldz, int zcol0, int C, const T* __restrict__ Wt,
                          int64_t ldwt, int wcol0, int r, int rp, int R, int M, float* __restrict__ partial) {
   constexpr int N = Vec16<T>::N;
@@ -44,8 +59,12 @@ lora_grad_partial_kernel(const T* __restrict__ Z, int64_t ldz, int zcol0, int C,
     for (int m = m0 + ty; m < m1; m += LG_RL) {
       Vec16<T> v; v.load(Z + (size_t)m * ldz + zcol0 + c);
       float w[RJ];
+      if (VEC4) {
+        load4<T>(Wt + (size_t)m * ldwt + wc[0], w);     // r % 4 == 0: the four columns are adjacent
+      } else {
 #pragma unroll
-      for (int j = 0; j < RJ; ++j) w[j] = wc[j] >= 0 ? to_f<T>(Wt[(size_t)m * ldwt + wc[j]]) : 0.f;
+        for (int j = 0; j < RJ; ++j) w[j] = wc[j] >= 0 ? to_f<T>(Wt[(size_t)m * ldwt + wc[j]]) : 0.f;
+      }
 #pragma unroll
       for (int i = 0; i < N; ++i) {
         float zv = v.get(i);
@@ -85,28 +104,40 @@ lora_grad_partial_kernel(const T* __restrict__ Z, int64_t ldz, int zcol0, int C,
   }
 }
 
-__global__ void lora_grad_reduce_kernel(const float* __restrict__ partial, int r, int R, int C, int chunks_per_group,
-                                        float scale, float* __restrict__ out, int64_t out_group_stride,
-                                        int64_t out_target_stride, int64_t out_sj, int64_t out_sc) {
-  int idx = blockIdx.x * blockDim.x + threadIdx.x;   // over R*C
-  int g = blockIdx.y;
-  if (idx >= R * C) return;
-  int j = idx / C, c = idx % C;
+// 32 outputs per block (threadIdx.x), RED_LANES chunk lanes (threadIdx.y) combined in lane order.
+__global__ void __launch_bounds__(32 * RED_LANES)
+lora_grad_reduce_kernel(const float* __restrict__ partial, int r, int R, int C, int chunks_per_group, float scale,
+                        float* __restrict__ out, int64_t out_group_stride, int64_t out_target_stride,
+                        int64_t out_sj, int64_t out_sc) {
+  __shared__ float red[RED_LANES][32];
+  const int idx = blockIdx.x * 32 + threadIdx.x;   // over R*C
+  const int g = blockIdx.y;
+  const bool active = idx < R * C;
   float s = 0.f;
-  for (int k = 0; k < chunks_per_group; ++k)
-    s += partial[((size_t)(g * chunks_per_group + k) * R + j) * C + c];
-  out[(size_t)g * out_group_stride + (size_t)(j / r) * out_target_stride + (size_t)(j % r) * out_sj +
-      (size_t)c * out_sc] = scale * s;
+  if (active) {
+    const float* p = partial + (size_t)g * chunks_per_group * R * C + idx;
+    for (int k = threadIdx.y; k < chunks_per_group; k += RED_LANES) s += p[(size_t)k * R * C];
+  }
+  red[threadIdx.y][threadIdx.x] = s;
+  __syncthreads();
+  if (threadIdx.y == 0 && active) {
+    float t = 0.f;
+#pragma unroll
+    for (int l = 0; l < RED_LANES; ++l) t += red[l][threadIdx.x];
+    const int j = idx / C, c = idx % C;
+    out[(size_t)g * out_group_stride + (size_t)(j / r) * out_target_stride + (size_t)(j % r) * out_sj +
+        (size_t)c * out_sc] = scale * t;
+  }
 }
 
 template <typename T>
-void launch_partial(dim3 grid, cudaStream_t st, int RJ, const void* Z, int64_t ldz, int zcol0, int C, const void* Wt,
+void launch_partial(dim3 grid, cudaStream_t st, bool vec4, const void* Z, int64_t ldz, int zcol0, int C, const void* Wt,
                     int64_t ldwt, int wcol0, int r, int rp, int R, int M, float* partial) {
   dim3 block(LG_CT, LG_RL);
-  if (RJ == 8)
-    lora_grad_partial_kernel<T, 8><<<grid, block, 0, st>>>((const T*)Z, ldz, zcol0, C, (const T*)Wt, ldwt, wcol0, r, rp, R, M, partial);
+  if (vec4)
+    lora_grad_partial_kernel<T, true><<<grid, block, 0, st>>>((const T*)Z, ldz, zcol0, C, (const T*)Wt, ldwt, wcol0, r, rp, R, M, partial);
   else
-    lora_grad_partial_kernel<T, 4><<<grid, block, 0, st>>>((const T*)Z, ldz, zcol0, C, (const T*)Wt, ldwt, wcol0, r, rp, R, M, partial);
+    lora_grad_partial_kernel<T, false><<<grid, block, 0, st>>>((const T*)Z, ldz, zcol0, C, (const T*)Wt, ldwt, wcol0, r, rp, R, M, partial);
 }
 
 }  // namespace
@@ -131,14 +162,15 @@ cudaError_t lora_grad(int dt, const void* Z, int64_t ldz, int zcol0, int C, cons
     groups = M / rpg; chunks_per_group = rpg / LG_ROWS;
   }
   if (C % n != 0 || R < 1) return cudaErrorInvalidValue;
-  const int RJ = (dt == DT_BF16) ? (R > 4 ? 8 : 4) : 4;     // fp32 vectors are 4 wide: keep registers in check
+  // vector loads of four adjacent weights need r % 4 == 0 and aligned rows / column offsets
+  const bool vec4 = (r % 4 == 0) && (wcol0 % 4 == 0) && (rp % 4 == 0) && (ldwt % 4 == 0);
   const int cvec = C / n;
   dim3 grid((cvec + LG_CT - 1) / LG_CT, chunks, (R + RJ - 1) / RJ);
-  if (dt == DT_BF16) launch_partial<bf16>(grid, st, RJ, Z, ldz, zcol0, C, Wt, ldwt, wcol0, r, rp, R, M, partial);
-  else launch_partial<float>(grid, st, RJ, Z, ldz, zcol0, C, Wt, ldwt, wcol0, r, rp, R, M, partial);
-  dim3 g2((R * C + 255) / 256, groups);
-  lora_grad_reduce_kernel<<<g2, 256, 0, st>>>(partial, r, R, C, chunks_per_group, scale, out, out_group_stride,
-                                              out_target_stride, out_sj, out_sc);
+  if (dt == DT_BF16) launch_partial<bf16>(grid, st, vec4, Z, ldz, zcol0, C, Wt, ldwt, wcol0, r, rp, R, M, partial);
+  else launch_partial<float>(grid, st, vec4, Z, ldz, zcol0, C, Wt, ldwt, wcol0, r, rp, R, M, partial);
+  dim3 g2((R * C + 31) / 32, groups), b2(32, RED_LANES);
+  lora_grad_reduce_kernel<<<g2, b2, 0, st>>>(partial, r, R, C, chunks_per_group, scale, out, out_group_stride,
+                                             out_target_stride, out_sj, out_sc);
   return cudaGetLastError();
 }
 
