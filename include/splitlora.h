@@ -196,6 +196,16 @@ int splitlora_lora_linear_bwd(int dtype, int use_tensor_cores, const void* x, co
                               const float* A, const float* B, float alpha, int M, int n_in, int n_out,
                               int r, int G, void* dx, float* dA, float* dB,
                               void* workspace, size_t workspace_bytes, void* stream);
+/* Frozen linear layer with a fused epilogue (the un-adapted projections of a block and their
+ * backward products; W is frozen, so the backward is the same call on the transposed weight):
+ *   epilogue 0: y = x W^T + bias                 1: z = x W^T + bias, y = gelu(z)
+ *            2: y = x W^T + bias + r             3: y = (x W^T) * gelu'(r)
+ * x [M, in], W [out, in], bias [out] or NULL, r / z / y [M, out], all in `dtype`.  status_word is a
+ * zero-initialised device int that receives a code if a bounded wait inside the tensor-core kernel
+ * expires (required when use_tensor_cores != 0 and dtype is bf16). */
+int splitlora_linear(int dtype, int use_tensor_cores, const void* x, const void* W, const void* bias,
+                     int epilogue, const void* r, void* z, int gelu_tanh, int M, int n_in, int n_out,
+                     void* y, int* status_word, void* stream);
 /* out [cols, rows] = in [rows, cols]^T in `dtype` (for building Wt). */
 int splitlora_transpose(int dtype, const void* in, int rows, int cols, void* out, void* stream);
 

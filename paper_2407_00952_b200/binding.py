@@ -27,7 +27,7 @@ EXPORTS = [
     "splitlora_device_status", "splitlora_launch_count", "splitlora_profile_enable", "splitlora_profile_report",
     "splitlora_lora_linear_workspace_bytes", "splitlora_lora_linear_fwd", "splitlora_lora_linear_bwd",
     "splitlora_transpose", "splitlora_aggregate_buffers", "splitlora_attention_fwd", "splitlora_attention_bwd",
-    "splitlora_attention_bwd_static",
+    "splitlora_attention_bwd_static", "splitlora_linear",
 ]
 
 
@@ -277,6 +277,28 @@ def lora_linear_bwd(x, Wt, dy, A, B, alpha, workspace=None, use_tensor_cores=Tru
                                       _ptr(B), C.c_float(alpha), M, n_in, n_out, r, G, _ptr(dx), _ptr(dA), _ptr(dB),
                                       _ptr(workspace), C.c_size_t(workspace.numel()), _stream_ptr()), "lora_linear_bwd")
     return dx, dA, dB
+
+
+EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_RESID, EPI_MUL_GELUGRAD = 0, 1, 2, 3
+_status_words = {}
+
+
+def linear(x, W, bias=None, epilogue=EPI_BIAS, r=None, y=None, z=None, gelu_tanh=True, use_tensor_cores=True):
+    """Frozen linear layer with fused epilogue (splitlora_linear).  Returns y, or (y, z) for the GELU epilogue."""
+    lib = load()
+    M, n_in = x.shape
+    n_out = W.shape[0]
+    if y is None:
+        y = torch.empty(M, n_out, dtype=x.dtype, device="cuda")
+    if epilogue == EPI_BIAS_GELU and z is None:
+        z = torch.empty(M, n_out, dtype=x.dtype, device="cuda")
+    dev = torch.cuda.current_device()
+    if dev not in _status_words:
+        _status_words[dev] = torch.zeros(64, dtype=torch.int32, device="cuda")
+    _rc(lib.splitlora_linear(_dt(x), 1 if use_tensor_cores else 0, _ptr(x), _ptr(W), _ptr(bias), epilogue, _ptr(r),
+                             _ptr(z), 1 if gelu_tanh else 0, M, n_in, n_out, _ptr(y), _ptr(_status_words[dev]),
+                             _stream_ptr()), "linear")
+    return (y, z) if epilogue == EPI_BIAS_GELU else y
 
 
 def transpose(t: torch.Tensor) -> torch.Tensor:

@@ -155,25 +155,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
     int as = 0; uint32_t aphase = 0;
     const bool tanh_form = p.gelu_tanh != 0;
     const uint32_t stage = epi_base + (uint32_t)(warp - 2) * 4096u;   // this warp's two staging buffers
-    int buf = 0;
+    EpiState est;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
       int tm, tn; tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
       const int m_warp0 = tm * BM + q * 32;
-      const int m = m_warp0 + lane;
       const int n0 = tn * BN;
+      int m_next = -1, n_next = 0;
+      if (tile + (int)gridDim.x < num_tiles) {
+        int tm2, tn2; tile_coords(tile + gridDim.x, p.tiles_m, p.tiles_n, tm2, tn2);
+        m_next = tm2 * BM + q * 32; n_next = tn2 * BN + c_begin;
+      }
       if (!mbar_wait(tfull_bar(as), aphase, abort_flag, p.status, 4)) { ok = false; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN);
-#pragma unroll 1
-      for (int c = c_begin; c < c_end; c += 32) {
-        const int n = n0 + c;
-        if (n >= p.N) break;                    // warp-uniform
-        float v[32];
-        tc_ld32(t_row + (uint32_t)c, v);
-        tc_wait_ld();
-        epilogue_chunk(p, v, m, n, tanh_form, stage, buf, &mapY, &mapZ, m_warp0, lane);
-      }
+      epilogue_tile(p, t_row, m_warp0, lane, n0, c_begin, c_end, m_next, n_next, tanh_form, stage, est, &mapY, &mapZ);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(as));
@@ -321,25 +317,21 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     int as = 0; uint32_t aphase = 0;
     const bool tanh_form = p.gelu_tanh != 0;
     const uint32_t stage = epi_base + (uint32_t)(warp - 2) * 4096u;   // this warp's two staging buffers
-    int buf = 0;
+    EpiState est;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
       int tm, tn; tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
       const int m_warp0 = tm * 2 * BM + (int)rank * BM + q * 32;
-      const int m = m_warp0 + lane;
       const int n0 = tn * BN;
+      int m_next = -1, n_next = 0;
+      if (tile + npairs < num_tiles) {
+        int tm2, tn2; tile_coords(tile + npairs, p.tiles_m, p.tiles_n, tm2, tn2);
+        m_next = tm2 * 2 * BM + (int)rank * BM + q * 32; n_next = tn2 * BN + c_begin;
+      }
       if (!mbar_wait(tfull_bar(as), aphase, abort_flag, p.status, 14)) { ok = false; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN);
-#pragma unroll 1
-      for (int c = c_begin; c < c_end; c += 32) {
-        const int n = n0 + c;
-        if (n >= p.N) break;
-        float v[32];
-        tc_ld32(t_row + (uint32_t)c, v);
-        tc_wait_ld();
-        epilogue_chunk(p, v, m, n, tanh_form, stage, buf, &mapY, &mapZ, m_warp0, lane);
-      }
+      epilogue_tile(p, t_row, m_warp0, lane, n0, c_begin, c_end, m_next, n_next, tanh_form, stage, est, &mapY, &mapZ);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(as), 0));   // 16 arrivals free the stage

@@ -192,3 +192,21 @@ int splitlora_attention_bwd(int dtype, int use_tc, const void* qkv, const void* 
 }
 
 }  // extern "C"
+
+// Frozen linear layer with a fused epilogue (steps a4 / a11), stand-alone.
+extern "C" int splitlora_linear(int dtype, int use_tc, const void* x, const void* W, const void* bias, int epilogue,
+                                const void* r, void* z, int gelu_tanh, int M, int n_in, int n_out, void* y,
+                                int* status_word, void* stream) {
+  if (!x || !W || !y || M < 1 || n_in < 8 || n_out < 8 || n_in % 8 || n_out % 8 || (dtype != DT_F32 && dtype != DT_BF16))
+    return SPLITLORA_ERR_ARG;
+  if (epilogue < EPI_BIAS || epilogue > EPI_MUL_GELUGRAD) return SPLITLORA_ERR_ARG;
+  if ((epilogue == EPI_BIAS_RESID || epilogue == EPI_MUL_GELUGRAD) && !r) return SPLITLORA_ERR_ARG;
+  if (epilogue == EPI_BIAS_GELU && !z) return SPLITLORA_ERR_ARG;
+  if (use_tc && dtype == DT_BF16 && !status_word) return SPLITLORA_ERR_ARG;
+  if (gemm_tc_init() != 0) return SPLITLORA_ERR_CUDA;
+  GemmArgs a;
+  a.dtype = dtype; a.X = x; a.ldx = n_in; a.W = W; a.ldw = n_in; a.Y = y; a.ldy = n_out;
+  a.M = M; a.N = n_out; a.K = n_in; a.bias = bias; a.epi = epilogue; a.R = r; a.ldr = n_out; a.Z = z; a.ldz = n_out;
+  a.gelu_tanh = gelu_tanh;
+  return run_gemm(use_tc, a, status_word, (cudaStream_t)stream) == cudaSuccess ? SPLITLORA_OK : SPLITLORA_ERR_CUDA;
+}

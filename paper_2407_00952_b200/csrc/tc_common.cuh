@@ -226,9 +226,21 @@ __device__ __forceinline__ void epilogue_drain(int lane) {
   __syncwarp();
 }
 
+// The second epilogue operand (residual, or the saved pre-activation) of columns [n, n+32) of row m.
+// Issued one chunk ahead of its use so that its latency overlaps the previous chunk's work.
+__device__ __forceinline__ void load_r_chunk(const TcParams& p, int m, int n, uint4* r) {
+  const bf16* rrow = p.R + (size_t)m * p.ldr + n;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (n + 8 * j < p.N) r[j] = *reinterpret_cast<const uint4*>(rrow + 8 * j);
+    else r[j] = make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+
 // Epilogue of 32 accumulator columns [n, n+32) of row m (= m_warp0 + lane): bias, activation /
-// residual, bf16 output through the staging buffers `stage` (this warp's two 2 KB buffers).
-__device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, int m, int n, bool tanh_form,
+// residual (rpre: the row's second operand, loaded by load_r_chunk), bf16 output through the
+// staging buffers `stage` (this warp's two 2 KB buffers).
+__device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, const uint4* rpre, int n, bool tanh_form,
                                                uint32_t stage, int& buf, const CUtensorMap* mapY,
                                                const CUtensorMap* mapZ, int m_warp0, int lane) {
   if (p.bias && p.epi != EPI_MUL_GELUGRAD) {
@@ -254,12 +266,10 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, int 
     stage_and_store(stage + (uint32_t)buf * 2048u, mapZ, packed, lane, n, m_warp0);
     buf ^= 1;
   } else if (p.epi == EPI_BIAS_RESID || p.epi == EPI_MUL_GELUGRAD) {
-    const bf16* rrow = p.R + (size_t)m * p.ldr + n;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       if (n + 8 * j < p.N) {
-        uint4 rw = *reinterpret_cast<const uint4*>(rrow + 8 * j);
-        const bf16* rp = reinterpret_cast<const bf16*>(&rw);
+        const bf16* rp = reinterpret_cast<const bf16*>(&rpre[j]);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           float rv = __bfloat162float(rp[i]);
@@ -276,6 +286,49 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, int 
   }
   stage_and_store(stage + (uint32_t)buf * 2048u, mapY, packed, lane, n, m_warp0);
   buf ^= 1;
+}
+
+// Per-warp epilogue state carried across tiles: staging buffer in use and the prefetched second
+// operand (valid for the chunk at row block pm, column pn).
+struct EpiState {
+  uint4 rnext[4];
+  int pm = -1, pn = -1;
+  int buf = 0;
+};
+
+// This warp's share of one output tile: columns [n0 + c_begin, n0 + c_end) of the 32 rows starting
+// at m_warp0, accumulator lanes at tensor-memory address t_row.  (m_next, n_next) is the first chunk
+// this warp will process in its next tile (m_next < 0: none); its second operand is requested while
+// the last chunk of this tile is being worked on.
+__device__ __forceinline__ void epilogue_tile(const TcParams& p, uint32_t t_row, int m_warp0, int lane, int n0,
+                                              int c_begin, int c_end, int m_next, int n_next, bool tanh_form,
+                                              uint32_t stage, EpiState& st, const CUtensorMap* mapY,
+                                              const CUtensorMap* mapZ) {
+  const bool need_r = p.epi == EPI_BIAS_RESID || p.epi == EPI_MUL_GELUGRAD;
+  const int m = m_warp0 + lane;
+#pragma unroll 1
+  for (int c = c_begin; c < c_end; c += 32) {
+    const int n = n0 + c;
+    if (n >= p.N) break;                    // warp-uniform
+    uint4 rcur[4];
+    if (need_r) {
+      if (st.pm == m_warp0 && st.pn == n) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) rcur[j] = st.rnext[j];
+      } else {
+        load_r_chunk(p, m, n, rcur);
+      }
+      if (c + 32 < c_end && n + 32 < p.N) {
+        load_r_chunk(p, m, n + 32, st.rnext); st.pm = m_warp0; st.pn = n + 32;
+      } else if (m_next >= 0 && n_next < p.N) {
+        load_r_chunk(p, m_next + lane, n_next, st.rnext); st.pm = m_next; st.pn = n_next;
+      }
+    }
+    float v[32];
+    tc_ld32(t_row + (uint32_t)c, v);
+    tc_wait_ld();
+    epilogue_chunk(p, v, rcur, n, tanh_form, stage, st.buf, mapY, mapZ, m_warp0, lane);
+  }
 }
 
 }  // namespace tc

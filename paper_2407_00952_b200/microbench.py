@@ -73,6 +73,35 @@ def bench_linear(M, n_in, n_out, r, G, iters=20, backward=True, tc=True):
     return out
 
 
+def bench_epilogues(M, d, F, iters=20):
+    """The un-adapted linear layers of one block (forward and backward), each with its epilogue."""
+    _, tflops, src = _peaks()
+    g = torch.Generator(device="cuda").manual_seed(2)
+    mk = lambda *s, sc=1.0: (torch.randn(*s, device="cuda", generator=g) * sc).bfloat16()
+    xd, xF = mk(M, d), mk(M, F)
+    rd, rF = mk(M, d), mk(M, F)
+    yd, yF, zF = (torch.empty(M, d, device="cuda", dtype=torch.bfloat16), torch.empty(M, F, device="cuda", dtype=torch.bfloat16),
+                  torch.empty(M, F, device="cuda", dtype=torch.bfloat16))
+    Wdd, WFd, WdF = mk(d, d, sc=d ** -0.5), mk(F, d, sc=d ** -0.5), mk(d, F, sc=F ** -0.5)
+    bd, bF = mk(d), mk(F)
+    cases = [
+        ("proj fwd  (bias+resid)", lambda i: B.linear(xd, Wdd, bd, B.EPI_BIAS_RESID, r=rd, y=yd), d, d),
+        ("fc1 fwd   (bias+gelu)", lambda i: B.linear(xd, WFd, bF, B.EPI_BIAS_GELU, y=yF, z=zF), d, F),
+        ("fc2 fwd   (bias+resid)", lambda i: B.linear(xF, WdF, bd, B.EPI_BIAS_RESID, r=rd, y=yd), F, d),
+        ("fc2 bwd   (x gelu')", lambda i: B.linear(xd, WFd, None, B.EPI_MUL_GELUGRAD, r=rF, y=yF), d, F),
+        ("fc1 bwd   (plain)", lambda i: B.linear(xF, WdF, None, B.EPI_BIAS, y=yd), F, d),
+        ("proj bwd  (plain)", lambda i: B.linear(xd, Wdd, None, B.EPI_BIAS, y=yd), d, d),
+    ]
+    out = []
+    for name, fn, k, n in cases:
+        ms = _time(fn, iters)
+        fl = 2.0 * M * k * n
+        out.append({"op": "linear", "case": name, "M": M, "K": k, "N": n, "us": round(ms * 1e3, 1),
+                    "tflops": round(fl / ms / 1e9, 1), "frac_of_bf16_peak": round(fl / ms / 1e9 / tflops, 3),
+                    "peak_source": src + " burst"})
+    return out
+
+
 def bench_aggregate(K, P, iters=50):
     hbm, _, src = _peaks()
     nset = max(1, min(8, -(-2 * L2_BYTES // (K * P * 4))))
@@ -100,7 +129,7 @@ def bench_attention(nseq, T, heads, iters=10):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["linear", "linear-sweep", "aggregate", "aggregate-sweep", "attention"])
+    ap.add_argument("what", choices=["linear", "linear-sweep", "epilogues", "aggregate", "aggregate-sweep", "attention"])
     ap.add_argument("--M", type=int, default=32768)
     ap.add_argument("--n-in", type=int, default=1024)
     ap.add_argument("--n-out", type=int, default=3072)
@@ -131,6 +160,9 @@ def main():
                     for r in rs:
                         for G in Gs:
                             print(json.dumps(bench_linear(M, n_in, n_out, r, G, 10)), flush=True)
+    elif a.what == "epilogues":
+        for row in bench_epilogues(a.M, a.n_in, 4 * a.n_in, a.iters):
+            print(json.dumps(row), flush=True)
     elif a.what == "aggregate":
         print(json.dumps(bench_aggregate(a.K, a.P, a.iters)))
     elif a.what == "aggregate-sweep":

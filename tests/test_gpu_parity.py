@@ -296,3 +296,27 @@ def test_error_paths():
         eng.bind_frozen("wte", torch.zeros(8, dtype=torch.float32, device="cuda"))
     assert e.value.code == -1
     assert eng.device_status() == 0
+
+
+@pytest.mark.parametrize("M,n_in,n_out", [(256, 128, 512), (1024, 1024, 1000), (512, 256, 64)])
+def test_linear_epilogues_bf16(M, n_in, n_out):
+    """Frozen linear with each fused epilogue (pair kernel, single-CTA kernel, ragged width)
+    against fp64: bias, bias + GELU (pre-activation saved), bias + residual, product with GELU'."""
+    rng = np.random.default_rng(M + n_out)
+    bfv = lambda a: synth._to_bf16_values(a.astype(np.float32))
+    x, W = bfv(rng.normal(size=(M, n_in))), bfv(rng.normal(size=(n_out, n_in)) / np.sqrt(n_in))
+    bias, r = bfv(rng.normal(size=n_out) * 0.1), bfv(rng.normal(size=(M, n_out)))
+    dev = lambda a: torch.from_numpy(a).cuda().bfloat16()
+    xd, Wd, bd, rd = dev(x), dev(W), dev(bias), dev(r)
+    acc = x.astype(np.float64) @ W.astype(np.float64).T
+    y = B.linear(xd, Wd, bd, B.EPI_BIAS)
+    assert H.rel_err(H.tnp(y), acc + bias) <= TOL_BF16
+    y, z = B.linear(xd, Wd, bd, B.EPI_BIAS_GELU)
+    assert H.rel_err(H.tnp(z), acc + bias) <= TOL_BF16
+    assert H.rel_err(H.tnp(y), O.gelu_fwd(acc + bias)) <= TOL_BF16
+    y = B.linear(xd, Wd, bd, B.EPI_BIAS_RESID, r=rd)
+    assert H.rel_err(H.tnp(y), acc + bias + r) <= TOL_BF16
+    y = B.linear(xd, Wd, None, B.EPI_MUL_GELUGRAD, r=rd)
+    assert H.rel_err(H.tnp(y), acc * O.gelu_grad(r.astype(np.float64))) <= TOL_BF16
+    y2 = B.linear(xd, Wd, None, B.EPI_MUL_GELUGRAD, r=rd, use_tensor_cores=False)
+    assert H.rel_err(H.tnp(y2), acc * O.gelu_grad(r.astype(np.float64))) <= TOL_BF16
