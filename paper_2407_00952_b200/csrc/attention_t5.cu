@@ -1,0 +1,363 @@
+// Causal multi-head attention forward on the 5th-generation tensor cores (tcgen05 + TMEM + TMA),
+// bf16, head width 64, sequence length a multiple of 128.
+//
+// One CTA per (sequence, head): it walks the 128-row query tiles of that head one after another
+// (set-up cost is paid once per head, K/V tiles are re-read from L2); two CTAs fit on an SM so that
+// the softmax of one overlaps the products of the other.  Per 128-row key tile:
+//   S  = Q K^T      tcgen05.mma M128 N128 K16 x4, both operands K-major from TMA-swizzled tiles
+//   softmax         one thread per query row reads S from tensor memory (twice: row max, then
+//                   exponentials), keeps the running max / sum, writes P (bf16) to shared memory
+//   O' = P V        tcgen05.mma M128 N64 K16 x8; V is used as loaded ([key, feature] rows, i.e. an
+//                   MN-major operand), no transpose
+//   O  = O*corr+O'  in registers of the row's thread
+// Warp roles (192 threads): warp 0 TMA producer, warp 1 tensor-memory owner + MMA issuer,
+// warps 2..5 softmax (warp w owns accumulator lanes 32*(w%4)..+31).
+// All mbarrier waits are bounded (see tc_common.cuh); on expiry a code is left in `status`.
+#include "tc_common.cuh"
+
+namespace sl {
+namespace {
+
+using namespace tc;
+
+constexpr int DH = 64;
+constexpr int BQ = 128;                   // query rows per tile
+constexpr int BKV = 128;                  // key rows per step
+constexpr int TILE = BQ * DH * 2;         // 16 KB: one [128 x 64] bf16 tile
+constexpr int T5_THREADS = 192;
+constexpr int OFF_Q = 0, OFF_K = TILE, OFF_V = 3 * TILE, OFF_P = 4 * TILE, OFF_BAR = 6 * TILE;
+constexpr int T5_SMEM = 6 * TILE + 256 + 1024;     // tiles + barriers + alignment slack
+constexpr int TMEM_COLS = 256;            // S at columns [0,128), O' at [128,192)
+constexpr uint32_t IDESC_S = make_idesc(BQ, BKV);
+constexpr uint32_t IDESC_PV = make_idesc(BQ, DH) | (1u << 16);   // B operand MN-major
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float LN2 = 0.6931471805599453f;
+
+// barrier slots
+enum { Q_FULL = 0, Q_EMPTY = 1, K_FULL = 2 /*+stage*/, K_EMPTY = 4 /*+stage*/, V_FULL = 6, V_EMPTY = 7,
+       S_FULL = 8, S_FREE = 9, P_READY = 10, O_FULL = 11, O_FREE = 12, N_BARS = 13 };
+
+// Shared-memory descriptor of an MN-major operand tile stored as [k rows][64 elements] with
+// 128-byte rows and 128-byte swizzle: groups of 8 k-rows are 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;                        // leading byte offset: unused (one 64-element block along MN)
+  d |= (uint64_t)(1024 >> 4) << 32;              // stride between 8-row groups along K
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;                        // 128-byte swizzle
+  return d;
+}
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct T5Params {
+  int T, H, d;
+  float scale_log2;
+  float* lse;
+  int* status;
+};
+
+// The CTA's work is a flat sequence of (query tile, key tile) steps: query tiles nq-1 .. 0, for
+// each the key tiles 0 .. qt.  `it` counts steps, `iq` counts query tiles; barrier parities derive
+// from these counters so that every role stays in lock step without sharing state.
+__global__ void __launch_bounds__(T5_THREADS, 2)
+attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapO, T5Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - raw);
+  const uint32_t bar = base + OFF_BAR;
+  auto B = [&](int i) { return bar + 8u * i; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + OFF_BAR + 8 * N_BARS);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + OFF_BAR + 8 * N_BARS + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int h = blockIdx.x, b = blockIdx.y;
+  const int nq = p.T / BQ;
+  const int seq_row0 = b * p.T;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < N_BARS; ++i) mbar_init(B(i), (i == S_FREE || i == P_READY || i == O_FREE) ? 128 : 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32((const void*)tmem_slot)), "r"((uint32_t)TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tS = tmem_base, tO = tmem_base + 128u;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0;                                   // running step index of the K loads issued
+      auto load_K = [&](int step, int j) -> bool {
+        const int s = step & 1;
+        if (!mbar_wait(B(K_EMPTY + s), (((uint32_t)(step >> 1)) & 1u) ^ 1u, abort_flag, p.status, 21)) return false;
+        mbar_expect_tx(B(K_FULL + s), TILE);
+        tma_load_2d(base + OFF_K + s * TILE, &mapQKV, B(K_FULL + s), p.d + h * DH, seq_row0 + j * BKV);
+        return true;
+      };
+      for (int iq = 0; iq < nq && ok; ++iq) {
+        const int qt = nq - 1 - iq;
+        // Q of this query tile (the buffer is free once the previous tile's last S product is done)
+        if (!mbar_wait(B(Q_EMPTY), ((uint32_t)iq & 1u) ^ 1u, abort_flag, p.status, 20)) { ok = false; break; }
+        mbar_expect_tx(B(Q_FULL), TILE);
+        tma_load_2d(base + OFF_Q, &mapQKV, B(Q_FULL), h * DH, seq_row0 + qt * BQ);
+        if (iq == 0) ok = load_K(0, 0);              // K runs one step ahead of V
+        for (int j = 0; j <= qt && ok; ++j, ++it) {
+          // next step's K: the next key tile, or key tile 0 of the next query tile
+          if (j < qt) ok = load_K(it + 1, j + 1);
+          else if (iq + 1 < nq) ok = load_K(it + 1, 0);
+          if (!ok) break;
+          if (!mbar_wait(B(V_EMPTY), ((uint32_t)it & 1u) ^ 1u, abort_flag, p.status, 22)) { ok = false; break; }
+          mbar_expect_tx(B(V_FULL), TILE);
+          tma_load_2d(base + OFF_V, &mapQKV, B(V_FULL), 2 * p.d + h * DH, seq_row0 + j * BKV);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      bool ok = true;
+      const uint64_t qdesc = make_smem_desc(base + OFF_Q);
+      // S of step `step`; first_of_q: wait for the query tile iq; last_of_q: release the Q buffer
+      auto issue_S = [&](int step, int iq, bool first_of_q, bool last_of_q) -> bool {
+        const int s = step & 1;
+        if (first_of_q && !mbar_wait(B(Q_FULL), (uint32_t)iq & 1u, abort_flag, p.status, 25)) return false;
+        if (!mbar_wait(B(K_FULL + s), (uint32_t)(step >> 1) & 1u, abort_flag, p.status, 23)) return false;
+        if (!mbar_wait(B(S_FREE), ((uint32_t)step & 1u) ^ 1u, abort_flag, p.status, 24)) return false;
+        tc_fence_after();
+        const uint64_t kdesc = make_smem_desc(base + OFF_K + s * TILE);
+#pragma unroll
+        for (int k = 0; k < DH / UMMA_K; ++k)
+          tc_mma_bf16(tS, qdesc + (uint64_t)(2 * k), kdesc + (uint64_t)(2 * k), IDESC_S, k != 0 ? 1u : 0u);
+        tc_commit(B(K_EMPTY + s));
+        if (last_of_q) tc_commit(B(Q_EMPTY));
+        tc_commit(B(S_FULL));
+        return true;
+      };
+      int it = 0;
+      ok = issue_S(0, 0, true, nq - 1 == 0);
+      for (int iq = 0; iq < nq && ok; ++iq) {
+        const int qt = nq - 1 - iq;
+        for (int j = 0; j <= qt && ok; ++j, ++it) {
+          // next step's S overlaps this step's softmax
+          if (j < qt) ok = issue_S(it + 1, iq, false, j + 1 == qt);
+          else if (iq + 1 < nq) ok = issue_S(it + 1, iq + 1, true, qt - 1 == 0);
+          if (!ok) break;
+          if (!mbar_wait(B(P_READY), (uint32_t)it & 1u, abort_flag, p.status, 26)) { ok = false; break; }
+          if (!mbar_wait(B(V_FULL), (uint32_t)it & 1u, abort_flag, p.status, 27)) { ok = false; break; }
+          if (!mbar_wait(B(O_FREE), ((uint32_t)it & 1u) ^ 1u, abort_flag, p.status, 28)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t vdesc = make_smem_desc_mn(base + OFF_V);
+#pragma unroll
+          for (int k = 0; k < BKV / UMMA_K; ++k) {
+            // P is two [128 x 64] K-major blocks; inside a block 16 columns = 32 bytes
+            const uint64_t pdesc = make_smem_desc(base + OFF_P + (k >> 2) * TILE) + (uint64_t)(2 * (k & 3));
+            // V advances 16 key rows = 2048 bytes per step
+            tc_mma_bf16(tO, pdesc, vdesc + (uint64_t)(128 * k), IDESC_PV, k != 0 ? 1u : 0u);
+          }
+          tc_commit(B(V_EMPTY));      // V (and P) reusable
+          tc_commit(B(O_FULL));       // O' complete
+        }
+      }
+    }
+  } else {
+    // ---------------- softmax / output: one thread per query row ----------------
+    const int q = warp & 3;
+    const int r = q * 32 + lane;                 // row inside the tile = accumulator lane
+    const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+    bool ok = true;
+    int it = 0;
+    for (int iq = 0; iq < nq; ++iq) {
+      const int qt = nq - 1 - iq;
+      float o_acc[DH];
+#pragma unroll
+      for (int i = 0; i < DH; ++i) o_acc[i] = 0.f;
+      float m_run = -INFINITY, l_run = 0.f;
+      for (int j = 0; j <= qt && ok; ++j, ++it) {
+        if (!mbar_wait(B(S_FULL), (uint32_t)it & 1u, abort_flag, p.status, 29)) { ok = false; break; }
+        tc_fence_after();
+        const bool diag = (j == qt);
+        // On the diagonal tile only columns <= r count; whole 32-column chunks beyond the row are
+        // skipped (their probabilities are zero), the chunk that holds the diagonal is masked.
+        const int c_last = diag ? (r & ~31) : (BKV - 32);       // last chunk with a live column
+        // pass 1: row maximum of the raw scores (the scale is positive)
+        float mx = -INFINITY;
+#pragma unroll 1
+        for (int c = 0; c <= c_last; c += 32) {
+          float v[32];
+          tc_ld32(tS + lane_off + (uint32_t)c, v);
+          tc_wait_ld();
+          if (diag && c == c_last) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (c + i > r) ? -INFINITY : v[i]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, v[i]);
+          }
+        }
+        const float m_new = fmaxf(m_run, mx * p.scale_log2);   // finite: column 0 is never masked
+        const float corr = ex2(m_run - m_new);
+        // pass 2: exponentials, row sum, P to shared memory
+        float psum = 0.f;
+#pragma unroll 1
+        for (int c = 0; c < BKV; c += 32) {
+          uint32_t pk[16];
+          if (c <= c_last) {
+            float v[32];
+            tc_ld32(tS + lane_off + (uint32_t)c, v);
+            tc_wait_ld();
+            const bool mask = diag && c == c_last;
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              float p0 = ex2(fmaf(v[i], p.scale_log2, -m_new)), p1 = ex2(fmaf(v[i + 1], p.scale_log2, -m_new));
+              if (mask) { if (c + i > r) p0 = 0.f; if (c + i + 1 > r) p1 = 0.f; }
+              psum += p0 + p1;
+              __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+              pk[i >> 1] = *reinterpret_cast<uint32_t*>(&pb);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+          }
+          const uint32_t prow = base + OFF_P + (uint32_t)(c >> 6) * TILE + (uint32_t)r * 128u;
+          const uint32_t cbase = (uint32_t)((c & 63) >> 3);          // first 16-byte chunk of these 32 columns
+#pragma unroll
+          for (uint32_t jj = 0; jj < 4; ++jj) {
+            const uint32_t chunk = (cbase + jj) ^ ((uint32_t)r & 7u);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(prow + (chunk << 4)), "r"(pk[4 * jj]),
+                         "r"(pk[4 * jj + 1]), "r"(pk[4 * jj + 2]), "r"(pk[4 * jj + 3]) : "memory");
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(B(S_FREE));                      // S may be overwritten
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(B(P_READY));                     // P visible to the tensor core
+        l_run = l_run * corr + psum;
+        m_run = m_new;
+        // O = O * corr + O'
+        if (!mbar_wait(B(O_FULL), (uint32_t)it & 1u, abort_flag, p.status, 30)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < DH; c += 32) {
+          float v[32];
+          tc_ld32(tO + lane_off + (uint32_t)c, v);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o_acc[c + i] = o_acc[c + i] * corr + v[i];
+        }
+        tc_fence_before();
+        mbar_arrive(B(O_FREE));                      // O' may be overwritten
+      }
+      // normalise, stage the [128 x 64] output tile in the P buffer (free: its last product is
+      // done), one TMA store per query tile
+      if (ok) {
+        const float inv = 1.0f / l_run;
+        const uint32_t orow = base + OFF_P + (uint32_t)r * 128u;
+#pragma unroll
+        for (uint32_t jj = 0; jj < 8; ++jj) {
+          uint32_t w[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 ob = __floats2bfloat162_rn(o_acc[8 * jj + 2 * i] * inv, o_acc[8 * jj + 2 * i + 1] * inv);
+            w[i] = *reinterpret_cast<uint32_t*>(&ob);
+          }
+          const uint32_t chunk = jj ^ ((uint32_t)r & 7u);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(orow + (chunk << 4)), "r"(w[0]), "r"(w[1]),
+                       "r"(w[2]), "r"(w[3]) : "memory");
+        }
+        p.lse[((size_t)b * p.H + h) * p.T + (size_t)qt * BQ + r] = (m_run + log2f(l_run)) * LN2;
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("bar.sync 1, 128;" ::: "memory");         // the four softmax warps (always reached)
+      if (ok && warp == 2 && lane == 0) {
+        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                     ::"l"(&mapO), "r"(base + OFF_P), "r"(h * DH), "r"(seq_row0 + qt * BQ) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging reusable for the next P
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
+    if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
+  // ---------------- teardown ----------------
+  __syncwarp();
+  if (*abort_flag) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+int* g_status = nullptr;      // device word for expired waits when the caller gives none
+__device__ int g_t5_status[4];
+
+bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool init_once() {
+  if (g_encode) return true;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
+      q != cudaDriverEntryPointSuccess)
+    return false;
+  if (cudaGetSymbolAddress((void**)&g_status, g_t5_status) != cudaSuccess) return false;
+  if (cudaMemset(g_status, 0, sizeof(int) * 4) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(attn_fwd_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T5_SMEM) != cudaSuccess) return false;
+  g_encode = (EncodeTiledFn)fn;
+  return true;
+}
+
+}  // namespace
+
+bool attention_t5_supported(int dt, int T, int H, int d) {
+  return dt == DT_BF16 && H > 0 && d % H == 0 && d / H == DH && T >= BQ && T % BQ == 0;
+}
+
+cudaError_t attention_fwd_t5(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, int* status,
+                             cudaStream_t st) {
+  if (!attention_t5_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
+  if (!init_once()) return cudaErrorInitializationError;
+  CUtensorMap mQKV, mO;
+  if (!make_map(&mQKV, qkv, (uint64_t)nseq * T, (uint64_t)3 * d, BQ)) return cudaErrorInvalidValue;
+  if (!make_map(&mO, o, (uint64_t)nseq * T, (uint64_t)d, BQ)) return cudaErrorInvalidValue;
+  T5Params p;
+  p.T = T; p.H = H; p.d = d; p.scale_log2 = LOG2E / sqrtf((float)DH); p.lse = lse;
+  p.status = status ? status : g_status;
+  dim3 grid(H, nseq);
+  attn_fwd_t5_kernel<<<grid, T5_THREADS, T5_SMEM, st>>>(mQKV, mO, p);
+  return cudaGetLastError();
+}
+
+}  // namespace sl

@@ -6,6 +6,8 @@
 //   backward: rowdot = sum(dO*O); a dQ kernel per query tile (loops over key tiles) and a dK/dV
 //             kernel per key tile (loops over query tiles).  No atomics: results are bit-reproducible.
 // Products use mma.sync m16n8k16 with ldmatrix-fed fragments from XOR-swizzled shared tiles.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "kernels.h"
 
@@ -377,8 +379,18 @@ bool attention_tc_supported(int dt, int T, int H, int d) {
   return dt == DT_BF16 && H > 0 && d % H == 0 && d / H == DH && T >= BT && T % BT == 0;
 }
 
+// SPLITLORA_ATTENTION_MMA_SYNC=1 keeps the mma.sync kernels even where the tcgen05 ones apply
+// (debugging aid / second opinion).
+static bool prefer_mma_sync() {
+  static int v = -1;
+  if (v < 0) { const char* e = std::getenv("SPLITLORA_ATTENTION_MMA_SYNC"); v = (e && e[0] == '1') ? 1 : 0; }
+  return v == 1;
+}
+
 cudaError_t attention_fwd_tc(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, cudaStream_t st) {
   if (!attention_tc_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
+  if (attention_t5_supported(DT_BF16, T, H, d) && !prefer_mma_sync())
+    return attention_fwd_t5(qkv, nseq, T, H, d, o, lse, nullptr, st);
   dim3 grid(T / BT, H, nseq);
   const float scale_log2 = LOG2E / sqrtf((float)DH);
   static bool attr = false;
