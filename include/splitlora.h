@@ -160,6 +160,33 @@ int splitlora_round(splitlora_ctx* ctx, const int32_t* tokens, const int32_t* la
 int splitlora_round_host(splitlora_ctx* ctx, const int32_t* tokens_host, const int32_t* labels_host,
                          const int64_t* sample_counts, float* loss_out);
 
+/* ---- sharding the clients of a round over several devices ----------------------------------
+ * Clients are independent on the client side (step a1, a5) and the server loss is a mean over the
+ * concatenated batch (step a3), so a device can own a subset of the clients and the matching rows
+ * of S^t.  Every device holds the same frozen weights and the same server adapters and runs the
+ * three calls on its own clients; two sums over devices make the result equal to the one-device
+ * round: the server adapter gradients before the server update, and the weighted adapter sums of
+ * Eq. 8-9 at aggregation.  The library does no communication itself; the caller reduces the
+ * buffers below (e.g. with an NCCL all-reduce on the context stream). */
+
+/* Number of valid label positions of the WHOLE concatenated batch (all devices).  When > 0 it
+ * replaces the local count as the normaliser of the loss and of dL/dlogits in server_step, so that
+ * local losses and gradients add up to the global ones.  0 restores the local count. */
+int splitlora_set_loss_normalizer(splitlora_ctx* ctx, int64_t n_valid_global);
+/* on != 0: server_step stops after the backward pass (gradients in the server gradient buffer) and
+ * leaves Eq. 4-5 to a later splitlora_server_update, after the caller has summed the gradients. */
+int splitlora_set_deferred_server_update(splitlora_ctx* ctx, int on);
+int splitlora_server_update(splitlora_ctx* ctx);
+/* Device pointer and element count of an adapter arena: side SPLITLORA_SIDE_*, kind 0 = fp32
+ * parameters, 1 = fp32 gradients.  Client arenas are [K, per-client]; the pointer stays valid while
+ * the workspace is bound.  After writing parameters call splitlora_adapters_changed(side). */
+int splitlora_adapter_buffer(splitlora_ctx* ctx, int side, int kind, float** dev, int64_t* count);
+int splitlora_adapters_changed(splitlora_ctx* ctx, int side);
+/* Eq. 8-9 for the local clients of one device: every local client A and B becomes
+ * sum_{i local} (|D_i| / total_count) P_i, total_count = |D| over ALL devices' clients.  Summing
+ * the client parameter buffers over devices afterwards gives every client the global average. */
+int splitlora_aggregate_partial(splitlora_ctx* ctx, const int64_t* sample_counts, int64_t total_count);
+
 /* Device loss of the last server_step (fp32 scalar, DEVICE pointer into the workspace). */
 int splitlora_loss_device(splitlora_ctx* ctx, const float** loss_dev);
 

@@ -27,7 +27,9 @@ EXPORTS = [
     "splitlora_device_status", "splitlora_launch_count", "splitlora_profile_enable", "splitlora_profile_report",
     "splitlora_lora_linear_workspace_bytes", "splitlora_lora_linear_fwd", "splitlora_lora_linear_bwd",
     "splitlora_transpose", "splitlora_aggregate_buffers", "splitlora_attention_fwd", "splitlora_attention_bwd",
-    "splitlora_attention_bwd_static", "splitlora_linear",
+    "splitlora_attention_bwd_static", "splitlora_linear", "splitlora_set_loss_normalizer",
+    "splitlora_set_deferred_server_update", "splitlora_server_update", "splitlora_adapter_buffer",
+    "splitlora_adapters_changed", "splitlora_aggregate_partial",
 ]
 
 
@@ -207,6 +209,37 @@ class SplitLoRA:
                                                   C.c_void_p(labels_host.data_ptr()), arr,
                                                   C.byref(loss) if want_loss else None))
         return loss.value if want_loss else None
+
+    # ---- sharding hooks ----
+    def set_loss_normalizer(self, n_valid_global: int):
+        self._check(self.lib.splitlora_set_loss_normalizer(self.ctx, C.c_int64(n_valid_global)))
+
+    def set_deferred_server_update(self, on: bool):
+        self._check(self.lib.splitlora_set_deferred_server_update(self.ctx, 1 if on else 0))
+
+    def server_update(self):
+        self._check(self.lib.splitlora_server_update(self.ctx))
+
+    def adapter_buffer(self, side: int, kind: int) -> torch.Tensor:
+        """fp32 view (no copy) of an adapter arena inside the workspace: kind 0 parameters, 1 gradients."""
+        ptr, n = C.c_void_p(0), C.c_int64(0)
+        self._check(self.lib.splitlora_adapter_buffer(self.ctx, side, kind, C.byref(ptr), C.byref(n)))
+        off = ptr.value - self.workspace.data_ptr()
+        return self.workspace[off:off + 4 * n.value].view(torch.float32)
+
+    def adapters_changed(self, side: int):
+        self._check(self.lib.splitlora_adapters_changed(self.ctx, side))
+
+    def aggregate_partial(self, counts, total_count: int):
+        arr = (C.c_int64 * len(counts))(*[int(x) for x in counts])
+        self._check(self.lib.splitlora_aggregate_partial(self.ctx, arr, C.c_int64(total_count)))
+
+    def loss_tensor(self) -> torch.Tensor:
+        """fp32 view of the device loss scalar of the last server_step."""
+        ptr = C.c_void_p(0)
+        self._check(self.lib.splitlora_loss_device(self.ctx, C.byref(ptr)))
+        off = ptr.value - self.workspace.data_ptr()
+        return self.workspace[off:off + 4].view(torch.float32)
 
     def device_status(self) -> int:
         code = C.c_int32(0)

@@ -117,9 +117,100 @@ __global__ void ln_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ x,
   }
 }
 
+// Register-resident variants for rows of exactly NV vectors per lane (d = NV * 32 * vector width):
+// the row is read from memory once and kept in registers between the statistics and the output.
+template <typename T, int NV>
+__global__ void __launch_bounds__(256) ln_fwd_reg_kernel(const T* __restrict__ x, const T* __restrict__ g,
+                                                         const T* __restrict__ b, T* __restrict__ y,
+                                                         float* __restrict__ mean, float* __restrict__ rstd, int M,
+                                                         int d, float eps) {
+  constexpr int N = Vec16<T>::N;
+  int row = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+  int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  const T* xr = x + (size_t)row * d;
+  Vec16<T> xv[NV];
+#pragma unroll
+  for (int k = 0; k < NV; ++k) xv[k].load(xr + (k * 32 + lane) * N);
+  float s = 0.f;
+#pragma unroll
+  for (int k = 0; k < NV; ++k)
+#pragma unroll
+    for (int i = 0; i < N; ++i) s += xv[k].get(i);
+  const float mu = warp_sum(s) / d;
+  float q = 0.f;
+#pragma unroll
+  for (int k = 0; k < NV; ++k)
+#pragma unroll
+    for (int i = 0; i < N; ++i) { float t = xv[k].get(i) - mu; q += t * t; }
+  const float rs = rsqrtf(warp_sum(q) / d + eps);
+  T* yr = y + (size_t)row * d;
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    const int c = (k * 32 + lane) * N;
+    Vec16<T> gv, bv, o;
+    gv.load(g + c); bv.load(b + c);
+#pragma unroll
+    for (int i = 0; i < N; ++i) o.set(i, (xv[k].get(i) - mu) * rs * gv.get(i) + bv.get(i));
+    o.store(yr + c);
+  }
+  if (lane == 0) { mean[row] = mu; rstd[row] = rs; }
+}
+
+template <typename T, int NV>
+__global__ void __launch_bounds__(256) ln_bwd_reg_kernel(const T* __restrict__ dy, const T* __restrict__ x,
+                                                         const T* __restrict__ g, const float* __restrict__ mean,
+                                                         const float* __restrict__ rstd, const T* __restrict__ resid,
+                                                         T* __restrict__ dx, int M, int d) {
+  constexpr int N = Vec16<T>::N;
+  int row = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+  int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  const size_t off = (size_t)row * d;
+  const float mu = mean[row], rs = rstd[row];
+  Vec16<T> xv[NV], dv[NV];
+#pragma unroll
+  for (int k = 0; k < NV; ++k) { xv[k].load(x + off + (k * 32 + lane) * N); dv[k].load(dy + off + (k * 32 + lane) * N); }
+  float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    Vec16<T> gv; gv.load(g + (k * 32 + lane) * N);
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      float dxh = dv[k].get(i) * gv.get(i);
+      s1 += dxh;
+      s2 += dxh * (xv[k].get(i) - mu) * rs;
+    }
+  }
+  const float m1 = warp_sum(s1) / d, m2 = warp_sum(s2) / d;
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    const int c = (k * 32 + lane) * N;
+    Vec16<T> gv, rv, o;
+    gv.load(g + c);
+    if (resid) rv.load(resid + off + c);
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      float xh = (xv[k].get(i) - mu) * rs;
+      float v = (dv[k].get(i) * gv.get(i) - m1 - xh * m2) * rs;
+      if (resid) v += rv.get(i);
+      o.set(i, v);
+    }
+    o.store(dx + off + c);
+  }
+}
+
 cudaError_t layernorm_fwd(int dt, const void* x, const void* g, const void* b, void* y, float* mean, float* rstd,
                           int M, int d, float eps, cudaStream_t st) {
   int blocks = (M + 7) / 8;
+  if (dt == DT_BF16 && d == 1024) {
+    ln_fwd_reg_kernel<bf16, 4><<<blocks, 256, 0, st>>>((const bf16*)x, (const bf16*)g, (const bf16*)b, (bf16*)y, mean, rstd, M, d, eps);
+    return cudaGetLastError();
+  }
+  if (dt == DT_BF16 && d == 768) {
+    ln_fwd_reg_kernel<bf16, 3><<<blocks, 256, 0, st>>>((const bf16*)x, (const bf16*)g, (const bf16*)b, (bf16*)y, mean, rstd, M, d, eps);
+    return cudaGetLastError();
+  }
   if (dt == DT_BF16)
     ln_fwd_kernel<bf16><<<blocks, 256, 0, st>>>((const bf16*)x, (const bf16*)g, (const bf16*)b, (bf16*)y, mean, rstd, M, d, eps);
   else
@@ -130,6 +221,14 @@ cudaError_t layernorm_fwd(int dt, const void* x, const void* g, const void* b, v
 cudaError_t layernorm_bwd(int dt, const void* dy, const void* x, const void* g, const float* mean,
                           const float* rstd, const void* resid, void* dx, int M, int d, cudaStream_t st) {
   int blocks = (M + 7) / 8;
+  if (dt == DT_BF16 && d == 1024) {
+    ln_bwd_reg_kernel<bf16, 4><<<blocks, 256, 0, st>>>((const bf16*)dy, (const bf16*)x, (const bf16*)g, mean, rstd, (const bf16*)resid, (bf16*)dx, M, d);
+    return cudaGetLastError();
+  }
+  if (dt == DT_BF16 && d == 768) {
+    ln_bwd_reg_kernel<bf16, 3><<<blocks, 256, 0, st>>>((const bf16*)dy, (const bf16*)x, (const bf16*)g, mean, rstd, (const bf16*)resid, (bf16*)dx, M, d);
+    return cudaGetLastError();
+  }
   if (dt == DT_BF16)
     ln_bwd_kernel<bf16><<<blocks, 256, 0, st>>>((const bf16*)dy, (const bf16*)x, (const bf16*)g, mean, rstd, (const bf16*)resid, (bf16*)dx, M, d);
   else
@@ -141,7 +240,12 @@ cudaError_t layernorm_bwd(int dt, const void* dy, const void* x, const void* g, 
 // cross-entropy: one block per row.  Pass 1: online max / sum of exp; pass 2: overwrite the row
 // with (softmax - onehot) / n_valid.  Pad columns [V, ld) are written as zero.
 // ------------------------------------------------------------------------------------------
-__global__ void count_valid_kernel(const int32_t* __restrict__ labels, int M, int* __restrict__ n_valid) {
+__global__ void count_valid_kernel(const int32_t* __restrict__ labels, int M, int* __restrict__ n_valid,
+                                   int normalizer_override) {
+  if (normalizer_override > 0) {       // the batch is one shard of a larger one: use the global count
+    if (threadIdx.x == 0) *n_valid = normalizer_override;
+    return;
+  }
   __shared__ int sh[32];
   int c = 0;
   for (int i = threadIdx.x; i < M; i += blockDim.x) c += labels[i] >= 0 ? 1 : 0;
@@ -175,14 +279,14 @@ __global__ void ce_kernel(T* __restrict__ logits, int64_t ld, const int32_t* __r
     float nm = fmaxf(mx, lm);
     float acc = 0.f;
 #pragma unroll
-    for (int i = 0; i < N; ++i) acc += expf(v.get(i) - nm);
-    sm = sm * expf(mx - nm) + acc;
+    for (int i = 0; i < N; ++i) acc += __expf(v.get(i) - nm);
+    sm = sm * __expf(mx - nm) + acc;
     mx = nm;
   }
   for (int c = Vv + threadIdx.x; c < V; c += blockDim.x) {
     float zc = to_f<T>(z[c]);
     float nm = fmaxf(mx, zc);
-    sm = sm * expf(mx - nm) + expf(zc - nm);
+    sm = sm * __expf(mx - nm) + __expf(zc - nm);
     mx = nm;
   }
   // combine (max, sum) pairs across the warp, then across warps
@@ -190,8 +294,8 @@ __global__ void ce_kernel(T* __restrict__ logits, int64_t ld, const int32_t* __r
   for (int o = 16; o > 0; o >>= 1) {
     float om = __shfl_xor_sync(0xffffffffu, mx, o), os = __shfl_xor_sync(0xffffffffu, sm, o);
     float nm = fmaxf(mx, om);
-    float a = (mx == -INFINITY) ? 0.f : sm * expf(mx - nm);
-    float b = (om == -INFINITY) ? 0.f : os * expf(om - nm);
+    float a = (mx == -INFINITY) ? 0.f : sm * __expf(mx - nm);
+    float b = (om == -INFINITY) ? 0.f : os * __expf(om - nm);
     sm = a + b; mx = nm;
   }
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
@@ -203,8 +307,8 @@ __global__ void ce_kernel(T* __restrict__ logits, int64_t ld, const int32_t* __r
     for (int o = 16; o > 0; o >>= 1) {
       float om = __shfl_xor_sync(0xffffffffu, m2, o), os = __shfl_xor_sync(0xffffffffu, s2, o);
       float nm = fmaxf(m2, om);
-      float a = (m2 == -INFINITY) ? 0.f : s2 * expf(m2 - nm);
-      float b = (om == -INFINITY) ? 0.f : os * expf(om - nm);
+      float a = (m2 == -INFINITY) ? 0.f : s2 * __expf(m2 - nm);
+      float b = (om == -INFINITY) ? 0.f : os * __expf(om - nm);
       s2 = a + b; m2 = nm;
     }
     if (lane == 0) {
@@ -224,7 +328,7 @@ __global__ void ce_kernel(T* __restrict__ logits, int64_t ld, const int32_t* __r
 #pragma unroll
     for (int i = 0; i < N; ++i) {
       int col = c + i;
-      float p = col < V ? expf(v.get(i) - lse) : 0.f;
+      float p = col < V ? __expf(v.get(i) - lse) : 0.f;
       if (col == y) p -= 1.0f;
       o.set(i, p * inv);
     }
@@ -249,8 +353,8 @@ __global__ void loss_reduce_kernel(const float* __restrict__ row_loss, int M, co
 }
 
 cudaError_t cross_entropy(int dt, void* logits, int64_t ld, const int32_t* labels, int M, int V, float* row_loss,
-                          int* n_valid, float* loss, cudaStream_t st) {
-  count_valid_kernel<<<1, 1024, 0, st>>>(labels, M, n_valid);
+                          int* n_valid, float* loss, int normalizer_override, cudaStream_t st) {
+  count_valid_kernel<<<1, 1024, 0, st>>>(labels, M, n_valid, normalizer_override);
   if (dt == DT_BF16) ce_kernel<bf16><<<M, 256, 0, st>>>((bf16*)logits, ld, labels, V, row_loss, n_valid);
   else ce_kernel<float><<<M, 256, 0, st>>>((float*)logits, ld, labels, V, row_loss, n_valid);
   loss_reduce_kernel<<<1, 1024, 0, st>>>(row_loss, M, n_valid, loss);

@@ -63,8 +63,9 @@ cudaError_t layernorm_bwd(int dt, const void* dy, const void* x, const void* g, 
 
 // Cross-entropy over logits [M, ld] (V valid columns): writes per-row losses, then overwrites the
 // logits with d loss / d logits (zero in the pad columns) and reduces the mean loss.
+// normalizer_override > 0 replaces the count of valid labels (the batch is a shard of a larger one).
 cudaError_t cross_entropy(int dt, void* logits, int64_t ld, const int32_t* labels, int M, int V,
-                          float* row_loss, int* n_valid, float* loss, cudaStream_t st);
+                          float* row_loss, int* n_valid, float* loss, int normalizer_override, cudaStream_t st);
 
 // Attention, fused qkv layout [nseq*T, 3d]; heads are contiguous slices of width d/H.
 cudaError_t attention_fwd_simt(int dt, const void* qkv, int nseq, int T, int H, int d, void* o, float* lse,

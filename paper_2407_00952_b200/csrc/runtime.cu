@@ -85,6 +85,9 @@ struct splitlora_ctx {
   // state
   bool client_copies_dirty = true, server_copies_dirty = true;
   bool have_client_fwd = false;
+  // sharding over devices: global loss normaliser (0: local count) and server update left to the caller
+  int64_t loss_normalizer = 0;
+  bool defer_server_update = false;
   int64_t round_index = 0, server_steps = 0, client_steps = 0;
   int64_t launches = 0;
   // profiling
@@ -621,7 +624,8 @@ int splitlora_server_step(splitlora_ctx* c, const void* act_in, const int32_t* l
     a.w_rows = c->V;
     CK(c, linear(c, "head_fwd", a)); }
   { Scope s(c, "cross_entropy", 3);
-    CK(c, cross_entropy(c->dt, c->logits, c->Vpad, labels, M, c->V, c->row_loss, c->n_valid, c->loss_dev, c->st)); }
+    CK(c, cross_entropy(c->dt, c->logits, c->Vpad, labels, M, c->V, c->row_loss, c->n_valid, c->loss_dev,
+                        (int)c->loss_normalizer, c->st)); }
   // backward: head, final norm, blocks L-1 .. cut
   { GemmArgs a = base_args(c, c->logits, c->Vpad, c->wteT, c->Vpad, c->g_a, d, M, d, c->Vpad);
     CK(c, linear(c, "head_bwd", a)); }
@@ -635,8 +639,10 @@ int splitlora_server_step(splitlora_ctx* c, const void* act_in, const int32_t* l
     other = cur; cur = dst;
   }
   // Eq. 4-5: server update
-  CK(c, run_optimizer(c, false));
-  c->server_copies_dirty = true;
+  if (!c->defer_server_update) {
+    CK(c, run_optimizer(c, false));
+    c->server_copies_dirty = true;
+  }
   if (loss_out) {
     CK(c, cudaMemcpyAsync(loss_out, c->loss_dev, 4, cudaMemcpyDeviceToHost, c->st));
     CK(c, cudaStreamSynchronize(c->st));
@@ -667,7 +673,7 @@ int splitlora_client_bwd(splitlora_ctx* c, const void* act_grad_in) {
   return SPLITLORA_OK;
 }
 
-int splitlora_aggregate(splitlora_ctx* c, const int64_t* counts) {
+static int aggregate_with_total(splitlora_ctx* c, const int64_t* counts, double total_override) {
   if (!c) return SPLITLORA_ERR_ARG;
   if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
   if (!counts) return fail(c, SPLITLORA_ERR_ARG, "null counts");
@@ -676,12 +682,63 @@ int splitlora_aggregate(splitlora_ctx* c, const int64_t* counts) {
     if (counts[i] < 0) return fail(c, SPLITLORA_ERR_COUNTS, "negative sample count");
     total += (double)counts[i];
   }
+  if (total_override > 0.0) {
+    if (total > total_override) return fail(c, SPLITLORA_ERR_COUNTS, "local counts exceed the global total");
+    total = total_override;
+  }
   if (!(total > 0.0)) return fail(c, SPLITLORA_ERR_COUNTS, "all sample counts are zero");
   float w[AGG_MAX_CLIENTS];
   for (int i = 0; i < c->K; ++i) w[i] = (float)((double)counts[i] / total);
   { Scope s(c, "aggregate", 1);
     CK(c, aggregate(c->cp, c->K, c->Pc, w, c->st)); }
   c->client_copies_dirty = true;
+  return SPLITLORA_OK;
+}
+
+int splitlora_aggregate(splitlora_ctx* c, const int64_t* counts) { return aggregate_with_total(c, counts, 0.0); }
+
+// ---- hooks for sharding the clients over several devices --------------------------------------
+
+int splitlora_aggregate_partial(splitlora_ctx* c, const int64_t* counts, int64_t total_count) {
+  if (total_count <= 0) return fail(c, SPLITLORA_ERR_COUNTS, "total_count must be positive");
+  return aggregate_with_total(c, counts, (double)total_count);
+}
+
+int splitlora_set_loss_normalizer(splitlora_ctx* c, int64_t n_valid_global) {
+  if (!c || n_valid_global < 0 || n_valid_global > 2147483647LL) return SPLITLORA_ERR_ARG;
+  c->loss_normalizer = n_valid_global;
+  return SPLITLORA_OK;
+}
+
+int splitlora_set_deferred_server_update(splitlora_ctx* c, int on) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  c->defer_server_update = on != 0;
+  return SPLITLORA_OK;
+}
+
+int splitlora_server_update(splitlora_ctx* c) {
+  int rc = check_ready(c);
+  if (rc) return rc;
+  CK(c, run_optimizer(c, false));
+  c->server_copies_dirty = true;
+  return SPLITLORA_OK;
+}
+
+int splitlora_adapter_buffer(splitlora_ctx* c, int side, int kind, float** dev, int64_t* count) {
+  if (!c || !dev || !count) return SPLITLORA_ERR_ARG;
+  if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
+  if (kind != 0 && kind != 1) return fail(c, SPLITLORA_ERR_ARG, "kind must be 0 (parameters) or 1 (gradients)");
+  if (side == SPLITLORA_SIDE_CLIENT) { *dev = kind ? c->cg : c->cp; *count = (int64_t)c->K * c->Pc; }
+  else if (side == SPLITLORA_SIDE_SERVER) { *dev = kind ? c->sg : c->sp; *count = c->Ps; }
+  else return fail(c, SPLITLORA_ERR_ARG, "bad side");
+  return SPLITLORA_OK;
+}
+
+int splitlora_adapters_changed(splitlora_ctx* c, int side) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  if (side == SPLITLORA_SIDE_CLIENT) c->client_copies_dirty = true;
+  else if (side == SPLITLORA_SIDE_SERVER) c->server_copies_dirty = true;
+  else return fail(c, SPLITLORA_ERR_ARG, "bad side");
   return SPLITLORA_OK;
 }
 
