@@ -1,0 +1,538 @@
+// Causal multi-head attention backward on the 5th-generation tensor cores (tcgen05 + TMEM + TMA),
+// bf16, head width 64, sequence length a multiple of 128.  Two kernels, no atomics, bit-reproducible:
+//
+//   attn_bwd_dkv_t5_kernel   one CTA per (sequence, head); for each 128-row key tile it walks the
+//       query tiles i >= key tile and keeps dK, dV as fp32 accumulators in tensor memory:
+//         S^T = K Q^T, dP^T = V dO^T                (M128 N128 K16 x4 each, operands K-major)
+//         P^T = exp(S^T/sqrt(dh) - lse[q]),  dS^T = P^T (dP^T - D[q])      (one thread per key row)
+//         dV += P^T dO,  dK += dS^T Q               (M128 N64 K16 x8 each; dO, Q used as loaded:
+//                                                    MN-major right operands)
+//   attn_bwd_dq_t5_kernel    one CTA per (sequence, head); for each 128-row query tile it walks the
+//       key tiles j <= query tile and keeps dQ in tensor memory:
+//         S = Q K^T, dP = dO V^T,  dS = P (dP - D[row]),  dQ += dS K   (K as loaded: MN-major)
+//
+// D[row] = sum(dO * O) comes from a small pre-pass.  Warp roles (192 threads): warp 0 TMA producer,
+// warp 1 tensor-memory owner + MMA issuer, warps 2..5 element-wise work (thread = accumulator lane).
+// All mbarrier waits are bounded (tc_common.cuh); on expiry a code is left in `status`.
+#include "tc_common.cuh"
+
+namespace sl {
+namespace {
+
+using namespace tc;
+
+constexpr int DH = 64;
+constexpr int BT = 128;                   // rows of a query tile and of a key tile
+constexpr int TILE = BT * DH * 2;         // 16 KB: one [128 x 64] bf16 tile
+constexpr int NTHREADS = 320;             // 2 service warps + 8 element-wise warps
+constexpr int EW_THREADS = 256;           // two warps per accumulator lane quarter, 64 columns each
+constexpr int TMEM_COLS = 512;
+constexpr uint32_t IDESC_128 = make_idesc(BT, BT);                    // [128 x 128] products, both K-major
+constexpr uint32_t IDESC_64MN = make_idesc(BT, DH) | (1u << 16);      // [128 x 64] products, right operand MN-major
+constexpr float LOG2E = 1.4426950408889634f;
+
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+// one row (lane r) of a [128 x 64] bf16 tile in the 128-byte-swizzled layout: 16-byte chunk jj
+__device__ __forceinline__ void st_row_chunk(uint32_t tile, int r, uint32_t jj, const uint32_t* w) {
+  const uint32_t addr = tile + (uint32_t)r * 128u + ((jj ^ ((uint32_t)r & 7u)) << 4);
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+}
+// 32 bf16 values (16 packed words) of row r, columns [c, c+32) of a [128 x 128] operand kept as two
+// [128 x 64] K-major blocks
+__device__ __forceinline__ void st_operand_chunk(uint32_t base2, int r, int c, const uint32_t* pk) {
+  const uint32_t tile = base2 + (uint32_t)(c >> 6) * TILE;
+  const uint32_t cb = (uint32_t)((c & 63) >> 3);
+#pragma unroll
+  for (uint32_t jj = 0; jj < 4; ++jj) st_row_chunk(tile, r, cb + jj, pk + 4 * jj);
+}
+// 8 products [128 x 64] += A[128 x 128] (two K-major blocks at a2) * B (MN-major tile at b)
+__device__ __forceinline__ void mma_acc_128x64(uint32_t d_tmem, uint32_t a2, uint32_t b, bool fresh) {
+  const uint64_t bdesc = make_smem_desc_mn(b);
+#pragma unroll
+  for (int k = 0; k < BT / UMMA_K; ++k) {
+    const uint64_t adesc = make_smem_desc(a2 + (k >> 2) * TILE) + (uint64_t)(2 * (k & 3));
+    tc_mma_bf16(d_tmem, adesc, bdesc + (uint64_t)(128 * k), IDESC_64MN, (fresh && k == 0) ? 0u : 1u);
+  }
+}
+// 4 products [128 x 128] = A[128 x 64] * B[128 x 64]^T, both K-major
+__device__ __forceinline__ void mma_128x128(uint32_t d_tmem, uint32_t a, uint32_t b) {
+  const uint64_t adesc = make_smem_desc(a), bdesc = make_smem_desc(b);
+#pragma unroll
+  for (int k = 0; k < DH / UMMA_K; ++k)
+    tc_mma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), IDESC_128, k != 0 ? 1u : 0u);
+}
+
+struct BwdParams {
+  int T, H, d;
+  float scale;             // 1/sqrt(dh)
+  const float* lse;        // [nseq, H, T] natural log
+  const float* rowdot;     // [nseq, H, T]
+  int* status;
+};
+
+#define T5_SETUP(NBARS, CNT128_A, CNT128_B, CNT128_C)                                                     \
+  extern __shared__ uint8_t smem_raw[];                                                                   \
+  const uint32_t raw = smem_u32(smem_raw);                                                                \
+  const uint32_t base = (raw + 1023u) & ~1023u;                                                           \
+  uint8_t* base_ptr = smem_raw + (base - raw);                                                            \
+  const uint32_t bar = base + OFF_BAR;                                                                    \
+  auto B = [&](int i) { return bar + 8u * i; };                                                           \
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + OFF_BAR + 8 * NBARS);    \
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + OFF_BAR + 8 * NBARS + 8);         \
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;                                             \
+  if (threadIdx.x == 0) {                                                                                 \
+    for (int i = 0; i < NBARS; ++i)                                                                       \
+      mbar_init(B(i), (i == CNT128_A || i == CNT128_B || i == CNT128_C) ? EW_THREADS : 1);                \
+    *abort_flag = 0;                                                                                      \
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");                                    \
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");                                          \
+  }                                                                                                       \
+  if (warp == 1) {                                                                                        \
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"                      \
+                 ::"r"(smem_u32((const void*)tmem_slot)), "r"((uint32_t)TMEM_COLS) : "memory");           \
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");              \
+  }                                                                                                       \
+  tc_fence_before();                                                                                      \
+  __syncthreads();                                                                                        \
+  tc_fence_after();                                                                                       \
+  const uint32_t tmem_base = *tmem_slot;
+
+#define T5_TEARDOWN()                                                                                     \
+  __syncwarp();                                                                                           \
+  if (*abort_flag) { for (int i = 0; i < 2000; ++i) __nanosleep(1000); }                                  \
+  tc_fence_before();                                                                                      \
+  __syncthreads();                                                                                        \
+  if (warp == 1) {                                                                                        \
+    tc_fence_after();                                                                                     \
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory"); \
+  }
+
+// parity to wait on for "the n-th completion (0-based) of this barrier has happened"
+__device__ __forceinline__ uint32_t done(int n) { return (uint32_t)n & 1u; }
+// parity to wait on before the n-th use of a slot whose release is signalled once per use
+__device__ __forceinline__ uint32_t freed(int n) { return ((uint32_t)n & 1u) ^ 1u; }
+
+// ==========================================================================================
+// dK, dV
+// ==========================================================================================
+namespace dkv {
+enum { KV_FULL = 0, KV_EMPTY, QD_FULL /*+s*/, QD_FULL1, QD_EMPTY /*+s*/, QD_EMPTY1, S_FULL, S_FREE, P_READY, P_FREE,
+       ACC_FULL, ACC_FREE, N_BARS };
+constexpr int OFF_K = 0, OFF_V = TILE, OFF_QD = 2 * TILE /* stage s: Q at +s*2*TILE, dO after it */,
+              OFF_PT = 6 * TILE, OFF_DST = 8 * TILE, OFF_STAT = 10 * TILE /* stage s: lse at +s*1024, D at +512 */,
+              OFF_BAR = 10 * TILE + 2048;
+constexpr int SMEM = OFF_BAR + 256 + 1024;
+}  // namespace dkv
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
+                       const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
+  using namespace dkv;
+  T5_SETUP(N_BARS, S_FREE, P_READY, ACC_FREE)
+  const int h = blockIdx.x, b = blockIdx.y;
+  const int nq = p.T / BT;
+  const int seq_row0 = b * p.T;
+  const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+  const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDV = tmem_base + 256u, tDK = tmem_base + 320u;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0;
+      for (int kt = 0; kt < nq && ok; ++kt) {
+        if (!mbar_wait(B(KV_EMPTY), freed(kt), abort_flag, p.status, 41)) { ok = false; break; }
+        mbar_expect_tx(B(KV_FULL), 2 * TILE);
+        tma_load_2d(base + OFF_K, &mapQKV, B(KV_FULL), p.d + h * DH, seq_row0 + kt * BT);
+        tma_load_2d(base + OFF_V, &mapQKV, B(KV_FULL), 2 * p.d + h * DH, seq_row0 + kt * BT);
+        for (int i = kt; i < nq; ++i, ++it) {
+          const int s = it & 1;
+          if (!mbar_wait(B(QD_EMPTY + s), freed(it >> 1), abort_flag, p.status, 42)) { ok = false; break; }
+          mbar_expect_tx(B(QD_FULL + s), 2 * TILE + 1024);
+          tma_load_2d(base + OFF_QD + s * 2 * TILE, &mapQKV, B(QD_FULL + s), h * DH, seq_row0 + i * BT);
+          tma_load_2d(base + OFF_QD + s * 2 * TILE + TILE, &mapDO, B(QD_FULL + s), h * DH, seq_row0 + i * BT);
+          bulk_load(base + OFF_STAT + s * 1024, p.lse + stat0 + (size_t)i * BT, 512, B(QD_FULL + s));
+          bulk_load(base + OFF_STAT + s * 1024 + 512, p.rowdot + stat0 + (size_t)i * BT, 512, B(QD_FULL + s));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0;
+      // S^T and dP^T of step `step` (needs its Q/dO stage and the previous step's reads of S^T, dP^T done)
+      auto issue_SdP = [&](int step) -> bool {
+        const int s = step & 1;
+        if (!mbar_wait(B(QD_FULL + s), done(step >> 1), abort_flag, p.status, 43)) return false;
+        if (!mbar_wait(B(S_FREE), freed(step), abort_flag, p.status, 44)) return false;
+        tc_fence_after();
+        mma_128x128(tS, base + OFF_K, base + OFF_QD + s * 2 * TILE);
+        mma_128x128(tDP, base + OFF_V, base + OFF_QD + s * 2 * TILE + TILE);
+        tc_commit(B(S_FULL));
+        return true;
+      };
+      for (int kt = 0; kt < nq && ok; ++kt) {
+        const int steps = nq - kt;
+        if (!mbar_wait(B(KV_FULL), done(kt), abort_flag, p.status, 45)) { ok = false; break; }
+        if (!mbar_wait(B(ACC_FREE), freed(kt), abort_flag, p.status, 46)) { ok = false; break; }
+        if (!issue_SdP(it)) { ok = false; break; }
+        for (int st = 0; st < steps; ++st, ++it) {
+          if (st + 1 < steps && !issue_SdP(it + 1)) { ok = false; break; }
+          if (!mbar_wait(B(P_READY), done(it), abort_flag, p.status, 47)) { ok = false; break; }
+          tc_fence_after();
+          const int s = it & 1;
+          mma_acc_128x64(tDV, base + OFF_PT, base + OFF_QD + s * 2 * TILE + TILE, st == 0);   // dV += P^T dO
+          mma_acc_128x64(tDK, base + OFF_DST, base + OFF_QD + s * 2 * TILE, st == 0);         // dK += dS^T Q
+          tc_commit(B(P_FREE));
+          tc_commit(B(QD_EMPTY + s));
+          if (st + 1 == steps) { tc_commit(B(ACC_FULL)); tc_commit(B(KV_EMPTY)); }
+        }
+      }
+    }
+  } else {
+    const int q4 = warp & 3;
+    const int c_lo = ((warp - 2) >> 2) * 64;     // this warp's 64 of the 128 score columns
+    const int r = q4 * 32 + lane;                // key row inside the tile = accumulator lane
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    const float scale_log2 = p.scale * LOG2E;
+    bool ok = true;
+    int it = 0;
+    for (int kt = 0; kt < nq; ++kt) {
+      for (int i = kt; i < nq && ok; ++i, ++it) {
+        const int s = it & 1;
+        const float* Ls = reinterpret_cast<const float*>(base_ptr + OFF_STAT + s * 1024);
+        const float* Ds = Ls + 128;
+        if (!mbar_wait(B(QD_FULL + s), done(it >> 1), abort_flag, p.status, 48)) { ok = false; break; }
+        if (!mbar_wait(B(S_FULL), done(it), abort_flag, p.status, 49)) { ok = false; break; }
+        if (!mbar_wait(B(P_FREE), freed(it), abort_flag, p.status, 50)) { ok = false; break; }
+        tc_fence_after();
+        const bool diag = (i == kt);
+        // on the diagonal tile only queries >= this key count: chunks wholly before the warp's rows are zero
+        const int c_first = diag ? q4 * 32 : 0;
+#pragma unroll 1
+        for (int c = c_lo; c < c_lo + 64; c += 32) {
+          uint32_t pk[16], dk[16];
+          if (c >= c_first) {
+            float sv[32], dv[32];
+            tc_ld32(tS + lane_off + (uint32_t)c, sv);
+            tc_ld32(tDP + lane_off + (uint32_t)c, dv);
+            tc_wait_ld();
+            const bool mask = diag && c == c_first;
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              float p0 = ex2(fmaf(sv[e], scale_log2, -Ls[c + e] * LOG2E));
+              float p1 = ex2(fmaf(sv[e + 1], scale_log2, -Ls[c + e + 1] * LOG2E));
+              if (mask) { if (c + e < r) p0 = 0.f; if (c + e + 1 < r) p1 = 0.f; }
+              const float d0 = p0 * (dv[e] - Ds[c + e]), d1 = p1 * (dv[e + 1] - Ds[c + e + 1]);
+              __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1), db = __floats2bfloat162_rn(d0, d1);
+              pk[e >> 1] = *reinterpret_cast<uint32_t*>(&pb);
+              dk[e >> 1] = *reinterpret_cast<uint32_t*>(&db);
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) { pk[e] = 0u; dk[e] = 0u; }
+          }
+          st_operand_chunk(base + OFF_PT, r, c, pk);
+          st_operand_chunk(base + OFF_DST, r, c, dk);
+        }
+        tc_fence_before();
+        mbar_arrive(B(S_FREE));
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(B(P_READY));
+      }
+      // dK (scaled) and dV of this key tile: tensor memory -> bf16 -> staged in the P^T buffer -> TMA stores
+      if (ok && !mbar_wait(B(ACC_FULL), done(kt), abort_flag, p.status, 51)) ok = false;
+      if (ok) {
+        tc_fence_after();
+        {
+          const int half = c_lo >> 6;                  // warps of the first half write dK, the others dV
+          const uint32_t tsrc = half == 0 ? tDK : tDV;
+          const float mul = half == 0 ? p.scale : 1.0f;
+#pragma unroll
+          for (int c = 0; c < DH; c += 32) {
+            float v[32];
+            tc_ld32(tsrc + lane_off + (uint32_t)c, v);
+            tc_wait_ld();
+#pragma unroll
+            for (uint32_t jj = 0; jj < 4; ++jj) {
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                __nv_bfloat162 ob = __floats2bfloat162_rn(v[8 * jj + 2 * e] * mul, v[8 * jj + 2 * e + 1] * mul);
+                w[e] = *reinterpret_cast<uint32_t*>(&ob);
+              }
+              st_row_chunk(base + OFF_PT + half * TILE, r, (uint32_t)(c >> 3) + jj, w);
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(B(ACC_FREE));
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (ok && warp == 2 && lane == 0) {
+        tma_store_2d(&mapDQKV, base + OFF_PT, p.d + h * DH, seq_row0 + kt * BT);
+        tma_store_2d(&mapDQKV, base + OFF_PT + TILE, 2 * p.d + h * DH, seq_row0 + kt * BT);
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+    }
+    if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+  T5_TEARDOWN()
+}
+
+// ==========================================================================================
+// dQ
+// ==========================================================================================
+namespace dq {
+enum { QO_FULL = 0, QO_EMPTY, KV_FULL /*+s*/, KV_FULL1, KV_EMPTY /*+s*/, KV_EMPTY1, S_FULL, S_FREE, P_READY, P_FREE,
+       ACC_FULL, ACC_FREE, N_BARS };
+constexpr int OFF_Q = 0, OFF_DO = TILE, OFF_KV = 2 * TILE /* stage s: K at +s*2*TILE, V after it */,
+              OFF_DS = 6 * TILE, OFF_BAR = 8 * TILE;
+constexpr int SMEM = OFF_BAR + 256 + 1024;
+}  // namespace dq
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
+                      const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
+  using namespace dq;
+  T5_SETUP(N_BARS, S_FREE, P_READY, ACC_FREE)
+  const int h = blockIdx.x, b = blockIdx.y;
+  const int nq = p.T / BT;
+  const int seq_row0 = b * p.T;
+  const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+  const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDQ = tmem_base + 256u;
+
+  // query tiles are walked from the last (most key tiles) to the first
+  if (warp == 0) {
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0;
+      for (int qi = 0; qi < nq && ok; ++qi) {
+        const int i = nq - 1 - qi;
+        if (!mbar_wait(B(QO_EMPTY), freed(qi), abort_flag, p.status, 61)) { ok = false; break; }
+        mbar_expect_tx(B(QO_FULL), 2 * TILE);
+        tma_load_2d(base + OFF_Q, &mapQKV, B(QO_FULL), h * DH, seq_row0 + i * BT);
+        tma_load_2d(base + OFF_DO, &mapDO, B(QO_FULL), h * DH, seq_row0 + i * BT);
+        for (int j = 0; j <= i; ++j, ++it) {
+          const int s = it & 1;
+          if (!mbar_wait(B(KV_EMPTY + s), freed(it >> 1), abort_flag, p.status, 62)) { ok = false; break; }
+          mbar_expect_tx(B(KV_FULL + s), 2 * TILE);
+          tma_load_2d(base + OFF_KV + s * 2 * TILE, &mapQKV, B(KV_FULL + s), p.d + h * DH, seq_row0 + j * BT);
+          tma_load_2d(base + OFF_KV + s * 2 * TILE + TILE, &mapQKV, B(KV_FULL + s), 2 * p.d + h * DH, seq_row0 + j * BT);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0;
+      auto issue_SdP = [&](int step) -> bool {
+        const int s = step & 1;
+        if (!mbar_wait(B(KV_FULL + s), done(step >> 1), abort_flag, p.status, 63)) return false;
+        if (!mbar_wait(B(S_FREE), freed(step), abort_flag, p.status, 64)) return false;
+        tc_fence_after();
+        mma_128x128(tS, base + OFF_Q, base + OFF_KV + s * 2 * TILE);                // S  = Q K^T
+        mma_128x128(tDP, base + OFF_DO, base + OFF_KV + s * 2 * TILE + TILE);       // dP = dO V^T
+        tc_commit(B(S_FULL));
+        return true;
+      };
+      for (int qi = 0; qi < nq && ok; ++qi) {
+        const int steps = nq - qi;               // key tiles 0 .. i, i = nq-1-qi
+        if (!mbar_wait(B(QO_FULL), done(qi), abort_flag, p.status, 65)) { ok = false; break; }
+        if (!mbar_wait(B(ACC_FREE), freed(qi), abort_flag, p.status, 66)) { ok = false; break; }
+        if (!issue_SdP(it)) { ok = false; break; }
+        for (int st = 0; st < steps; ++st, ++it) {
+          if (st + 1 < steps && !issue_SdP(it + 1)) { ok = false; break; }
+          if (!mbar_wait(B(P_READY), done(it), abort_flag, p.status, 67)) { ok = false; break; }
+          tc_fence_after();
+          const int s = it & 1;
+          mma_acc_128x64(tDQ, base + OFF_DS, base + OFF_KV + s * 2 * TILE, st == 0);     // dQ += dS K
+          tc_commit(B(P_FREE));
+          tc_commit(B(KV_EMPTY + s));
+          if (st + 1 == steps) { tc_commit(B(ACC_FULL)); tc_commit(B(QO_EMPTY)); }
+        }
+      }
+    }
+  } else {
+    const int q4 = warp & 3;
+    const int c_lo = ((warp - 2) >> 2) * 64;     // this warp's 64 of the 128 score columns
+    const int r = q4 * 32 + lane;                // query row inside the tile
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    const float scale_log2 = p.scale * LOG2E;
+    bool ok = true;
+    int it = 0;
+    for (int qi = 0; qi < nq; ++qi) {
+      const int i = nq - 1 - qi;
+      const float L2 = p.lse[stat0 + (size_t)i * BT + r] * LOG2E;
+      const float Dr = p.rowdot[stat0 + (size_t)i * BT + r];
+      for (int j = 0; j <= i && ok; ++j, ++it) {
+        if (!mbar_wait(B(S_FULL), done(it), abort_flag, p.status, 68)) { ok = false; break; }
+        if (!mbar_wait(B(P_FREE), freed(it), abort_flag, p.status, 69)) { ok = false; break; }
+        tc_fence_after();
+        const bool diag = (j == i);
+        // on the diagonal tile only keys <= this query count: chunks wholly after the warp's rows are zero
+        const int c_last = diag ? q4 * 32 : BT - 32;
+#pragma unroll 1
+        for (int c = c_lo; c < c_lo + 64; c += 32) {
+          uint32_t dk[16];
+          if (c <= c_last) {
+            float sv[32], dv[32];
+            tc_ld32(tS + lane_off + (uint32_t)c, sv);
+            tc_ld32(tDP + lane_off + (uint32_t)c, dv);
+            tc_wait_ld();
+            const bool mask = diag && c == c_last;
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              float p0 = ex2(fmaf(sv[e], scale_log2, -L2)), p1 = ex2(fmaf(sv[e + 1], scale_log2, -L2));
+              if (mask) { if (c + e > r) p0 = 0.f; if (c + e + 1 > r) p1 = 0.f; }
+              __nv_bfloat162 db = __floats2bfloat162_rn(p0 * (dv[e] - Dr), p1 * (dv[e + 1] - Dr));
+              dk[e >> 1] = *reinterpret_cast<uint32_t*>(&db);
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) dk[e] = 0u;
+          }
+          st_operand_chunk(base + OFF_DS, r, c, dk);
+        }
+        tc_fence_before();
+        mbar_arrive(B(S_FREE));
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(B(P_READY));
+      }
+      if (ok && !mbar_wait(B(ACC_FULL), done(qi), abort_flag, p.status, 70)) ok = false;
+      if (ok) {
+        tc_fence_after();
+        {
+          const int c = c_lo >> 1;                     // each of the two warps of a lane quarter takes 32 of the 64 columns
+          float v[32];
+          tc_ld32(tDQ + lane_off + (uint32_t)c, v);
+          tc_wait_ld();
+#pragma unroll
+          for (uint32_t jj = 0; jj < 4; ++jj) {
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              __nv_bfloat162 ob = __floats2bfloat162_rn(v[8 * jj + 2 * e] * p.scale, v[8 * jj + 2 * e + 1] * p.scale);
+              w[e] = *reinterpret_cast<uint32_t*>(&ob);
+            }
+            st_row_chunk(base + OFF_DS, r, (uint32_t)(c >> 3) + jj, w);
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(B(ACC_FREE));
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (ok && warp == 2 && lane == 0) {
+        tma_store_2d(&mapDQKV, base + OFF_DS, h * DH, seq_row0 + i * BT);
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+    }
+    if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+  T5_TEARDOWN()
+}
+
+// rowdot[b, h, i] = sum_c dO[i, c] O[i, c] over the head's 64 columns; 8 lanes per row
+__global__ void attn_rowdot_t5_kernel(const bf16* __restrict__ o, const bf16* __restrict__ d_o, int nseq, int T, int H,
+                                      int d, float* __restrict__ rowdot) {
+  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  int64_t rowhead = idx >> 3;
+  int part = (int)(idx & 7);
+  if (rowhead >= (int64_t)nseq * T * H) return;
+  int h = (int)(rowhead % H);
+  int64_t row = rowhead / H;
+  size_t off = (size_t)row * d + (size_t)h * DH + part * 8;
+  uint4 a = *reinterpret_cast<const uint4*>(o + off), bb = *reinterpret_cast<const uint4*>(d_o + off);
+  const bf16* ap = reinterpret_cast<const bf16*>(&a);
+  const bf16* bp = reinterpret_cast<const bf16*>(&bb);
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) s = fmaf(__bfloat162float(ap[i]), __bfloat162float(bp[i]), s);
+  s += __shfl_xor_sync(0xffffffffu, s, 1); s += __shfl_xor_sync(0xffffffffu, s, 2); s += __shfl_xor_sync(0xffffffffu, s, 4);
+  if (part == 0) {
+    int bq = (int)(row / T), i = (int)(row % T);
+    rowdot[((size_t)bq * H + h) * T + i] = s;
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+int* g_status = nullptr;
+__device__ int g_t5b_status[4];
+
+bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)BT};
+  cuuint32_t estr[2] = {1, 1};
+  return g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool init_once() {
+  if (g_encode) return true;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
+      q != cudaDriverEntryPointSuccess)
+    return false;
+  if (cudaGetSymbolAddress((void**)&g_status, g_t5b_status) != cudaSuccess) return false;
+  if (cudaMemset(g_status, 0, sizeof(int) * 4) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(attn_bwd_dkv_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dkv::SMEM) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(attn_bwd_dq_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dq::SMEM) != cudaSuccess) return false;
+  g_encode = (EncodeTiledFn)fn;
+  return true;
+}
+
+}  // namespace
+
+cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq, int T, int H,
+                             int d, void* dqkv, float* rowdot, int* status, cudaStream_t st) {
+  if (!attention_t5_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
+  if (!init_once()) return cudaErrorInitializationError;
+  CUtensorMap mQKV, mDO, mDQKV;
+  const uint64_t rows = (uint64_t)nseq * T;
+  if (!make_map(&mQKV, qkv, rows, (uint64_t)3 * d) || !make_map(&mDO, d_o, rows, (uint64_t)d) ||
+      !make_map(&mDQKV, dqkv, rows, (uint64_t)3 * d))
+    return cudaErrorInvalidValue;
+  int64_t threads = (int64_t)nseq * T * H * 8;
+  attn_rowdot_t5_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>((const bf16*)o, (const bf16*)d_o, nseq, T, H, d, rowdot);
+  BwdParams p;
+  p.T = T; p.H = H; p.d = d; p.scale = 1.0f / sqrtf((float)DH); p.lse = lse; p.rowdot = rowdot;
+  p.status = status ? status : g_status;
+  dim3 grid(H, nseq);
+  attn_bwd_dkv_t5_kernel<<<grid, NTHREADS, dkv::SMEM, st>>>(mQKV, mDO, mDQKV, p);
+  attn_bwd_dq_t5_kernel<<<grid, NTHREADS, dq::SMEM, st>>>(mQKV, mDO, mDQKV, p);
+  return cudaGetLastError();
+}
+
+}  // namespace sl

@@ -406,6 +406,8 @@ cudaError_t attention_fwd_tc(const void* qkv, int nseq, int T, int H, int d, voi
 cudaError_t attention_bwd_tc(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq, int T, int H,
                              int d, void* dqkv, float* rowdot, cudaStream_t st) {
   if (!attention_tc_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
+  if (attention_t5_supported(DT_BF16, T, H, d) && !prefer_mma_sync())
+    return attention_bwd_t5(qkv, o, lse, d_o, nseq, T, H, d, dqkv, rowdot, nullptr, st);
   static bool attr = false;
   if (!attr) {
     cudaError_t e = cudaFuncSetAttribute(attn_bwd_dq_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM);

@@ -77,6 +77,8 @@ cudaError_t attention_bwd_simt(int dt, const void* qkv, const void* o, const flo
 bool attention_t5_supported(int dt, int T, int H, int d);
 cudaError_t attention_fwd_t5(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, int* status,
                              cudaStream_t st);
+cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq, int T, int H,
+                             int d, void* dqkv, float* rowdot, int* status, cudaStream_t st);
 bool attention_tc_supported(int dt, int T, int H, int d);
 cudaError_t attention_fwd_tc(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, cudaStream_t st);
 cudaError_t attention_bwd_tc(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq,
