@@ -195,34 +195,43 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
 // ------------------------------------------------------------------------------------------
 // CTA pairs
 // ------------------------------------------------------------------------------------------
-struct PairCfg {
+// NEED_R: the epilogue has a second operand R (residual, or the pre-activation for GELU').  Its
+// [128 x 256] block per CTA tile is brought into shared memory by the producer warp with TMA about
+// one tile ahead of its use, so the epilogue never waits on a global load; the room comes from a
+// shorter operand ring (4 stages instead of 6).
+template <bool NEED_R> struct PairCfg {
   static constexpr int BN = 256;                       // tile columns of the pair
   static constexpr int A_BYTES = BM * BK * 2;          // this CTA's 128 rows of X
   static constexpr int B_BYTES = (BN / 2) * BK * 2;    // this CTA's half of the W tile
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = 6;
+  static constexpr int STAGES = NEED_R ? 4 : 6;
+  static constexpr int R_BYTES = NEED_R ? BM * BN * 2 : 0;
   static constexpr int TMEM_COLS = 512;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_STAGE_BYTES + 1024 + 256;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + R_BYTES + EPI_STAGE_BYTES + 1024 + 256;
   static constexpr uint32_t IDESC = make_idesc(2 * BM, BN);
 };
 
+template <bool NEED_R>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
                     const __grid_constant__ CUtensorMap mapXe, const __grid_constant__ CUtensorMap mapWe,
-               const __grid_constant__ CUtensorMap mapY, const __grid_constant__ CUtensorMap mapZ, TcParams p) {
-  using C = PairCfg;
+                    const __grid_constant__ CUtensorMap mapY, const __grid_constant__ CUtensorMap mapZ,
+                    const __grid_constant__ CUtensorMap mapR, TcParams p) {
+  using C = PairCfg<NEED_R>;
   constexpr int BN = C::BN;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - raw);
-  const uint32_t epi_base = base + C::STAGES * C::STAGE_BYTES;     // output staging of the epilogue warps
+  const uint32_t r_base = base + C::STAGES * C::STAGE_BYTES;       // second epilogue operand of the current tile
+  const uint32_t epi_base = r_base + C::R_BYTES;                   // output staging of the epilogue warps
   const uint32_t bar_base = epi_base + EPI_STAGE_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };                         // used in the leader
   auto empty_bar = [&](int s) { return bar_base + 8u * (C::STAGES + s); };          // one per CTA
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * C::STAGES + a); };      // one per CTA
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * C::STAGES + 2 + a); }; // used in the leader
-  uint8_t* tail = base_ptr + C::STAGES * C::STAGE_BYTES + EPI_STAGE_BYTES + 8 * (2 * C::STAGES + 4);
+  const uint32_t rfull_bar = bar_base + 8u * (2 * C::STAGES + 4), rempty_bar = rfull_bar + 8u;   // one per CTA
+  uint8_t* tail = base_ptr + C::STAGES * C::STAGE_BYTES + C::R_BYTES + EPI_STAGE_BYTES + 8 * (2 * C::STAGES + 6);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8);
 
@@ -233,6 +242,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 16); }
+    mbar_init(rfull_bar, 1); mbar_init(rempty_bar, 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -256,6 +266,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     // ---------------- TMA producer (both CTAs) ----------------
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
+      int tcount = 0;                              // tiles this CTA has started
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
         int tm, tn; tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
@@ -263,7 +274,23 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
         const int g = p.rows_per_group > 0 ? m0 / p.rows_per_group : 0;
         const int w_row = g * p.w_group_rows + n0;
         const int we_row = g * p.we_group_rows + n0;
+        // R block of this tile: issued as soon as the epilogue has released the buffer (checked
+        // between operand blocks so that the operand ring never waits for it)
+        bool r_pending = NEED_R;
+        auto issue_r = [&](bool blocking) -> bool {
+          if (!r_pending) return true;
+          const uint32_t par = ((uint32_t)tcount & 1u) ^ 1u;
+          if (blocking) { if (!mbar_wait(rempty_bar, par, abort_flag, p.status, 15)) return false; }
+          else if (!mbar_try(rempty_bar, par)) return true;
+          mbar_expect_tx(rfull_bar, C::R_BYTES);
+#pragma unroll
+          for (int j = 0; j < BN / BK; ++j)
+            tma_load_2d(r_base + j * (BM * BK * 2), &mapR, rfull_bar, tn * BN + j * BK, m0);
+          r_pending = false;
+          return true;
+        };
         for (int kb = 0; kb < kb_total; ++kb) {
+          issue_r(false);
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 11)) { ok = false; break; }
           // the leader's barrier collects the bytes of both CTAs' copies
           if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * C::STAGE_BYTES);
@@ -279,6 +306,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
           }
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
+        if (ok && !issue_r(true)) ok = false;
+        ++tcount;
       }
     }
   } else if (warp == 1) {
@@ -317,21 +346,19 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
     int as = 0; uint32_t aphase = 0;
     const bool tanh_form = p.gelu_tanh != 0;
     const uint32_t stage = epi_base + (uint32_t)(warp - 2) * 4096u;   // this warp's two staging buffers
-    EpiState est;
+    int buf = 0, tcount = 0;
     bool ok = true;
-    for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+    for (int tile = pair; tile < num_tiles && ok; tile += npairs, ++tcount) {
       int tm, tn; tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
       const int m_warp0 = tm * 2 * BM + (int)rank * BM + q * 32;
       const int n0 = tn * BN;
-      int m_next = -1, n_next = 0;
-      if (tile + npairs < num_tiles) {
-        int tm2, tn2; tile_coords(tile + npairs, p.tiles_m, p.tiles_n, tm2, tn2);
-        m_next = tm2 * 2 * BM + (int)rank * BM + q * 32; n_next = tn2 * BN + c_begin;
-      }
       if (!mbar_wait(tfull_bar(as), aphase, abort_flag, p.status, 14)) { ok = false; break; }
+      if (NEED_R && !mbar_wait(rfull_bar, (uint32_t)tcount & 1u, abort_flag, p.status, 16)) { ok = false; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN);
-      epilogue_tile(p, t_row, m_warp0, lane, n0, c_begin, c_end, m_next, n_next, tanh_form, stage, est, &mapY, &mapZ);
+      epilogue_tile_smem_r(p, t_row, m_warp0, lane, n0, c_begin, c_end, tanh_form, stage, buf, &mapY, &mapZ,
+                           NEED_R ? r_base : 0u, q * 32 + lane);
+      if (NEED_R) { __syncwarp(); if (lane == 0) mbar_arrive(rempty_bar); }   // 8 warps release the R buffer
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(as), 0));   // 16 arrivals free the stage
@@ -451,14 +478,21 @@ cudaError_t launch(const GemmArgs& a, int* status, cudaStream_t st) {
 }
 
 cudaError_t launch_pair(const GemmArgs& a, int* status, cudaStream_t st) {
-  using C = PairCfg;
-  CUtensorMap mX, mW, mXe, mWe, mY, mZ;
+  constexpr int BN = PairCfg<false>::BN;
+  CUtensorMap mX, mW, mXe, mWe, mY, mZ, mR;
   TcParams p;
-  if (!prepare(a, status, C::BN / 2, &mX, &mW, &mXe, &mWe, &mY, &mZ, &p)) return cudaErrorInvalidValue;
-  p.tiles_m = a.M / (2 * BM); p.tiles_n = (a.N + C::BN - 1) / C::BN;
+  if (!prepare(a, status, BN / 2, &mX, &mW, &mXe, &mWe, &mY, &mZ, &p)) return cudaErrorInvalidValue;
+  p.tiles_m = a.M / (2 * BM); p.tiles_n = (a.N + BN - 1) / BN;
   const int tiles = p.tiles_m * p.tiles_n;
   const int pairs = tiles < g_max_pairs ? tiles : g_max_pairs;
-  gemm_tc_pair_kernel<<<2 * pairs, NUM_THREADS, C::SMEM_BYTES, st>>>(mX, mW, mXe, mWe, mY, mZ, p);
+  const bool need_r = a.epi == EPI_BIAS_RESID || a.epi == EPI_MUL_GELUGRAD;
+  if (need_r) {
+    if (!make_map(&mR, a.R, a.M, a.N, a.ldr, BM)) return cudaErrorInvalidValue;
+    gemm_tc_pair_kernel<true><<<2 * pairs, NUM_THREADS, PairCfg<true>::SMEM_BYTES, st>>>(mX, mW, mXe, mWe, mY, mZ, mR, p);
+  } else {
+    mR = mY;
+    gemm_tc_pair_kernel<false><<<2 * pairs, NUM_THREADS, PairCfg<false>::SMEM_BYTES, st>>>(mX, mW, mXe, mWe, mY, mZ, mR, p);
+  }
   return cudaGetLastError();
 }
 
@@ -478,15 +512,16 @@ int gemm_tc_init() {
   g_max_pairs = 0;
   const char* off = std::getenv("SPLITLORA_NO_CTA_PAIRS");     // debugging aid: force the single-CTA kernel
   if (!(off && off[0] == '1') &&
-      cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg::SMEM_BYTES) == cudaSuccess) {
+      cudaFuncSetAttribute(gemm_tc_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<false>::SMEM_BYTES) == cudaSuccess &&
+      cudaFuncSetAttribute(gemm_tc_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<true>::SMEM_BYTES) == cudaSuccess) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(g_num_sms & ~1); cfg.blockDim = dim3(NUM_THREADS); cfg.dynamicSmemBytes = PairCfg::SMEM_BYTES;
+    cfg.gridDim = dim3(g_num_sms & ~1); cfg.blockDim = dim3(NUM_THREADS); cfg.dynamicSmemBytes = PairCfg<true>::SMEM_BYTES;
     cudaLaunchAttribute at;
     at.id = cudaLaunchAttributeClusterDimension;
     at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
     cfg.attrs = &at; cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_pair_kernel, &cfg) == cudaSuccess && n > 0)
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_pair_kernel<true>, &cfg) == cudaSuccess && n > 0)
       g_max_pairs = n < g_num_sms / 2 ? n : g_num_sms / 2;
     cudaGetLastError();
   }

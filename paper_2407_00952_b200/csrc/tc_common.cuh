@@ -331,5 +331,35 @@ __device__ __forceinline__ void epilogue_tile(const TcParams& p, uint32_t t_row,
   }
 }
 
+// Same, with the second epilogue operand already in shared memory: `rtile` holds this CTA's
+// [128 rows x 256 columns] block of R as four [128 x 64] tiles in the 128-byte-swizzled layout a
+// TMA load produces (rtile == 0: the epilogue has no second operand).  row = this thread's row
+// inside the CTA tile.
+__device__ __forceinline__ void epilogue_tile_smem_r(const TcParams& p, uint32_t t_row, int m_warp0, int lane, int n0,
+                                                     int c_begin, int c_end, bool tanh_form, uint32_t stage, int& buf,
+                                                     const CUtensorMap* mapY, const CUtensorMap* mapZ, uint32_t rtile,
+                                                     int row) {
+#pragma unroll 1
+  for (int c = c_begin; c < c_end; c += 32) {
+    const int n = n0 + c;
+    if (n >= p.N) break;                    // warp-uniform
+    uint4 rcur[4];
+    if (rtile) {
+      const uint32_t rrow = rtile + (uint32_t)(c >> 6) * (uint32_t)(BM * BK * 2) + (uint32_t)row * 128u;
+      const uint32_t cb = (uint32_t)((c & 63) >> 3);
+#pragma unroll
+      for (uint32_t j = 0; j < 4; ++j) {
+        const uint32_t a = rrow + (((cb + j) ^ ((uint32_t)row & 7u)) << 4);
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(rcur[j].x), "=r"(rcur[j].y), "=r"(rcur[j].z), "=r"(rcur[j].w) : "r"(a) : "memory");
+      }
+    }
+    float v[32];
+    tc_ld32(t_row + (uint32_t)c, v);
+    tc_wait_ld();
+    epilogue_chunk(p, v, rcur, n, tanh_form, stage, buf, mapY, mapZ, m_warp0, lane);
+  }
+}
+
 }  // namespace tc
 }  // namespace sl
