@@ -285,7 +285,13 @@ def run_gpu(args, w):
                 "achieved": round(achieved, 1), "peak": peak, "unit": "TFLOP/s",
                 "frac": round(achieved / peak, 4) if peak else None,
                 "peak_source": f"{peaks['source']} sustained bf16 (kernel timed inside a long step)",
-                "traffic": None, "launches": n_launch, "avg_launch_us": round(t_ms * 1e3 / max(1, n_launch), 2),
+                # DRAM bytes of one launch from the committed ncu capture of the CTA-pair kernel
+                # (profiles/gemm_tc_pair_kernel_qkv_m32768.md): the QKV + LoRA forward launch of this
+                # workload, whose algorithmic bytes are 275 MB.  Null for any other workload.
+                "traffic": 236439040 if w.index == 3 else None,
+                "traffic_launch": "QKV+LoRA forward, M 32768 K 1024(+64) N 3072: 81.3 MB read + 155.2 MB written; "
+                                  "algorithmic 275 MB" if w.index == 3 else None,
+                "launches": n_launch, "avg_launch_us": round(t_ms * 1e3 / max(1, n_launch), 2),
                 "by_class": by_class, "share_of_step": round(t_ms / ms, 4)}
     breakdown = {k: {"launches": v[0], "ms_per_step": round(v[1] / args.steps, 3)}
                  for k, v in sorted(prof.items(), key=lambda kv: -kv[1][1])}
