@@ -17,7 +17,11 @@ design notes):
     (paper Sec. II-C: W + dW with dW a product of two rank-r factors);
   * the model is a pre-LN GPT-style decoder; the fused attention projection
     'attn.qkv.w' is [3d, d] with the q, k, v slices stacked in that order and
-    adapters sit on the slices named in cfg.targets.
+    adapters sit on the slices named in cfg.targets;
+  * cfg.arch = "llama" selects a second block shape that the paper does not describe (it only
+    cites Llama-2 as an LLM): RMSNorm, rotary positions on q and k (pairs (j, j + dh/2)),
+    SwiGLU, no biases, no learned positions, a head separate from wte, and "o" (the attention
+    output projection) as a fourth possible adapter target.
 
 Parity status: every function below is pinned by tests/test_oracle_*.py
 (library routines + autograd in fp64, finite differences, closed forms,
@@ -66,6 +70,11 @@ class OracleConfig:
     agg_interval: int = 1         # I of Algorithm 1
     norm_eps: float = 1e-5
     gelu_tanh: bool = True
+    # "gpt": LayerNorm, learned positions, GELU MLP, biases, head tied to wte (the paper's GPT-2).
+    # "llama": RMSNorm, rotary positions on q and k, SwiGLU MLP, no biases, separate head.  The
+    # paper only cites Llama-2 as an LLM; this shape is defined by this file (see the notes).
+    arch: str = "gpt"
+    rope_theta: float = 10000.0
 
     @property
     def scale(self) -> float:
@@ -155,6 +164,51 @@ def gelu_grad(z, tanh_form=True):
     return 0.5 * (1.0 + erf(z / math.sqrt(2.0))) + z * np.exp(-0.5 * z * z) / math.sqrt(2.0 * math.pi)
 
 
+def rmsnorm_fwd(x, g, eps):
+    """Row-wise RMSNorm: x / sqrt(mean(x^2) + eps) * g  (no centring, no bias)."""
+    ms = (x * x).mean(axis=-1, keepdims=True)
+    rstd = 1.0 / np.sqrt(ms + eps)
+    xhat = x * rstd
+    return xhat * g, (xhat, rstd, g)
+
+
+def rmsnorm_bwd(dy, cache):
+    """Gradient of rmsnorm_fwd w.r.t. x only (the gain is frozen)."""
+    xhat, rstd, g = cache
+    dxhat = dy * g
+    m2 = (dxhat * xhat).mean(axis=-1, keepdims=True)
+    return (dxhat - xhat * m2) * rstd
+
+
+def rope_rotate(x, n_head, theta, sign=1.0):
+    """Rotary position embedding on x [nseq, T, d], heads split d contiguously.
+
+    Inside each head of width dh, element j < dh/2 is paired with element j + dh/2; at position t
+    the pair is rotated by the angle sign * t * theta^(-2j/dh).  sign=-1 is the inverse rotation,
+    which is also the gradient map (the rotation matrix is orthogonal).
+    """
+    nseq, T, d = x.shape
+    dh = d // n_head
+    half = dh // 2
+    j = np.arange(half, dtype=F64)
+    inv_freq = theta ** (-2.0 * j / dh)
+    ang = sign * np.arange(T, dtype=F64)[:, None] * inv_freq[None, :]       # [T, half]
+    cos, sin = np.cos(ang)[None, :, None, :], np.sin(ang)[None, :, None, :]
+    xh = x.reshape(nseq, T, n_head, dh)
+    lo, hi = xh[..., :half], xh[..., half:]
+    out = np.concatenate([lo * cos - hi * sin, hi * cos + lo * sin], axis=-1)
+    return out.reshape(nseq, T, d)
+
+
+def silu(z):
+    return z / (1.0 + np.exp(-z))
+
+
+def silu_grad(z):
+    sg = 1.0 / (1.0 + np.exp(-z))
+    return sg * (1.0 + z * (1.0 - sg))
+
+
 def causal_attention_fwd(q, k, v, n_head):
     """Multi-head causal softmax attention.  q, k, v [nseq, T, d]; heads split d contiguously.
 
@@ -233,6 +287,8 @@ def block_fwd(cfg: OracleConfig, params, l: int, adapters, x):
 
     adapters[(l, target)] = {"A": [r, d], "B": [d, r]} for each target in cfg.targets.
     """
+    if cfg.arch == "llama":
+        return llama_block_fwd(cfg, params, l, adapters, x)
     nseq, T, d = x.shape
     s = cfg.scale
     x2 = x.reshape(nseq * T, d)
@@ -261,6 +317,8 @@ def block_fwd(cfg: OracleConfig, params, l: int, adapters, x):
 
 def block_bwd(cfg: OracleConfig, params, l: int, adapters, dy, cache):
     """Back-propagate dy [nseq, T, d] through block l.  Returns dx and {(l, target): (dA, dB)}."""
+    if cfg.arch == "llama":
+        return llama_block_bwd(cfg, params, l, adapters, dy, cache)
     nseq, T, d = cache["shape"]
     s = cfg.scale
     dy2 = dy.reshape(nseq * T, d)
@@ -288,11 +346,89 @@ def block_bwd(cfg: OracleConfig, params, l: int, adapters, dy, cache):
 
 
 # --------------------------------------------------------------------------
+# the Llama-shaped block (not in the paper: RMSNorm, rotary q/k, SwiGLU, no biases; adapters on
+# any of q, k, v and the attention output projection o)
+# --------------------------------------------------------------------------
+def llama_block_fwd(cfg: OracleConfig, params, l: int, adapters, x):
+    nseq, T, d = x.shape
+    s = cfg.scale
+    x2 = x.reshape(nseq * T, d)
+    u, n1 = rmsnorm_fwd(x2, params[_pname(l, "ln1.g")], cfg.norm_eps)
+    qkv = u @ params[_pname(l, "attn.qkv.w")].T
+    for t in cfg.targets:
+        if t == "o":
+            continue
+        ad = adapters[(l, t)]
+        j = TARGET_SLICE[t]
+        qkv[:, j * d:(j + 1) * d] += s * ((u @ ad["A"].T) @ ad["B"].T)
+    q_pre = qkv[:, 0:d].reshape(nseq, T, d)
+    k_pre = qkv[:, d:2 * d].reshape(nseq, T, d)
+    v = qkv[:, 2 * d:3 * d].reshape(nseq, T, d)
+    q = rope_rotate(q_pre, cfg.n_head, cfg.rope_theta)
+    k = rope_rotate(k_pre, cfg.n_head, cfg.rope_theta)
+    o, probs = causal_attention_fwd(q, k, v, cfg.n_head)
+    o2 = o.reshape(nseq * T, d)
+    if "o" in cfg.targets:
+        ad = adapters[(l, "o")]
+        attn_out, _ = lora_linear_fwd(o2, params[_pname(l, "attn.proj.w")], None, ad["A"], ad["B"], s)
+    else:
+        attn_out = o2 @ params[_pname(l, "attn.proj.w")].T
+    x_mid = x2 + attn_out
+    u2, n2 = rmsnorm_fwd(x_mid, params[_pname(l, "ln2.g")], cfg.norm_eps)
+    zg = u2 @ params[_pname(l, "mlp.gate.w")].T
+    zu = u2 @ params[_pname(l, "mlp.up.w")].T
+    a = silu(zg) * zu
+    y = x_mid + a @ params[_pname(l, "mlp.down.w")].T
+    cache = dict(n1=n1, u=u, q=q, k=k, v=v, probs=probs, o2=o2, n2=n2, zg=zg, zu=zu, shape=(nseq, T, d))
+    return y.reshape(nseq, T, d), cache
+
+
+def llama_block_bwd(cfg: OracleConfig, params, l: int, adapters, dy, cache):
+    nseq, T, d = cache["shape"]
+    s = cfg.scale
+    dy2 = dy.reshape(nseq * T, d)
+    grads = {}
+    # MLP branch
+    da = dy2 @ params[_pname(l, "mlp.down.w")]
+    dzu = da * silu(cache["zg"])
+    dzg = da * cache["zu"] * silu_grad(cache["zg"])
+    du2 = dzg @ params[_pname(l, "mlp.gate.w")] + dzu @ params[_pname(l, "mlp.up.w")]
+    dx_mid = dy2 + rmsnorm_bwd(du2, cache["n2"])
+    # attention branch
+    if "o" in cfg.targets:
+        ad = adapters[(l, "o")]
+        do2, dA, dB = lora_linear_bwd(dx_mid, cache["o2"], params[_pname(l, "attn.proj.w")], ad["A"], ad["B"], s)
+        grads[(l, "o")] = (dA, dB)
+    else:
+        do2 = dx_mid @ params[_pname(l, "attn.proj.w")]
+    dq, dk, dv = causal_attention_bwd(do2.reshape(nseq, T, d), cache["q"], cache["k"], cache["v"],
+                                      cache["probs"], cfg.n_head)
+    dq = rope_rotate(dq, cfg.n_head, cfg.rope_theta, sign=-1.0)
+    dk = rope_rotate(dk, cfg.n_head, cfg.rope_theta, sign=-1.0)
+    dqkv = np.concatenate([dq.reshape(-1, d), dk.reshape(-1, d), dv.reshape(-1, d)], axis=1)
+    u = cache["u"]
+    du = dqkv @ params[_pname(l, "attn.qkv.w")]
+    for t in cfg.targets:
+        if t == "o":
+            continue
+        ad = adapters[(l, t)]
+        j = TARGET_SLICE[t]
+        dyt = dqkv[:, j * d:(j + 1) * d]
+        dh = s * (dyt @ ad["B"])
+        du = du + dh @ ad["A"]
+        grads[(l, t)] = (dh.T @ u, s * (dyt.T @ (u @ ad["A"].T)))
+    dx = dx_mid + rmsnorm_bwd(du, cache["n1"])
+    return dx.reshape(nseq, T, d), grads
+
+
+# --------------------------------------------------------------------------
 # the three split-fine-tuning calls (Algorithm 1, stage a)
 # --------------------------------------------------------------------------
 def embed(cfg: OracleConfig, params, tokens):
     """x0[b, t, :] = wte[tokens[b, t], :] + wpe[t, :]  (input side of the client sub-model)."""
     nseq, T = tokens.shape
+    if cfg.arch == "llama":        # positions enter through the rotation of q and k instead
+        return params["wte"][tokens].astype(F64)
     # stored values (fp32 or bf16-exact) are widened to fp64 before the first addition
     return params["wte"][tokens].astype(F64) + params["wpe"][:T][None, :, :].astype(F64)
 
@@ -331,12 +467,15 @@ def server_fwd_bwd(cfg: OracleConfig, params, server_adapters: dict, S, labels):
     for l in range(cfg.cut, cfg.n_layer):
         x, c = block_fwd(cfg, params, l, server_adapters, x)
         caches.append(c)
-    xf, lnf = layernorm_fwd(x.reshape(-1, d), params["lnf.g"], params["lnf.b"], cfg.norm_eps)
+    if cfg.arch == "llama":
+        xf, lnf = rmsnorm_fwd(x.reshape(-1, d), params["lnf.g"], cfg.norm_eps)
+    else:
+        xf, lnf = layernorm_fwd(x.reshape(-1, d), params["lnf.g"], params["lnf.b"], cfg.norm_eps)
     head = params.get("head.w", params["wte"])   # tied head unless a separate one is given
     z = xf @ head.T
     loss, dz = cross_entropy_fwd_bwd(z, labels.reshape(-1))
     dxf = dz @ head
-    dx = layernorm_bwd(dxf, lnf).reshape(K * b, T, d)
+    dx = (rmsnorm_bwd(dxf, lnf) if cfg.arch == "llama" else layernorm_bwd(dxf, lnf)).reshape(K * b, T, d)
     grads = {}
     for l in range(cfg.n_layer - 1, cfg.cut - 1, -1):
         dx, g = block_bwd(cfg, params, l, server_adapters, dx, caches[l - cfg.cut])

@@ -43,6 +43,9 @@ class Workload:
     counts: Optional[Tuple[int, ...]] = None   # fixed sample counts, else drawn in [200, 1000]
     rounds: int = 1
     agg_interval: int = 1
+    arch: str = "gpt"     # "gpt": LayerNorm / learned positions / GELU / biases / tied head;
+                          # "llama": RMSNorm / rotary q,k / SwiGLU / no biases / separate head
+    rope_theta: float = 10000.0
 
     @property
     def tokens_per_round(self) -> int:
@@ -56,6 +59,8 @@ WORKLOADS: Dict[int, Workload] = {
                 4, 8, 512, "bf16", 2e-4, True, None, 10),
     3: Workload(3, "gpt2-medium-shaped", 24, 6, 1024, 16, 4096, 50257, 512, 4, 32.0, ("q", "v"),
                 8, 8, 512, "bf16", 2e-4, True, None, 10),
+    5: Workload(5, "llama2-7b-shaped", 32, 4, 4096, 32, 11008, 32000, 1024, 16, 32.0, ("q", "k", "v", "o"),
+                4, 2, 1024, "bf16", 2e-4, True, None, 1, arch="llama"),
 }
 
 
@@ -75,6 +80,17 @@ def _to_bf16_values(a: np.ndarray) -> np.ndarray:
 def frozen_param_names(w: Workload) -> List[Tuple[str, Tuple[int, ...], str]]:
     """(name, shape, kind) of every frozen tensor, in the order that fixes the seeds."""
     d, F, V = w.d_model, w.d_ff, w.vocab
+    if w.arch == "llama":
+        out = [("wte", (V, d), "w"), ("head.w", (V, d), "w")]
+        for l in range(w.n_layer):
+            p = f"h.{l}."
+            out += [
+                (p + "ln1.g", (d,), "gain"), (p + "attn.qkv.w", (3 * d, d), "w"),
+                (p + "attn.proj.w", (d, d), "w"), (p + "ln2.g", (d,), "gain"),
+                (p + "mlp.gate.w", (F, d), "w"), (p + "mlp.up.w", (F, d), "w"),
+                (p + "mlp.down.w", (d, F), "w"),
+            ]
+        return out + [("lnf.g", (d,), "gain")]
     out = [("wte", (V, d), "w"), ("wpe", (w.max_seq, d), "w")]
     for l in range(w.n_layer):
         p = f"h.{l}."

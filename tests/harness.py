@@ -13,7 +13,7 @@ def oracle_config(w, optimizer="adamw", **kw):
              max_seq=w.max_seq, lora_r=w.lora_r, lora_alpha=w.lora_alpha, targets=w.targets,
              n_clients=w.n_clients, batch_per_client=w.batch_per_client, seq=w.seq,
              bf16_handoff=(w.dtype == "bf16"), optimizer=optimizer, lr_client=w.lr, lr_server=w.lr,
-             agg_interval=w.agg_interval)
+             agg_interval=w.agg_interval, arch=w.arch, rope_theta=w.rope_theta)
     d.update(kw)
     return O.OracleConfig(**d)
 
