@@ -53,6 +53,13 @@ extern "C" {
 #define SPLITLORA_TARGET_Q 1u         /* bits of lora_targets: which slices of the fused qkv        */
 #define SPLITLORA_TARGET_K 2u         /* projection carry an adapter                                */
 #define SPLITLORA_TARGET_V 4u
+#define SPLITLORA_TARGET_O 8u         /* the attention output projection                            */
+
+#define SPLITLORA_ARCH_GPT   0        /* LayerNorm, learned positions, GELU MLP, biases, head tied to
+                                         wte: the paper's GPT-2 (Sec. IV-A)                          */
+#define SPLITLORA_ARCH_LLAMA 1        /* RMSNorm, rotary positions on q and k (pairs j, j + dh/2),
+                                         SwiGLU MLP, no biases, separate head.  The paper cites
+                                         Llama-2 only as an LLM and does not describe this shape    */
 
 #define SPLITLORA_SIDE_CLIENT 0
 #define SPLITLORA_SIDE_SERVER 1
@@ -79,6 +86,8 @@ typedef struct {
   int32_t gelu_tanh;         /* 1: tanh form of GELU (GPT-2), 0: erf form                   */
   int32_t use_tensor_cores;  /* bf16 only: 1 = tcgen05 GEMMs + tensor-core attention (default),
                                 0 = plain FMA kernels (a second opinion for debugging)      */
+  int32_t arch;              /* SPLITLORA_ARCH_*                                            */
+  float   rope_theta;        /* base of the rotary frequencies (ARCH_LLAMA only), e.g. 1e4  */
 } splitlora_config;
 
 /* ---- context ------------------------------------------------------------------------------ */
@@ -100,7 +109,11 @@ int splitlora_bind_workspace(splitlora_ctx* ctx, void* dev, size_t bytes);
  *   "h.<l>.ln1.g" "h.<l>.ln1.b" [d]          "h.<l>.attn.qkv.w" [3d, d]  "h.<l>.attn.qkv.b" [3d]
  *   "h.<l>.attn.proj.w" [d, d] "h.<l>.attn.proj.b" [d]   "h.<l>.ln2.g" "h.<l>.ln2.b" [d]
  *   "h.<l>.mlp.fc1.w" [d_ff, d] "h.<l>.mlp.fc1.b" [d_ff] "h.<l>.mlp.fc2.w" [d, d_ff] "h.<l>.mlp.fc2.b" [d]
- * The LM head is tied to "wte".  Tensors are borrowed and never written.  `bytes` must equal the
+ * The LM head is tied to "wte".  With ARCH_LLAMA the set is instead
+ *   "wte" [vocab, d]   "head.w" [vocab, d]   "lnf.g" [d]
+ *   "h.<l>.ln1.g" [d]  "h.<l>.attn.qkv.w" [3d, d]  "h.<l>.attn.proj.w" [d, d]  "h.<l>.ln2.g" [d]
+ *   "h.<l>.mlp.gate_up.w" [2*d_ff, d] (rows 0..d_ff-1 gate, the rest up)  "h.<l>.mlp.down.w" [d, d_ff]
+ * Tensors are borrowed and never written.  `bytes` must equal the
  * size implied by the shape.  Requires a bound workspace (transposed copies for the backward
  * products are made at bind time, on the context stream). */
 int splitlora_bind_frozen(splitlora_ctx* ctx, const char* name, const void* dev, size_t bytes);

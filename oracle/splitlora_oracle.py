@@ -297,6 +297,8 @@ def block_fwd(cfg: OracleConfig, params, l: int, adapters, x):
     bqkv = params[_pname(l, "attn.qkv.b")]
     qkv = u @ Wqkv.T + bqkv
     for t in cfg.targets:
+        if t == "o":
+            continue
         ad = adapters[(l, t)]
         j = TARGET_SLICE[t]
         # the slice [j*d, (j+1)*d) of the fused projection is a LoRA layer of its own
@@ -306,12 +308,18 @@ def block_fwd(cfg: OracleConfig, params, l: int, adapters, x):
     v = qkv[:, 2 * d:3 * d].reshape(nseq, T, d)
     o, probs = causal_attention_fwd(q, k, v, cfg.n_head)
     o2 = o.reshape(nseq * T, d)
-    x_mid = x2 + o2 @ params[_pname(l, "attn.proj.w")].T + params[_pname(l, "attn.proj.b")]
+    if "o" in cfg.targets:     # the output projection as a LoRA layer
+        ad = adapters[(l, "o")]
+        proj, _ = lora_linear_fwd(o2, params[_pname(l, "attn.proj.w")], params[_pname(l, "attn.proj.b")],
+                                  ad["A"], ad["B"], s)
+        x_mid = x2 + proj
+    else:
+        x_mid = x2 + o2 @ params[_pname(l, "attn.proj.w")].T + params[_pname(l, "attn.proj.b")]
     u2, ln2 = layernorm_fwd(x_mid, params[_pname(l, "ln2.g")], params[_pname(l, "ln2.b")], cfg.norm_eps)
     z = u2 @ params[_pname(l, "mlp.fc1.w")].T + params[_pname(l, "mlp.fc1.b")]
     a = gelu_fwd(z, cfg.gelu_tanh)
     y = x_mid + a @ params[_pname(l, "mlp.fc2.w")].T + params[_pname(l, "mlp.fc2.b")]
-    cache = dict(ln1=ln1, u=u, q=q, k=k, v=v, probs=probs, ln2=ln2, z=z, shape=(nseq, T, d))
+    cache = dict(ln1=ln1, u=u, q=q, k=k, v=v, probs=probs, o2=o2, ln2=ln2, z=z, shape=(nseq, T, d))
     return y.reshape(nseq, T, d), cache
 
 
@@ -328,13 +336,21 @@ def block_bwd(cfg: OracleConfig, params, l: int, adapters, dy, cache):
     du2 = dz @ params[_pname(l, "mlp.fc1.w")]
     dx_mid = dy2 + layernorm_bwd(du2, cache["ln2"])
     # attention branch
-    do = (dx_mid @ params[_pname(l, "attn.proj.w")]).reshape(nseq, T, d)
+    grads = {}
+    if "o" in cfg.targets:
+        ad = adapters[(l, "o")]
+        do2, dAo, dBo = lora_linear_bwd(dx_mid, cache["o2"], params[_pname(l, "attn.proj.w")], ad["A"], ad["B"], s)
+        grads[(l, "o")] = (dAo, dBo)
+        do = do2.reshape(nseq, T, d)
+    else:
+        do = (dx_mid @ params[_pname(l, "attn.proj.w")]).reshape(nseq, T, d)
     dq, dk, dv = causal_attention_bwd(do, cache["q"], cache["k"], cache["v"], cache["probs"], cfg.n_head)
     dqkv = np.concatenate([dq.reshape(-1, d), dk.reshape(-1, d), dv.reshape(-1, d)], axis=1)
     u = cache["u"]
     du = dqkv @ params[_pname(l, "attn.qkv.w")]
-    grads = {}
     for t in cfg.targets:
+        if t == "o":
+            continue
         ad = adapters[(l, t)]
         j = TARGET_SLICE[t]
         dyt = dqkv[:, j * d:(j + 1) * d]

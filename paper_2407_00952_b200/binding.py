@@ -16,7 +16,9 @@ DTYPE_FP32, DTYPE_BF16 = 0, 1
 OPT_SGD, OPT_ADAMW = 0, 1
 TARGET_Q, TARGET_K, TARGET_V = 1, 2, 4
 SIDE_CLIENT, SIDE_SERVER = 0, 1
-TARGET_BITS = {"q": TARGET_Q, "k": TARGET_K, "v": TARGET_V}
+TARGET_O = 8
+ARCH_GPT, ARCH_LLAMA = 0, 1
+TARGET_BITS = {"q": TARGET_Q, "k": TARGET_K, "v": TARGET_V, "o": TARGET_O}
 
 EXPORTS = [
     "splitlora_create", "splitlora_destroy", "splitlora_workspace_bytes", "splitlora_bind_workspace",
@@ -48,6 +50,7 @@ class Config(C.Structure):
         ("lr_client", C.c_float), ("lr_server", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
         ("adam_eps", C.c_float), ("weight_decay", C.c_float), ("agg_interval", C.c_int32),
         ("norm_eps", C.c_float), ("gelu_tanh", C.c_int32), ("use_tensor_cores", C.c_int32),
+        ("arch", C.c_int32), ("rope_theta", C.c_float),
     ]
 
 
@@ -75,7 +78,9 @@ def config_from_workload(w, optimizer: str = "adamw", use_tensor_cores: bool = T
         batch_per_client=w.batch_per_client, seq=w.seq, dtype=DTYPE_BF16 if w.dtype == "bf16" else DTYPE_FP32,
         optimizer=OPT_ADAMW if optimizer == "adamw" else OPT_SGD, lr_client=w.lr, lr_server=w.lr, beta1=0.9,
         beta2=0.999, adam_eps=1e-8, weight_decay=0.01, agg_interval=w.agg_interval, norm_eps=1e-5, gelu_tanh=1,
-        use_tensor_cores=1 if use_tensor_cores else 0)
+        use_tensor_cores=1 if use_tensor_cores else 0,
+        arch=ARCH_LLAMA if getattr(w, "arch", "gpt") == "llama" else ARCH_GPT,
+        rope_theta=float(getattr(w, "rope_theta", 10000.0)))
     for k, v in over.items():
         setattr(cfg, k, v)
     return cfg

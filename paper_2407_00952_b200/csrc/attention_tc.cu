@@ -1,5 +1,5 @@
 // Causal multi-head attention on tensor cores (bf16 operands, fp32 softmax and accumulation),
-// head width 64, sequence length a multiple of 64.  Flash-style: scores are never written to
+// head width 64 or 128, sequence length a multiple of 64.  Flash-style: scores are never written to
 // memory; the forward keeps only the log-sum-exp per row, the backward recomputes probabilities.
 //   forward : one CTA per (sequence, head, 64-row query tile), 4 warps x 16 rows, K/V tiles double
 //             buffered in shared memory with cp.async, online softmax in registers.
@@ -14,19 +14,23 @@
 namespace sl {
 namespace {
 
-constexpr int DH = 64;
 constexpr int BT = 64;            // rows of a query tile and of a key tile
 constexpr int NT = 128;           // threads per CTA
-constexpr int TILE_BYTES = BT * DH * 2;
-constexpr int FWD_SMEM = 5 * TILE_BYTES, DQ_SMEM = 6 * TILE_BYTES, DKV_SMEM = 6 * TILE_BYTES + 4 * BT * 4;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
+template <int DH> struct Sizes {
+  static constexpr int TILE = BT * DH * 2;     // bytes of one [64][DH] bf16 tile
+  static constexpr int FWD = 5 * TILE, DQ = 6 * TILE, DKV = 6 * TILE + 4 * BT * 4;
+};
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-// byte offset of element (r, c) in a [64][64] bf16 tile whose 16-byte chunks are XOR-swizzled by row
-__device__ __forceinline__ uint32_t swz(int r, int c) {
-  return (uint32_t)(r * 128 + ((((c >> 3) ^ (r & 7)) << 4) | ((c & 7) << 1)));
+// byte offset of element (r, c) in a [64][DH] bf16 tile; the 16-byte chunks of every 128-byte
+// segment of a row are XOR-swizzled by the row index
+template <int DH> __device__ __forceinline__ uint32_t swz(int r, int c) {
+  int ch = c >> 3;
+  return (uint32_t)(r * (DH * 2) + ((((ch & ~7) | ((ch & 7) ^ (r & 7))) << 4) | ((c & 7) << 1)));
 }
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -35,12 +39,13 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
 __device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// 64 x 64 bf16 tile, global rows `ld` elements apart -> swizzled shared tile
-__device__ __forceinline__ void load_tile(uint32_t sbase, const bf16* g, int64_t ld) {
+// 64 x DH bf16 tile, global rows `ld` elements apart -> swizzled shared tile
+template <int DH> __device__ __forceinline__ void load_tile(uint32_t sbase, const bf16* g, int64_t ld) {
+  constexpr int CH = DH / 8;
 #pragma unroll
-  for (int i = threadIdx.x; i < BT * 8; i += NT) {
-    int r = i >> 3, ch = i & 7;
-    cp_async16(sbase + r * 128 + ((ch ^ (r & 7)) << 4), g + (size_t)r * ld + ch * 8);
+  for (int i = threadIdx.x; i < BT * CH; i += NT) {
+    int r = i / CH, ch = i % CH;
+    cp_async16(sbase + swz<DH>(r, ch * 8), g + (size_t)r * ld + ch * 8);
   }
 }
 
@@ -63,38 +68,40 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// A fragment (16 x 16) of a row-major [rows][64] tile at (row0, k0)
-__device__ __forceinline__ void load_a(uint32_t* a, uint32_t sbase, int row0, int k0) {
+// A fragment (16 x 16) of a row-major [rows][DH] tile at (row0, k0)
+template <int DH> __device__ __forceinline__ void load_a(uint32_t* a, uint32_t sbase, int row0, int k0) {
   int l = threadIdx.x & 31;
-  ldsm4(a, sbase + swz(row0 + (l & 7) + ((l >> 3) & 1) * 8, k0 + (l >> 4) * 8));
+  ldsm4(a, sbase + swz<DH>(row0 + (l & 7) + ((l >> 3) & 1) * 8, k0 + (l >> 4) * 8));
 }
 // B fragments for two n-tiles (n0, n0+8) x k16 from a tile stored [n][k]: b[0],b[1] -> n0 ; b[2],b[3] -> n0+8
-__device__ __forceinline__ void load_b_nk(uint32_t* b, uint32_t sbase, int n0, int k0) {
+template <int DH> __device__ __forceinline__ void load_b_nk(uint32_t* b, uint32_t sbase, int n0, int k0) {
   int l = threadIdx.x & 31;
-  ldsm4(b, sbase + swz(n0 + (l & 7) + (l >> 4) * 8, k0 + ((l >> 3) & 1) * 8));
+  ldsm4(b, sbase + swz<DH>(n0 + (l & 7) + (l >> 4) * 8, k0 + ((l >> 3) & 1) * 8));
 }
 // B fragments for two n-tiles (n0, n0+8) x k16 from a tile stored [k][n]
-__device__ __forceinline__ void load_b_kn(uint32_t* b, uint32_t sbase, int k0, int n0) {
+template <int DH> __device__ __forceinline__ void load_b_kn(uint32_t* b, uint32_t sbase, int k0, int n0) {
   int l = threadIdx.x & 31;
-  ldsm4t(b, sbase + swz(k0 + (l & 7) + ((l >> 3) & 1) * 8, n0 + (l >> 4) * 8));
+  ldsm4t(b, sbase + swz<DH>(k0 + (l & 7) + ((l >> 3) & 1) * 8, n0 + (l >> 4) * 8));
 }
 
-// acc[8][4] (16 x 64) += A(16 x 64 from `a_tile` rows row0..) * B^T where B tile is stored [n][k]
+// acc[8][4] (16 x 64) += A(16 x DH from `a_tile` rows row0..) * B^T where the B tile is stored [64][DH]
+template <int DH>
 __device__ __forceinline__ void mma_a_smem_b_nk(float (*acc)[4], uint32_t a_tile, int row0, uint32_t b_tile) {
 #pragma unroll
-  for (int ks = 0; ks < 4; ++ks) {
+  for (int ks = 0; ks < DH / 16; ++ks) {
     uint32_t a[4];
-    load_a(a, a_tile, row0, ks * 16);
+    load_a<DH>(a, a_tile, row0, ks * 16);
 #pragma unroll
     for (int np = 0; np < 4; ++np) {
       uint32_t b[4];
-      load_b_nk(b, b_tile, np * 16, ks * 16);
+      load_b_nk<DH>(b, b_tile, np * 16, ks * 16);
       mma16816(acc[2 * np], a, b[0], b[1]);
       mma16816(acc[2 * np + 1], a, b[2], b[3]);
     }
   }
 }
-// acc[8][4] (16 x 64) += P(16 x 64, fp32 accumulator layout, converted to bf16) * B where B tile is stored [k][n]
+// acc[DH/8][4] (16 x DH) += P(16 x 64, fp32 accumulator layout, converted to bf16) * B, B tile stored [64][DH]
+template <int DH>
 __device__ __forceinline__ void mma_p_regs_b_kn(float (*acc)[4], const float (*p)[4], uint32_t b_tile) {
 #pragma unroll
   for (int ks = 0; ks < 4; ++ks) {
@@ -104,18 +111,18 @@ __device__ __forceinline__ void mma_p_regs_b_kn(float (*acc)[4], const float (*p
     a[2] = pack2(p[2 * ks + 1][0], p[2 * ks + 1][1]);
     a[3] = pack2(p[2 * ks + 1][2], p[2 * ks + 1][3]);
 #pragma unroll
-    for (int np = 0; np < 4; ++np) {
+    for (int np = 0; np < DH / 16; ++np) {
       uint32_t b[4];
-      load_b_kn(b, b_tile, ks * 16, np * 16);
+      load_b_kn<DH>(b, b_tile, ks * 16, np * 16);
       mma16816(acc[2 * np], a, b[0], b[1]);
       mma16816(acc[2 * np + 1], a, b[2], b[3]);
     }
   }
 }
 
-__device__ __forceinline__ void zero_acc(float (*a)[4]) {
+template <int N> __device__ __forceinline__ void zero_acc(float (*a)[4]) {
 #pragma unroll
-  for (int i = 0; i < 8; ++i)
+  for (int i = 0; i < N; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) a[i][j] = 0.f;
 }
@@ -123,8 +130,10 @@ __device__ __forceinline__ void zero_acc(float (*a)[4]) {
 // ------------------------------------------------------------------------------------------
 // forward
 // ------------------------------------------------------------------------------------------
+template <int DH>
 __global__ void __launch_bounds__(NT) attn_fwd_tc_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ o,
                                                          float* __restrict__ lse, int T, int H, int d, float scale_log2) {
+  constexpr int TILE_BYTES = Sizes<DH>::TILE;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sQ = smem_u32(smem), sK0 = sQ + TILE_BYTES, sV0 = sQ + 3 * TILE_BYTES;
   const int qt = gridDim.x - 1 - blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -133,19 +142,19 @@ __global__ void __launch_bounds__(NT) attn_fwd_tc_kernel(const bf16* __restrict_
   const bf16* qbase = qkv + ((size_t)b * T + (size_t)qt * BT) * ld + (size_t)h * DH;
   const bf16* kbase = qkv + (size_t)b * T * ld + d + (size_t)h * DH;
   const bf16* vbase = kbase + d;
-  load_tile(sQ, qbase, ld);
-  load_tile(sK0, kbase, ld);
-  load_tile(sV0, vbase, ld);
+  load_tile<DH>(sQ, qbase, ld);
+  load_tile<DH>(sK0, kbase, ld);
+  load_tile<DH>(sV0, vbase, ld);
   cp_commit();
-  float oacc[8][4];
-  zero_acc(oacc);
+  float oacc[DH / 8][4];
+  zero_acc<DH / 8>(oacc);
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
   const int r0 = warp * 16 + g, r1 = r0 + 8;
   for (int j = 0; j <= qt; ++j) {
     const uint32_t sK = sK0 + (j & 1) * TILE_BYTES, sV = sV0 + (j & 1) * TILE_BYTES;
     if (j < qt) {
-      load_tile(sK0 + ((j + 1) & 1) * TILE_BYTES, kbase + (size_t)(j + 1) * BT * ld, ld);
-      load_tile(sV0 + ((j + 1) & 1) * TILE_BYTES, vbase + (size_t)(j + 1) * BT * ld, ld);
+      load_tile<DH>(sK0 + ((j + 1) & 1) * TILE_BYTES, kbase + (size_t)(j + 1) * BT * ld, ld);
+      load_tile<DH>(sV0 + ((j + 1) & 1) * TILE_BYTES, vbase + (size_t)(j + 1) * BT * ld, ld);
       cp_commit();
       cp_wait<1>();
     } else {
@@ -153,8 +162,8 @@ __global__ void __launch_bounds__(NT) attn_fwd_tc_kernel(const bf16* __restrict_
     }
     __syncthreads();
     float s[8][4];
-    zero_acc(s);
-    mma_a_smem_b_nk(s, sQ, warp * 16, sK);
+    zero_acc<8>(s);
+    mma_a_smem_b_nk<DH>(s, sQ, warp * 16, sK);
     float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
@@ -178,11 +187,12 @@ __global__ void __launch_bounds__(NT) attn_fwd_tc_kernel(const bf16* __restrict_
       s[n][0] = exp2f(s[n][0] - nm0); s[n][1] = exp2f(s[n][1] - nm0);
       s[n][2] = exp2f(s[n][2] - nm1); s[n][3] = exp2f(s[n][3] - nm1);
       ps0 += s[n][0] + s[n][1]; ps1 += s[n][2] + s[n][3];
-      oacc[n][0] *= c0; oacc[n][1] *= c0; oacc[n][2] *= c1; oacc[n][3] *= c1;
     }
+#pragma unroll
+    for (int n = 0; n < DH / 8; ++n) { oacc[n][0] *= c0; oacc[n][1] *= c0; oacc[n][2] *= c1; oacc[n][3] *= c1; }
     l0 = l0 * c0 + ps0; l1 = l1 * c1 + ps1;
     m0 = nm0; m1 = nm1;
-    mma_p_regs_b_kn(oacc, s, sV);
+    mma_p_regs_b_kn<DH>(oacc, s, sV);
     __syncthreads();
   }
   l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
@@ -191,7 +201,7 @@ __global__ void __launch_bounds__(NT) attn_fwd_tc_kernel(const bf16* __restrict_
   bf16* o0 = o + ((size_t)b * T + (size_t)qt * BT + r0) * d + (size_t)h * DH;
   bf16* o1 = o + ((size_t)b * T + (size_t)qt * BT + r1) * d + (size_t)h * DH;
 #pragma unroll
-  for (int n = 0; n < 8; ++n) {
+  for (int n = 0; n < DH / 8; ++n) {
     *reinterpret_cast<uint32_t*>(o0 + n * 8 + 2 * t) = pack2(oacc[n][0] * i0, oacc[n][1] * i0);
     *reinterpret_cast<uint32_t*>(o1 + n * 8 + 2 * t) = pack2(oacc[n][2] * i1, oacc[n][3] * i1);
   }
@@ -202,12 +212,14 @@ __global__ void __launch_bounds__(NT) attn_fwd_tc_kernel(const bf16* __restrict_
   }
 }
 
-// rowdot[b, h, i] = sum_c dO[i, c] O[i, c] over the head's 64 columns; 8 lanes per row
+// rowdot[b, h, i] = sum_c dO[i, c] O[i, c] over the head's DH columns; DH/8 lanes per row
+template <int DH>
 __global__ void attn_rowdot_tc_kernel(const bf16* __restrict__ o, const bf16* __restrict__ d_o, int nseq, int T, int H,
                                       int d, float* __restrict__ rowdot) {
+  constexpr int LPR = DH / 8;
   int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  int64_t rowhead = idx >> 3;
-  int part = (int)(idx & 7);
+  int64_t rowhead = idx / LPR;
+  int part = (int)(idx % LPR);
   if (rowhead >= (int64_t)nseq * T * H) return;
   int h = (int)(rowhead % H);
   int64_t row = rowhead / H;
@@ -218,7 +230,8 @@ __global__ void attn_rowdot_tc_kernel(const bf16* __restrict__ o, const bf16* __
   float s = 0.f;
 #pragma unroll
   for (int i = 0; i < 8; ++i) s = fmaf(__bfloat162float(ap[i]), __bfloat162float(bp[i]), s);
-  s += __shfl_xor_sync(0xffffffffu, s, 1); s += __shfl_xor_sync(0xffffffffu, s, 2); s += __shfl_xor_sync(0xffffffffu, s, 4);
+#pragma unroll
+  for (int m = 1; m < LPR; m <<= 1) s += __shfl_xor_sync(0xffffffffu, s, m);
   if (part == 0) {
     int bq = (int)(row / T), i = (int)(row % T);
     rowdot[((size_t)bq * H + h) * T + i] = s;
@@ -228,9 +241,11 @@ __global__ void attn_rowdot_tc_kernel(const bf16* __restrict__ o, const bf16* __
 // ------------------------------------------------------------------------------------------
 // backward, dQ: one CTA per query tile, loops over key tiles j <= qt
 // ------------------------------------------------------------------------------------------
+template <int DH>
 __global__ void __launch_bounds__(NT) attn_bwd_dq_tc_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ d_o,
                                                             const float* __restrict__ lse, const float* __restrict__ rowdot,
                                                             bf16* __restrict__ dqkv, int T, int H, int d, float scale) {
+  constexpr int TILE_BYTES = Sizes<DH>::TILE;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sQ = smem_u32(smem), sdO = sQ + TILE_BYTES, sK0 = sQ + 2 * TILE_BYTES, sV0 = sQ + 4 * TILE_BYTES;
   const int qt = gridDim.x - 1 - blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -240,23 +255,23 @@ __global__ void __launch_bounds__(NT) attn_bwd_dq_tc_kernel(const bf16* __restri
   const bf16* kbase = qkv + (size_t)b * T * ld + d + (size_t)h * DH;
   const bf16* vbase = kbase + d;
   const bf16* dobase = d_o + ((size_t)b * T + (size_t)qt * BT) * d + (size_t)h * DH;
-  load_tile(sQ, qbase, ld);
-  load_tile(sdO, dobase, d);
-  load_tile(sK0, kbase, ld);
-  load_tile(sV0, vbase, ld);
+  load_tile<DH>(sQ, qbase, ld);
+  load_tile<DH>(sdO, dobase, d);
+  load_tile<DH>(sK0, kbase, ld);
+  load_tile<DH>(sV0, vbase, ld);
   cp_commit();
   const int r0 = warp * 16 + g, r1 = r0 + 8;
   const size_t stat = ((size_t)b * H + h) * T + (size_t)qt * BT;
   const float L0 = lse[stat + r0] * LOG2E, L1 = lse[stat + r1] * LOG2E;
   const float D0 = rowdot[stat + r0], D1 = rowdot[stat + r1];
   const float scale_log2 = scale * LOG2E;
-  float dq[8][4];
-  zero_acc(dq);
+  float dq[DH / 8][4];
+  zero_acc<DH / 8>(dq);
   for (int j = 0; j <= qt; ++j) {
     const uint32_t sK = sK0 + (j & 1) * TILE_BYTES, sV = sV0 + (j & 1) * TILE_BYTES;
     if (j < qt) {
-      load_tile(sK0 + ((j + 1) & 1) * TILE_BYTES, kbase + (size_t)(j + 1) * BT * ld, ld);
-      load_tile(sV0 + ((j + 1) & 1) * TILE_BYTES, vbase + (size_t)(j + 1) * BT * ld, ld);
+      load_tile<DH>(sK0 + ((j + 1) & 1) * TILE_BYTES, kbase + (size_t)(j + 1) * BT * ld, ld);
+      load_tile<DH>(sV0 + ((j + 1) & 1) * TILE_BYTES, vbase + (size_t)(j + 1) * BT * ld, ld);
       cp_commit();
       cp_wait<1>();
     } else {
@@ -264,10 +279,10 @@ __global__ void __launch_bounds__(NT) attn_bwd_dq_tc_kernel(const bf16* __restri
     }
     __syncthreads();
     float s[8][4], dp[8][4];
-    zero_acc(s);
-    mma_a_smem_b_nk(s, sQ, warp * 16, sK);       // S = Q K^T
-    zero_acc(dp);
-    mma_a_smem_b_nk(dp, sdO, warp * 16, sV);     // dP = dO V^T
+    zero_acc<8>(s);
+    mma_a_smem_b_nk<DH>(s, sQ, warp * 16, sK);       // S = Q K^T
+    zero_acc<8>(dp);
+    mma_a_smem_b_nk<DH>(dp, sdO, warp * 16, sV);     // dP = dO V^T
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
 #pragma unroll
@@ -279,13 +294,13 @@ __global__ void __launch_bounds__(NT) attn_bwd_dq_tc_kernel(const bf16* __restri
         s[n][e] = p * (dp[n][e] - ((e < 2) ? D0 : D1));    // dS (without the 1/sqrt(dh) factor)
       }
     }
-    mma_p_regs_b_kn(dq, s, sK);                  // dQ += dS K
+    mma_p_regs_b_kn<DH>(dq, s, sK);                  // dQ += dS K
     __syncthreads();
   }
   bf16* q0 = dqkv + ((size_t)b * T + (size_t)qt * BT + r0) * ld + (size_t)h * DH;
   bf16* q1 = dqkv + ((size_t)b * T + (size_t)qt * BT + r1) * ld + (size_t)h * DH;
 #pragma unroll
-  for (int n = 0; n < 8; ++n) {
+  for (int n = 0; n < DH / 8; ++n) {
     *reinterpret_cast<uint32_t*>(q0 + n * 8 + 2 * t) = pack2(dq[n][0] * scale, dq[n][1] * scale);
     *reinterpret_cast<uint32_t*>(q1 + n * 8 + 2 * t) = pack2(dq[n][2] * scale, dq[n][3] * scale);
   }
@@ -296,9 +311,11 @@ __global__ void __launch_bounds__(NT) attn_bwd_dq_tc_kernel(const bf16* __restri
 // Works on the transposed score tile S^T = K Q^T so that P^T and dS^T land in the register layout
 // the next product needs as its left operand.
 // ------------------------------------------------------------------------------------------
+template <int DH>
 __global__ void __launch_bounds__(NT) attn_bwd_dkv_tc_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ d_o,
                                                              const float* __restrict__ lse, const float* __restrict__ rowdot,
                                                              bf16* __restrict__ dqkv, int T, int H, int d, float scale) {
+  constexpr int TILE_BYTES = Sizes<DH>::TILE;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sK = smem_u32(smem), sV = sK + TILE_BYTES, sQ0 = sK + 2 * TILE_BYTES, sdO0 = sK + 4 * TILE_BYTES;
   float* sL = reinterpret_cast<float*>(smem + 6 * TILE_BYTES);     // [2][64] lse * log2e
@@ -311,10 +328,10 @@ __global__ void __launch_bounds__(NT) attn_bwd_dkv_tc_kernel(const bf16* __restr
   const bf16* kbase = qhead + (size_t)kt * BT * ld + d;
   const bf16* dohead = d_o + (size_t)b * T * d + (size_t)h * DH;
   const size_t stat = ((size_t)b * H + h) * T;
-  load_tile(sK, kbase, ld);
-  load_tile(sV, kbase + d, ld);
-  load_tile(sQ0 + (kt & 1) * TILE_BYTES, qhead + (size_t)kt * BT * ld, ld);
-  load_tile(sdO0 + (kt & 1) * TILE_BYTES, dohead + (size_t)kt * BT * d, d);
+  load_tile<DH>(sK, kbase, ld);
+  load_tile<DH>(sV, kbase + d, ld);
+  load_tile<DH>(sQ0 + (kt & 1) * TILE_BYTES, qhead + (size_t)kt * BT * ld, ld);
+  load_tile<DH>(sdO0 + (kt & 1) * TILE_BYTES, dohead + (size_t)kt * BT * d, d);
   cp_commit();
   if (threadIdx.x < BT) {
     sL[(kt & 1) * BT + threadIdx.x] = lse[stat + (size_t)kt * BT + threadIdx.x] * LOG2E;
@@ -322,15 +339,15 @@ __global__ void __launch_bounds__(NT) attn_bwd_dkv_tc_kernel(const bf16* __restr
   }
   const float scale_log2 = scale * LOG2E;
   const int r0 = warp * 16 + g, r1 = r0 + 8;       // key rows of this thread inside the tile
-  float dk[8][4], dv[8][4];
-  zero_acc(dk); zero_acc(dv);
+  float dk[DH / 8][4], dv[DH / 8][4];
+  zero_acc<DH / 8>(dk); zero_acc<DH / 8>(dv);
   for (int i = kt; i < nT; ++i) {
     const uint32_t sQ = sQ0 + (i & 1) * TILE_BYTES, sdO = sdO0 + (i & 1) * TILE_BYTES;
     const float* Lq = sL + (i & 1) * BT;
     const float* Dq = sD + (i & 1) * BT;
     if (i + 1 < nT) {
-      load_tile(sQ0 + ((i + 1) & 1) * TILE_BYTES, qhead + (size_t)(i + 1) * BT * ld, ld);
-      load_tile(sdO0 + ((i + 1) & 1) * TILE_BYTES, dohead + (size_t)(i + 1) * BT * d, d);
+      load_tile<DH>(sQ0 + ((i + 1) & 1) * TILE_BYTES, qhead + (size_t)(i + 1) * BT * ld, ld);
+      load_tile<DH>(sdO0 + ((i + 1) & 1) * TILE_BYTES, dohead + (size_t)(i + 1) * BT * d, d);
       cp_commit();
       if (threadIdx.x < BT) {
         sL[((i + 1) & 1) * BT + threadIdx.x] = lse[stat + (size_t)(i + 1) * BT + threadIdx.x] * LOG2E;
@@ -342,10 +359,10 @@ __global__ void __launch_bounds__(NT) attn_bwd_dkv_tc_kernel(const bf16* __restr
     }
     __syncthreads();
     float st[8][4], dpt[8][4];
-    zero_acc(st);
-    mma_a_smem_b_nk(st, sK, warp * 16, sQ);       // S^T = K Q^T   (rows: keys, columns: queries)
-    zero_acc(dpt);
-    mma_a_smem_b_nk(dpt, sV, warp * 16, sdO);     // dP^T = V dO^T
+    zero_acc<8>(st);
+    mma_a_smem_b_nk<DH>(st, sK, warp * 16, sQ);       // S^T = K Q^T   (rows: keys, columns: queries)
+    zero_acc<8>(dpt);
+    mma_a_smem_b_nk<DH>(dpt, sV, warp * 16, sdO);     // dP^T = V dO^T
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
 #pragma unroll
@@ -358,14 +375,14 @@ __global__ void __launch_bounds__(NT) attn_bwd_dkv_tc_kernel(const bf16* __restr
         dpt[n][e] = p * (dpt[n][e] - Dq[qcol]);     // dS^T (without the 1/sqrt(dh) factor)
       }
     }
-    mma_p_regs_b_kn(dv, st, sdO);                 // dV += P^T dO
-    mma_p_regs_b_kn(dk, dpt, sQ);                 // dK += dS^T Q
+    mma_p_regs_b_kn<DH>(dv, st, sdO);                 // dV += P^T dO
+    mma_p_regs_b_kn<DH>(dk, dpt, sQ);                 // dK += dS^T Q
     __syncthreads();
   }
   bf16* k0 = dqkv + ((size_t)b * T + (size_t)kt * BT + r0) * ld + d + (size_t)h * DH;
   bf16* k1 = dqkv + ((size_t)b * T + (size_t)kt * BT + r1) * ld + d + (size_t)h * DH;
 #pragma unroll
-  for (int n = 0; n < 8; ++n) {
+  for (int n = 0; n < DH / 8; ++n) {
     *reinterpret_cast<uint32_t*>(k0 + n * 8 + 2 * t) = pack2(dk[n][0] * scale, dk[n][1] * scale);
     *reinterpret_cast<uint32_t*>(k1 + n * 8 + 2 * t) = pack2(dk[n][2] * scale, dk[n][3] * scale);
     *reinterpret_cast<uint32_t*>(k0 + d + n * 8 + 2 * t) = pack2(dv[n][0], dv[n][1]);
@@ -373,10 +390,44 @@ __global__ void __launch_bounds__(NT) attn_bwd_dkv_tc_kernel(const bf16* __restr
   }
 }
 
+template <int DH>
+cudaError_t launch_fwd(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, cudaStream_t st) {
+  static bool attr = false;
+  if (!attr) {
+    cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, Sizes<DH>::FWD);
+    if (e != cudaSuccess) return e;
+    attr = true;
+  }
+  dim3 grid(T / BT, H, nseq);
+  attn_fwd_tc_kernel<DH><<<grid, NT, Sizes<DH>::FWD, st>>>((const bf16*)qkv, (bf16*)o, lse, T, H, d,
+                                                          LOG2E / sqrtf((float)DH));
+  return cudaGetLastError();
+}
+
+template <int DH>
+cudaError_t launch_bwd(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq, int T, int H, int d,
+                       void* dqkv, float* rowdot, cudaStream_t st) {
+  static bool attr = false;
+  if (!attr) {
+    cudaError_t e = cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, Sizes<DH>::DQ);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_bwd_dkv_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, Sizes<DH>::DKV);
+    if (e != cudaSuccess) return e;
+    attr = true;
+  }
+  int64_t threads = (int64_t)nseq * T * H * (DH / 8);
+  attn_rowdot_tc_kernel<DH><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>((const bf16*)o, (const bf16*)d_o, nseq, T, H, d, rowdot);
+  dim3 grid(T / BT, H, nseq);
+  const float scale = 1.0f / sqrtf((float)DH);
+  attn_bwd_dq_tc_kernel<DH><<<grid, NT, Sizes<DH>::DQ, st>>>((const bf16*)qkv, (const bf16*)d_o, lse, rowdot, (bf16*)dqkv, T, H, d, scale);
+  attn_bwd_dkv_tc_kernel<DH><<<grid, NT, Sizes<DH>::DKV, st>>>((const bf16*)qkv, (const bf16*)d_o, lse, rowdot, (bf16*)dqkv, T, H, d, scale);
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 bool attention_tc_supported(int dt, int T, int H, int d) {
-  return dt == DT_BF16 && H > 0 && d % H == 0 && d / H == DH && T >= BT && T % BT == 0;
+  return dt == DT_BF16 && H > 0 && d % H == 0 && (d / H == 64 || d / H == 128) && T >= BT && T % BT == 0;
 }
 
 // SPLITLORA_ATTENTION_MMA_SYNC=1 keeps the mma.sync kernels even where the tcgen05 ones apply
@@ -391,16 +442,7 @@ cudaError_t attention_fwd_tc(const void* qkv, int nseq, int T, int H, int d, voi
   if (!attention_tc_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
   if (attention_t5_supported(DT_BF16, T, H, d) && !prefer_mma_sync())
     return attention_fwd_t5(qkv, nseq, T, H, d, o, lse, nullptr, st);
-  dim3 grid(T / BT, H, nseq);
-  const float scale_log2 = LOG2E / sqrtf((float)DH);
-  static bool attr = false;
-  if (!attr) {
-    cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM);
-    if (e != cudaSuccess) return e;
-    attr = true;
-  }
-  attn_fwd_tc_kernel<<<grid, NT, FWD_SMEM, st>>>((const bf16*)qkv, (bf16*)o, lse, T, H, d, scale_log2);
-  return cudaGetLastError();
+  return d / H == 64 ? launch_fwd<64>(qkv, nseq, T, H, d, o, lse, st) : launch_fwd<128>(qkv, nseq, T, H, d, o, lse, st);
 }
 
 cudaError_t attention_bwd_tc(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq, int T, int H,
@@ -408,21 +450,8 @@ cudaError_t attention_bwd_tc(const void* qkv, const void* o, const float* lse, c
   if (!attention_tc_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
   if (attention_t5_supported(DT_BF16, T, H, d) && !prefer_mma_sync())
     return attention_bwd_t5(qkv, o, lse, d_o, nseq, T, H, d, dqkv, rowdot, nullptr, st);
-  static bool attr = false;
-  if (!attr) {
-    cudaError_t e = cudaFuncSetAttribute(attn_bwd_dq_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_bwd_dkv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DKV_SMEM);
-    if (e != cudaSuccess) return e;
-    attr = true;
-  }
-  int64_t threads = (int64_t)nseq * T * H * 8;
-  attn_rowdot_tc_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>((const bf16*)o, (const bf16*)d_o, nseq, T, H, d, rowdot);
-  dim3 grid(T / BT, H, nseq);
-  const float scale = 1.0f / sqrtf((float)DH);
-  attn_bwd_dq_tc_kernel<<<grid, NT, DQ_SMEM, st>>>((const bf16*)qkv, (const bf16*)d_o, lse, rowdot, (bf16*)dqkv, T, H, d, scale);
-  attn_bwd_dkv_tc_kernel<<<grid, NT, DKV_SMEM, st>>>((const bf16*)qkv, (const bf16*)d_o, lse, rowdot, (bf16*)dqkv, T, H, d, scale);
-  return cudaGetLastError();
+  return d / H == 64 ? launch_bwd<64>(qkv, o, lse, d_o, nseq, T, H, d, dqkv, rowdot, st)
+                     : launch_bwd<128>(qkv, o, lse, d_o, nseq, T, H, d, dqkv, rowdot, st);
 }
 
 }  // namespace sl

@@ -23,6 +23,10 @@ __global__ void embed_kernel(const int32_t* __restrict__ tok, const T* __restric
   t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
   Vec16<T> a, b, o;
   a.load(wte + (size_t)t * d + c);
+  if (wpe == nullptr) {             // no learned positions (rotary models): plain gather
+    a.store(out + (size_t)m * d + c);
+    return;
+  }
   b.load(wpe + (size_t)(m % Tseq) * d + c);
 #pragma unroll
   for (int i = 0; i < N; ++i) o.set(i, a.get(i) + b.get(i));

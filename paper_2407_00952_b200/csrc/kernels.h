@@ -61,6 +61,21 @@ cudaError_t layernorm_fwd(int dt, const void* x, const void* g, const void* b, v
 cudaError_t layernorm_bwd(int dt, const void* dy, const void* x, const void* g, const float* mean,
                           const float* rstd, const void* resid, void* dx, int M, int d, cudaStream_t st);
 
+// Llama-shaped block pieces.  RMSNorm: y = x * rsqrt(mean(x^2) + eps) * g, saves rstd [M];
+// backward gives dx = resid + d/dx (resid may be null).
+cudaError_t rmsnorm_fwd(int dt, const void* x, const void* g, void* y, float* rstd, int M, int d, float eps,
+                        cudaStream_t st);
+cudaError_t rmsnorm_bwd(int dt, const void* dy, const void* x, const void* g, const float* rstd, const void* resid,
+                        void* dx, int M, int d, cudaStream_t st);
+// Rotates the q and k slices of qkv [M, 3d] in place; table [T, d/H/2] of (cos, sin) pairs as
+// float2; sign +1 forward, -1 inverse (= gradient).  Needs d/H/2 to be a multiple of the 16-byte
+// vector width.
+cudaError_t rope_inplace(int dt, void* qkv, const float* table, int M, int T, int H, int d, float sign,
+                         cudaStream_t st);
+// z [M, 2F] = (gate | up).  act [M, F] = silu(gate) * up;  dz [M, 2F] from dact [M, F].
+cudaError_t swiglu_fwd(int dt, const void* z, void* act, int M, int F, cudaStream_t st);
+cudaError_t swiglu_bwd(int dt, const void* dact, const void* z, void* dz, int M, int F, cudaStream_t st);
+
 // Cross-entropy over logits [M, ld] (V valid columns): writes per-row losses, then overwrites the
 // logits with d loss / d logits (zero in the pad columns) and reduces the mean loss.
 // normalizer_override > 0 replaces the count of valid labels (the batch is a shard of a larger one).

@@ -34,6 +34,8 @@ struct LayerBuf {
   const void* x_in = nullptr;
   // adapter compute copies of this layer (all groups stacked)
   void *Acat = nullptr, *AcatT = nullptr, *Bext = nullptr, *BextT = nullptr;
+  // the same for an adapter on the attention output projection, and its down-projected input
+  void *AcatO = nullptr, *AcatOT = nullptr, *BextO = nullptr, *BextOT = nullptr, *hcat_o = nullptr;
 };
 
 struct ProfRec { int cls; cudaEvent_t a, b; };
@@ -59,13 +61,20 @@ struct splitlora_ctx {
   int dt = 0; size_t es = 4;
   int M = 0, nseq = 0, d = 0, F = 0, V = 0, Vpad = 0, L = 0, cut = 0, K = 0, rows_per_client = 0;
   int r = 0, rp = 0, ext = 0, ke = 0, n_targets = 0;
+  int nq = 0;                 // adapted slices of the fused qkv projection (targets 0..nq-1)
+  bool has_o = false;         // adapter on the attention output projection (target index nq)
+  int ext_o = 0;
+  bool llama = false;
+  int Fz = 0;                 // width of the saved MLP pre-activation: d_ff, or 2*d_ff (gate | up)
   int slice_idx[4] = {0, 0, 0, 0};
   uint32_t target_bit[4] = {0, 0, 0, 0};
   float scale = 1.f;
   bool tc = false;
   // frozen
-  const void *wte = nullptr, *wpe = nullptr, *lnfg = nullptr, *lnfb = nullptr;
-  void* wteT = nullptr;
+  const void *wte = nullptr, *wpe = nullptr, *lnfg = nullptr, *lnfb = nullptr, *headw = nullptr;
+  void* wteT = nullptr;       // transposed head [d, Vpad]
+  float* rope_table = nullptr;
+  std::vector<float> rope_host;
   std::vector<FrozenLayer> fl;
   int n_bound = 0;
   // workspace
@@ -79,7 +88,7 @@ struct splitlora_ctx {
         *grad_scratch = nullptr;
   int *n_valid = nullptr, *status = nullptr;
   void *g_a = nullptr, *g_b = nullptr, *g_dz = nullptr, *g_du2 = nullptr, *g_dxmid = nullptr, *g_do = nullptr,
-       *g_dqkv = nullptr, *g_dhcat = nullptr, *g_du = nullptr;
+       *g_dqkv = nullptr, *g_dhcat = nullptr, *g_du = nullptr, *g_dhcat_o = nullptr;
   void *S = nullptr, *dS = nullptr;
   int32_t *tok_dev = nullptr, *lab_dev = nullptr;
   // state
@@ -123,7 +132,14 @@ int validate(const splitlora_config* c, std::string* why) {
   if (c->d_model / c->n_head > 128) return bad("head width above 128");
   if (c->vocab < 2 || c->max_seq < 1 || c->seq < 1 || c->seq > c->max_seq) return bad("bad vocab / seq");
   if (c->lora_r < 1 || c->lora_r > 64) return bad("lora_r must be in 1..64");
-  if ((c->lora_targets & 7u) == 0 || (c->lora_targets & ~7u)) return bad("lora_targets must name q, k and/or v");
+  if ((c->lora_targets & 7u) == 0 || (c->lora_targets & ~15u))
+    return bad("lora_targets must name at least one of q, k, v, and optionally o");
+  if (c->arch != SPLITLORA_ARCH_GPT && c->arch != SPLITLORA_ARCH_LLAMA) return bad("bad arch");
+  if (c->arch == SPLITLORA_ARCH_LLAMA) {
+    const int dh = c->d_model / c->n_head, vec = c->dtype == SPLITLORA_DTYPE_BF16 ? 8 : 4;
+    if (dh % 2 != 0 || (dh / 2) % vec != 0) return bad("half the head width must be a multiple of the 16-byte vector width");
+    if (!(c->rope_theta > 0.f)) return bad("rope_theta must be positive");
+  }
   if (c->n_clients < 1 || c->n_clients > AGG_MAX_CLIENTS) return bad("n_clients must be in 1..64");
   if (c->batch_per_client < 1) return bad("batch_per_client must be positive");
   if (((int64_t)c->batch_per_client * c->seq) % 256 != 0 && c->n_clients > 1)
@@ -148,8 +164,14 @@ void derive(splitlora_ctx* c) {
   c->n_targets = 0;
   for (int s = 0; s < 3; ++s)
     if (g.lora_targets & (1u << s)) { c->slice_idx[c->n_targets] = s; c->target_bit[c->n_targets] = 1u << s; c->n_targets++; }
-  c->ke = c->n_targets * c->rp;
+  c->nq = c->n_targets;
+  c->has_o = (g.lora_targets & SPLITLORA_TARGET_O) != 0;
+  if (c->has_o) { c->slice_idx[c->n_targets] = 0; c->target_bit[c->n_targets] = SPLITLORA_TARGET_O; c->n_targets++; }
+  c->ke = c->nq * c->rp;
   c->ext = (int)align_up((size_t)c->ke, EXT_BLOCK);
+  c->ext_o = c->has_o ? (int)align_up((size_t)c->rp, EXT_BLOCK) : 0;
+  c->llama = g.arch == SPLITLORA_ARCH_LLAMA;
+  c->Fz = c->llama ? 2 * g.d_ff : g.d_ff;
   c->scale = g.lora_alpha / (float)g.lora_r;
   c->per_layer = (int64_t)c->n_targets * 2 * c->r * c->d;
   c->Pc = c->per_layer * c->cut;
@@ -161,10 +183,11 @@ void derive(splitlora_ctx* c) {
 size_t plan(splitlora_ctx* c, char* ws) {
   Arena a(ws);
   const size_t es = c->es;
-  const size_t M = c->M, d = c->d, F = c->F, ext = c->ext;
+  const size_t M = c->M, d = c->d, F = c->F, ext = c->ext, Fz = c->Fz, ext_o = c->ext_o;
   c->status = (int*)a.take(256);
   c->loss_dev = (float*)a.take(256);
   c->n_valid = (int*)a.take(256);
+  if (c->llama) c->rope_table = (float*)a.take((size_t)c->cfg.seq * (d / c->cfg.n_head / 2) * 8);
   // adapters: masters, gradients, moments
   c->cp = (float*)a.take((size_t)c->K * c->Pc * 4); c->cg = (float*)a.take((size_t)c->K * c->Pc * 4);
   c->cm = (float*)a.take((size_t)c->K * c->Pc * 4); c->cv = (float*)a.take((size_t)c->K * c->Pc * 4);
@@ -175,13 +198,18 @@ size_t plan(splitlora_ctx* c, char* ws) {
   for (int l = 0; l < c->L; ++l) {
     FrozenLayer& f = c->fl[l];
     f.qkvwT = a.take(3 * d * d * es); f.projwT = a.take(d * d * es);
-    f.fc1wT = a.take(F * d * es); f.fc2wT = a.take(d * F * es);
+    f.fc1wT = a.take(Fz * d * es); f.fc2wT = a.take(d * F * es);
     LayerBuf& b = c->lb[l];
     const size_t G = l < c->cut ? c->K : 1;
     b.Acat = a.take(G * ext * d * es); b.AcatT = a.take(G * d * ext * es);
     b.Bext = a.take(G * 3 * d * ext * es); b.BextT = a.take(G * ext * 3 * d * es);
+    if (c->has_o) {
+      b.AcatO = a.take(G * ext_o * d * es); b.AcatOT = a.take(G * d * ext_o * es);
+      b.BextO = a.take(G * d * ext_o * es); b.BextOT = a.take(G * ext_o * d * es);
+      b.hcat_o = a.take(M * ext_o * es);
+    }
     b.u = a.take(M * d * es); b.hcat = a.take(M * ext * es); b.qkv = a.take(M * 3 * d * es);
-    b.o = a.take(M * d * es); b.x_mid = a.take(M * d * es); b.z = a.take(M * F * es);
+    b.o = a.take(M * d * es); b.x_mid = a.take(M * d * es); b.z = a.take(M * Fz * es);
     b.x_out = a.take(M * d * es);
     b.mean1 = (float*)a.take(M * 4); b.rstd1 = (float*)a.take(M * 4);
     b.mean2 = (float*)a.take(M * 4); b.rstd2 = (float*)a.take(M * 4);
@@ -192,8 +220,9 @@ size_t plan(splitlora_ctx* c, char* ws) {
   c->xf = a.take(M * d * es); c->logits = a.take(M * (size_t)c->Vpad * es);
   c->meanf = (float*)a.take(M * 4); c->rstdf = (float*)a.take(M * 4); c->row_loss = (float*)a.take(M * 4);
   c->rowdot = (float*)a.take((size_t)c->nseq * c->cfg.n_head * c->cfg.seq * 4);
-  c->grad_scratch = (float*)a.take(lora_grad_scratch_floats(c->M, c->n_targets * c->r, c->d) * 4);
-  c->g_a = a.take(M * d * es); c->g_b = a.take(M * d * es); c->g_dz = a.take(M * F * es);
+  c->grad_scratch = (float*)a.take(lora_grad_scratch_floats(c->M, c->nq * c->r, c->d) * 4);
+  if (c->has_o) c->g_dhcat_o = a.take(M * ext_o * es);
+  c->g_a = a.take(M * d * es); c->g_b = a.take(M * d * es); c->g_dz = a.take(M * Fz * es);
   c->g_du2 = a.take(M * d * es); c->g_dxmid = a.take(M * d * es); c->g_do = a.take(M * d * es);
   c->g_dqkv = a.take(M * 3 * d * es); c->g_dhcat = a.take(M * ext * es); c->g_du = a.take(M * d * es);
   c->S = a.take(M * d * es); c->dS = a.take(M * d * es);
@@ -242,28 +271,52 @@ GemmArgs base_args(splitlora_ctx* c, const void* X, int64_t ldx, const void* W, 
   return a;
 }
 
-bool all_frozen_bound(const splitlora_ctx* c) { return c->n_bound == 4 + 12 * c->L; }
+bool all_frozen_bound(const splitlora_ctx* c) { return c->n_bound == (c->llama ? 3 + 6 * c->L : 4 + 12 * c->L); }
 
 cudaError_t refresh_side(splitlora_ctx* c, bool client) {
   AdapterCopyArgs a;
   a.dtype = c->dt;
   a.a_gs = a.b_gs = client ? c->Pc : 0;
   a.a_ts = a.b_ts = (int64_t)2 * c->r * c->d;
-  a.n_targets = c->n_targets; a.r = c->r; a.rp = c->rp; a.d_in = c->d; a.d_out = c->d; a.n_out = 3 * c->d;
-  a.ext = c->ext;
-  for (int t = 0; t < 4; ++t) a.slice_off[t] = c->slice_idx[t] * c->d;
+  a.r = c->r; a.rp = c->rp; a.d_in = c->d; a.d_out = c->d;
   a.scale = c->scale;
   a.G = client ? c->K : 1;
   const int l0 = client ? 0 : c->cut, l1 = client ? c->cut : c->L;
   for (int l = l0; l < l1; ++l) {
-    a.A = (client ? c->cp : c->sp) + (size_t)(l - l0) * c->per_layer;
-    a.B = a.A + (size_t)c->r * c->d;
-    a.Acat = c->lb[l].Acat; a.AcatT = c->lb[l].AcatT; a.Bext = c->lb[l].Bext; a.BextT = c->lb[l].BextT;
-    Scope s(c, "adapter_copies", 1);
-    cudaError_t e = refresh_adapter_copies(a, c->st);
-    if (e != cudaSuccess) return e;
+    const float* base = (client ? c->cp : c->sp) + (size_t)(l - l0) * c->per_layer;
+    {  // the adapted slices of the fused qkv projection
+      a.A = base; a.B = a.A + (size_t)c->r * c->d;
+      a.n_targets = c->nq; a.n_out = 3 * c->d; a.ext = c->ext;
+      for (int t = 0; t < 4; ++t) a.slice_off[t] = c->slice_idx[t] * c->d;
+      a.Acat = c->lb[l].Acat; a.AcatT = c->lb[l].AcatT; a.Bext = c->lb[l].Bext; a.BextT = c->lb[l].BextT;
+      Scope s(c, "adapter_copies", 1);
+      cudaError_t e = refresh_adapter_copies(a, c->st);
+      if (e != cudaSuccess) return e;
+    }
+    if (c->has_o) {  // the output projection: a LoRA layer of its own
+      a.A = base + (size_t)c->nq * 2 * c->r * c->d; a.B = a.A + (size_t)c->r * c->d;
+      a.n_targets = 1; a.n_out = c->d; a.ext = c->ext_o;
+      for (int t = 0; t < 4; ++t) a.slice_off[t] = 0;
+      a.Acat = c->lb[l].AcatO; a.AcatT = c->lb[l].AcatOT; a.Bext = c->lb[l].BextO; a.BextT = c->lb[l].BextOT;
+      Scope s(c, "adapter_copies", 1);
+      cudaError_t e = refresh_adapter_copies(a, c->st);
+      if (e != cudaSuccess) return e;
+    }
   }
   return cudaSuccess;
+}
+
+// LayerNorm or RMSNorm, by architecture (mean is unused by RMSNorm)
+cudaError_t norm_forward(splitlora_ctx* c, const void* x, const void* g, const void* b, void* y, float* mean, float* rstd) {
+  Scope s(c, "layernorm_fwd", 1);
+  if (c->llama) return rmsnorm_fwd(c->dt, x, g, y, rstd, c->M, c->d, c->cfg.norm_eps, c->st);
+  return layernorm_fwd(c->dt, x, g, b, y, mean, rstd, c->M, c->d, c->cfg.norm_eps, c->st);
+}
+cudaError_t norm_backward(splitlora_ctx* c, const void* dy, const void* x, const void* g, const float* mean,
+                          const float* rstd, const void* resid, void* dx) {
+  Scope s(c, "layernorm_bwd", 1);
+  if (c->llama) return rmsnorm_bwd(c->dt, dy, x, g, rstd, resid, dx, c->M, c->d, c->st);
+  return layernorm_bwd(c->dt, dy, x, g, mean, rstd, resid, dx, c->M, c->d, c->st);
 }
 
 // ---- one block -----------------------------------------------------------------------------
@@ -276,8 +329,7 @@ cudaError_t block_forward(splitlora_ctx* c, int l, const void* x_in, void* x_out
   LayerBuf& b = c->lb[l];
   b.x_in = x_in;
   cudaError_t e;
-  { Scope s(c, "layernorm_fwd", 1);
-    if ((e = layernorm_fwd(c->dt, x_in, f.ln1g, f.ln1b, b.u, b.mean1, b.rstd1, M, d, c->cfg.norm_eps, c->st))) return e; }
+  if ((e = norm_forward(c, x_in, f.ln1g, f.ln1b, b.u, b.mean1, b.rstd1))) return e;
   {  // h = u A_g^T for every target of the layer, one padded block of `ext` columns
     GemmArgs a = base_args(c, b.u, d, b.Acat, d, b.hcat, ext, M, ext, d);
     a.rows_per_group = rpg; a.w_grouped = grouped;
@@ -289,20 +341,39 @@ cudaError_t block_forward(splitlora_ctx* c, int l, const void* x_in, void* x_out
     a.Xe = b.hcat; a.ldxe = ext; a.We = b.Bext; a.ldwe = ext; a.Ke = c->ke; a.we_grouped = grouped;
     if ((e = linear(c, "lora_linear_fwd", a))) return e;
   }
+  if (c->llama) {
+    Scope s(c, "rope", 1);
+    if ((e = rope_inplace(c->dt, b.qkv, c->rope_table, M, c->cfg.seq, c->cfg.n_head, d, 1.0f, c->st))) return e;
+  }
   { Scope s(c, "attention_fwd", 1);
     if (c->tc && attention_tc_supported(c->dt, c->cfg.seq, c->cfg.n_head, d))
       e = attention_fwd_tc(b.qkv, c->nseq, c->cfg.seq, c->cfg.n_head, d, b.o, b.lse, c->st);
     else
       e = attention_fwd_simt(c->dt, b.qkv, c->nseq, c->cfg.seq, c->cfg.n_head, d, b.o, b.lse, c->st);
     if (e) return e; }
+  if (c->has_o) {  // h_o = o A_o,g^T
+    GemmArgs a = base_args(c, b.o, d, b.AcatO, d, b.hcat_o, c->ext_o, M, c->ext_o, d);
+    a.rows_per_group = rpg; a.w_grouped = grouped;
+    if ((e = linear(c, "lora_down_fwd", a))) return e;
+  }
   { GemmArgs a = base_args(c, b.o, d, f.projw, d, b.x_mid, d, M, d, d);
     a.bias = f.projb; a.epi = EPI_BIAS_RESID; a.R = x_in; a.ldr = d;
-    if ((e = linear(c, "linear_fwd", a))) return e; }
-  { Scope s(c, "layernorm_fwd", 1);
-    if ((e = layernorm_fwd(c->dt, b.x_mid, f.ln2g, f.ln2b, c->u2, b.mean2, b.rstd2, M, d, c->cfg.norm_eps, c->st))) return e; }
-  { GemmArgs a = base_args(c, c->u2, d, f.fc1w, d, c->act, F, M, F, d);
+    if (c->has_o) {
+      a.rows_per_group = rpg;
+      a.Xe = b.hcat_o; a.ldxe = c->ext_o; a.We = b.BextO; a.ldwe = c->ext_o; a.Ke = c->rp; a.we_grouped = grouped;
+    }
+    if ((e = linear(c, c->has_o ? "lora_linear_fwd" : "linear_fwd", a))) return e; }
+  if ((e = norm_forward(c, b.x_mid, f.ln2g, f.ln2b, c->u2, b.mean2, b.rstd2))) return e;
+  if (c->llama) {
+    { GemmArgs a = base_args(c, c->u2, d, f.fc1w, d, b.z, 2 * F, M, 2 * F, d);     // (gate | up)
+      if ((e = linear(c, "linear_fwd", a))) return e; }
+    { Scope s(c, "swiglu_fwd", 1);
+      if ((e = swiglu_fwd(c->dt, b.z, c->act, M, F, c->st))) return e; }
+  } else {
+    GemmArgs a = base_args(c, c->u2, d, f.fc1w, d, c->act, F, M, F, d);
     a.bias = f.fc1b; a.epi = EPI_BIAS_GELU; a.Z = b.z; a.ldz = F;
-    if ((e = linear(c, "linear_fwd", a))) return e; }
+    if ((e = linear(c, "linear_fwd", a))) return e;
+  }
   { GemmArgs a = base_args(c, c->act, F, f.fc2w, F, x_out, d, M, d, F);
     a.bias = f.fc2b; a.epi = EPI_BIAS_RESID; a.R = b.x_mid; a.ldr = d;
     if ((e = linear(c, "linear_fwd", a))) return e; }
@@ -319,33 +390,61 @@ cudaError_t block_backward(splitlora_ctx* c, int l, const void* dy, void* dx) {
   const FrozenLayer& f = c->fl[l];
   LayerBuf& b = c->lb[l];
   cudaError_t e;
-  { GemmArgs a = base_args(c, dy, d, f.fc2wT, d, c->g_dz, F, M, F, d);
+  const int Fz = c->Fz;
+  float* gbase = client ? c->cg + (size_t)l * c->per_layer : c->sg + (size_t)(l - c->cut) * c->per_layer;
+  const int64_t gstride = client ? c->Pc : 0;
+  if (c->llama) {
+    { GemmArgs a = base_args(c, dy, d, f.fc2wT, d, c->act, F, M, F, d);               // d act
+      if ((e = linear(c, "linear_bwd", a))) return e; }
+    { Scope s(c, "swiglu_bwd", 1);
+      if ((e = swiglu_bwd(c->dt, c->act, b.z, c->g_dz, M, F, c->st))) return e; }
+  } else {
+    GemmArgs a = base_args(c, dy, d, f.fc2wT, d, c->g_dz, F, M, F, d);
     a.epi = EPI_MUL_GELUGRAD; a.R = b.z; a.ldr = F;
+    if ((e = linear(c, "linear_bwd", a))) return e;
+  }
+  { GemmArgs a = base_args(c, c->g_dz, Fz, f.fc1wT, Fz, c->g_du2, d, M, d, Fz);
     if ((e = linear(c, "linear_bwd", a))) return e; }
-  { GemmArgs a = base_args(c, c->g_dz, F, f.fc1wT, F, c->g_du2, d, M, d, F);
-    if ((e = linear(c, "linear_bwd", a))) return e; }
-  { Scope s(c, "layernorm_bwd", 1);
-    if ((e = layernorm_bwd(c->dt, c->g_du2, b.x_mid, f.ln2g, b.mean2, b.rstd2, dy, c->g_dxmid, M, d, c->st))) return e; }
+  if ((e = norm_backward(c, c->g_du2, b.x_mid, f.ln2g, b.mean2, b.rstd2, dy, c->g_dxmid))) return e;
+  if (c->has_o) {
+    // dh_o = (alpha/r) dx_mid B_o,g ;  G_A = dh_o^T o ;  G_B = (alpha/r) dx_mid^T h_o   (Eq. 4-7)
+    { GemmArgs a = base_args(c, c->g_dxmid, d, b.BextOT, d, c->g_dhcat_o, c->ext_o, M, c->ext_o, d);
+      a.rows_per_group = rpg; a.w_grouped = grouped;
+      if ((e = linear(c, "lora_down_bwd", a))) return e; }
+    float* gA = gbase + (size_t)c->nq * 2 * c->r * d;
+    { Scope s(c, "lora_grad", 2);
+      if ((e = lora_grad(c->dt, b.o, d, 0, d, c->g_dhcat_o, c->ext_o, 0, c->r, c->rp, 1, M, rpg, 1.0f, gA, gstride, 0, d,
+                         1, c->grad_scratch, c->st))) return e; }
+    { Scope s(c, "lora_grad", 2);
+      if ((e = lora_grad(c->dt, c->g_dxmid, d, 0, d, b.hcat_o, c->ext_o, 0, c->r, c->rp, 1, M, rpg, c->scale,
+                         gA + (size_t)c->r * d, gstride, 0, 1, c->r, c->grad_scratch, c->st))) return e; }
+  }
   { GemmArgs a = base_args(c, c->g_dxmid, d, f.projwT, d, c->g_do, d, M, d, d);
-    if ((e = linear(c, "linear_bwd", a))) return e; }
+    if (c->has_o) {
+      a.rows_per_group = rpg;
+      a.Xe = c->g_dhcat_o; a.ldxe = c->ext_o; a.We = b.AcatOT; a.ldwe = c->ext_o; a.Ke = c->rp; a.we_grouped = grouped;
+    }
+    if ((e = linear(c, c->has_o ? "lora_linear_bwd" : "linear_bwd", a))) return e; }
   { Scope s(c, "attention_bwd", 3);
     if (c->tc && attention_tc_supported(c->dt, c->cfg.seq, c->cfg.n_head, d))
       e = attention_bwd_tc(b.qkv, b.o, b.lse, c->g_do, c->nseq, c->cfg.seq, c->cfg.n_head, d, c->g_dqkv, c->rowdot, c->st);
     else
       e = attention_bwd_simt(c->dt, b.qkv, b.o, b.lse, c->g_do, c->nseq, c->cfg.seq, c->cfg.n_head, d, c->g_dqkv, c->rowdot, c->st);
     if (e) return e; }
+  if (c->llama) {  // the gradient of a rotation is the inverse rotation
+    Scope s(c, "rope", 1);
+    if ((e = rope_inplace(c->dt, c->g_dqkv, c->rope_table, M, c->cfg.seq, c->cfg.n_head, d, -1.0f, c->st))) return e;
+  }
   {  // dh = (alpha/r) dqkv B_g for every target (the scale lives in the compute copy)
     GemmArgs a = base_args(c, c->g_dqkv, 3 * d, b.BextT, 3 * d, c->g_dhcat, ext, M, ext, 3 * d);
     a.rows_per_group = rpg; a.w_grouped = grouped;
     if ((e = linear(c, "lora_down_bwd", a))) return e;
   }
   // G_A = dh^T u, G_B = (alpha/r) dy^T h, per group (Eq. 4-7)
-  float* gbase = client ? c->cg + (size_t)l * c->per_layer : c->sg + (size_t)(l - c->cut) * c->per_layer;
-  const int64_t gstride = client ? c->Pc : 0;
-  { Scope s(c, "lora_grad", 2);   // every target's G_A in one pass over u
-    if ((e = lora_grad(c->dt, b.u, d, 0, d, c->g_dhcat, ext, 0, c->r, c->rp, c->n_targets, M, rpg, 1.0f, gbase,
+  { Scope s(c, "lora_grad", 2);   // every qkv target's G_A in one pass over u
+    if ((e = lora_grad(c->dt, b.u, d, 0, d, c->g_dhcat, ext, 0, c->r, c->rp, c->nq, M, rpg, 1.0f, gbase,
                        gstride, (int64_t)2 * c->r * d, d, 1, c->grad_scratch, c->st))) return e; }
-  for (int t = 0; t < c->n_targets; ++t) {
+  for (int t = 0; t < c->nq; ++t) {
     float* gB = gbase + (size_t)t * 2 * c->r * d + (size_t)c->r * d;
     Scope s(c, "lora_grad", 2);
     if ((e = lora_grad(c->dt, c->g_dqkv, 3 * d, c->slice_idx[t] * d, d, b.hcat, ext, t * c->rp, c->r, c->rp, 1, M,
@@ -356,8 +455,7 @@ cudaError_t block_backward(splitlora_ctx* c, int l, const void* dy, void* dx) {
     a.rows_per_group = rpg;
     a.Xe = c->g_dhcat; a.ldxe = ext; a.We = b.AcatT; a.ldwe = ext; a.Ke = c->ke; a.we_grouped = grouped;
     if ((e = linear(c, "lora_linear_bwd", a))) return e;
-    Scope s(c, "layernorm_bwd", 1);
-    if ((e = layernorm_bwd(c->dt, c->g_du, b.x_in, f.ln1g, b.mean1, b.rstd1, c->g_dxmid, dx, M, d, c->st))) return e;
+    if ((e = norm_backward(c, c->g_du, b.x_in, f.ln1g, b.mean1, b.rstd1, c->g_dxmid, dx))) return e;
   }
   return cudaSuccess;
 }
@@ -464,6 +562,20 @@ int splitlora_bind_workspace(splitlora_ctx* c, void* dev, size_t bytes) {
     CK(c, cudaMemsetAsync(c->lb[l].AcatT, 0, G * ext * d * es, c->st));
     CK(c, cudaMemsetAsync(c->lb[l].Bext, 0, G * 3 * d * ext * es, c->st));
     CK(c, cudaMemsetAsync(c->lb[l].BextT, 0, G * 3 * d * ext * es, c->st));
+    if (c->has_o)
+      for (void* p : {c->lb[l].AcatO, c->lb[l].AcatOT, c->lb[l].BextO, c->lb[l].BextOT})
+        CK(c, cudaMemsetAsync(p, 0, G * (size_t)c->ext_o * d * es, c->st));
+  }
+  if (c->llama) {  // (cos, sin) of t * theta^(-2j/dh), evaluated in double
+    const int half = c->d / c->cfg.n_head / 2, T = c->cfg.seq;
+    c->rope_host.resize((size_t)T * half * 2);
+    for (int t = 0; t < T; ++t)
+      for (int j = 0; j < half; ++j) {
+        const double ang = (double)t * std::pow((double)c->cfg.rope_theta, -2.0 * j / (2.0 * half));
+        c->rope_host[((size_t)t * half + j) * 2] = (float)std::cos(ang);
+        c->rope_host[((size_t)t * half + j) * 2 + 1] = (float)std::sin(ang);
+      }
+    CK(c, cudaMemcpyAsync(c->rope_table, c->rope_host.data(), c->rope_host.size() * 4, cudaMemcpyHostToDevice, c->st));
   }
   CK(c, cudaMemsetAsync(c->wteT, 0, (size_t)c->d * c->Vpad * c->es, c->st));
   c->client_copies_dirty = c->server_copies_dirty = true;
@@ -481,30 +593,39 @@ int splitlora_bind_frozen(splitlora_ctx* c, const char* name, const void* dev, s
   auto bad_size = [&]() { return fail(c, SPLITLORA_ERR_ARG, std::string("wrong byte size for ") + name); };
   auto set = [&](const void** slot) { if (!*slot) c->n_bound++; *slot = dev; };
   std::string n(name);
-  if (n == "wte") {
+  if (n == "wte" || (c->llama && n == "head.w")) {
     if (!expect((size_t)c->V * d)) return bad_size();
-    set(&c->wte);
-    Scope s(c, "transpose", 1);
-    CK(c, transpose(c->dt, dev, c->V, c->d, c->wteT, c->Vpad, c->st));
+    if (n == "wte") set(&c->wte);
+    if (n == "head.w" || !c->llama) {      // the head: tied to wte unless the architecture has its own
+      if (c->llama) set(&c->headw); else c->headw = dev;
+      Scope s(c, "transpose", 1);
+      CK(c, transpose(c->dt, dev, c->V, c->d, c->wteT, c->Vpad, c->st));
+    }
     return SPLITLORA_OK;
   }
-  if (n == "wpe") { if (!expect((size_t)c->cfg.max_seq * d)) return bad_size(); set(&c->wpe); return SPLITLORA_OK; }
   if (n == "lnf.g") { if (!expect(d)) return bad_size(); set(&c->lnfg); return SPLITLORA_OK; }
-  if (n == "lnf.b") { if (!expect(d)) return bad_size(); set(&c->lnfb); return SPLITLORA_OK; }
+  if (!c->llama) {
+    if (n == "wpe") { if (!expect((size_t)c->cfg.max_seq * d)) return bad_size(); set(&c->wpe); return SPLITLORA_OK; }
+    if (n == "lnf.b") { if (!expect(d)) return bad_size(); set(&c->lnfb); return SPLITLORA_OK; }
+  }
   int l = -1; char rest[64];
   if (sscanf(name, "h.%d.%63s", &l, rest) != 2 || l < 0 || l >= c->L) return fail(c, SPLITLORA_ERR_ARG, std::string("unknown tensor ") + name);
   FrozenLayer& f = c->fl[l];
   std::string r(rest);
-  struct Ent { const char* nm; const void** slot; size_t elems; void* tr; int rows, cols; };
+  struct Ent { const char* nm; const void** slot; size_t elems; void* tr; int rows, cols; bool gpt, llama; };
   Ent ents[] = {
-      {"ln1.g", &f.ln1g, d, nullptr, 0, 0}, {"ln1.b", &f.ln1b, d, nullptr, 0, 0},
-      {"attn.qkv.w", &f.qkvw, 3 * d * d, f.qkvwT, 3 * c->d, c->d}, {"attn.qkv.b", &f.qkvb, 3 * d, nullptr, 0, 0},
-      {"attn.proj.w", &f.projw, d * d, f.projwT, c->d, c->d}, {"attn.proj.b", &f.projb, d, nullptr, 0, 0},
-      {"ln2.g", &f.ln2g, d, nullptr, 0, 0}, {"ln2.b", &f.ln2b, d, nullptr, 0, 0},
-      {"mlp.fc1.w", &f.fc1w, F * d, f.fc1wT, c->F, c->d}, {"mlp.fc1.b", &f.fc1b, F, nullptr, 0, 0},
-      {"mlp.fc2.w", &f.fc2w, d * F, f.fc2wT, c->d, c->F}, {"mlp.fc2.b", &f.fc2b, d, nullptr, 0, 0}};
+      {"ln1.g", &f.ln1g, d, nullptr, 0, 0, true, true}, {"ln1.b", &f.ln1b, d, nullptr, 0, 0, true, false},
+      {"attn.qkv.w", &f.qkvw, 3 * d * d, f.qkvwT, 3 * c->d, c->d, true, true},
+      {"attn.qkv.b", &f.qkvb, 3 * d, nullptr, 0, 0, true, false},
+      {"attn.proj.w", &f.projw, d * d, f.projwT, c->d, c->d, true, true},
+      {"attn.proj.b", &f.projb, d, nullptr, 0, 0, true, false},
+      {"ln2.g", &f.ln2g, d, nullptr, 0, 0, true, true}, {"ln2.b", &f.ln2b, d, nullptr, 0, 0, true, false},
+      {"mlp.fc1.w", &f.fc1w, F * d, f.fc1wT, c->F, c->d, true, false}, {"mlp.fc1.b", &f.fc1b, F, nullptr, 0, 0, true, false},
+      {"mlp.fc2.w", &f.fc2w, d * F, f.fc2wT, c->d, c->F, true, false}, {"mlp.fc2.b", &f.fc2b, d, nullptr, 0, 0, true, false},
+      {"mlp.gate_up.w", &f.fc1w, 2 * F * d, f.fc1wT, 2 * c->F, c->d, false, true},
+      {"mlp.down.w", &f.fc2w, d * F, f.fc2wT, c->d, c->F, false, true}};
   for (auto& e : ents) {
-    if (r == e.nm) {
+    if (r == e.nm && (c->llama ? e.llama : e.gpt)) {
       if (!expect(e.elems)) return bad_size();
       set(e.slot);
       if (e.tr) {
@@ -618,9 +739,8 @@ int splitlora_server_step(splitlora_ctx* c, const void* act_in, const int32_t* l
     CK(c, block_forward(c, l, x, c->lb[l].x_out));
     x = c->lb[l].x_out;
   }
-  { Scope s(c, "layernorm_fwd", 1);
-    CK(c, layernorm_fwd(c->dt, x, c->lnfg, c->lnfb, c->xf, c->meanf, c->rstdf, M, d, c->cfg.norm_eps, c->st)); }
-  { GemmArgs a = base_args(c, c->xf, d, c->wte, d, c->logits, c->Vpad, M, c->Vpad, d);
+  CK(c, norm_forward(c, x, c->lnfg, c->lnfb, c->xf, c->meanf, c->rstdf));
+  { GemmArgs a = base_args(c, c->xf, d, c->headw, d, c->logits, c->Vpad, M, c->Vpad, d);
     a.w_rows = c->V;
     CK(c, linear(c, "head_fwd", a)); }
   { Scope s(c, "cross_entropy", 3);
@@ -630,8 +750,7 @@ int splitlora_server_step(splitlora_ctx* c, const void* act_in, const int32_t* l
   { GemmArgs a = base_args(c, c->logits, c->Vpad, c->wteT, c->Vpad, c->g_a, d, M, d, c->Vpad);
     CK(c, linear(c, "head_bwd", a)); }
   void* cur = c->g_b;
-  { Scope s(c, "layernorm_bwd", 1);
-    CK(c, layernorm_bwd(c->dt, c->g_a, x, c->lnfg, c->meanf, c->rstdf, nullptr, cur, M, d, c->st)); }
+  CK(c, norm_backward(c, c->g_a, x, c->lnfg, c->meanf, c->rstdf, nullptr, cur));
   void* other = c->g_a;
   for (int l = c->L - 1; l >= c->cut; --l) {
     void* dst = (l == c->cut) ? act_grad_out : other;

@@ -18,6 +18,11 @@ def make_engine(w, frozen, client_adapters, server_adapters, optimizer="adamw", 
     cfg = B.config_from_workload(w, optimizer=optimizer, use_tensor_cores=use_tensor_cores, **over)
     eng = B.SplitLoRA(cfg)
     for name, arr in frozen.items():
+        if name.endswith("mlp.up.w"):
+            continue                      # bound together with the gate, below
+        if name.endswith("mlp.gate.w"):   # the library takes gate and up stacked as one [2F, d] tensor
+            up = frozen[name[:-len("gate.w")] + "up.w"]
+            name, arr = name[:-len("gate.w")] + "gate_up.w", np.concatenate([arr, up], axis=0)
         eng.bind_frozen(name, to_device(arr, eng.act_dtype))
     for i, ca in enumerate(client_adapters):
         for (l, t), ad in ca.items():

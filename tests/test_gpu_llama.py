@@ -1,0 +1,95 @@
+"""GPU parity of the Llama-shaped block (RMSNorm, rotary q/k, SwiGLU, adapters on q, k, v, o, separate
+head) and of an adapter on the output projection of the GPT-shaped block, against the CPU oracle.
+Same tolerances as test_gpu_parity.py."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import splitlora_oracle as O
+from paper_2407_00952_b200 import binding as B
+from paper_2407_00952_b200 import runner, synth
+import harness as H
+from test_gpu_parity import TOL_AGG, TOL_BF16, TOL_FP32, TOL_LOSS, check_three_calls
+
+pytestmark = pytest.mark.gpu
+
+
+def tiny_llama(**kw):
+    base = dict(index=1, name="tiny-llama", n_layer=2, cut=1, d_model=64, n_head=2, d_ff=96, vocab=1024, max_seq=64,
+                lora_r=4, lora_alpha=8.0, n_clients=2, batch_per_client=4, seq=64, dtype="fp32", lr=1e-3, zipf=False,
+                counts=(3, 5))
+    base.update(kw)
+    return synth.scaled(synth.WORKLOADS[5], **base)
+
+
+def test_tiny_llama_fp32_three_calls():
+    check_three_calls(tiny_llama(), TOL_FP32)
+
+
+@pytest.mark.parametrize("targets", [("q", "v"), ("k", "o"), ("q", "k", "v")])
+def test_tiny_llama_fp32_target_sets(targets):
+    check_three_calls(tiny_llama(targets=targets, n_layer=3, cut=2), TOL_FP32)
+
+
+def test_gpt_shaped_with_output_projection_adapter():
+    w = synth.scaled(synth.WORKLOADS[1], targets=("q", "v", "o"))
+    check_three_calls(w, TOL_FP32)
+
+
+def test_tiny_llama_zero_b():
+    """B = 0: every dA vanishes, the o adapter included."""
+    w = tiny_llama()
+    case = H.build_case(w, nonzero_b=False, distinct_clients=False)
+    eng = check_three_calls(w, TOL_FP32, case=case)
+    gA, gB = eng.get_adapter_grad(B.SIDE_SERVER, 0, 1, B.TARGET_O)
+    assert float(gA.abs().max()) == 0.0 and float(gB.abs().max()) > 0.0
+
+
+def test_tiny_llama_full_round_adamw_and_aggregation():
+    w = tiny_llama()
+    frozen, cads, sads, tokens, labels = H.build_case(w)
+    counts = synth.make_counts(w)
+    eng = runner.make_engine(w, frozen, cads, sads, optimizer="adamw")
+    loss = eng.round(torch.from_numpy(tokens).cuda(), torch.from_numpy(labels).cuda(), counts)
+    cfg = H.oracle_config(w, optimizer="adamw")
+    st = O.OracleState(client_adapters=[H.ads64(a) for a in cads], server_adapters=H.ads64(sads))
+    loss_ref, info = O.split_round(cfg, H.f64(frozen), st, tokens, labels, counts)
+    assert info["aggregated"]
+    assert abs(loss - loss_ref) <= TOL_LOSS * abs(loss_ref)
+    for i in range(w.n_clients):
+        for (l, t), ad in st.client_adapters[i].items():
+            A, Bm = eng.get_adapter(B.SIDE_CLIENT, i, l, B.TARGET_BITS[t])
+            gs = [info["client_grads"][k][(l, t)] for k in range(w.n_clients)]
+            for got, ref, gi in ((A, ad["A"], 0), (Bm, ad["B"], 1)):
+                mask = np.ones_like(ref, dtype=bool)
+                for g in gs:
+                    mask &= np.abs(g[gi]) > 1e-3 * np.abs(g[gi]).max()
+                err = np.abs(H.tnp(got) - ref)[mask].max() / np.abs(ref).max()
+                assert err <= 1e-4, (i, l, t, gi, err)
+    A0, B0 = eng.get_adapter(B.SIDE_CLIENT, 0, 0, B.TARGET_O)
+    A1, B1 = eng.get_adapter(B.SIDE_CLIENT, 1, 0, B.TARGET_O)
+    assert torch.equal(A0, A1) and torch.equal(B0, B1)
+
+
+@pytest.mark.parametrize("use_tc", [True, False])
+def test_llama_shaped_reduced_bf16(use_tc):
+    """Head width 128, rank 16, adapters on q, k, v, o, at reduced width and depth, bf16."""
+    w = synth.scaled(synth.WORKLOADS[5], n_layer=3, cut=1, d_model=512, n_head=4, d_ff=1280, vocab=8192,
+                     n_clients=2, batch_per_client=1, seq=256, max_seq=256)
+    check_three_calls(w, TOL_BF16, use_tc=use_tc)
+
+
+def test_llama_shaped_full_width_one_block_each_bf16():
+    """Full width (d 4096, 32 heads, d_ff 11008, rank 16), one client block and one server block, short
+    sequences and a reduced vocabulary so that the oracle finishes in about a minute.
+
+    Activations, activation gradients, loss and the v / o adapter gradients keep the 2e-2 bound.  The q / k
+    adapter gradients get 4e-2: with N(0, 0.02) weights at width 4096 the attention logits have a standard
+    deviation of 1.7, and at that scale the attention backward turns a relative noise eps on q, k, v, dO
+    into about 2.5 eps on dq, dk (CPU experiment with the oracle); rounding every stored tensor of one
+    block to bf16 in the oracle's own fp64 arithmetic already gives eps = 1.0 % on the block output, so
+    2.5 % is what the storage format allows, whatever the kernels do.  The plain-FMA kernels (fp32
+    arithmetic, same bf16 storage points) land on the same errors as the tensor-core ones."""
+    w = synth.scaled(synth.WORKLOADS[5], n_layer=2, cut=1, vocab=4096, n_clients=2, batch_per_client=1, seq=256,
+                     max_seq=256)
+    check_three_calls(w, TOL_BF16, tol_qk=4e-2)

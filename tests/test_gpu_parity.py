@@ -26,8 +26,10 @@ TOL_AGG = 1e-6
 TOL_LOSS = 1e-3
 
 
-def check_three_calls(w, tol, use_tc=True, case=None):
+def check_three_calls(w, tol, use_tc=True, case=None, tol_qk=None):
+    """tol_qk: bound for the q and k adapter gradients where it differs from tol (see the caller)."""
     case = case or H.build_case(w)
+    tol_of = lambda t: tol_qk if (tol_qk is not None and t in ("q", "k")) else tol
     eng, S, dS, loss = H.run_three_calls(w, *case, optimizer="sgd", use_tensor_cores=use_tc)
     cfg, params, c64, s64, S_ref, dS_ref, loss_ref, sg, cg = H.oracle_three_calls(w, *case, optimizer="sgd")
     assert abs(loss - loss_ref) <= TOL_LOSS * abs(loss_ref)
@@ -35,13 +37,13 @@ def check_three_calls(w, tol, use_tc=True, case=None):
     assert H.rel_err(H.tnp(dS), dS_ref) <= tol
     for (l, t), (dA, dB) in sg.items():
         gA, gB = eng.get_adapter_grad(B.SIDE_SERVER, 0, l, B.TARGET_BITS[t])
-        assert H.rel_err(H.tnp(gA), dA) <= tol, ("server dA", l, t)
-        assert H.rel_err(H.tnp(gB), dB) <= tol, ("server dB", l, t)
+        assert H.rel_err(H.tnp(gA), dA) <= tol_of(t), ("server dA", l, t)
+        assert H.rel_err(H.tnp(gB), dB) <= tol_of(t), ("server dB", l, t)
     for i in range(w.n_clients):
         for (l, t), (dA, dB) in cg[i].items():
             gA, gB = eng.get_adapter_grad(B.SIDE_CLIENT, i, l, B.TARGET_BITS[t])
-            assert H.rel_err(H.tnp(gA), dA) <= tol, ("client dA", i, l, t)
-            assert H.rel_err(H.tnp(gB), dB) <= tol, ("client dB", i, l, t)
+            assert H.rel_err(H.tnp(gA), dA) <= tol_of(t), ("client dA", i, l, t)
+            assert H.rel_err(H.tnp(gB), dB) <= tol_of(t), ("client dB", i, l, t)
     # SGD update is the literal rule of Eq. 4-7: P_new = P - lr * G (on every element)
     for (l, t), (dA, dB) in sg.items():
         A, Bm = eng.get_adapter(B.SIDE_SERVER, 0, l, B.TARGET_BITS[t])
@@ -223,9 +225,10 @@ def test_lora_linear_fp32():
 
 
 @pytest.mark.parametrize("nseq,T,Hh,d,use_tc", [(2, 64, 2, 128, True), (2, 256, 3, 192, True),
-                                                (1, 512, 2, 128, True), (3, 40, 4, 96, False)])
+                                                (1, 512, 2, 128, True), (3, 40, 4, 96, False),
+                                                (2, 192, 2, 256, True), (1, 1024, 1, 128, True)])
 def test_attention_bf16(nseq, T, Hh, d, use_tc):
-    """Causal attention forward/backward: tensor-core kernels (head width 64) and the plain kernels
+    """Causal attention forward/backward: tensor-core kernels (head width 64 and 128) and the plain kernels
     (any head width, ragged length) against the oracle."""
     torch.manual_seed(T + d)
     qkv = torch.randn(nseq * T, 3 * d, device="cuda").bfloat16()

@@ -70,13 +70,18 @@ def torch_block(cfg, P, l, ads, x):
     s = cfg.scale
     parts = {"q": q, "k": k, "v": v}
     for t in cfg.targets:
-        A, B = ads[(l, t)]
-        parts[t] = parts[t] + s * F.linear(F.linear(u, A), B)
+        if t != "o":
+            A, B = ads[(l, t)]
+            parts[t] = parts[t] + s * F.linear(F.linear(u, A), B)
     nseq, T, _ = x.shape
     sh = lambda z: z.reshape(nseq, T, H, d // H).transpose(1, 2)
     o = F.scaled_dot_product_attention(sh(parts["q"]), sh(parts["k"]), sh(parts["v"]), is_causal=True)
     o = o.transpose(1, 2).reshape(nseq, T, d)
-    x = x + F.linear(o, P[f"h.{l}.attn.proj.w"], P[f"h.{l}.attn.proj.b"])
+    Wo = P[f"h.{l}.attn.proj.w"]
+    if "o" in cfg.targets:
+        A, B = ads[(l, "o")]
+        Wo = Wo + s * B @ A            # the update folded into the weight
+    x = x + F.linear(o, Wo, P[f"h.{l}.attn.proj.b"])
     u2 = F.layer_norm(x, (d,), P[f"h.{l}.ln2.g"], P[f"h.{l}.ln2.b"], cfg.norm_eps)
     z = F.linear(u2, P[f"h.{l}.mlp.fc1.w"], P[f"h.{l}.mlp.fc1.b"])
     a = F.gelu(z, approximate="tanh" if cfg.gelu_tanh else "none")
@@ -189,9 +194,9 @@ def test_lora_linear_equals_merged_weight():
 
 
 # ------------------------------------------------------------------ whole split model
-@pytest.mark.parametrize("cut", [1, 2])
-def test_split_model_matches_autograd(cut):
-    w = tiny_workload(cut=cut)
+@pytest.mark.parametrize("cut,targets", [(1, ("q", "v")), (2, ("q", "v")), (1, ("q", "k", "v", "o"))])
+def test_split_model_matches_autograd(cut, targets):
+    w = tiny_workload(cut=cut, targets=targets)
     cfg = ocfg(w)
     params, cads, sads, tokens, labels = setup(w)
     labels = labels.copy()
