@@ -49,12 +49,17 @@ def workload_description(w):
 def gemm_flops_per_round(w):
     """Algorithmic FLOPs of the tensor-core linear layers per round, by launch class (no dW)."""
     M, d, F, V, L = w.tokens_per_round, w.d_model, w.d_ff, w.vocab, w.n_layer
-    nt, r = len(w.targets), w.lora_r
+    r = w.lora_r
+    nq = len([t for t in w.targets if t != "o"])
+    has_o = "o" in w.targets
+    mlp = (6.0 if w.arch == "llama" else 4.0) * M * d * F          # gate, up, down / fc1, fc2
+    proj = 2.0 * M * d * d + (2.0 * M * r * d if has_o else 0.0)   # output projection (+ its rank-r term)
+    qkv = 2.0 * M * d * 3 * d + 2.0 * M * r * d * nq
     return {
-        "lora_linear_fwd": L * (2.0 * M * d * 3 * d + 2.0 * M * r * d * nt),
-        "linear_fwd": L * (2.0 * M * d * d + 4.0 * M * d * F),
-        "linear_bwd": L * (2.0 * M * d * d + 4.0 * M * d * F),
-        "lora_linear_bwd": (L - 1) * (2.0 * M * 3 * d * d + 2.0 * M * r * d * nt),
+        "lora_linear_fwd": L * (qkv + (proj if has_o else 0.0)),
+        "linear_fwd": L * (mlp + (0.0 if has_o else proj)),
+        "linear_bwd": L * (mlp + (0.0 if has_o else proj)),
+        "lora_linear_bwd": (L - 1) * qkv + (L * proj if has_o else 0.0),
         "head_fwd": 2.0 * M * d * V,
         "head_bwd": 2.0 * M * d * V,
     }
@@ -102,7 +107,11 @@ class ClockSampler:
 
 
 def oracle_sample_workload(w):
-    """The bounded sample the CPU oracle is timed on: same model, 2 clients x 1 sequence."""
+    """The bounded sample the CPU oracle is timed on: same model, 2 clients x 1 sequence.  A model whose
+    fp64 round would take many minutes even so (width 4096) is cut to one client block and one server
+    block on one sequence; time_oracle_rounds scales the time back up to the full depth."""
+    if w.d_model >= 2048:
+        return synth.scaled(w, n_layer=2, cut=1, n_clients=1, batch_per_client=1, counts=None)
     return synth.scaled(w, n_clients=min(2, w.n_clients), batch_per_client=1, counts=None)
 
 
@@ -119,7 +128,7 @@ def time_oracle_rounds(w, steps, warmup):
                          vocab=ws.vocab, max_seq=ws.max_seq, lora_r=ws.lora_r, lora_alpha=ws.lora_alpha,
                          targets=ws.targets, n_clients=ws.n_clients, batch_per_client=ws.batch_per_client, seq=ws.seq,
                          bf16_handoff=(ws.dtype == "bf16"), optimizer="adamw", lr_client=ws.lr, lr_server=ws.lr,
-                         agg_interval=ws.agg_interval)
+                         agg_interval=ws.agg_interval, arch=ws.arch, rope_theta=ws.rope_theta)
     counts = synth.make_counts(ws)
     times = []
     for s in range(warmup + steps):
@@ -134,13 +143,16 @@ def time_oracle_rounds(w, steps, warmup):
         threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
     except Exception:
         threads = os.cpu_count() or 1
-    sec = float(np.mean(times))
+    sec = float(np.mean(times)) * (w.n_layer / ws.n_layer)     # depth-reduced sample: linear in depth
     return ws.tokens_per_round / sec, sec, threads, ws
 
 
 def sample_text(ws, sec=None):
     s = (f"one oracle round (numpy fp64) of the same model on {ws.n_clients} clients x {ws.batch_per_client} "
          f"sequence x {ws.seq} tokens = {ws.tokens_per_round} tokens")
+    if ws.n_layer == 2 and ws.d_model >= 2048:
+        s += (" with one client block and one server block at full width, the time multiplied by (blocks of the "
+              "full model / 2): an extrapolation that also multiplies the head's share")
     return s + (f" ({sec:.1f} s)" if sec is not None else "")
 
 
@@ -169,11 +181,9 @@ def run_gpu(args, w):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    frozen = synth.make_frozen(w)
     cads = [synth.make_adapters(w, range(w.cut)) for _ in range(w.n_clients)]
     sads = synth.make_adapters(w, range(w.cut, w.n_layer))
-    eng = runner.make_engine(w, frozen, cads, sads, optimizer="adamw")
-    del frozen
+    eng = runner.make_engine(w, synth.iter_frozen(w), cads, sads, optimizer="adamw")   # uploaded as drawn
     counts = synth.make_counts(w)
     nbatch = 4
     host_tok, host_lab, dev_tok, dev_lab = [], [], [], []

@@ -108,7 +108,15 @@ size_t lora_grad_scratch_floats(int M, int R, int C);
 cudaError_t lora_grad(int dt, const void* Z, int64_t ldz, int zcol0, int C, const void* Wt, int64_t ldwt,
                       int wcol0, int r, int rp, int nt, int M, int rows_per_group, float scale, float* out,
                       int64_t out_group_stride, int64_t out_target_stride, int64_t out_sj, int64_t out_sc,
-                      float* partial, cudaStream_t st);
+                      float* partial, cudaStream_t st, int* status = nullptr, bool use_tc = false);
+// The same reduction as a tcgen05 product with both operands MN-major (bf16, rp in {16, 32, 64},
+// ldwt a multiple of 64, the wanted weight columns inside one 64-column tile).  Writes per-chunk
+// partials [chunk][nt*r][C]; lora_grad adds them.  status: device word for an expired bounded wait.
+bool lora_grad_tc_supported(int dt, const void* Z, int64_t ldz, int zcol0, int C, const void* Wt, int64_t ldwt,
+                            int wcol0, int r, int rp, int nt, int M, int rows_per_group);
+cudaError_t lora_grad_tc_partial(const void* Z, int64_t ldz, int zcol0, int C, const void* Wt, int64_t ldwt, int wcol0,
+                                 int r, int rp, int nt, int M, int rows_per_group, float* partial, int* status,
+                                 int* chunks_per_group, cudaStream_t st);
 
 struct OptArgs {
   int optimizer; float lr, beta1, beta2, eps, wd; float bc1, bc2;   // bc = 1 - beta^step

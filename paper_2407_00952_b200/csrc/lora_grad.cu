@@ -150,7 +150,29 @@ size_t lora_grad_scratch_floats(int M, int R, int C) {
 cudaError_t lora_grad(int dt, const void* Z, int64_t ldz, int zcol0, int C, const void* Wt, int64_t ldwt, int wcol0,
                       int r, int rp, int nt, int M, int rows_per_group, float scale, float* out,
                       int64_t out_group_stride, int64_t out_target_stride, int64_t out_sj, int64_t out_sc,
-                      float* partial, cudaStream_t st) {
+                      float* partial, cudaStream_t st, int* status, bool use_tc) {
+  if (use_tc && status && dt == DT_BF16 && (rp == 16 || rp == 32 || rp == 64)) {
+    // tensor-core path, in windows of the targets whose weight columns share one 64-column tile
+    const int tw = 64 / rp;
+    bool ok = true;
+    for (int t0 = 0; t0 < nt && ok; t0 += tw)
+      ok = lora_grad_tc_supported(dt, Z, ldz, zcol0, C, Wt, ldwt, wcol0 + t0 * rp, r, rp, min(tw, nt - t0), M,
+                                  rows_per_group);
+    if (ok) {
+      const int groups = rows_per_group > 0 && rows_per_group < M ? M / rows_per_group : 1;
+      for (int t0 = 0; t0 < nt; t0 += tw) {
+        const int ntw = min(tw, nt - t0), Rw = ntw * r;
+        int cpg = 0;
+        cudaError_t e = lora_grad_tc_partial(Z, ldz, zcol0, C, Wt, ldwt, wcol0 + t0 * rp, r, rp, ntw, M, rows_per_group,
+                                             partial, status, &cpg, st);
+        if (e != cudaSuccess) return e;
+        dim3 g2((Rw * C + 31) / 32, groups), b2(32, RED_LANES);
+        lora_grad_reduce_kernel<<<g2, b2, 0, st>>>(partial, r, Rw, C, cpg, scale, out + (size_t)t0 * out_target_stride,
+                                                   out_group_stride, out_target_stride, out_sj, out_sc);
+      }
+      return cudaGetLastError();
+    }
+  }
   const int R = nt * r;
   const int rpg = rows_per_group > 0 ? rows_per_group : M;
   const int n = dt == DT_BF16 ? 8 : 4;

@@ -147,9 +147,9 @@ int splitlora_lora_linear_bwd(int dtype, int use_tc, const void* x, const void* 
   if (run_gemm(use_tc, a, status, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
   float* scratch = (float*)(ws + p.off_scratch);
   if (lora_grad(dtype, x, n_in, 0, n_in, ws + p.off_dh, p.ext, 0, r, p.rp, 1, M, rpg, 1.0f, dA, (int64_t)r * n_in, 0, n_in, 1,
-                scratch, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
+                scratch, st, status, use_tc != 0) != cudaSuccess) return SPLITLORA_ERR_CUDA;
   if (lora_grad(dtype, dy, n_out, 0, n_out, ws + p.off_h, p.ext, 0, r, p.rp, 1, M, rpg, s, dB, (int64_t)n_out * r, 0, 1, r,
-                scratch, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
+                scratch, st, status, use_tc != 0) != cudaSuccess) return SPLITLORA_ERR_CUDA;
   return SPLITLORA_OK;
 }
 

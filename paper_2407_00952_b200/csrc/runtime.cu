@@ -414,10 +414,10 @@ cudaError_t block_backward(splitlora_ctx* c, int l, const void* dy, void* dx) {
     float* gA = gbase + (size_t)c->nq * 2 * c->r * d;
     { Scope s(c, "lora_grad", 2);
       if ((e = lora_grad(c->dt, b.o, d, 0, d, c->g_dhcat_o, c->ext_o, 0, c->r, c->rp, 1, M, rpg, 1.0f, gA, gstride, 0, d,
-                         1, c->grad_scratch, c->st))) return e; }
+                         1, c->grad_scratch, c->st, c->status, c->tc))) return e; }
     { Scope s(c, "lora_grad", 2);
       if ((e = lora_grad(c->dt, c->g_dxmid, d, 0, d, b.hcat_o, c->ext_o, 0, c->r, c->rp, 1, M, rpg, c->scale,
-                         gA + (size_t)c->r * d, gstride, 0, 1, c->r, c->grad_scratch, c->st))) return e; }
+                         gA + (size_t)c->r * d, gstride, 0, 1, c->r, c->grad_scratch, c->st, c->status, c->tc))) return e; }
   }
   { GemmArgs a = base_args(c, c->g_dxmid, d, f.projwT, d, c->g_do, d, M, d, d);
     if (c->has_o) {
@@ -443,12 +443,12 @@ cudaError_t block_backward(splitlora_ctx* c, int l, const void* dy, void* dx) {
   // G_A = dh^T u, G_B = (alpha/r) dy^T h, per group (Eq. 4-7)
   { Scope s(c, "lora_grad", 2);   // every qkv target's G_A in one pass over u
     if ((e = lora_grad(c->dt, b.u, d, 0, d, c->g_dhcat, ext, 0, c->r, c->rp, c->nq, M, rpg, 1.0f, gbase,
-                       gstride, (int64_t)2 * c->r * d, d, 1, c->grad_scratch, c->st))) return e; }
+                       gstride, (int64_t)2 * c->r * d, d, 1, c->grad_scratch, c->st, c->status, c->tc))) return e; }
   for (int t = 0; t < c->nq; ++t) {
     float* gB = gbase + (size_t)t * 2 * c->r * d + (size_t)c->r * d;
     Scope s(c, "lora_grad", 2);
     if ((e = lora_grad(c->dt, c->g_dqkv, 3 * d, c->slice_idx[t] * d, d, b.hcat, ext, t * c->rp, c->r, c->rp, 1, M,
-                       rpg, c->scale, gB, gstride, 0, 1, c->r, c->grad_scratch, c->st))) return e;
+                       rpg, c->scale, gB, gstride, 0, 1, c->r, c->grad_scratch, c->st, c->status, c->tc))) return e;
   }
   if (dx) {
     GemmArgs a = base_args(c, c->g_dqkv, 3 * d, f.qkvwT, 3 * d, c->g_du, d, M, d, 3 * d);

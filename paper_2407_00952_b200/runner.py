@@ -13,17 +13,23 @@ def to_device(a: np.ndarray, dtype: torch.dtype) -> torch.Tensor:
 
 
 def make_engine(w, frozen, client_adapters, server_adapters, optimizer="adamw", use_tensor_cores=True, **over):
-    """frozen: {name: fp32 ndarray}; client_adapters: list (one per client) of {(layer, target): {"A","B"}};
+    """frozen: {name: fp32 ndarray} or an iterable of (name, array) pairs in which a layer's "mlp.up.w"
+    follows its "mlp.gate.w"; client_adapters: list (one per client) of {(layer, target): {"A","B"}};
     server_adapters: {(layer, target): {"A","B"}}."""
     cfg = B.config_from_workload(w, optimizer=optimizer, use_tensor_cores=use_tensor_cores, **over)
     eng = B.SplitLoRA(cfg)
-    for name, arr in frozen.items():
-        if name.endswith("mlp.up.w"):
-            continue                      # bound together with the gate, below
+    gate = None
+    for name, arr in (frozen.items() if hasattr(frozen, "items") else frozen):
         if name.endswith("mlp.gate.w"):   # the library takes gate and up stacked as one [2F, d] tensor
-            up = frozen[name[:-len("gate.w")] + "up.w"]
-            name, arr = name[:-len("gate.w")] + "gate_up.w", np.concatenate([arr, up], axis=0)
-        eng.bind_frozen(name, to_device(arr, eng.act_dtype))
+            gate = to_device(arr, eng.act_dtype)
+            continue
+        if name.endswith("mlp.up.w"):
+            name = name[:-len("up.w")] + "gate_up.w"
+            dev = torch.cat([gate, to_device(arr, eng.act_dtype)], dim=0)
+            gate = None
+        else:
+            dev = to_device(arr, eng.act_dtype)
+        eng.bind_frozen(name, dev)
     for i, ca in enumerate(client_adapters):
         for (l, t), ad in ca.items():
             eng.set_adapter(B.SIDE_CLIENT, i, l, B.TARGET_BITS[t], to_device(ad["A"], torch.float32),

@@ -112,7 +112,12 @@ def make_frozen(w: Workload, randomize_affine: bool = False) -> Dict[str, np.nda
     Weights ~ N(0, 0.02); biases 0 and LayerNorm gain 1 / bias 0 unless `randomize_affine`,
     which draws them (used by tests so that no term is hidden by a zero).
     """
-    params = {}
+    return dict(iter_frozen(w, randomize_affine))
+
+
+def iter_frozen(w: Workload, randomize_affine: bool = False):
+    """The tensors of make_frozen one at a time, as (name, array): a workload whose weights do not
+    fit in host memory at once (13.5 GB in bf16 for the Llama-2-7B shape) is uploaded as it is drawn."""
     for idx, (name, shape, kind) in enumerate(frozen_param_names(w)):
         rng = np.random.default_rng(1234 + 1000 * w.index + idx)
         if kind == "w":
@@ -125,8 +130,7 @@ def make_frozen(w: Workload, randomize_affine: bool = False) -> Dict[str, np.nda
                 else np.zeros(shape, np.float32)
         if w.dtype == "bf16":
             a = _to_bf16_values(a)
-        params[name] = a
-    return params
+        yield name, a
 
 
 def make_adapters(w: Workload, layers, nonzero_b: bool = False, salt: int = 0):
