@@ -69,7 +69,11 @@ typedef struct splitlora_ctx splitlora_ctx;   /* opaque */
 /* Inputs of Algorithm 1 (b, I, gamma_c, gamma_s, N) plus the model shape.  Plain data. */
 typedef struct {
   int32_t n_layer;           /* blocks in the whole model                                   */
-  int32_t cut;               /* blocks 0..cut-1 run on the clients; 1 <= cut < n_layer      */
+  int32_t cut;               /* blocks 0..cut-1 run on the clients; 1 <= cut <= n_layer.
+                                cut == n_layer: every block is client-side and aggregated,
+                                the server keeps only the final norm and the head (the
+                                federated-LoRA baseline of Sec. IV-A); n_clients == 1 is
+                                the centralised baseline                                    */
   int32_t d_model, n_head, d_ff, vocab, max_seq;
   int32_t lora_r;            /* rank r, 1..64                                               */
   float   lora_alpha;        /* scaling alpha; the update is scaled by alpha / r            */

@@ -401,6 +401,7 @@ __global__ void optimizer_kernel(float* __restrict__ p, const float* __restrict_
 cudaError_t optimizer_step(float* p, const float* g, float* m, float* v, int64_t n, const OptArgs& o,
                            cudaStream_t st) {
   if (n % 4 != 0) return cudaErrorInvalidValue;
+  if (n == 0) return cudaSuccess;     // a side without adapters (all blocks on the clients)
   int64_t n4 = n / 4;
   optimizer_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(p, g, m, v, n4, o);
   return cudaGetLastError();

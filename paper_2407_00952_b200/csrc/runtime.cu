@@ -126,7 +126,9 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 int validate(const splitlora_config* c, std::string* why) {
   auto bad = [&](const char* m) { *why = m; return SPLITLORA_ERR_ARG; };
   if (!c) return bad("null config");
-  if (c->n_layer < 2 || c->cut < 1 || c->cut >= c->n_layer) return bad("need 1 <= cut < n_layer");
+  // cut == n_layer puts every block on the clients (the server keeps the final norm and the head):
+  // the federated-LoRA baseline of Sec. IV as a degenerate case of the same round
+  if (c->n_layer < 1 || c->cut < 1 || c->cut > c->n_layer) return bad("need 1 <= cut <= n_layer");
   if (c->d_model < 8 || c->n_head < 1 || c->d_model % c->n_head != 0) return bad("d_model must be a multiple of n_head");
   if (c->d_model % 8 != 0 || c->d_ff % 8 != 0) return bad("d_model and d_ff must be multiples of 8");
   if (c->d_model / c->n_head > 128) return bad("head width above 128");
@@ -749,7 +751,7 @@ int splitlora_server_step(splitlora_ctx* c, const void* act_in, const int32_t* l
   // backward: head, final norm, blocks L-1 .. cut
   { GemmArgs a = base_args(c, c->logits, c->Vpad, c->wteT, c->Vpad, c->g_a, d, M, d, c->Vpad);
     CK(c, linear(c, "head_bwd", a)); }
-  void* cur = c->g_b;
+  void* cur = (c->cut == c->L) ? act_grad_out : c->g_b;     // no server block: this is dL/dS already
   CK(c, norm_backward(c, c->g_a, x, c->lnfg, c->meanf, c->rstdf, nullptr, cur));
   void* other = c->g_a;
   for (int l = c->L - 1; l >= c->cut; --l) {

@@ -127,9 +127,38 @@ def bench_attention(nseq, T, heads, iters=10):
             "bwd_tflops_algorithmic": round(2.5 * fl / b / 1e9, 1), "peak_source": src}
 
 
+def bench_split(config: int, cut: int, agg_interval: int, n_clients: int, steps: int):
+    """One workload at another split point / aggregation interval / client count: tokens per second of
+    whole rounds, the bytes that cross the client-server boundary per round (S and dL/dS, Sec. III-B
+    steps a2 and a4, plus labels), the adapter bytes of an aggregation (b1 + b3) and the share of the
+    blocks that run on the clients.  cut == n_layer is the federated baseline, n_clients == 1 the
+    centralised one (Sec. IV-A)."""
+    from . import runner, synth
+    w = synth.scaled(synth.WORKLOADS[config], cut=cut, agg_interval=agg_interval, n_clients=n_clients)
+    cads = [synth.make_adapters(w, range(w.cut)) for _ in range(w.n_clients)]
+    sads = synth.make_adapters(w, range(w.cut, w.n_layer))
+    eng = runner.make_engine(w, synth.iter_frozen(w), cads, sads, optimizer="adamw")
+    counts = synth.make_counts(w)
+    batches = []
+    for s in range(2):
+        t, l = synth.make_tokens(w, round_index=s)
+        batches.append((torch.from_numpy(t).cuda(), torch.from_numpy(l).cuda()))
+    ms = _time(lambda i: eng.round(*batches[i % 2], counts, want_loss=False), steps, warmup=3)
+    assert eng.device_status() == 0
+    M, es = w.tokens_per_round, 2 if w.dtype == "bf16" else 4
+    per_client = w.cut * len(w.targets) * 2 * w.lora_r * w.d_model * 4
+    return {"op": "split_round", "config": config, "cut": cut, "n_layer": w.n_layer, "I": agg_interval,
+            "K": w.n_clients, "tokens_per_round": M, "ms_per_round": round(ms, 3),
+            "tokens_per_s": round(M / ms * 1e3, 1), "client_block_share": round(w.cut / w.n_layer, 4),
+            "handoff_bytes_per_round": 2 * M * w.d_model * es + M * 4,
+            "aggregation_bytes_per_client": 2 * per_client, "aggregations_per_round": round(1.0 / agg_interval, 3)}
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["linear", "linear-sweep", "epilogues", "aggregate", "aggregate-sweep", "attention"])
+    ap.add_argument("what", choices=["linear", "linear-sweep", "epilogues", "aggregate", "aggregate-sweep", "attention",
+                                     "split-sweep"])
+    ap.add_argument("--config", type=int, default=3)
     ap.add_argument("--M", type=int, default=32768)
     ap.add_argument("--n-in", type=int, default=1024)
     ap.add_argument("--n-out", type=int, default=3072)
@@ -170,6 +199,15 @@ def main():
             for lg in range(17, 27 if K == 32 else 29, 2):
                 print(json.dumps(bench_aggregate(K, 1 << lg)), flush=True)
         print(json.dumps(dict(bench_aggregate(8, 98304), note="GPT-2-medium-shaped client adapter set")))
+    elif a.what == "split-sweep":
+        from . import synth
+        w = synth.WORKLOADS[a.config]
+        L = w.n_layer
+        cuts = sorted({1, w.cut, L // 4, L // 2, L})
+        for cut in cuts:                                   # split point, the paper's aggregation interval I
+            for I in (1, 10):
+                print(json.dumps(bench_split(a.config, cut, I, w.n_clients, 5)), flush=True)
+        print(json.dumps(dict(bench_split(a.config, w.cut, 1, 1, 5), note="one client: centralised baseline")), flush=True)
     else:
         print(json.dumps(bench_attention(a.nseq, a.T, a.heads, a.iters)))
 

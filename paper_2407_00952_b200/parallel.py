@@ -41,7 +41,8 @@ class ShardedRound:
         engine.set_deferred_server_update(True)
 
     def _sum(self, t: torch.Tensor):
-        dist.all_reduce(t, op=dist.ReduceOp.SUM, group=self.group)
+        if t.numel() > 0:       # no server adapters when every block is client-side
+            dist.all_reduce(t, op=dist.ReduceOp.SUM, group=self.group)
 
     def round(self, tokens, labels, S, dS, local_counts, total_count: int, n_valid_global: int):
         """tokens, labels: this rank's [K_local, b, T]; S, dS: hand-off buffers [K_local, b, T, d];

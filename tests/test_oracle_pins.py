@@ -270,7 +270,7 @@ def test_every_cut_gives_the_unsplit_model():
     layer_ads = ads64(synth.make_adapters(base, range(L), nonzero_b=True, salt=3))
     tokens, labels = synth.make_tokens(base)
     ref = None
-    for cut in range(1, L):
+    for cut in range(1, L + 1):          # cut == L: every block on the clients, the server keeps the head
         w = tiny_workload(n_layer=L, cut=cut)
         cfg = ocfg(w)
         cads = [{k: v for k, v in layer_ads.items() if k[0] < cut} for _ in range(w.n_clients)]
@@ -287,6 +287,35 @@ def test_every_cut_gives_the_unsplit_model():
             for key in per_layer:
                 assert np.allclose(per_layer[key][0], ref[1][key][0], rtol=1e-9, atol=1e-14)
                 assert np.allclose(per_layer[key][1], ref[1][key][1], rtol=1e-9, atol=1e-14)
+
+
+def test_all_blocks_on_clients_is_local_training_per_client():
+    """cut == L is the federated baseline of Sec. IV-A: client i's adapter gradients are those of
+    training the whole model on client i's data alone, up to the ratio of the loss normalisers
+    (the round's loss is one mean over the concatenated batch)."""
+    L = 2
+    w = tiny_workload(n_layer=L, cut=L)
+    cfg = ocfg(w)
+    params, cads, _, tokens, labels = setup(w)
+    labels = labels.copy()
+    labels[1, 0, :3] = -1
+    loss, S, dS, sg, cg = oracle_grads(cfg, params, cads, {}, tokens, labels)
+    assert sg == {}
+    n_all = int((labels >= 0).sum())
+    total = 0.0
+    for i in range(w.n_clients):
+        w1 = tiny_workload(n_layer=L, cut=1, n_clients=1)         # centralised: K = 1, any cut
+        ads = cads[i]
+        li, _, _, sgi, cgi = oracle_grads(ocfg(w1), params, [{k: v for k, v in ads.items() if k[0] < 1}],
+                                          {k: v for k, v in ads.items() if k[0] >= 1}, tokens[i:i + 1], labels[i:i + 1])
+        n_i = int((labels[i] >= 0).sum())
+        total += li * n_i / n_all
+        local = dict(sgi)
+        local.update(cgi[0])
+        for key, (dA, dB) in cg[i].items():
+            assert np.allclose(dA * n_all / n_i, local[key][0], rtol=1e-9, atol=1e-14)
+            assert np.allclose(dB * n_all / n_i, local[key][1], rtol=1e-9, atol=1e-14)
+    assert abs(total - loss) < 1e-12
 
 
 def test_initial_loss_is_ln_vocab():
