@@ -204,11 +204,15 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
           tc_wait_ld();
           if (diag && c == c_last) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (c + i > r) ? -INFINITY : v[i]);
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, v[i]);
+            for (int i = 0; i < 32; ++i) v[i] = (c + i > r) ? -INFINITY : v[i];
           }
+          float m4[4] = {v[0], v[1], v[2], v[3]};          // four short chains instead of one of 32
+#pragma unroll
+          for (int i = 4; i < 32; i += 4) {
+            m4[0] = fmaxf(m4[0], v[i]); m4[1] = fmaxf(m4[1], v[i + 1]);
+            m4[2] = fmaxf(m4[2], v[i + 2]); m4[3] = fmaxf(m4[3], v[i + 3]);
+          }
+          mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
         }
         const float m_new = fmaxf(m_run, mx * p.scale_log2);   // finite: column 0 is never masked
         const float corr = ex2(m_run - m_new);
@@ -221,11 +225,13 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
             float v[32];
             tc_ld32(tS + lane_off + (uint32_t)c, v);
             tc_wait_ld();
-            const bool mask = diag && c == c_last;
+            if (diag && c == c_last) {          // mask on the scores: the element loop stays free of tests
+#pragma unroll
+              for (int i = 0; i < 32; ++i) v[i] = (c + i > r) ? -INFINITY : v[i];
+            }
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
-              float p0 = ex2(fmaf(v[i], p.scale_log2, -m_new)), p1 = ex2(fmaf(v[i + 1], p.scale_log2, -m_new));
-              if (mask) { if (c + i > r) p0 = 0.f; if (c + i + 1 > r) p1 = 0.f; }
+              const float p0 = ex2(fmaf(v[i], p.scale_log2, -m_new)), p1 = ex2(fmaf(v[i + 1], p.scale_log2, -m_new));
               psum += p0 + p1;
               __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
               pk[i >> 1] = *reinterpret_cast<uint32_t*>(&pb);

@@ -237,16 +237,28 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
             tc_ld32(tS + lane_off + (uint32_t)c, sv);
             tc_ld32(tDP + lane_off + (uint32_t)c, dv);
             tc_wait_ld();
-            const bool mask = diag && c == c_first;
+            // The causal mask goes onto the scores first (exp2(-inf) = 0), so that the element loop
+            // below has no test in it: with one, every element is a basic block of its own and the
+            // 32 independent chains run one after another instead of interleaved.
+            if (diag && c == c_first) {
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-              float p0 = ex2(fmaf(sv[e], scale_log2, -Ls[c + e] * LOG2E));
-              float p1 = ex2(fmaf(sv[e + 1], scale_log2, -Ls[c + e + 1] * LOG2E));
-              if (mask) { if (c + e < r) p0 = 0.f; if (c + e + 1 < r) p1 = 0.f; }
-              const float d0 = p0 * (dv[e] - Ds[c + e]), d1 = p1 * (dv[e + 1] - Ds[c + e + 1]);
-              __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1), db = __floats2bfloat162_rn(d0, d1);
-              pk[e >> 1] = *reinterpret_cast<uint32_t*>(&pb);
-              dk[e >> 1] = *reinterpret_cast<uint32_t*>(&db);
+              for (int e = 0; e < 32; ++e) sv[e] = (c + e < r) ? -INFINITY : sv[e];
+            }
+#pragma unroll
+            for (int e = 0; e < 32; e += 4) {
+              const float4 l4 = *reinterpret_cast<const float4*>(Ls + c + e);
+              const float4 d4 = *reinterpret_cast<const float4*>(Ds + c + e);
+              const float p0 = ex2(fmaf(sv[e], scale_log2, -l4.x * LOG2E));
+              const float p1 = ex2(fmaf(sv[e + 1], scale_log2, -l4.y * LOG2E));
+              const float p2 = ex2(fmaf(sv[e + 2], scale_log2, -l4.z * LOG2E));
+              const float p3 = ex2(fmaf(sv[e + 3], scale_log2, -l4.w * LOG2E));
+              __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
+              __nv_bfloat162 da = __floats2bfloat162_rn(p0 * (dv[e] - d4.x), p1 * (dv[e + 1] - d4.y));
+              __nv_bfloat162 db = __floats2bfloat162_rn(p2 * (dv[e + 2] - d4.z), p3 * (dv[e + 3] - d4.w));
+              pk[e >> 1] = *reinterpret_cast<uint32_t*>(&pa);
+              pk[(e >> 1) + 1] = *reinterpret_cast<uint32_t*>(&pb);
+              dk[e >> 1] = *reinterpret_cast<uint32_t*>(&da);
+              dk[(e >> 1) + 1] = *reinterpret_cast<uint32_t*>(&db);
             }
           } else {
 #pragma unroll
@@ -403,11 +415,13 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
             tc_ld32(tS + lane_off + (uint32_t)c, sv);
             tc_ld32(tDP + lane_off + (uint32_t)c, dv);
             tc_wait_ld();
-            const bool mask = diag && c == c_last;
+            if (diag && c == c_last) {          // mask on the scores: the element loop stays free of tests
+#pragma unroll
+              for (int e = 0; e < 32; ++e) sv[e] = (c + e > r) ? -INFINITY : sv[e];
+            }
 #pragma unroll
             for (int e = 0; e < 32; e += 2) {
-              float p0 = ex2(fmaf(sv[e], scale_log2, -L2)), p1 = ex2(fmaf(sv[e + 1], scale_log2, -L2));
-              if (mask) { if (c + e > r) p0 = 0.f; if (c + e + 1 > r) p1 = 0.f; }
+              const float p0 = ex2(fmaf(sv[e], scale_log2, -L2)), p1 = ex2(fmaf(sv[e + 1], scale_log2, -L2));
               __nv_bfloat162 db = __floats2bfloat162_rn(p0 * (dv[e] - Dr), p1 * (dv[e + 1] - Dr));
               dk[e >> 1] = *reinterpret_cast<uint32_t*>(&db);
             }

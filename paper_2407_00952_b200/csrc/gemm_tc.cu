@@ -352,12 +352,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
       int tm, tn; tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
       const int m_warp0 = tm * 2 * BM + (int)rank * BM + q * 32;
       const int n0 = tn * BN;
+      uint4 bfirst[4];
+      load_bias_chunk(p, n0 + c_begin, bfirst);       // in flight while the accumulator is awaited
       if (!mbar_wait(tfull_bar(as), aphase, abort_flag, p.status, 14)) { ok = false; break; }
       if (NEED_R && !mbar_wait(rfull_bar, (uint32_t)tcount & 1u, abort_flag, p.status, 16)) { ok = false; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN);
       epilogue_tile_smem_r(p, t_row, m_warp0, lane, n0, c_begin, c_end, tanh_form, stage, buf, &mapY, &mapZ,
-                           NEED_R ? r_base : 0u, q * 32 + lane);
+                           NEED_R ? r_base : 0u, q * 32 + lane, bfirst);
       if (NEED_R) { __syncwarp(); if (lane == 0) mbar_arrive(rempty_bar); }   // 8 warps release the R buffer
       tc_fence_before();
       __syncwarp();

@@ -149,6 +149,20 @@ __device__ __forceinline__ float tanh_fast(float x) {
   asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// tanh-form GELU and its derivative without a test of the form (see epilogue_chunk)
+__device__ __forceinline__ float gelu_tanh_tc(float z) {
+  const float u = z * fmaf(0.7978845608028654f * 0.044715f, z * z, 0.7978845608028654f);
+  const float hz = 0.5f * z;
+  return fmaf(hz, tanh_fast(u), hz);
+}
+__device__ __forceinline__ float gelu_grad_tanh_tc(float z) {
+  const float z2 = z * z;
+  const float u = z * fmaf(0.7978845608028654f * 0.044715f, z2, 0.7978845608028654f);
+  const float t = tanh_fast(u);
+  const float du = fmaf(0.7978845608028654f * 0.134145f, z2, 0.7978845608028654f);
+  const float hz = 0.5f * z;
+  return fmaf(hz * du, fmaf(-t, t, 1.0f), fmaf(0.5f, t, 0.5f));
+}
 __device__ __forceinline__ float gelu_tc(float z, bool tanh_form) {
   if (tanh_form) {
     float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);
@@ -237,45 +251,74 @@ __device__ __forceinline__ void load_r_chunk(const TcParams& p, int m, int n, ui
   }
 }
 
-// Epilogue of 32 accumulator columns [n, n+32) of row m (= m_warp0 + lane): bias, activation /
-// residual (rpre: the row's second operand, loaded by load_r_chunk), bf16 output through the
-// staging buffers `stage` (this warp's two 2 KB buffers).
-__device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, const uint4* rpre, int n, bool tanh_form,
-                                               uint32_t stage, int& buf, const CUtensorMap* mapY,
+// Bias of columns [n, n+32) (zeros past the last column, or when the layer has none).  Every lane
+// reads the same 64 bytes; issued ahead of its use because nothing hides a global load's latency
+// inside a chunk.
+__device__ __forceinline__ void load_bias_chunk(const TcParams& p, int n, uint4* b) {
+  const bool have = p.bias != nullptr && p.epi != EPI_MUL_GELUGRAD;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (have && n + 8 * j < p.N) b[j] = __ldg(reinterpret_cast<const uint4*>(p.bias + n + 8 * j));
+    else b[j] = make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+
+// Epilogue of 32 accumulator columns [n, n+32) of row m (= m_warp0 + lane): bias (bcur, from
+// load_bias_chunk), activation / residual (rpre: the row's second operand, zero past the last
+// column), bf16 output through the staging buffers `stage` (this warp's two 2 KB buffers).
+// Every per-element loop below is free of branches: the form of the epilogue is tested once per
+// chunk, so that the 32 independent element chains can be interleaved by the instruction scheduler
+// (with a test inside the loop each element is a basic block of its own and runs serially).
+// Columns past N carry garbage that the TMA store clips.
+__device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, const uint4* bcur, const uint4* rpre, int n,
+                                               bool tanh_form, uint32_t stage, int& buf, const CUtensorMap* mapY,
                                                const CUtensorMap* mapZ, int m_warp0, int lane) {
-  if (p.bias && p.epi != EPI_MUL_GELUGRAD) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (n + 8 * j < p.N) {
-        uint4 bw = __ldg(reinterpret_cast<const uint4*>(p.bias + n + 8 * j));
-        const bf16* bp = reinterpret_cast<const bf16*>(&bw);
+  for (int j = 0; j < 4; ++j) {
+    const bf16* bp = reinterpret_cast<const bf16*>(&bcur[j]);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[8 * j + i] += __bfloat162float(bp[i]);
-      }
-    }
+    for (int i = 0; i < 8; ++i) v[8 * j + i] += __bfloat162float(bp[i]);
   }
   uint32_t packed[16];
   if (p.epi == EPI_BIAS_GELU) {
+    float zr[32];                       // the pre-activation as stored (rounded to bf16)
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
       __nv_bfloat162 z2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
       packed[i] = *reinterpret_cast<uint32_t*>(&z2);
-      v[2 * i] = gelu_tc(__low2float(z2), tanh_form);
-      v[2 * i + 1] = gelu_tc(__high2float(z2), tanh_form);
+      zr[2 * i] = __low2float(z2);
+      zr[2 * i + 1] = __high2float(z2);
+    }
+    if (tanh_form) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = gelu_tanh_tc(zr[i]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = gelu_f(zr[i], false);
     }
     stage_and_store(stage + (uint32_t)buf * 2048u, mapZ, packed, lane, n, m_warp0);
     buf ^= 1;
-  } else if (p.epi == EPI_BIAS_RESID || p.epi == EPI_MUL_GELUGRAD) {
+  } else if (p.epi == EPI_BIAS_RESID) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      if (n + 8 * j < p.N) {
+      const bf16* rp = reinterpret_cast<const bf16*>(&rpre[j]);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[8 * j + i] += __bfloat162float(rp[i]);
+    }
+  } else if (p.epi == EPI_MUL_GELUGRAD) {
+    if (tanh_form) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
         const bf16* rp = reinterpret_cast<const bf16*>(&rpre[j]);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          float rv = __bfloat162float(rp[i]);
-          if (p.epi == EPI_BIAS_RESID) v[8 * j + i] += rv;
-          else v[8 * j + i] *= gelu_grad_tc(rv, tanh_form);
-        }
+        for (int i = 0; i < 8; ++i) v[8 * j + i] *= gelu_grad_tanh_tc(__bfloat162float(rp[i]));
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const bf16* rp = reinterpret_cast<const bf16*>(&rpre[j]);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[8 * j + i] *= gelu_grad_f(__bfloat162float(rp[i]), false);
       }
     }
   }
@@ -324,10 +367,12 @@ __device__ __forceinline__ void epilogue_tile(const TcParams& p, uint32_t t_row,
         load_r_chunk(p, m_next + lane, n_next, st.rnext); st.pm = m_next; st.pn = n_next;
       }
     }
+    uint4 bcur[4];
+    load_bias_chunk(p, n, bcur);
     float v[32];
     tc_ld32(t_row + (uint32_t)c, v);
     tc_wait_ld();
-    epilogue_chunk(p, v, rcur, n, tanh_form, stage, st.buf, mapY, mapZ, m_warp0, lane);
+    epilogue_chunk(p, v, bcur, rcur, n, tanh_form, stage, st.buf, mapY, mapZ, m_warp0, lane);
   }
 }
 
@@ -338,11 +383,17 @@ __device__ __forceinline__ void epilogue_tile(const TcParams& p, uint32_t t_row,
 __device__ __forceinline__ void epilogue_tile_smem_r(const TcParams& p, uint32_t t_row, int m_warp0, int lane, int n0,
                                                      int c_begin, int c_end, bool tanh_form, uint32_t stage, int& buf,
                                                      const CUtensorMap* mapY, const CUtensorMap* mapZ, uint32_t rtile,
-                                                     int row) {
+                                                     int row, const uint4* bfirst) {
+  uint4 bcur[4], bnext[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) bnext[j] = bfirst[j];
 #pragma unroll 1
   for (int c = c_begin; c < c_end; c += 32) {
     const int n = n0 + c;
     if (n >= p.N) break;                    // warp-uniform
+#pragma unroll
+    for (int j = 0; j < 4; ++j) bcur[j] = bnext[j];
+    if (c + 32 < c_end) load_bias_chunk(p, n + 32, bnext);
     uint4 rcur[4];
     if (rtile) {
       const uint32_t rrow = rtile + (uint32_t)(c >> 6) * (uint32_t)(BM * BK * 2) + (uint32_t)row * 128u;
@@ -357,7 +408,7 @@ __device__ __forceinline__ void epilogue_tile_smem_r(const TcParams& p, uint32_t
     float v[32];
     tc_ld32(t_row + (uint32_t)c, v);
     tc_wait_ld();
-    epilogue_chunk(p, v, rcur, n, tanh_form, stage, buf, mapY, mapZ, m_warp0, lane);
+    epilogue_chunk(p, v, bcur, rcur, n, tanh_form, stage, buf, mapY, mapZ, m_warp0, lane);
   }
 }
 
