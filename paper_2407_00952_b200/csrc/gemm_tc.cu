@@ -123,23 +123,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
       int stage = 0; uint32_t phase = 0;
       int as = 0; uint32_t aphase = 0;
       bool ok = true;
+      const uint32_t a_lo0 = desc_lo(base);
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         if (!mbar_wait(tempty_bar(as), aphase ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * BN);
-        for (int kb = 0; kb < kb_total; ++kb) {
+        // main contraction: four products per block, issued back to back (advancing 16 elements
+        // along K inside the swizzled row = +32 bytes = +2 in descriptor units)
+        for (int kb = 0; kb < p.num_kb; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
-          const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);
-          int nmma = BK / UMMA_K;
-          if (kb >= p.num_kb && kb == kb_total - 1) nmma = p.ext_last_mmas;
-#pragma unroll 1
-          for (int k = 0; k < nmma; ++k) {
-            // advancing 16 elements along K inside the swizzled row = +32 bytes = +2 in descriptor units
-            tc_mma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), C::IDESC, (kb | k) != 0 ? 1u : 0u);
-          }
+          const uint32_t alo = a_lo0 + (uint32_t)stage * (uint32_t)(C::STAGE_BYTES >> 4);
+          const uint32_t blo = alo + (uint32_t)(C::A_BYTES >> 4);
+          tc_mma_lo(d_tmem, alo, blo, C::IDESC, (uint32_t)kb);
+          tc_mma_lo_acc(d_tmem, alo + 2, blo + 2, C::IDESC);
+          tc_mma_lo_acc(d_tmem, alo + 4, blo + 4, C::IDESC);
+          tc_mma_lo_acc(d_tmem, alo + 6, blo + 6, C::IDESC);
           tc_commit(empty_bar(stage));          // frees the stage once these products have read it
+          if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+        }
+        // rank-r extension: the last block may hold fewer than four products
+        for (int kb = p.num_kb; kb < kb_total && ok; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { ok = false; break; }
+          const uint32_t alo = a_lo0 + (uint32_t)stage * (uint32_t)(C::STAGE_BYTES >> 4);
+          const uint32_t blo = alo + (uint32_t)(C::A_BYTES >> 4);
+          const int nmma = kb == kb_total - 1 ? p.ext_last_mmas : BK / UMMA_K;
+#pragma unroll 1
+          for (int k = 0; k < nmma; ++k) tc_mma_lo_acc(d_tmem, alo + 2 * k, blo + 2 * k, C::IDESC);
+          tc_commit(empty_bar(stage));
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
@@ -316,21 +326,30 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
       int stage = 0; uint32_t phase = 0;
       int as = 0; uint32_t aphase = 0;
       bool ok = true;
+      const uint32_t a_lo0 = desc_lo(base);
       for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
         if (!mbar_wait(tempty_bar(as), aphase ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * BN);
-        for (int kb = 0; kb < kb_total; ++kb) {
+        for (int kb = 0; kb < p.num_kb; ++kb) {    // four products per block, issued back to back
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 13)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
-          const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);
-          int nmma = BK / UMMA_K;
-          if (kb >= p.num_kb && kb == kb_total - 1) nmma = p.ext_last_mmas;
-#pragma unroll 1
-          for (int k = 0; k < nmma; ++k)
-            tc_mma_bf16_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), C::IDESC, (kb | k) != 0 ? 1u : 0u);
+          const uint32_t alo = a_lo0 + (uint32_t)stage * (uint32_t)(C::STAGE_BYTES >> 4);
+          const uint32_t blo = alo + (uint32_t)(C::A_BYTES >> 4);
+          tc_mma_pair_lo(d_tmem, alo, blo, C::IDESC, (uint32_t)kb);
+          tc_mma_pair_lo_acc(d_tmem, alo + 2, blo + 2, C::IDESC);
+          tc_mma_pair_lo_acc(d_tmem, alo + 4, blo + 4, C::IDESC);
+          tc_mma_pair_lo_acc(d_tmem, alo + 6, blo + 6, C::IDESC);
           tc_commit_pair(empty_bar(stage), 3);     // frees the stage in both CTAs
+          if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+        }
+        for (int kb = p.num_kb; kb < kb_total && ok; ++kb) {   // rank-r extension
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 13)) { ok = false; break; }
+          const uint32_t alo = a_lo0 + (uint32_t)stage * (uint32_t)(C::STAGE_BYTES >> 4);
+          const uint32_t blo = alo + (uint32_t)(C::A_BYTES >> 4);
+          const int nmma = kb == kb_total - 1 ? p.ext_last_mmas : BK / UMMA_K;
+#pragma unroll 1
+          for (int k = 0; k < nmma; ++k) tc_mma_pair_lo_acc(d_tmem, alo + 2 * k, blo + 2 * k, C::IDESC);
+          tc_commit_pair(empty_bar(stage), 3);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
