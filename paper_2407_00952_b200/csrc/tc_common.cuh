@@ -47,9 +47,12 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// arrive on a barrier given by a shared::cluster address (own CTA or the peer of a CTA pair)
+// Arrive on a barrier given by a shared::cluster address (own CTA or the peer of a CTA pair).
+// Default (CTA-scope) release: what the arrival publishes are tensor-memory reads, which the
+// tcgen05 fence before it orders.  A cluster-scope release here waited for the warp's output
+// stores in flight, about 2,600 cycles per tile.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
 // shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
@@ -318,11 +321,13 @@ __device__ __forceinline__ void load_bias_chunk(const TcParams& p, int n, uint4*
 __device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, const uint4* bcur, const uint4* rpre, int n,
                                                bool tanh_form, uint32_t stage, int& buf, const CUtensorMap* mapY,
                                                const CUtensorMap* mapZ, int m_warp0, int lane) {
+  if (p.bias != nullptr && p.epi != EPI_MUL_GELUGRAD) {      // warp-uniform; layers without a bias skip 64 instructions
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const bf16* bp = reinterpret_cast<const bf16*>(&bcur[j]);
+    for (int j = 0; j < 4; ++j) {
+      const bf16* bp = reinterpret_cast<const bf16*>(&bcur[j]);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[8 * j + i] += __bfloat162float(bp[i]);
+      for (int i = 0; i < 8; ++i) v[8 * j + i] += __bfloat162float(bp[i]);
+    }
   }
   uint32_t packed[16];
   if (p.epi == EPI_BIAS_GELU) {
