@@ -37,18 +37,10 @@ constexpr float LN2 = 0.6931471805599453f;
 enum { Q_FULL = 0, Q_EMPTY = 1, K_FULL = 2 /*+stage*/, K_EMPTY = 4 /*+stage*/, V_FULL = 6, V_EMPTY = 7,
        S_FULL = 8, S_FREE = 9, P_READY = 10, O_FULL = 11, O_FREE = 12, N_BARS = 13 };
 
-// Shared-memory descriptor of an MN-major operand tile stored as [k rows][64 elements] with
-// 128-byte rows and 128-byte swizzle: groups of 8 k-rows are 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)1 << 16;                        // leading byte offset: unused (one 64-element block along MN)
-  d |= (uint64_t)(1024 >> 4) << 32;              // stride between 8-row groups along K
-  d |= (uint64_t)1 << 46;
-  d |= (uint64_t)2 << 61;                        // 128-byte swizzle
-  return d;
-}
-
+// Operand descriptors are passed to the products as their address-carrying lower halves (desc_lo);
+// the upper half is the same constant for the K-major tiles (Q, K, P) and for V, which is used as
+// loaded ([key, feature] rows = an MN-major right operand with 128-byte rows and 128-byte swizzle,
+// groups of 8 key rows 1024 bytes apart).
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -132,7 +124,9 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       bool ok = true;
-      const uint64_t qdesc = make_smem_desc(base + OFF_Q);
+      const uint32_t lo_q = desc_lo(base + OFF_Q), lo_k0 = desc_lo(base + OFF_K), lo_v = desc_lo(base + OFF_V);
+      const uint32_t lo_p = desc_lo(base + OFF_P);
+      constexpr uint32_t TILE16 = TILE >> 4;
       // S of step `step`; first_of_q: wait for the query tile iq; last_of_q: release the Q buffer
       auto issue_S = [&](int step, int iq, bool first_of_q, bool last_of_q) -> bool {
         const int s = step & 1;
@@ -140,10 +134,11 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         if (!mbar_wait(B(K_FULL + s), (uint32_t)(step >> 1) & 1u, abort_flag, p.status, 23)) return false;
         if (!mbar_wait(B(S_FREE), ((uint32_t)step & 1u) ^ 1u, abort_flag, p.status, 24)) return false;
         tc_fence_after();
-        const uint64_t kdesc = make_smem_desc(base + OFF_K + s * TILE);
-#pragma unroll
-        for (int k = 0; k < DH / UMMA_K; ++k)
-          tc_mma_bf16(tS, qdesc + (uint64_t)(2 * k), kdesc + (uint64_t)(2 * k), IDESC_S, k != 0 ? 1u : 0u);
+        const uint32_t lo_k = lo_k0 + (uint32_t)s * TILE16;
+        tc_mma_lo(tS, lo_q, lo_k, IDESC_S, 0u);              // 16 elements along K = +32 bytes = +2 units
+        tc_mma_lo_acc(tS, lo_q + 2, lo_k + 2, IDESC_S);
+        tc_mma_lo_acc(tS, lo_q + 4, lo_k + 4, IDESC_S);
+        tc_mma_lo_acc(tS, lo_q + 6, lo_k + 6, IDESC_S);
         tc_commit(B(K_EMPTY + s));
         if (last_of_q) tc_commit(B(Q_EMPTY));
         tc_commit(B(S_FULL));
@@ -162,14 +157,12 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
           if (!mbar_wait(B(V_FULL), (uint32_t)it & 1u, abort_flag, p.status, 27)) { ok = false; break; }
           if (!mbar_wait(B(O_FREE), ((uint32_t)it & 1u) ^ 1u, abort_flag, p.status, 28)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t vdesc = make_smem_desc_mn(base + OFF_V);
+          // P is two [128 x 64] K-major blocks (inside a block 16 columns = 32 bytes = 2 units);
+          // V advances 16 key rows = 2048 bytes = 128 units per product
+          tc_mma_lo(tO, lo_p, lo_v, IDESC_PV, 0u);
 #pragma unroll
-          for (int k = 0; k < BKV / UMMA_K; ++k) {
-            // P is two [128 x 64] K-major blocks; inside a block 16 columns = 32 bytes
-            const uint64_t pdesc = make_smem_desc(base + OFF_P + (k >> 2) * TILE) + (uint64_t)(2 * (k & 3));
-            // V advances 16 key rows = 2048 bytes per step
-            tc_mma_bf16(tO, pdesc, vdesc + (uint64_t)(128 * k), IDESC_PV, k != 0 ? 1u : 0u);
-          }
+          for (int k = 1; k < BKV / UMMA_K; ++k)
+            tc_mma_lo_acc(tO, lo_p + (uint32_t)((k >> 2) * (int)TILE16 + 2 * (k & 3)), lo_v + (uint32_t)(128 * k), IDESC_PV);
           tc_commit(B(V_EMPTY));      // V (and P) reusable
           tc_commit(B(O_FULL));       // O' complete
         }

@@ -24,22 +24,14 @@ using namespace tc;
 constexpr int DH = 64;
 constexpr int BT = 128;                   // rows of a query tile and of a key tile
 constexpr int TILE = BT * DH * 2;         // 16 KB: one [128 x 64] bf16 tile
-constexpr int NTHREADS = 320;             // 2 service warps + 8 element-wise warps
+constexpr int NTHREADS = 352;             // TMA warp, two MMA-issuing warps (1 and 10), 8 element-wise warps
+constexpr int ACC_WARP = 10;              // issues the products that accumulate dK, dV / dQ
 constexpr int EW_THREADS = 256;           // two warps per accumulator lane quarter, 64 columns each
 constexpr int TMEM_COLS = 512;
-constexpr uint32_t IDESC_128 = make_idesc(BT, BT);                    // [128 x 128] products, both K-major
+constexpr uint32_t IDESC_64KK = make_idesc(BT, DH);                   // [128 x 64] products, both operands K-major
 constexpr uint32_t IDESC_64MN = make_idesc(BT, DH) | (1u << 16);      // [128 x 64] products, right operand MN-major
 constexpr float LOG2E = 1.4426950408889634f;
 
-__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)1 << 16;
-  d |= (uint64_t)(1024 >> 4) << 32;
-  d |= (uint64_t)1 << 46;
-  d |= (uint64_t)2 << 61;
-  return d;
-}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -66,21 +58,27 @@ __device__ __forceinline__ void st_operand_chunk(uint32_t base2, int r, int c, c
 #pragma unroll
   for (uint32_t jj = 0; jj < 4; ++jj) st_row_chunk(tile, r, cb + jj, pk + 4 * jj);
 }
-// 8 products [128 x 64] += A[128 x 128] (two K-major blocks at a2) * B (MN-major tile at b)
-__device__ __forceinline__ void mma_acc_128x64(uint32_t d_tmem, uint32_t a2, uint32_t b, bool fresh) {
-  const uint64_t bdesc = make_smem_desc_mn(b);
-#pragma unroll
-  for (int k = 0; k < BT / UMMA_K; ++k) {
-    const uint64_t adesc = make_smem_desc(a2 + (k >> 2) * TILE) + (uint64_t)(2 * (k & 3));
-    tc_mma_bf16(d_tmem, adesc, bdesc + (uint64_t)(128 * k), IDESC_64MN, (fresh && k == 0) ? 0u : 1u);
-  }
+// Operand descriptors are passed as their address-carrying lower halves (desc_lo); the upper half
+// is the same constant for the K-major tiles and for the MN-major ones (128-byte rows, 128-byte
+// swizzle, 8-row groups 1024 bytes apart), so a product costs the issuing thread two adds.
+//
+// 4 products [128 x 64] += A-block [128 x 64] (K-major, lower half alo) * B rows [64h, 64h + 64) of an
+// MN-major tile (lower half blo of the tile): one half of the contraction over a 128-row tile.
+__device__ __forceinline__ void mma_acc_half(uint32_t d_tmem, uint32_t alo, uint32_t blo, int h, bool fresh) {
+  const uint32_t b0 = blo + (uint32_t)(512 * h);          // 16 rows of the right operand = 2048 bytes = 128 units
+  tc_mma_lo(d_tmem, alo, b0, IDESC_64MN, fresh ? 0u : 1u);
+  tc_mma_lo_acc(d_tmem, alo + 2, b0 + 128, IDESC_64MN);
+  tc_mma_lo_acc(d_tmem, alo + 4, b0 + 256, IDESC_64MN);
+  tc_mma_lo_acc(d_tmem, alo + 6, b0 + 384, IDESC_64MN);
 }
-// 4 products [128 x 128] = A[128 x 64] * B[128 x 64]^T, both K-major
-__device__ __forceinline__ void mma_128x128(uint32_t d_tmem, uint32_t a, uint32_t b) {
-  const uint64_t adesc = make_smem_desc(a), bdesc = make_smem_desc(b);
-#pragma unroll
-  for (int k = 0; k < DH / UMMA_K; ++k)
-    tc_mma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), IDESC_128, k != 0 ? 1u : 0u);
+// 4 products [128 x 64] = A[128 x 64] * (rows [64h, 64h + 64) of the K-major tile at blo)^T:
+// one half (64 columns) of a [128 x 128] score tile.  64 rows of 128 bytes = 512 descriptor units.
+__device__ __forceinline__ void mma_score_half(uint32_t d_tmem, uint32_t alo, uint32_t blo, int h) {
+  const uint32_t b0 = blo + (uint32_t)(512 * h);
+  tc_mma_lo(d_tmem, alo, b0, IDESC_64KK, 0u);
+  tc_mma_lo_acc(d_tmem, alo + 2, b0 + 2, IDESC_64KK);
+  tc_mma_lo_acc(d_tmem, alo + 4, b0 + 4, IDESC_64KK);
+  tc_mma_lo_acc(d_tmem, alo + 6, b0 + 6, IDESC_64KK);
 }
 
 struct BwdParams {
@@ -91,7 +89,7 @@ struct BwdParams {
   int* status;
 };
 
-#define T5_SETUP(NBARS, CNT128_A, CNT128_B, CNT128_C)                                                     \
+#define T5_SETUP(NBARS, CNT128_A, CNT128_B, CNT128_C, CNT128_D, CNT128_E, CNT2_A, CNT2_B)                                                     \
   extern __shared__ uint8_t smem_raw[];                                                                   \
   const uint32_t raw = smem_u32(smem_raw);                                                                \
   const uint32_t base = (raw + 1023u) & ~1023u;                                                           \
@@ -103,7 +101,8 @@ struct BwdParams {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;                                             \
   if (threadIdx.x == 0) {                                                                                 \
     for (int i = 0; i < NBARS; ++i)                                                                       \
-      mbar_init(B(i), (i == CNT128_A || i == CNT128_B || i == CNT128_C) ? EW_THREADS : 1);                \
+      mbar_init(B(i), (i == CNT128_A || i == CNT128_B || i == CNT128_C || i == CNT128_D || i == CNT128_E) ? EW_THREADS \
+                      : (i == CNT2_A || i == CNT2_B) ? 2 : 1);                                            \
     *abort_flag = 0;                                                                                      \
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");                                    \
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");                                          \
@@ -137,8 +136,8 @@ __device__ __forceinline__ uint32_t freed(int n) { return ((uint32_t)n & 1u) ^ 1
 // dK, dV
 // ==========================================================================================
 namespace dkv {
-enum { KV_FULL = 0, KV_EMPTY, QD_FULL /*+s*/, QD_FULL1, QD_EMPTY /*+s*/, QD_EMPTY1, S_FULL, S_FREE, P_READY, P_FREE,
-       ACC_FULL, ACC_FREE, N_BARS };
+enum { KV_FULL = 0, KV_EMPTY, QD_FULL /*+s*/, QD_FULL1, QD_EMPTY /*+s*/, QD_EMPTY1, S_FULL /*+half*/, S_FULL1,
+       S_FREE /*+half*/, S_FREE1, P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, N_BARS };
 constexpr int OFF_K = 0, OFF_V = TILE, OFF_QD = 2 * TILE /* stage s: Q at +s*2*TILE, dO after it */,
               OFF_PT = 6 * TILE, OFF_DST = 8 * TILE, OFF_STAT = 10 * TILE /* stage s: lse at +s*1024, D at +512 */,
               OFF_BAR = 10 * TILE + 2048;
@@ -149,7 +148,7 @@ __global__ void __launch_bounds__(NTHREADS, 1)
 attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
                        const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dkv;
-  T5_SETUP(N_BARS, S_FREE, P_READY, ACC_FREE)
+  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, QD_EMPTY, QD_EMPTY1)
   const int h = blockIdx.x, b = blockIdx.y;
   const int nq = p.T / BT;
   const int seq_row0 = b * p.T;
@@ -177,41 +176,66 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       }
     }
   } else if (warp == 1) {
+    // ---------------- score products: S^T = K Q^T, dP^T = V dO^T ----------------
+    // Half hh (64 query columns) of a step needs the step's Q/dO stage and the previous step's reads
+    // of that half done.  The halves are separate products so that the next step's first half is
+    // computed while the element-wise warps still work on this step's second.  The accumulating
+    // products are issued by another thread (warp ACC_WARP): one thread cannot issue 32 products of
+    // 48 cycles each per step next to eight busy element-wise warps.
     if (lane == 0) {
       bool ok = true;
       int it = 0;
-      // S^T and dP^T of step `step` (needs its Q/dO stage and the previous step's reads of S^T, dP^T done)
-      auto issue_SdP = [&](int step) -> bool {
-        const int s = step & 1;
-        if (!mbar_wait(B(QD_FULL + s), done(step >> 1), abort_flag, p.status, 43)) return false;
-        if (!mbar_wait(B(S_FREE), freed(step), abort_flag, p.status, 44)) return false;
-        tc_fence_after();
-        mma_128x128(tS, base + OFF_K, base + OFF_QD + s * 2 * TILE);
-        mma_128x128(tDP, base + OFF_V, base + OFF_QD + s * 2 * TILE + TILE);
-        tc_commit(B(S_FULL));
-        return true;
-      };
+      const uint32_t lo_k = desc_lo(base + OFF_K), lo_v = desc_lo(base + OFF_V), lo_qd = desc_lo(base + OFF_QD);
+      constexpr uint32_t TILE16 = TILE >> 4;
       for (int kt = 0; kt < nq && ok; ++kt) {
-        const int steps = nq - kt;
         if (!mbar_wait(B(KV_FULL), done(kt), abort_flag, p.status, 45)) { ok = false; break; }
-        if (!mbar_wait(B(ACC_FREE), freed(kt), abort_flag, p.status, 46)) { ok = false; break; }
-        if (!issue_SdP(it)) { ok = false; break; }
-        for (int st = 0; st < steps; ++st, ++it) {
-          if (st + 1 < steps && !issue_SdP(it + 1)) { ok = false; break; }
-          if (!mbar_wait(B(P_READY), done(it), abort_flag, p.status, 47)) { ok = false; break; }
-          tc_fence_after();
+        for (int i = kt; i < nq && ok; ++i, ++it) {
           const int s = it & 1;
-          mma_acc_128x64(tDV, base + OFF_PT, base + OFF_QD + s * 2 * TILE + TILE, st == 0);   // dV += P^T dO
-          mma_acc_128x64(tDK, base + OFF_DST, base + OFF_QD + s * 2 * TILE, st == 0);         // dK += dS^T Q
-          tc_commit(B(P_FREE));
-          tc_commit(B(QD_EMPTY + s));
-          if (st + 1 == steps) { tc_commit(B(ACC_FULL)); tc_commit(B(KV_EMPTY)); }
+          const uint32_t lo_q = lo_qd + (uint32_t)s * 2u * TILE16;
+          if (!mbar_wait(B(QD_FULL + s), done(it >> 1), abort_flag, p.status, 43)) { ok = false; break; }
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            if (!mbar_wait(B(S_FREE + hh), freed(it), abort_flag, p.status, 44)) { ok = false; break; }
+            tc_fence_after();
+            mma_score_half(tS + 64u * hh, lo_k, lo_q, hh);
+            mma_score_half(tDP + 64u * hh, lo_v, lo_q + TILE16, hh);
+            tc_commit(B(S_FULL + hh));
+          }
+          if (ok) tc_commit(B(QD_EMPTY + s));        // second arrival comes from the accumulating thread
         }
+        if (ok) tc_commit(B(KV_EMPTY));              // K, V are read by these products only
+      }
+    }
+  } else if (warp == ACC_WARP) {
+    // ---------------- accumulating products: dV += P^T dO, dK += dS^T Q ----------------
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0;
+      const uint32_t lo_qd = desc_lo(base + OFF_QD), lo_pt = desc_lo(base + OFF_PT), lo_dst = desc_lo(base + OFF_DST);
+      constexpr uint32_t TILE16 = TILE >> 4;
+      for (int kt = 0; kt < nq && ok; ++kt) {
+        // the accumulators of the previous key tile must have been read
+        if (!mbar_wait(B(ACC_FREE), freed(kt), abort_flag, p.status, 46)) { ok = false; break; }
+        for (int i = kt; i < nq && ok; ++i, ++it) {
+          const int s = it & 1;
+          const uint32_t lo_q = lo_qd + (uint32_t)s * 2u * TILE16, lo_do = lo_q + TILE16;
+          if (!mbar_wait(B(QD_FULL + s), done(it >> 1), abort_flag, p.status, 43)) { ok = false; break; }
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            if (!mbar_wait(B(P_READY + hh), done(it), abort_flag, p.status, 47)) { ok = false; break; }
+            tc_fence_after();
+            mma_acc_half(tDV, lo_pt + (uint32_t)hh * TILE16, lo_do, hh, i == kt && hh == 0);
+            mma_acc_half(tDK, lo_dst + (uint32_t)hh * TILE16, lo_q, hh, i == kt && hh == 0);
+            tc_commit(B(P_FREE + hh));
+          }
+          if (ok) tc_commit(B(QD_EMPTY + s));
+        }
+        if (ok) tc_commit(B(ACC_FULL));
       }
     }
   } else {
     const int q4 = warp & 3;
-    const int c_lo = ((warp - 2) >> 2) * 64;     // this warp's 64 of the 128 score columns
+    const int wsel = (warp - 2) >> 2;            // which of the two warps of this accumulator lane quarter
     const int r = q4 * 32 + lane;                // key row inside the tile = accumulator lane
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     const float scale_log2 = p.scale * LOG2E;
@@ -223,14 +247,17 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
         const float* Ls = reinterpret_cast<const float*>(base_ptr + OFF_STAT + s * 1024);
         const float* Ds = Ls + 128;
         if (!mbar_wait(B(QD_FULL + s), done(it >> 1), abort_flag, p.status, 48)) { ok = false; break; }
-        if (!mbar_wait(B(S_FULL), done(it), abort_flag, p.status, 49)) { ok = false; break; }
-        if (!mbar_wait(B(P_FREE), freed(it), abort_flag, p.status, 50)) { ok = false; break; }
-        tc_fence_after();
         const bool diag = (i == kt);
         // on the diagonal tile only queries >= this key count: chunks wholly before the warp's rows are zero
         const int c_first = diag ? q4 * 32 : 0;
+        // The 128 query columns go in two halves of 64 (one 32-column chunk per warp and half): the
+        // products that contract over the first half run while the second half is being computed.
 #pragma unroll 1
-        for (int c = c_lo; c < c_lo + 64; c += 32) {
+        for (int hh = 0; hh < 2; ++hh) {
+          const int c = hh * 64 + wsel * 32;
+          if (!mbar_wait(B(S_FULL + hh), done(it), abort_flag, p.status, 49)) { ok = false; break; }
+          if (!mbar_wait(B(P_FREE + hh), freed(it), abort_flag, p.status, 50)) { ok = false; break; }
+          tc_fence_after();
           uint32_t pk[16], dk[16];
           if (c >= c_first) {
             float sv[32], dv[32];
@@ -266,18 +293,19 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
           }
           st_operand_chunk(base + OFF_PT, r, c, pk);
           st_operand_chunk(base + OFF_DST, r, c, dk);
+          tc_fence_before();
+          mbar_arrive(B(S_FREE + hh));                 // this half of S^T, dP^T may be overwritten
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          mbar_arrive(B(P_READY + hh));                // this half of P^T, dS^T is visible to the tensor core
         }
-        tc_fence_before();
-        mbar_arrive(B(S_FREE));
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(B(P_READY));
+        if (!ok) break;
       }
       // dK (scaled) and dV of this key tile: tensor memory -> bf16 -> staged in the P^T buffer -> TMA stores
       if (ok && !mbar_wait(B(ACC_FULL), done(kt), abort_flag, p.status, 51)) ok = false;
       if (ok) {
         tc_fence_after();
         {
-          const int half = c_lo >> 6;                  // warps of the first half write dK, the others dV
+          const int half = wsel;                       // the first warp of a lane quarter writes dK, the other dV
           const uint32_t tsrc = half == 0 ? tDK : tDV;
           const float mul = half == 0 ? p.scale : 1.0f;
 #pragma unroll
@@ -319,8 +347,8 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
 // dQ
 // ==========================================================================================
 namespace dq {
-enum { QO_FULL = 0, QO_EMPTY, KV_FULL /*+s*/, KV_FULL1, KV_EMPTY /*+s*/, KV_EMPTY1, S_FULL, S_FREE, P_READY, P_FREE,
-       ACC_FULL, ACC_FREE, N_BARS };
+enum { QO_FULL = 0, QO_EMPTY, KV_FULL /*+s*/, KV_FULL1, KV_EMPTY /*+s*/, KV_EMPTY1, S_FULL /*+half*/, S_FULL1,
+       S_FREE /*+half*/, S_FREE1, P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, N_BARS };
 constexpr int OFF_Q = 0, OFF_DO = TILE, OFF_KV = 2 * TILE /* stage s: K at +s*2*TILE, V after it */,
               OFF_DS = 6 * TILE, OFF_BAR = 8 * TILE;
 constexpr int SMEM = OFF_BAR + 256 + 1024;
@@ -330,7 +358,7 @@ __global__ void __launch_bounds__(NTHREADS, 1)
 attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
                       const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dq;
-  T5_SETUP(N_BARS, S_FREE, P_READY, ACC_FREE)
+  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, KV_EMPTY, KV_EMPTY1)
   const int h = blockIdx.x, b = blockIdx.y;
   const int nq = p.T / BT;
   const int seq_row0 = b * p.T;
@@ -358,39 +386,61 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       }
     }
   } else if (warp == 1) {
+    // ---------------- score products: S = Q K^T, dP = dO V^T, in halves of 64 key columns ----------------
     if (lane == 0) {
       bool ok = true;
       int it = 0;
-      auto issue_SdP = [&](int step) -> bool {
-        const int s = step & 1;
-        if (!mbar_wait(B(KV_FULL + s), done(step >> 1), abort_flag, p.status, 63)) return false;
-        if (!mbar_wait(B(S_FREE), freed(step), abort_flag, p.status, 64)) return false;
-        tc_fence_after();
-        mma_128x128(tS, base + OFF_Q, base + OFF_KV + s * 2 * TILE);                // S  = Q K^T
-        mma_128x128(tDP, base + OFF_DO, base + OFF_KV + s * 2 * TILE + TILE);       // dP = dO V^T
-        tc_commit(B(S_FULL));
-        return true;
-      };
+      const uint32_t lo_q = desc_lo(base + OFF_Q), lo_do = desc_lo(base + OFF_DO), lo_kv = desc_lo(base + OFF_KV);
+      constexpr uint32_t TILE16 = TILE >> 4;
       for (int qi = 0; qi < nq && ok; ++qi) {
         const int steps = nq - qi;               // key tiles 0 .. i, i = nq-1-qi
         if (!mbar_wait(B(QO_FULL), done(qi), abort_flag, p.status, 65)) { ok = false; break; }
-        if (!mbar_wait(B(ACC_FREE), freed(qi), abort_flag, p.status, 66)) { ok = false; break; }
-        if (!issue_SdP(it)) { ok = false; break; }
-        for (int st = 0; st < steps; ++st, ++it) {
-          if (st + 1 < steps && !issue_SdP(it + 1)) { ok = false; break; }
-          if (!mbar_wait(B(P_READY), done(it), abort_flag, p.status, 67)) { ok = false; break; }
-          tc_fence_after();
+        for (int st = 0; st < steps && ok; ++st, ++it) {
           const int s = it & 1;
-          mma_acc_128x64(tDQ, base + OFF_DS, base + OFF_KV + s * 2 * TILE, st == 0);     // dQ += dS K
-          tc_commit(B(P_FREE));
-          tc_commit(B(KV_EMPTY + s));
-          if (st + 1 == steps) { tc_commit(B(ACC_FULL)); tc_commit(B(QO_EMPTY)); }
+          const uint32_t lo_k = lo_kv + (uint32_t)s * 2u * TILE16;
+          if (!mbar_wait(B(KV_FULL + s), done(it >> 1), abort_flag, p.status, 63)) { ok = false; break; }
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            if (!mbar_wait(B(S_FREE + hh), freed(it), abort_flag, p.status, 64)) { ok = false; break; }
+            tc_fence_after();
+            mma_score_half(tS + 64u * hh, lo_q, lo_k, hh);
+            mma_score_half(tDP + 64u * hh, lo_do, lo_k + TILE16, hh);
+            tc_commit(B(S_FULL + hh));
+          }
+          if (ok) tc_commit(B(KV_EMPTY + s));        // second arrival comes from the accumulating thread
         }
+        if (ok) tc_commit(B(QO_EMPTY));              // Q, dO are read by these products only
+      }
+    }
+  } else if (warp == ACC_WARP) {
+    // ---------------- accumulating products: dQ += dS K ----------------
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0;
+      const uint32_t lo_kv = desc_lo(base + OFF_KV), lo_ds = desc_lo(base + OFF_DS);
+      constexpr uint32_t TILE16 = TILE >> 4;
+      for (int qi = 0; qi < nq && ok; ++qi) {
+        const int steps = nq - qi;
+        if (!mbar_wait(B(ACC_FREE), freed(qi), abort_flag, p.status, 66)) { ok = false; break; }
+        for (int st = 0; st < steps && ok; ++st, ++it) {
+          const int s = it & 1;
+          const uint32_t lo_k = lo_kv + (uint32_t)s * 2u * TILE16;
+          if (!mbar_wait(B(KV_FULL + s), done(it >> 1), abort_flag, p.status, 63)) { ok = false; break; }
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            if (!mbar_wait(B(P_READY + hh), done(it), abort_flag, p.status, 67)) { ok = false; break; }
+            tc_fence_after();
+            mma_acc_half(tDQ, lo_ds + (uint32_t)hh * TILE16, lo_k, hh, st == 0 && hh == 0);
+            tc_commit(B(P_FREE + hh));
+          }
+          if (ok) tc_commit(B(KV_EMPTY + s));
+        }
+        if (ok) tc_commit(B(ACC_FULL));
       }
     }
   } else {
     const int q4 = warp & 3;
-    const int c_lo = ((warp - 2) >> 2) * 64;     // this warp's 64 of the 128 score columns
+    const int wsel = (warp - 2) >> 2;            // which of the two warps of this accumulator lane quarter
     const int r = q4 * 32 + lane;                // query row inside the tile
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     const float scale_log2 = p.scale * LOG2E;
@@ -401,14 +451,15 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       const float L2 = p.lse[stat0 + (size_t)i * BT + r] * LOG2E;
       const float Dr = p.rowdot[stat0 + (size_t)i * BT + r];
       for (int j = 0; j <= i && ok; ++j, ++it) {
-        if (!mbar_wait(B(S_FULL), done(it), abort_flag, p.status, 68)) { ok = false; break; }
-        if (!mbar_wait(B(P_FREE), freed(it), abort_flag, p.status, 69)) { ok = false; break; }
-        tc_fence_after();
         const bool diag = (j == i);
         // on the diagonal tile only keys <= this query count: chunks wholly after the warp's rows are zero
         const int c_last = diag ? q4 * 32 : BT - 32;
 #pragma unroll 1
-        for (int c = c_lo; c < c_lo + 64; c += 32) {
+        for (int hh = 0; hh < 2; ++hh) {
+          const int c = hh * 64 + wsel * 32;
+          if (!mbar_wait(B(S_FULL + hh), done(it), abort_flag, p.status, 68)) { ok = false; break; }
+          if (!mbar_wait(B(P_FREE + hh), freed(it), abort_flag, p.status, 69)) { ok = false; break; }
+          tc_fence_after();
           uint32_t dk[16];
           if (c <= c_last) {
             float sv[32], dv[32];
@@ -430,17 +481,18 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
             for (int e = 0; e < 16; ++e) dk[e] = 0u;
           }
           st_operand_chunk(base + OFF_DS, r, c, dk);
+          tc_fence_before();
+          mbar_arrive(B(S_FREE + hh));
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          mbar_arrive(B(P_READY + hh));
         }
-        tc_fence_before();
-        mbar_arrive(B(S_FREE));
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(B(P_READY));
+        if (!ok) break;
       }
       if (ok && !mbar_wait(B(ACC_FULL), done(qi), abort_flag, p.status, 70)) ok = false;
       if (ok) {
         tc_fence_after();
         {
-          const int c = c_lo >> 1;                     // each of the two warps of a lane quarter takes 32 of the 64 columns
+          const int c = wsel * 32;                     // each of the two warps of a lane quarter takes 32 of the 64 columns
           float v[32];
           tc_ld32(tDQ + lane_off + (uint32_t)c, v);
           tc_wait_ld();
