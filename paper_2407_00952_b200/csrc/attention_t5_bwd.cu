@@ -4,8 +4,10 @@
 //   attn_bwd_dkv_t5_kernel   one CTA per (sequence, head); for each 128-row key tile it walks the
 //       query tiles i >= key tile and keeps dK, dV as fp32 accumulators in tensor memory:
 //         S^T = K Q^T, dP^T = V dO^T                (M128 N128 K16 x4 each, operands K-major)
-//         P^T = exp(S^T/sqrt(dh) - lse[q]),  dS^T = P^T (dP^T - D[q])      (one thread per key row)
-//         dV += P^T dO,  dK += dS^T Q               (M128 N64 K16 x8 each; dO, Q used as loaded:
+//         P^T = exp(S^T/sqrt(dh) - lse[q]),  dS^T = P^T (dP^T - D[q])      (one thread per key row; the
+//                                                    results go back to tensor memory as bf16)
+//         dV += P^T dO,  dK += dS^T Q               (M128 N64 K16 x8 each; left operand read from
+//                                                    tensor memory, dO and Q used as loaded:
 //                                                    MN-major right operands)
 //   attn_bwd_dq_t5_kernel    one CTA per (sequence, head); for each 128-row query tile it walks the
 //       key tiles j <= query tile and keeps dQ in tensor memory:
@@ -50,26 +52,20 @@ __device__ __forceinline__ void st_row_chunk(uint32_t tile, int r, uint32_t jj, 
   const uint32_t addr = tile + (uint32_t)r * 128u + ((jj ^ ((uint32_t)r & 7u)) << 4);
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
 }
-// 32 bf16 values (16 packed words) of row r, columns [c, c+32) of a [128 x 128] operand kept as two
-// [128 x 64] K-major blocks
-__device__ __forceinline__ void st_operand_chunk(uint32_t base2, int r, int c, const uint32_t* pk) {
-  const uint32_t tile = base2 + (uint32_t)(c >> 6) * TILE;
-  const uint32_t cb = (uint32_t)((c & 63) >> 3);
-#pragma unroll
-  for (uint32_t jj = 0; jj < 4; ++jj) st_row_chunk(tile, r, cb + jj, pk + 4 * jj);
-}
 // Operand descriptors are passed as their address-carrying lower halves (desc_lo); the upper half
 // is the same constant for the K-major tiles and for the MN-major ones (128-byte rows, 128-byte
 // swizzle, 8-row groups 1024 bytes apart), so a product costs the issuing thread two adds.
 //
-// 4 products [128 x 64] += A-block [128 x 64] (K-major, lower half alo) * B rows [64h, 64h + 64) of an
-// MN-major tile (lower half blo of the tile): one half of the contraction over a 128-row tile.
-__device__ __forceinline__ void mma_acc_half(uint32_t d_tmem, uint32_t alo, uint32_t blo, int h, bool fresh) {
-  const uint32_t b0 = blo + (uint32_t)(512 * h);          // 16 rows of the right operand = 2048 bytes = 128 units
-  tc_mma_lo(d_tmem, alo, b0, IDESC_64MN, fresh ? 0u : 1u);
-  tc_mma_lo_acc(d_tmem, alo + 2, b0 + 128, IDESC_64MN);
-  tc_mma_lo_acc(d_tmem, alo + 4, b0 + 256, IDESC_64MN);
-  tc_mma_lo_acc(d_tmem, alo + 6, b0 + 384, IDESC_64MN);
+// 4 products [128 x 64] += A[:, 64h .. 64h+63] * B rows [64h, 64h + 64): one half of the contraction
+// over a 128-row tile.  A (P^T, dS^T or dS, bf16) lives in tensor memory at a_tmem: 128 contraction
+// elements = 64 columns, so half h starts 32 columns in and each product advances 8 columns.  B is an
+// MN-major tile used as loaded (lower descriptor half blo); 16 of its rows = 2048 bytes = 128 units.
+__device__ __forceinline__ void mma_acc_half(uint32_t d_tmem, uint32_t a_tmem, uint32_t blo, int h, bool fresh) {
+  const uint32_t a0 = a_tmem + (uint32_t)(32 * h), b0 = blo + (uint32_t)(512 * h);
+  tc_mma_ts_lo(d_tmem, a0, b0, IDESC_64MN, fresh ? 0u : 1u);
+  tc_mma_ts_lo(d_tmem, a0 + 8, b0 + 128, IDESC_64MN, 1u);
+  tc_mma_ts_lo(d_tmem, a0 + 16, b0 + 256, IDESC_64MN, 1u);
+  tc_mma_ts_lo(d_tmem, a0 + 24, b0 + 384, IDESC_64MN, 1u);
 }
 // 4 products [128 x 64] = A[128 x 64] * (rows [64h, 64h + 64) of the K-major tile at blo)^T:
 // one half (64 columns) of a [128 x 128] score tile.  64 rows of 128 bytes = 512 descriptor units.
@@ -154,6 +150,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
   const int seq_row0 = b * p.T;
   const size_t stat0 = ((size_t)b * p.H + h) * p.T;
   const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDV = tmem_base + 256u, tDK = tmem_base + 320u;
+  const uint32_t tPT = tmem_base + 384u, tDST = tmem_base + 448u;     // P^T, dS^T: bf16, 64 columns each
 
   if (warp == 0) {
     if (lane == 0) {
@@ -211,7 +208,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     if (lane == 0) {
       bool ok = true;
       int it = 0;
-      const uint32_t lo_qd = desc_lo(base + OFF_QD), lo_pt = desc_lo(base + OFF_PT), lo_dst = desc_lo(base + OFF_DST);
+      const uint32_t lo_qd = desc_lo(base + OFF_QD);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int kt = 0; kt < nq && ok; ++kt) {
         // the accumulators of the previous key tile must have been read
@@ -224,8 +221,8 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
           for (int hh = 0; hh < 2; ++hh) {
             if (!mbar_wait(B(P_READY + hh), done(it), abort_flag, p.status, 47)) { ok = false; break; }
             tc_fence_after();
-            mma_acc_half(tDV, lo_pt + (uint32_t)hh * TILE16, lo_do, hh, i == kt && hh == 0);
-            mma_acc_half(tDK, lo_dst + (uint32_t)hh * TILE16, lo_q, hh, i == kt && hh == 0);
+            mma_acc_half(tDV, tPT, lo_do, hh, i == kt && hh == 0);
+            mma_acc_half(tDK, tDST, lo_q, hh, i == kt && hh == 0);
             tc_commit(B(P_FREE + hh));
           }
           if (ok) tc_commit(B(QD_EMPTY + s));
@@ -291,12 +288,12 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
 #pragma unroll
             for (int e = 0; e < 16; ++e) { pk[e] = 0u; dk[e] = 0u; }
           }
-          st_operand_chunk(base + OFF_PT, r, c, pk);
-          st_operand_chunk(base + OFF_DST, r, c, dk);
+          tc_st16(tPT + lane_off + (uint32_t)(c >> 1), pk);      // 32 bf16 = 16 columns
+          tc_st16(tDST + lane_off + (uint32_t)(c >> 1), dk);
+          tc_wait_st();
           tc_fence_before();
           mbar_arrive(B(S_FREE + hh));                 // this half of S^T, dP^T may be overwritten
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          mbar_arrive(B(P_READY + hh));                // this half of P^T, dS^T is visible to the tensor core
+          mbar_arrive(B(P_READY + hh));                // this half of P^T, dS^T is complete
         }
         if (!ok) break;
       }
@@ -364,6 +361,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
   const int seq_row0 = b * p.T;
   const size_t stat0 = ((size_t)b * p.H + h) * p.T;
   const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDQ = tmem_base + 256u;
+  const uint32_t tDS = tmem_base + 320u;                               // dS: bf16, 64 columns
 
   // query tiles are walked from the last (most key tiles) to the first
   if (warp == 0) {
@@ -417,7 +415,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
     if (lane == 0) {
       bool ok = true;
       int it = 0;
-      const uint32_t lo_kv = desc_lo(base + OFF_KV), lo_ds = desc_lo(base + OFF_DS);
+      const uint32_t lo_kv = desc_lo(base + OFF_KV);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int qi = 0; qi < nq && ok; ++qi) {
         const int steps = nq - qi;
@@ -430,7 +428,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
           for (int hh = 0; hh < 2; ++hh) {
             if (!mbar_wait(B(P_READY + hh), done(it), abort_flag, p.status, 67)) { ok = false; break; }
             tc_fence_after();
-            mma_acc_half(tDQ, lo_ds + (uint32_t)hh * TILE16, lo_k, hh, st == 0 && hh == 0);
+            mma_acc_half(tDQ, tDS, lo_k, hh, st == 0 && hh == 0);
             tc_commit(B(P_FREE + hh));
           }
           if (ok) tc_commit(B(KV_EMPTY + s));
@@ -480,10 +478,10 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
 #pragma unroll
             for (int e = 0; e < 16; ++e) dk[e] = 0u;
           }
-          st_operand_chunk(base + OFF_DS, r, c, dk);
+          tc_st16(tDS + lane_off + (uint32_t)(c >> 1), dk);
+          tc_wait_st();
           tc_fence_before();
           mbar_arrive(B(S_FREE + hh));
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           mbar_arrive(B(P_READY + hh));
         }
         if (!ok) break;

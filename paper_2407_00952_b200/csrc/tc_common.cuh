@@ -178,6 +178,24 @@ __device__ __forceinline__ void tc_mma_pair_lo_acc(uint32_t d_tmem, uint32_t alo
       "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}"
       ::"r"(d_tmem), "r"(alo), "r"(blo), "r"(DESC_HI), "r"(idesc) : "memory");
 }
+// Left operand taken from tensor memory (row = lane, two bf16 per 32-bit column, 16 elements of K
+// = 8 columns), right operand from shared memory through its descriptor's lower half.
+__device__ __forceinline__ void tc_mma_ts_lo(uint32_t d_tmem, uint32_t a_tmem, uint32_t blo, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(blo), "r"(DESC_HI), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 16 packed words of this thread's lane to 16 consecutive tensor-memory columns
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* w) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]),
+        "r"(w[8]), "r"(w[9]), "r"(w[10]), "r"(w[11]), "r"(w[12]), "r"(w[13]), "r"(w[14]), "r"(w[15]) : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
   uint32_t* r = reinterpret_cast<uint32_t*>(v);
   asm volatile(
