@@ -6,9 +6,9 @@
 // the softmax of one overlaps the products of the other.  Per 128-row key tile:
 //   S  = Q K^T      tcgen05.mma M128 N128 K16 x4, both operands K-major from TMA-swizzled tiles
 //   softmax         one thread per query row reads S from tensor memory (twice: row max, then
-//                   exponentials), keeps the running max / sum, writes P (bf16) to shared memory
-//   O' = P V        tcgen05.mma M128 N64 K16 x8; V is used as loaded ([key, feature] rows, i.e. an
-//                   MN-major operand), no transpose
+//                   exponentials), keeps the running max / sum, writes P (bf16) back to tensor memory
+//   O' = P V        tcgen05.mma M128 N64 K16 x8, P read from tensor memory; V is used as loaded
+//                   ([key, feature] rows, i.e. an MN-major operand), no transpose
 //   O  = O*corr+O'  in registers of the row's thread
 // Warp roles (192 threads): warp 0 TMA producer, warp 1 tensor-memory owner + MMA issuer,
 // warps 2..5 softmax (warp w owns accumulator lanes 32*(w%4)..+31).
@@ -25,9 +25,9 @@ constexpr int BQ = 128;                   // query rows per tile
 constexpr int BKV = 128;                  // key rows per step
 constexpr int TILE = BQ * DH * 2;         // 16 KB: one [128 x 64] bf16 tile
 constexpr int T5_THREADS = 192;
-constexpr int OFF_Q = 0, OFF_K = TILE, OFF_V = 3 * TILE, OFF_P = 4 * TILE, OFF_BAR = 6 * TILE;
-constexpr int T5_SMEM = 6 * TILE + 256 + 1024;     // tiles + barriers + alignment slack
-constexpr int TMEM_COLS = 256;            // S at columns [0,128), O' at [128,192)
+constexpr int OFF_Q = 0, OFF_K = TILE, OFF_V = 3 * TILE, OFF_P = 4 * TILE /* staging of the output tile */, OFF_BAR = 5 * TILE;
+constexpr int T5_SMEM = 5 * TILE + 256 + 1024;     // tiles + barriers + alignment slack
+constexpr int TMEM_COLS = 256;            // S at columns [0,128), O' at [128,192), P (bf16) at [192,256)
 constexpr uint32_t IDESC_S = make_idesc(BQ, BKV);
 constexpr uint32_t IDESC_PV = make_idesc(BQ, DH) | (1u << 16);   // B operand MN-major
 constexpr float LOG2E = 1.4426950408889634f;
@@ -88,7 +88,7 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tS = tmem_base, tO = tmem_base + 128u;
+  const uint32_t tS = tmem_base, tO = tmem_base + 128u, tP = tmem_base + 192u;
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -125,7 +125,6 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
     if (lane == 0) {
       bool ok = true;
       const uint32_t lo_q = desc_lo(base + OFF_Q), lo_k0 = desc_lo(base + OFF_K), lo_v = desc_lo(base + OFF_V);
-      const uint32_t lo_p = desc_lo(base + OFF_P);
       constexpr uint32_t TILE16 = TILE >> 4;
       // S of step `step`; first_of_q: wait for the query tile iq; last_of_q: release the Q buffer
       auto issue_S = [&](int step, int iq, bool first_of_q, bool last_of_q) -> bool {
@@ -157,12 +156,11 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
           if (!mbar_wait(B(V_FULL), (uint32_t)it & 1u, abort_flag, p.status, 27)) { ok = false; break; }
           if (!mbar_wait(B(O_FREE), ((uint32_t)it & 1u) ^ 1u, abort_flag, p.status, 28)) { ok = false; break; }
           tc_fence_after();
-          // P is two [128 x 64] K-major blocks (inside a block 16 columns = 32 bytes = 2 units);
+          // P is read from tensor memory (16 keys = 8 columns per product);
           // V advances 16 key rows = 2048 bytes = 128 units per product
-          tc_mma_lo(tO, lo_p, lo_v, IDESC_PV, 0u);
 #pragma unroll
-          for (int k = 1; k < BKV / UMMA_K; ++k)
-            tc_mma_lo_acc(tO, lo_p + (uint32_t)((k >> 2) * (int)TILE16 + 2 * (k & 3)), lo_v + (uint32_t)(128 * k), IDESC_PV);
+          for (int k = 0; k < BKV / UMMA_K; ++k)
+            tc_mma_ts_lo(tO, tP + (uint32_t)(8 * k), lo_v + (uint32_t)(128 * k), IDESC_PV, k != 0 ? 1u : 0u);
           tc_commit(B(V_EMPTY));      // V (and P) reusable
           tc_commit(B(O_FULL));       // O' complete
         }
@@ -233,19 +231,12 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
 #pragma unroll
             for (int i = 0; i < 16; ++i) pk[i] = 0u;
           }
-          const uint32_t prow = base + OFF_P + (uint32_t)(c >> 6) * TILE + (uint32_t)r * 128u;
-          const uint32_t cbase = (uint32_t)((c & 63) >> 3);          // first 16-byte chunk of these 32 columns
-#pragma unroll
-          for (uint32_t jj = 0; jj < 4; ++jj) {
-            const uint32_t chunk = (cbase + jj) ^ ((uint32_t)r & 7u);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(prow + (chunk << 4)), "r"(pk[4 * jj]),
-                         "r"(pk[4 * jj + 1]), "r"(pk[4 * jj + 2]), "r"(pk[4 * jj + 3]) : "memory");
-          }
+          tc_st16(tP + lane_off + (uint32_t)(c >> 1), pk);          // 32 bf16 = 16 columns of this row's lane
         }
+        tc_wait_st();
         tc_fence_before();
         mbar_arrive(B(S_FREE));                      // S may be overwritten
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(B(P_READY));                     // P visible to the tensor core
+        mbar_arrive(B(P_READY));                     // P complete in tensor memory
         l_run = l_run * corr + psum;
         m_run = m_new;
         // O = O * corr + O'

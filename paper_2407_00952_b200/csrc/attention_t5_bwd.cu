@@ -28,6 +28,7 @@ constexpr int BT = 128;                   // rows of a query tile and of a key t
 constexpr int TILE = BT * DH * 2;         // 16 KB: one [128 x 64] bf16 tile
 constexpr int NTHREADS = 352;             // TMA warp, two MMA-issuing warps (1 and 10), 8 element-wise warps
 constexpr int ACC_WARP = 10;              // issues the products that accumulate dK, dV / dQ
+constexpr int RING = 3;                   // stages of the per-step operand ring (Q/dO, resp. K/V)
 constexpr int EW_THREADS = 256;           // two warps per accumulator lane quarter, 64 columns each
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t IDESC_64KK = make_idesc(BT, DH);                   // [128 x 64] products, both operands K-major
@@ -85,7 +86,7 @@ struct BwdParams {
   int* status;
 };
 
-#define T5_SETUP(NBARS, CNT128_A, CNT128_B, CNT128_C, CNT128_D, CNT128_E, CNT2_A, CNT2_B)                                                     \
+#define T5_SETUP(NBARS, CNT128_A, CNT128_B, CNT128_C, CNT128_D, CNT128_E, CNT2_LO, CNT2_HI)                                                     \
   extern __shared__ uint8_t smem_raw[];                                                                   \
   const uint32_t raw = smem_u32(smem_raw);                                                                \
   const uint32_t base = (raw + 1023u) & ~1023u;                                                           \
@@ -98,7 +99,7 @@ struct BwdParams {
   if (threadIdx.x == 0) {                                                                                 \
     for (int i = 0; i < NBARS; ++i)                                                                       \
       mbar_init(B(i), (i == CNT128_A || i == CNT128_B || i == CNT128_C || i == CNT128_D || i == CNT128_E) ? EW_THREADS \
-                      : (i == CNT2_A || i == CNT2_B) ? 2 : 1);                                            \
+                      : (i >= CNT2_LO && i < CNT2_HI) ? 2 : 1);                                           \
     *abort_flag = 0;                                                                                      \
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");                                    \
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");                                          \
@@ -132,11 +133,16 @@ __device__ __forceinline__ uint32_t freed(int n) { return ((uint32_t)n & 1u) ^ 1
 // dK, dV
 // ==========================================================================================
 namespace dkv {
-enum { KV_FULL = 0, KV_EMPTY, QD_FULL /*+s*/, QD_FULL1, QD_EMPTY /*+s*/, QD_EMPTY1, S_FULL /*+half*/, S_FULL1,
-       S_FREE /*+half*/, S_FREE1, P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, N_BARS };
-constexpr int OFF_K = 0, OFF_V = TILE, OFF_QD = 2 * TILE /* stage s: Q at +s*2*TILE, dO after it */,
-              OFF_PT = 6 * TILE, OFF_DST = 8 * TILE, OFF_STAT = 10 * TILE /* stage s: lse at +s*1024, D at +512 */,
-              OFF_BAR = 10 * TILE + 2048;
+enum { KV_FULL = 0 /*+buffer*/, KV_FULL1, KV_EMPTY /*+buffer*/, KV_EMPTY1, QD_FULL /*+s*/, QD_FULL1, QD_FULL2,
+       QD_EMPTY /*+s*/, QD_EMPTY1, QD_EMPTY2, S_FULL /*+half*/, S_FULL1, S_FREE /*+half*/, S_FREE1,
+       P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, N_BARS };
+// K, V of a key tile are double buffered (the next key tile's arrive during this one's last steps);
+// Q, dO and the row statistics of a step go through a ring of RING stages.
+constexpr int OFF_KV = 0 /* buffer kb: K at +kb*2*TILE, V after it */,
+              OFF_QD = 4 * TILE /* stage s: Q at +s*2*TILE, dO after it */,
+              OFF_OUT = 10 * TILE /* dK, dV staged for the TMA stores */,
+              OFF_STAT = 12 * TILE /* stage s: lse at +s*1024, D at +512 */,
+              OFF_BAR = 12 * TILE + RING * 1024;
 constexpr int SMEM = OFF_BAR + 256 + 1024;
 }  // namespace dkv
 
@@ -144,7 +150,7 @@ __global__ void __launch_bounds__(NTHREADS, 1)
 attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
                        const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dkv;
-  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, QD_EMPTY, QD_EMPTY1)
+  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, QD_EMPTY, QD_EMPTY + RING)
   const int h = blockIdx.x, b = blockIdx.y;
   const int nq = p.T / BT;
   const int seq_row0 = b * p.T;
@@ -155,20 +161,21 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
   if (warp == 0) {
     if (lane == 0) {
       bool ok = true;
-      int it = 0;
+      int s = 0, n = 0;                            // ring stage and how often it has been used
       for (int kt = 0; kt < nq && ok; ++kt) {
-        if (!mbar_wait(B(KV_EMPTY), freed(kt), abort_flag, p.status, 41)) { ok = false; break; }
-        mbar_expect_tx(B(KV_FULL), 2 * TILE);
-        tma_load_2d(base + OFF_K, &mapQKV, B(KV_FULL), p.d + h * DH, seq_row0 + kt * BT);
-        tma_load_2d(base + OFF_V, &mapQKV, B(KV_FULL), 2 * p.d + h * DH, seq_row0 + kt * BT);
-        for (int i = kt; i < nq; ++i, ++it) {
-          const int s = it & 1;
-          if (!mbar_wait(B(QD_EMPTY + s), freed(it >> 1), abort_flag, p.status, 42)) { ok = false; break; }
+        const int kb = kt & 1;
+        if (!mbar_wait(B(KV_EMPTY + kb), freed(kt >> 1), abort_flag, p.status, 41)) { ok = false; break; }
+        mbar_expect_tx(B(KV_FULL + kb), 2 * TILE);
+        tma_load_2d(base + OFF_KV + kb * 2 * TILE, &mapQKV, B(KV_FULL + kb), p.d + h * DH, seq_row0 + kt * BT);
+        tma_load_2d(base + OFF_KV + kb * 2 * TILE + TILE, &mapQKV, B(KV_FULL + kb), 2 * p.d + h * DH, seq_row0 + kt * BT);
+        for (int i = kt; i < nq; ++i) {
+          if (!mbar_wait(B(QD_EMPTY + s), freed(n), abort_flag, p.status, 42)) { ok = false; break; }
           mbar_expect_tx(B(QD_FULL + s), 2 * TILE + 1024);
           tma_load_2d(base + OFF_QD + s * 2 * TILE, &mapQKV, B(QD_FULL + s), h * DH, seq_row0 + i * BT);
           tma_load_2d(base + OFF_QD + s * 2 * TILE + TILE, &mapDO, B(QD_FULL + s), h * DH, seq_row0 + i * BT);
           bulk_load(base + OFF_STAT + s * 1024, p.lse + stat0 + (size_t)i * BT, 512, B(QD_FULL + s));
           bulk_load(base + OFF_STAT + s * 1024 + 512, p.rowdot + stat0 + (size_t)i * BT, 512, B(QD_FULL + s));
+          if (++s == RING) { s = 0; ++n; }
         }
       }
     }
@@ -181,15 +188,16 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     // 48 cycles each per step next to eight busy element-wise warps.
     if (lane == 0) {
       bool ok = true;
-      int it = 0;
-      const uint32_t lo_k = desc_lo(base + OFF_K), lo_v = desc_lo(base + OFF_V), lo_qd = desc_lo(base + OFF_QD);
+      int it = 0, s = 0, n = 0;
+      const uint32_t lo_kv = desc_lo(base + OFF_KV), lo_qd = desc_lo(base + OFF_QD);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int kt = 0; kt < nq && ok; ++kt) {
-        if (!mbar_wait(B(KV_FULL), done(kt), abort_flag, p.status, 45)) { ok = false; break; }
+        const int kb = kt & 1;
+        const uint32_t lo_k = lo_kv + (uint32_t)kb * 2u * TILE16, lo_v = lo_k + TILE16;
+        if (!mbar_wait(B(KV_FULL + kb), done(kt >> 1), abort_flag, p.status, 45)) { ok = false; break; }
         for (int i = kt; i < nq && ok; ++i, ++it) {
-          const int s = it & 1;
           const uint32_t lo_q = lo_qd + (uint32_t)s * 2u * TILE16;
-          if (!mbar_wait(B(QD_FULL + s), done(it >> 1), abort_flag, p.status, 43)) { ok = false; break; }
+          if (!mbar_wait(B(QD_FULL + s), done(n), abort_flag, p.status, 43)) { ok = false; break; }
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             if (!mbar_wait(B(S_FREE + hh), freed(it), abort_flag, p.status, 44)) { ok = false; break; }
@@ -199,24 +207,24 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
             tc_commit(B(S_FULL + hh));
           }
           if (ok) tc_commit(B(QD_EMPTY + s));        // second arrival comes from the accumulating thread
+          if (++s == RING) { s = 0; ++n; }
         }
-        if (ok) tc_commit(B(KV_EMPTY));              // K, V are read by these products only
+        if (ok) tc_commit(B(KV_EMPTY + kb));         // K, V are read by these products only
       }
     }
   } else if (warp == ACC_WARP) {
     // ---------------- accumulating products: dV += P^T dO, dK += dS^T Q ----------------
     if (lane == 0) {
       bool ok = true;
-      int it = 0;
+      int it = 0, s = 0, n = 0;
       const uint32_t lo_qd = desc_lo(base + OFF_QD);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int kt = 0; kt < nq && ok; ++kt) {
         // the accumulators of the previous key tile must have been read
         if (!mbar_wait(B(ACC_FREE), freed(kt), abort_flag, p.status, 46)) { ok = false; break; }
         for (int i = kt; i < nq && ok; ++i, ++it) {
-          const int s = it & 1;
           const uint32_t lo_q = lo_qd + (uint32_t)s * 2u * TILE16, lo_do = lo_q + TILE16;
-          if (!mbar_wait(B(QD_FULL + s), done(it >> 1), abort_flag, p.status, 43)) { ok = false; break; }
+          if (!mbar_wait(B(QD_FULL + s), done(n), abort_flag, p.status, 43)) { ok = false; break; }
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             if (!mbar_wait(B(P_READY + hh), done(it), abort_flag, p.status, 47)) { ok = false; break; }
@@ -226,6 +234,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
             tc_commit(B(P_FREE + hh));
           }
           if (ok) tc_commit(B(QD_EMPTY + s));
+          if (++s == RING) { s = 0; ++n; }
         }
         if (ok) tc_commit(B(ACC_FULL));
       }
@@ -237,13 +246,12 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     const float scale_log2 = p.scale * LOG2E;
     bool ok = true;
-    int it = 0;
+    int it = 0, s = 0, n = 0;
     for (int kt = 0; kt < nq; ++kt) {
       for (int i = kt; i < nq && ok; ++i, ++it) {
-        const int s = it & 1;
         const float* Ls = reinterpret_cast<const float*>(base_ptr + OFF_STAT + s * 1024);
         const float* Ds = Ls + 128;
-        if (!mbar_wait(B(QD_FULL + s), done(it >> 1), abort_flag, p.status, 48)) { ok = false; break; }
+        if (!mbar_wait(B(QD_FULL + s), done(n), abort_flag, p.status, 48)) { ok = false; break; }
         const bool diag = (i == kt);
         // on the diagonal tile only queries >= this key count: chunks wholly before the warp's rows are zero
         const int c_first = diag ? q4 * 32 : 0;
@@ -296,6 +304,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
           mbar_arrive(B(P_READY + hh));                // this half of P^T, dS^T is complete
         }
         if (!ok) break;
+        if (++s == RING) { s = 0; ++n; }
       }
       // dK (scaled) and dV of this key tile: tensor memory -> bf16 -> staged in the P^T buffer -> TMA stores
       if (ok && !mbar_wait(B(ACC_FULL), done(kt), abort_flag, p.status, 51)) ok = false;
@@ -318,7 +327,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
                 __nv_bfloat162 ob = __floats2bfloat162_rn(v[8 * jj + 2 * e] * mul, v[8 * jj + 2 * e + 1] * mul);
                 w[e] = *reinterpret_cast<uint32_t*>(&ob);
               }
-              st_row_chunk(base + OFF_PT + half * TILE, r, (uint32_t)(c >> 3) + jj, w);
+              st_row_chunk(base + OFF_OUT + half * TILE, r, (uint32_t)(c >> 3) + jj, w);
             }
           }
         }
@@ -328,8 +337,8 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("bar.sync 1, 256;" ::: "memory");
       if (ok && warp == 2 && lane == 0) {
-        tma_store_2d(&mapDQKV, base + OFF_PT, p.d + h * DH, seq_row0 + kt * BT);
-        tma_store_2d(&mapDQKV, base + OFF_PT + TILE, 2 * p.d + h * DH, seq_row0 + kt * BT);
+        tma_store_2d(&mapDQKV, base + OFF_OUT, p.d + h * DH, seq_row0 + kt * BT);
+        tma_store_2d(&mapDQKV, base + OFF_OUT + TILE, 2 * p.d + h * DH, seq_row0 + kt * BT);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
       }
@@ -344,10 +353,13 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
 // dQ
 // ==========================================================================================
 namespace dq {
-enum { QO_FULL = 0, QO_EMPTY, KV_FULL /*+s*/, KV_FULL1, KV_EMPTY /*+s*/, KV_EMPTY1, S_FULL /*+half*/, S_FULL1,
-       S_FREE /*+half*/, S_FREE1, P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, N_BARS };
-constexpr int OFF_Q = 0, OFF_DO = TILE, OFF_KV = 2 * TILE /* stage s: K at +s*2*TILE, V after it */,
-              OFF_DS = 6 * TILE, OFF_BAR = 8 * TILE;
+enum { QO_FULL = 0 /*+buffer*/, QO_FULL1, QO_EMPTY /*+buffer*/, QO_EMPTY1, KV_FULL /*+s*/, KV_FULL1, KV_FULL2,
+       KV_EMPTY /*+s*/, KV_EMPTY1, KV_EMPTY2, S_FULL /*+half*/, S_FULL1, S_FREE /*+half*/, S_FREE1,
+       P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, N_BARS };
+// Q, dO of a query tile are double buffered; K, V of a step go through a ring of RING stages.
+constexpr int OFF_QO = 0 /* buffer qb: Q at +qb*2*TILE, dO after it */,
+              OFF_KV = 4 * TILE /* stage s: K at +s*2*TILE, V after it */,
+              OFF_OUT = 10 * TILE /* dQ staged for the TMA store */, OFF_BAR = 11 * TILE;
 constexpr int SMEM = OFF_BAR + 256 + 1024;
 }  // namespace dq
 
@@ -355,7 +367,7 @@ __global__ void __launch_bounds__(NTHREADS, 1)
 attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
                       const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dq;
-  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, KV_EMPTY, KV_EMPTY1)
+  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, KV_EMPTY, KV_EMPTY + RING)
   const int h = blockIdx.x, b = blockIdx.y;
   const int nq = p.T / BT;
   const int seq_row0 = b * p.T;
@@ -367,19 +379,19 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
   if (warp == 0) {
     if (lane == 0) {
       bool ok = true;
-      int it = 0;
+      int s = 0, n = 0;
       for (int qi = 0; qi < nq && ok; ++qi) {
-        const int i = nq - 1 - qi;
-        if (!mbar_wait(B(QO_EMPTY), freed(qi), abort_flag, p.status, 61)) { ok = false; break; }
-        mbar_expect_tx(B(QO_FULL), 2 * TILE);
-        tma_load_2d(base + OFF_Q, &mapQKV, B(QO_FULL), h * DH, seq_row0 + i * BT);
-        tma_load_2d(base + OFF_DO, &mapDO, B(QO_FULL), h * DH, seq_row0 + i * BT);
-        for (int j = 0; j <= i; ++j, ++it) {
-          const int s = it & 1;
-          if (!mbar_wait(B(KV_EMPTY + s), freed(it >> 1), abort_flag, p.status, 62)) { ok = false; break; }
+        const int i = nq - 1 - qi, qb = qi & 1;
+        if (!mbar_wait(B(QO_EMPTY + qb), freed(qi >> 1), abort_flag, p.status, 61)) { ok = false; break; }
+        mbar_expect_tx(B(QO_FULL + qb), 2 * TILE);
+        tma_load_2d(base + OFF_QO + qb * 2 * TILE, &mapQKV, B(QO_FULL + qb), h * DH, seq_row0 + i * BT);
+        tma_load_2d(base + OFF_QO + qb * 2 * TILE + TILE, &mapDO, B(QO_FULL + qb), h * DH, seq_row0 + i * BT);
+        for (int j = 0; j <= i; ++j) {
+          if (!mbar_wait(B(KV_EMPTY + s), freed(n), abort_flag, p.status, 62)) { ok = false; break; }
           mbar_expect_tx(B(KV_FULL + s), 2 * TILE);
           tma_load_2d(base + OFF_KV + s * 2 * TILE, &mapQKV, B(KV_FULL + s), p.d + h * DH, seq_row0 + j * BT);
           tma_load_2d(base + OFF_KV + s * 2 * TILE + TILE, &mapQKV, B(KV_FULL + s), 2 * p.d + h * DH, seq_row0 + j * BT);
+          if (++s == RING) { s = 0; ++n; }
         }
       }
     }
@@ -387,16 +399,17 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
     // ---------------- score products: S = Q K^T, dP = dO V^T, in halves of 64 key columns ----------------
     if (lane == 0) {
       bool ok = true;
-      int it = 0;
-      const uint32_t lo_q = desc_lo(base + OFF_Q), lo_do = desc_lo(base + OFF_DO), lo_kv = desc_lo(base + OFF_KV);
+      int it = 0, s = 0, n = 0;
+      const uint32_t lo_qo = desc_lo(base + OFF_QO), lo_kv = desc_lo(base + OFF_KV);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int qi = 0; qi < nq && ok; ++qi) {
         const int steps = nq - qi;               // key tiles 0 .. i, i = nq-1-qi
-        if (!mbar_wait(B(QO_FULL), done(qi), abort_flag, p.status, 65)) { ok = false; break; }
+        const int qb = qi & 1;
+        const uint32_t lo_q = lo_qo + (uint32_t)qb * 2u * TILE16, lo_do = lo_q + TILE16;
+        if (!mbar_wait(B(QO_FULL + qb), done(qi >> 1), abort_flag, p.status, 65)) { ok = false; break; }
         for (int st = 0; st < steps && ok; ++st, ++it) {
-          const int s = it & 1;
           const uint32_t lo_k = lo_kv + (uint32_t)s * 2u * TILE16;
-          if (!mbar_wait(B(KV_FULL + s), done(it >> 1), abort_flag, p.status, 63)) { ok = false; break; }
+          if (!mbar_wait(B(KV_FULL + s), done(n), abort_flag, p.status, 63)) { ok = false; break; }
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             if (!mbar_wait(B(S_FREE + hh), freed(it), abort_flag, p.status, 64)) { ok = false; break; }
@@ -406,24 +419,24 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
             tc_commit(B(S_FULL + hh));
           }
           if (ok) tc_commit(B(KV_EMPTY + s));        // second arrival comes from the accumulating thread
+          if (++s == RING) { s = 0; ++n; }
         }
-        if (ok) tc_commit(B(QO_EMPTY));              // Q, dO are read by these products only
+        if (ok) tc_commit(B(QO_EMPTY + qb));         // Q, dO are read by these products only
       }
     }
   } else if (warp == ACC_WARP) {
     // ---------------- accumulating products: dQ += dS K ----------------
     if (lane == 0) {
       bool ok = true;
-      int it = 0;
+      int it = 0, s = 0, n = 0;
       const uint32_t lo_kv = desc_lo(base + OFF_KV);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int qi = 0; qi < nq && ok; ++qi) {
         const int steps = nq - qi;
         if (!mbar_wait(B(ACC_FREE), freed(qi), abort_flag, p.status, 66)) { ok = false; break; }
         for (int st = 0; st < steps && ok; ++st, ++it) {
-          const int s = it & 1;
           const uint32_t lo_k = lo_kv + (uint32_t)s * 2u * TILE16;
-          if (!mbar_wait(B(KV_FULL + s), done(it >> 1), abort_flag, p.status, 63)) { ok = false; break; }
+          if (!mbar_wait(B(KV_FULL + s), done(n), abort_flag, p.status, 63)) { ok = false; break; }
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             if (!mbar_wait(B(P_READY + hh), done(it), abort_flag, p.status, 67)) { ok = false; break; }
@@ -432,6 +445,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
             tc_commit(B(P_FREE + hh));
           }
           if (ok) tc_commit(B(KV_EMPTY + s));
+          if (++s == RING) { s = 0; ++n; }
         }
         if (ok) tc_commit(B(ACC_FULL));
       }
@@ -502,7 +516,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
               __nv_bfloat162 ob = __floats2bfloat162_rn(v[8 * jj + 2 * e] * p.scale, v[8 * jj + 2 * e + 1] * p.scale);
               w[e] = *reinterpret_cast<uint32_t*>(&ob);
             }
-            st_row_chunk(base + OFF_DS, r, (uint32_t)(c >> 3) + jj, w);
+            st_row_chunk(base + OFF_OUT, r, (uint32_t)(c >> 3) + jj, w);
           }
         }
         tc_fence_before();
@@ -511,7 +525,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("bar.sync 1, 256;" ::: "memory");
       if (ok && warp == 2 && lane == 0) {
-        tma_store_2d(&mapDQKV, base + OFF_DS, h * DH, seq_row0 + i * BT);
+        tma_store_2d(&mapDQKV, base + OFF_OUT, h * DH, seq_row0 + i * BT);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
       }
