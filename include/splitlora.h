@@ -215,7 +215,9 @@ int splitlora_device_status(splitlora_ctx* ctx, int32_t* code);
 int splitlora_launch_count(const splitlora_ctx* ctx, int64_t* launches);
 /* Per-kernel-class device time: when enabled, each launch is bracketed by CUDA events on the
  * context stream; splitlora_profile_report copies up to `cap` entries of {name, launches,
- * milliseconds} into HOST arrays and returns the number of classes in *n. */
+ * milliseconds} into HOST arrays and returns the number of classes in *n.
+ * on: 0 off; 1 every launch class; 2 only the tensor-bound linear layers (classes "lora_linear_*",
+ * "linear_*", "head_*"), which leaves two thirds of a round's launches without events between them. */
 int splitlora_profile_enable(splitlora_ctx* ctx, int on);
 int splitlora_profile_report(splitlora_ctx* ctx, char (*names)[48], int64_t* launches, double* ms,
                              int cap, int* n);

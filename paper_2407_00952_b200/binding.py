@@ -256,8 +256,9 @@ class SplitLoRA:
         self._check(self.lib.splitlora_launch_count(self.ctx, C.byref(n)))
         return n.value
 
-    def profile_enable(self, on: bool):
-        self._check(self.lib.splitlora_profile_enable(self.ctx, 1 if on else 0))
+    def profile_enable(self, on):
+        """on: False / 0 off, True / 1 every launch class, 2 the tensor-bound linear layers only."""
+        self._check(self.lib.splitlora_profile_enable(self.ctx, int(on)))
 
     def profile_report(self):
         cap = 64

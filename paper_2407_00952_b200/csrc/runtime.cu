@@ -100,7 +100,7 @@ struct splitlora_ctx {
   int64_t round_index = 0, server_steps = 0, client_steps = 0;
   int64_t launches = 0;
   // profiling
-  bool prof_on = false;
+  int prof_on = 0;            // 0 off, 1 every launch class, 2 the tensor-bound linear classes only
   std::vector<std::string> prof_names;
   std::map<std::string, int> prof_ids;
   std::vector<ProfRec> prof_recs;
@@ -238,6 +238,7 @@ struct Scope {
   Scope(splitlora_ctx* ctx, const char* name, int kernels) : c(ctx) {
     c->launches += kernels;
     if (!c->prof_on) return;
+    if (c->prof_on == 2 && !std::strstr(name, "linear_") && std::strncmp(name, "head_", 5) != 0) return;
     auto it = c->prof_ids.find(name);
     if (it == c->prof_ids.end()) {
       cls = (int)c->prof_names.size();
@@ -919,7 +920,7 @@ int splitlora_launch_count(const splitlora_ctx* c, int64_t* launches) {
 
 int splitlora_profile_enable(splitlora_ctx* c, int on) {
   if (!c) return SPLITLORA_ERR_ARG;
-  c->prof_on = on != 0;
+  c->prof_on = on < 0 || on > 2 ? 1 : on;
   return SPLITLORA_OK;
 }
 

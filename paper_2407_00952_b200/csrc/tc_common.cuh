@@ -229,6 +229,61 @@ __device__ __forceinline__ float gelu_grad_tanh_tc(float z) {
   const float hz = 0.5f * z;
   return fmaf(hz * du, fmaf(-t, t, 1.0f), fmaf(0.5f, t, 0.5f));
 }
+// The same two functions on pairs of values with the packed fp32 instructions of this architecture
+// (one instruction per pair; the hyperbolic tangent stays one special-function instruction per
+// value).  The epilogue warps share their schedulers with the threads that feed the tensor pipe, so
+// every instruction saved here is issue time given back to them.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+// the two bf16 halves of a 32-bit word as a packed pair of floats
+__device__ __forceinline__ uint64_t bf16x2_to_f32x2(uint32_t w) {
+  return pack2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+__device__ __forceinline__ void gelu_tanh_pair(float& a, float& b) {
+  const uint64_t c1 = pack2(0.7978845608028654f, 0.7978845608028654f);
+  const uint64_t c2 = pack2(0.7978845608028654f * 0.044715f, 0.7978845608028654f * 0.044715f);
+  const uint64_t half = pack2(0.5f, 0.5f);
+  const uint64_t z = pack2(a, b);
+  const uint64_t u = mul2(z, fma2(mul2(z, z), c2, c1));
+  float u0, u1;
+  unpack2(u, u0, u1);
+  const uint64_t t = pack2(tanh_fast(u0), tanh_fast(u1));
+  const uint64_t hz = mul2(z, half);
+  unpack2(fma2(hz, t, hz), a, b);
+}
+// (a, b) *= gelu'(z) for the two bf16 values of zw
+__device__ __forceinline__ void mul_gelu_grad_tanh_pair(float& a, float& b, uint32_t zw) {
+  const uint64_t c1 = pack2(0.7978845608028654f, 0.7978845608028654f);
+  const uint64_t c2 = pack2(0.7978845608028654f * 0.044715f, 0.7978845608028654f * 0.044715f);
+  const uint64_t c3 = pack2(0.7978845608028654f * 0.134145f, 0.7978845608028654f * 0.134145f);
+  const uint64_t half = pack2(0.5f, 0.5f), one = pack2(1.0f, 1.0f), neg1 = pack2(-1.0f, -1.0f);
+  const uint64_t z = bf16x2_to_f32x2(zw);
+  const uint64_t z2 = mul2(z, z);
+  const uint64_t u = mul2(z, fma2(z2, c2, c1));
+  float u0, u1;
+  unpack2(u, u0, u1);
+  const uint64_t t = pack2(tanh_fast(u0), tanh_fast(u1));
+  const uint64_t hzdu = mul2(mul2(z, half), fma2(z2, c3, c1));
+  const uint64_t sech2 = fma2(mul2(t, t), neg1, one);
+  const uint64_t g = fma2(hzdu, sech2, fma2(t, half, half));
+  unpack2(mul2(pack2(a, b), g), a, b);
+}
 __device__ __forceinline__ float gelu_tc(float z, bool tanh_form) {
   if (tanh_form) {
     float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);
@@ -359,7 +414,7 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, cons
     }
     if (tanh_form) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) v[i] = gelu_tanh_tc(zr[i]);
+      for (int i = 0; i < 32; i += 2) { v[i] = zr[i]; v[i + 1] = zr[i + 1]; gelu_tanh_pair(v[i], v[i + 1]); }
     } else {
 #pragma unroll
       for (int i = 0; i < 32; ++i) v[i] = gelu_f(zr[i], false);
@@ -377,9 +432,9 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, cons
     if (tanh_form) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const bf16* rp = reinterpret_cast<const bf16*>(&rpre[j]);
+        const uint32_t* rw = reinterpret_cast<const uint32_t*>(&rpre[j]);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[8 * j + i] *= gelu_grad_tanh_tc(__bfloat162float(rp[i]));
+        for (int i = 0; i < 4; ++i) mul_gelu_grad_tanh_pair(v[8 * j + 2 * i], v[8 * j + 2 * i + 1], rw[i]);
       }
     } else {
 #pragma unroll
