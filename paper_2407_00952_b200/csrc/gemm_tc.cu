@@ -106,8 +106,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
           mbar_expect_tx(full_bar(stage), C::STAGE_BYTES);
           const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
           if (kb < p.num_kb) {
-            tma_load_2d(sa, &mapX, full_bar(stage), kb * BK, m0);
-            tma_load_2d(sb, &mapW, full_bar(stage), kb * BK, w_row);
+            const int kc = (kb < p.gap_kb_begin ? kb : kb + p.gap_kb) * BK;
+            tma_load_2d(sa, &mapX, full_bar(stage), kc, m0);
+            tma_load_2d(sb, &mapW, full_bar(stage), kc, w_row);
           } else {
             const int e = kb - p.num_kb;
             tma_load_2d(sa, &mapXe, full_bar(stage), e * BK, m0);
@@ -442,7 +443,7 @@ int pick_bn(const GemmArgs& a) {
 }
 
 bool pair_ok(const GemmArgs& a) {
-  if (g_max_pairs < 1) return false;
+  if (g_max_pairs < 1 || a.k_gap_len > 0) return false;
   if (a.M % (2 * BM) != 0 || a.N < 256) return false;
   if (a.rows_per_group > 0 && a.rows_per_group % (2 * BM) != 0) return false;
   return true;
@@ -453,9 +454,11 @@ bool prepare(const GemmArgs& a, int* status, int w_box_rows, CUtensorMap* mX, CU
              CUtensorMap* mWe, CUtensorMap* mY, CUtensorMap* mZ, TcParams* p) {
   const int G = a.rows_per_group > 0 ? a.M / a.rows_per_group : 1;
   const int w_rows = a.w_rows > 0 ? a.w_rows : a.N;
-  if (!make_map(mX, a.X, a.M, a.K, a.ldx, BM)) return false;
-  if (!make_map(mW, a.W, a.w_grouped ? (uint64_t)G * a.N : (uint64_t)w_rows, a.K, a.ldw, w_box_rows)) return false;
+  if (!make_map(mX, a.X, a.M, a.K + a.k_gap_len, a.ldx, BM)) return false;
+  if (!make_map(mW, a.W, a.w_grouped ? (uint64_t)G * a.N : (uint64_t)w_rows, a.K + a.k_gap_len, a.ldw, w_box_rows)) return false;
   p->M = a.M; p->N = a.N; p->K = a.K; p->num_kb = a.K / BK;
+  p->gap_kb = a.k_gap_len / BK;
+  p->gap_kb_begin = a.k_gap_len > 0 ? a.k_gap_begin / BK : p->num_kb;
   if (a.Ke > 0) {
     const uint64_t ke_cols = (uint64_t)((a.Ke + BK - 1) / BK) * BK;
     if (!make_map(mXe, a.Xe, a.M, ke_cols, a.ldxe, BM)) return false;
@@ -556,6 +559,7 @@ bool gemm_tc_supported(const GemmArgs& a) {
   if (a.M < BM || a.M % BM != 0 || a.K < BK || a.K % BK != 0 || a.N < 8 || a.N % 8 != 0) return false;
   if (a.rows_per_group > 0 && (a.rows_per_group % BM != 0 || a.M % a.rows_per_group != 0)) return false;
   if (a.ldx % 8 || a.ldw % 8 || a.ldy % 8) return false;
+  if (a.k_gap_len < 0 || a.k_gap_begin < 0 || a.k_gap_len % BK || a.k_gap_begin % BK || a.k_gap_begin > a.K) return false;
   if (!al16(a.X) || !al16(a.W) || !al16(a.Y)) return false;
   if (a.bias && !al16(a.bias)) return false;
   if (a.epi == EPI_BIAS_GELU && (!a.Z || a.ldz % 8 || !al16(a.Z))) return false;

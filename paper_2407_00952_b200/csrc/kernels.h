@@ -42,6 +42,9 @@ struct GemmArgs {
   const void* We = nullptr; int64_t ldwe = 0;
   int Ke = 0;               // 0: no extension; else a multiple of 16
   int we_grouped = 0;       // We is [G*N, Ke]
+  // Columns [k_gap_begin, k_gap_begin + k_gap_len) of X and W are left out of the contraction (both
+  // multiples of 64; K counts the contracted columns only).  Single-CTA tensor-core kernel only.
+  int k_gap_begin = 0, k_gap_len = 0;
 };
 
 // Plain-FMA tiled kernel, any shape, fp32 or bf16 storage with fp32 accumulation.

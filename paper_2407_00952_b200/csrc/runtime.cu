@@ -441,6 +441,17 @@ cudaError_t block_backward(splitlora_ctx* c, int l, const void* dy, void* dx) {
   {  // dh = (alpha/r) dqkv B_g for every target (the scale lives in the compute copy)
     GemmArgs a = base_args(c, c->g_dqkv, 3 * d, b.BextT, 3 * d, c->g_dhcat, ext, M, ext, 3 * d);
     a.rows_per_group = rpg; a.w_grouped = grouped;
+    if (c->tc && c->nq < 3) {
+      // only the adapted slices of dqkv contribute (the other rows of the compute copy are zero):
+      // contract over those columns alone, which is one third less to read for q and v
+      GemmArgs g = a;
+      const int lo = c->slice_idx[0], hi = c->slice_idx[c->nq - 1];
+      g.X = (const char*)a.X + (size_t)lo * d * c->es;
+      g.W = (const char*)a.W + (size_t)lo * d * c->es;
+      g.K = c->nq * d;
+      if (hi - lo + 1 > c->nq) { g.k_gap_begin = d; g.k_gap_len = d; }     // q and v: skip the k slice
+      if (gemm_tc_supported(g)) a = g;
+    }
     if ((e = linear(c, "lora_down_bwd", a))) return e;
   }
   // G_A = dh^T u, G_B = (alpha/r) dy^T h, per group (Eq. 4-7)

@@ -24,6 +24,7 @@ struct TcParams {
   int num_kb;                     // K / 64
   int ext_blocks;                 // blocks of 64 in the rank-r extension
   int ext_last_mmas;              // MMAs (of 16) in the last extension block
+  int gap_kb_begin, gap_kb;       // blocks of 64 columns skipped in X and W from block gap_kb_begin on
   int rows_per_group;             // 0: one group
   int w_group_rows;               // rows between groups in W (0: shared)
   int we_group_rows;              // rows between groups in We
