@@ -1,0 +1,81 @@
+"""The GPT-2-medium-shaped workload at its full size, in the launch configuration the benchmark
+times (24 blocks, 8 clients x 8 sequences x 512 tokens, vocabulary 50257, bf16).
+
+A full oracle round at this size takes hours, so the check uses what the method itself fixes:
+* sequences are independent on the client side (Sec. III-B step a1: clients run in parallel) and on
+  the server side up to the common loss normaliser, so the oracle can follow ONE sampled sequence
+  through all 24 blocks and the head by itself; its cut-layer activations and, scaled by
+  (its valid positions / all valid positions), its activation gradients must equal the rows the GPU
+  produced for that sequence inside the full batch;
+* the first loss of a model with N(0, 0.02) weights lies just above ln V (closed form);
+* Eq. 8-9 on the adapters the full-size round produced, against the weighted mean in fp64.
+"""
+import numpy as np
+import pytest
+import torch
+
+import harness as H
+from oracle import splitlora_oracle as O
+from paper_2407_00952_b200 import binding as B
+from paper_2407_00952_b200 import runner, synth
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+TOL_AGG = 1e-6
+
+
+def test_cfg3_full_size_sampled_sequence_loss_and_aggregation():
+    w = synth.WORKLOADS[3]
+    frozen = synth.make_frozen(w)
+    cads = [synth.make_adapters(w, range(w.cut), nonzero_b=True, salt=i + 1) for i in range(w.n_clients)]
+    sads = synth.make_adapters(w, range(w.cut, w.n_layer), nonzero_b=True, salt=77)
+    tokens, labels = synth.make_tokens(w)
+    counts = synth.make_counts(w)
+
+    eng = runner.make_engine(w, frozen, cads, sads, optimizer="adamw")
+    tok, lab = torch.from_numpy(tokens).cuda(), torch.from_numpy(labels).cuda()
+    S, dS = eng.new_activation_buffer(), eng.new_activation_buffer()
+    eng.client_fwd(tok, S)
+    loss = eng.server_step(S, lab, dS)
+    eng.client_bwd(dS)
+    torch.cuda.synchronize()
+    assert eng.device_status() == 0
+
+    # closed form: logits of a random small-weight model have variance d * 0.02^2 = 0.41, so the
+    # mean cross-entropy is ln V plus about half of that
+    assert np.log(w.vocab) < loss < np.log(w.vocab) + 0.6, loss
+
+    # sampled sequences through the oracle, each alone
+    params = H.f64(frozen)
+    del frozen
+    w1 = synth.scaled(w, n_clients=1, batch_per_client=1)
+    cfg1 = H.oracle_config(w1, optimizer="adamw")
+    n_all = int((labels >= 0).sum())
+    Sv = S.view(w.n_clients, w.batch_per_client, w.seq, w.d_model)
+    dSv = dS.view(w.n_clients, w.batch_per_client, w.seq, w.d_model)
+    for ci, si in ((5, 3), (0, 7)):
+        tok1, lab1 = tokens[ci:ci + 1, si:si + 1], labels[ci:ci + 1, si:si + 1]
+        S_ref, _ = O.client_fwd(cfg1, params, [H.ads64(cads[ci])], tok1)
+        loss1, dS_ref, _ = O.server_fwd_bwd(cfg1, params, H.ads64(sads), S_ref, lab1)
+        # the oracle normalised by this sequence's valid positions, the round by all of them
+        dS_ref = np.asarray(dS_ref) * (int((lab1 >= 0).sum()) / n_all)
+        assert H.rel_err(H.tnp(Sv[ci, si]), np.asarray(S_ref).reshape(w.seq, w.d_model)) <= TOL_BF16, (ci, si)
+        assert H.rel_err(H.tnp(dSv[ci, si]), dS_ref.reshape(w.seq, w.d_model)) <= TOL_BF16, (ci, si)
+        assert abs(loss1 - loss) < 0.5, (loss1, loss)    # one sequence's loss is a sample of the batch mean
+    del params
+
+    # Eq. 8-9 at full size, on the adapters this round left behind
+    before = [[eng.get_adapter(B.SIDE_CLIENT, i, l, B.TARGET_BITS[t]) for i in range(w.n_clients)]
+              for l in range(w.cut) for t in w.targets]
+    eng.aggregate(counts)
+    wts = O.aggregation_weights(counts)
+    k = 0
+    for l in range(w.cut):
+        for t in w.targets:
+            for part in (0, 1):
+                ref = sum(wts[i] * H.tnp(before[k][i][part]) for i in range(w.n_clients))
+                for i in (0, w.n_clients - 1):
+                    got = H.tnp(eng.get_adapter(B.SIDE_CLIENT, i, l, B.TARGET_BITS[t])[part])
+                    assert H.rel_err(got, ref) <= TOL_AGG, (l, t, part, i)
+            k += 1
