@@ -13,8 +13,10 @@
 //       key tiles j <= query tile and keeps dQ in tensor memory:
 //         S = Q K^T, dP = dO V^T,  dS = P (dP - D[row]),  dQ += dS K   (K as loaded: MN-major)
 //
-// D[row] = sum(dO * O) comes from a small pre-pass.  Warp roles (192 threads): warp 0 TMA producer,
-// warp 1 tensor-memory owner + MMA issuer, warps 2..5 element-wise work (thread = accumulator lane).
+// D[row] = sum(dO * O) is computed by the dQ kernel from its staged dO and O tiles and left in global
+// memory for the dK/dV kernel, which runs second.  Warp roles (352 threads): warp 0 TMA producer,
+// warp 1 tensor-memory owner + issuer of the score products, warp 10 issuer of the accumulating
+// products, warps 2..9 element-wise work (thread = accumulator lane, two warps per lane quarter).
 // All mbarrier waits are bounded (tc_common.cuh); on expiry a code is left in `status`.
 #include "tc_common.cuh"
 
@@ -82,7 +84,8 @@ struct BwdParams {
   int T, H, d;
   float scale;             // 1/sqrt(dh)
   const float* lse;        // [nseq, H, T] natural log
-  const float* rowdot;     // [nseq, H, T]
+  const float* rowdot;     // [nseq, H, T]: D[row] = sum(dO * O), read by the dK/dV kernel
+  float* rowdot_out;       // the same buffer, written by the dQ kernel (which runs first)
   int* status;
 };
 
@@ -356,16 +359,18 @@ namespace dq {
 enum { QO_FULL = 0 /*+buffer*/, QO_FULL1, QO_EMPTY /*+buffer*/, QO_EMPTY1, KV_FULL /*+s*/, KV_FULL1, KV_FULL2,
        KV_EMPTY /*+s*/, KV_EMPTY1, KV_EMPTY2, S_FULL /*+half*/, S_FULL1, S_FREE /*+half*/, S_FREE1,
        P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, N_BARS };
-// Q, dO of a query tile are double buffered; K, V of a step go through a ring of RING stages.
-constexpr int OFF_QO = 0 /* buffer qb: Q at +qb*2*TILE, dO after it */,
-              OFF_KV = 4 * TILE /* stage s: K at +s*2*TILE, V after it */,
-              OFF_OUT = 10 * TILE /* dQ staged for the TMA store */, OFF_BAR = 11 * TILE;
+// Q, dO and O of a query tile are double buffered (O only serves D[row] = sum(dO * O), which this
+// kernel computes for itself and leaves in global memory for the dK/dV kernel); K, V of a step go
+// through a ring of RING stages.
+constexpr int OFF_QO = 0 /* buffer qb: Q at +qb*3*TILE, then dO, then O */,
+              OFF_KV = 6 * TILE /* stage s: K at +s*2*TILE, V after it */,
+              OFF_OUT = 12 * TILE /* dQ staged for the TMA store */, OFF_BAR = 13 * TILE;
 constexpr int SMEM = OFF_BAR + 256 + 1024;
 }  // namespace dq
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
-                      const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
+                      const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dq;
   T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, KV_EMPTY, KV_EMPTY + RING)
   const int h = blockIdx.x, b = blockIdx.y;
@@ -383,9 +388,10 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       for (int qi = 0; qi < nq && ok; ++qi) {
         const int i = nq - 1 - qi, qb = qi & 1;
         if (!mbar_wait(B(QO_EMPTY + qb), freed(qi >> 1), abort_flag, p.status, 61)) { ok = false; break; }
-        mbar_expect_tx(B(QO_FULL + qb), 2 * TILE);
-        tma_load_2d(base + OFF_QO + qb * 2 * TILE, &mapQKV, B(QO_FULL + qb), h * DH, seq_row0 + i * BT);
-        tma_load_2d(base + OFF_QO + qb * 2 * TILE + TILE, &mapDO, B(QO_FULL + qb), h * DH, seq_row0 + i * BT);
+        mbar_expect_tx(B(QO_FULL + qb), 3 * TILE);
+        tma_load_2d(base + OFF_QO + qb * 3 * TILE, &mapQKV, B(QO_FULL + qb), h * DH, seq_row0 + i * BT);
+        tma_load_2d(base + OFF_QO + qb * 3 * TILE + TILE, &mapDO, B(QO_FULL + qb), h * DH, seq_row0 + i * BT);
+        tma_load_2d(base + OFF_QO + qb * 3 * TILE + 2 * TILE, &mapO, B(QO_FULL + qb), h * DH, seq_row0 + i * BT);
         for (int j = 0; j <= i; ++j) {
           if (!mbar_wait(B(KV_EMPTY + s), freed(n), abort_flag, p.status, 62)) { ok = false; break; }
           mbar_expect_tx(B(KV_FULL + s), 2 * TILE);
@@ -405,7 +411,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       for (int qi = 0; qi < nq && ok; ++qi) {
         const int steps = nq - qi;               // key tiles 0 .. i, i = nq-1-qi
         const int qb = qi & 1;
-        const uint32_t lo_q = lo_qo + (uint32_t)qb * 2u * TILE16, lo_do = lo_q + TILE16;
+        const uint32_t lo_q = lo_qo + (uint32_t)qb * 3u * TILE16, lo_do = lo_q + TILE16;
         if (!mbar_wait(B(QO_FULL + qb), done(qi >> 1), abort_flag, p.status, 65)) { ok = false; break; }
         for (int st = 0; st < steps && ok; ++st, ++it) {
           const uint32_t lo_k = lo_kv + (uint32_t)s * 2u * TILE16;
@@ -461,7 +467,31 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
     for (int qi = 0; qi < nq; ++qi) {
       const int i = nq - 1 - qi;
       const float L2 = p.lse[stat0 + (size_t)i * BT + r] * LOG2E;
-      const float Dr = p.rowdot[stat0 + (size_t)i * BT + r];
+      // D[row] = sum(dO * O) from the staged tiles: both have the same swizzle, so 16-byte chunk j of
+      // one row holds the same eight columns in both
+      float Dr = 0.f;
+      {
+        const int qb = qi & 1;
+        if (!mbar_wait(B(QO_FULL + qb), done(qi >> 1), abort_flag, p.status, 71)) ok = false;
+        if (ok) {
+          const uint8_t* dorow = base_ptr + OFF_QO + qb * 3 * TILE + TILE + r * 128;
+          const uint8_t* orow = dorow + TILE;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int jj = (j ^ (r & 7)) << 4;       // lanes of a warp spread over all banks
+            const uint4 a = *reinterpret_cast<const uint4*>(dorow + jj);
+            const uint4 bq = *reinterpret_cast<const uint4*>(orow + jj);
+            const uint32_t* aw = reinterpret_cast<const uint32_t*>(&a);
+            const uint32_t* bw = reinterpret_cast<const uint32_t*>(&bq);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              Dr = fmaf(__uint_as_float(aw[e] << 16), __uint_as_float(bw[e] << 16), Dr);
+              Dr = fmaf(__uint_as_float(aw[e] & 0xffff0000u), __uint_as_float(bw[e] & 0xffff0000u), Dr);
+            }
+          }
+          if (wsel == 0) p.rowdot_out[stat0 + (size_t)i * BT + r] = Dr;
+        }
+      }
       for (int j = 0; j <= i && ok; ++j, ++it) {
         const bool diag = (j == i);
         // on the diagonal tile only keys <= this query count: chunks wholly after the warp's rows are zero
@@ -536,29 +566,6 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
   T5_TEARDOWN()
 }
 
-// rowdot[b, h, i] = sum_c dO[i, c] O[i, c] over the head's 64 columns; 8 lanes per row
-__global__ void attn_rowdot_t5_kernel(const bf16* __restrict__ o, const bf16* __restrict__ d_o, int nseq, int T, int H,
-                                      int d, float* __restrict__ rowdot) {
-  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  int64_t rowhead = idx >> 3;
-  int part = (int)(idx & 7);
-  if (rowhead >= (int64_t)nseq * T * H) return;
-  int h = (int)(rowhead % H);
-  int64_t row = rowhead / H;
-  size_t off = (size_t)row * d + (size_t)h * DH + part * 8;
-  uint4 a = *reinterpret_cast<const uint4*>(o + off), bb = *reinterpret_cast<const uint4*>(d_o + off);
-  const bf16* ap = reinterpret_cast<const bf16*>(&a);
-  const bf16* bp = reinterpret_cast<const bf16*>(&bb);
-  float s = 0.f;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) s = fmaf(__bfloat162float(ap[i]), __bfloat162float(bp[i]), s);
-  s += __shfl_xor_sync(0xffffffffu, s, 1); s += __shfl_xor_sync(0xffffffffu, s, 2); s += __shfl_xor_sync(0xffffffffu, s, 4);
-  if (part == 0) {
-    int bq = (int)(row / T), i = (int)(row % T);
-    rowdot[((size_t)bq * H + h) * T + i] = s;
-  }
-}
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -597,19 +604,18 @@ cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, c
                              int d, void* dqkv, float* rowdot, int* status, cudaStream_t st) {
   if (!attention_t5_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
   if (!init_once()) return cudaErrorInitializationError;
-  CUtensorMap mQKV, mDO, mDQKV;
+  CUtensorMap mQKV, mDO, mO, mDQKV;
   const uint64_t rows = (uint64_t)nseq * T;
   if (!make_map(&mQKV, qkv, rows, (uint64_t)3 * d) || !make_map(&mDO, d_o, rows, (uint64_t)d) ||
-      !make_map(&mDQKV, dqkv, rows, (uint64_t)3 * d))
+      !make_map(&mO, o, rows, (uint64_t)d) || !make_map(&mDQKV, dqkv, rows, (uint64_t)3 * d))
     return cudaErrorInvalidValue;
-  int64_t threads = (int64_t)nseq * T * H * 8;
-  attn_rowdot_t5_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>((const bf16*)o, (const bf16*)d_o, nseq, T, H, d, rowdot);
   BwdParams p;
-  p.T = T; p.H = H; p.d = d; p.scale = 1.0f / sqrtf((float)DH); p.lse = lse; p.rowdot = rowdot;
+  p.T = T; p.H = H; p.d = d; p.scale = 1.0f / sqrtf((float)DH); p.lse = lse; p.rowdot = rowdot; p.rowdot_out = rowdot;
   p.status = status ? status : g_status;
   dim3 grid(H, nseq);
+  // dQ first: it leaves D[row] = sum(dO * O) in `rowdot` for the dK/dV kernel
+  attn_bwd_dq_t5_kernel<<<grid, NTHREADS, dq::SMEM, st>>>(mQKV, mDO, mO, mDQKV, p);
   attn_bwd_dkv_t5_kernel<<<grid, NTHREADS, dkv::SMEM, st>>>(mQKV, mDO, mDQKV, p);
-  attn_bwd_dq_t5_kernel<<<grid, NTHREADS, dq::SMEM, st>>>(mQKV, mDO, mDQKV, p);
   return cudaGetLastError();
 }
 

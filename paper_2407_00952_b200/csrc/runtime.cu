@@ -428,7 +428,7 @@ cudaError_t block_backward(splitlora_ctx* c, int l, const void* dy, void* dx) {
       a.Xe = c->g_dhcat_o; a.ldxe = c->ext_o; a.We = b.AcatOT; a.ldwe = c->ext_o; a.Ke = c->rp; a.we_grouped = grouped;
     }
     if ((e = linear(c, c->has_o ? "lora_linear_bwd" : "linear_bwd", a))) return e; }
-  { Scope s(c, "attention_bwd", 3);
+  { Scope s(c, "attention_bwd", c->tc && attention_t5_supported(c->dt, c->cfg.seq, c->cfg.n_head, d) ? 2 : 3);
     if (c->tc && attention_tc_supported(c->dt, c->cfg.seq, c->cfg.n_head, d))
       e = attention_bwd_tc(b.qkv, b.o, b.lse, c->g_do, c->nseq, c->cfg.seq, c->cfg.n_head, d, c->g_dqkv, c->rowdot, c->st);
     else
