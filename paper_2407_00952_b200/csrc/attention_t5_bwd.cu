@@ -14,9 +14,10 @@
 //         S = Q K^T, dP = dO V^T,  dS = P (dP - D[row]),  dQ += dS K   (K as loaded: MN-major)
 //
 // D[row] = sum(dO * O) is computed by the dQ kernel from its staged dO and O tiles and left in global
-// memory for the dK/dV kernel, which runs second.  Warp roles (352 threads): warp 0 TMA producer,
+// memory for the dK/dV kernel, which runs second.  Warp roles (480 threads): warp 0 TMA producer,
 // warp 1 tensor-memory owner + issuer of the score products, warp 10 issuer of the accumulating
-// products, warps 2..9 element-wise work (thread = accumulator lane, two warps per lane quarter).
+// products, warps 2..9 element-wise work (thread = accumulator lane, two warps per lane quarter),
+// warps 11..14 output of the finished accumulators.
 // All mbarrier waits are bounded (tc_common.cuh); on expiry a code is left in `status`.
 #include "tc_common.cuh"
 
@@ -28,7 +29,9 @@ using namespace tc;
 constexpr int DH = 64;
 constexpr int BT = 128;                   // rows of a query tile and of a key tile
 constexpr int TILE = BT * DH * 2;         // 16 KB: one [128 x 64] bf16 tile
-constexpr int NTHREADS = 352;             // TMA warp, two MMA-issuing warps (1 and 10), 8 element-wise warps
+constexpr int NTHREADS = 480;             // TMA warp, two MMA-issuing warps (1 and 10), 8 element-wise warps, 4 output warps
+constexpr int OUT_WARP0 = 11;             // warps 11..14 move finished accumulators to global memory
+constexpr int OUT_THREADS = 128;
 constexpr int ACC_WARP = 10;              // issues the products that accumulate dK, dV / dQ
 constexpr int RING = 3;                   // stages of the per-step operand ring (Q/dO, resp. K/V)
 constexpr int EW_THREADS = 256;           // two warps per accumulator lane quarter, 64 columns each
@@ -89,7 +92,7 @@ struct BwdParams {
   int* status;
 };
 
-#define T5_SETUP(NBARS, CNT128_A, CNT128_B, CNT128_C, CNT128_D, CNT128_E, CNT2_LO, CNT2_HI)                                                     \
+#define T5_SETUP(NBARS, CNT128_A, CNT128_B, CNT128_C, CNT128_D, CNT_OUT, CNT2_LO, CNT2_HI)                                                     \
   extern __shared__ uint8_t smem_raw[];                                                                   \
   const uint32_t raw = smem_u32(smem_raw);                                                                \
   const uint32_t base = (raw + 1023u) & ~1023u;                                                           \
@@ -101,7 +104,7 @@ struct BwdParams {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;                                             \
   if (threadIdx.x == 0) {                                                                                 \
     for (int i = 0; i < NBARS; ++i)                                                                       \
-      mbar_init(B(i), (i == CNT128_A || i == CNT128_B || i == CNT128_C || i == CNT128_D || i == CNT128_E) ? EW_THREADS \
+      mbar_init(B(i), (i == CNT128_A || i == CNT128_B || i == CNT128_C || i == CNT128_D) ? EW_THREADS : i == CNT_OUT ? OUT_THREADS \
                       : (i >= CNT2_LO && i < CNT2_HI) ? 2 : 1);                                           \
     *abort_flag = 0;                                                                                      \
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");                                    \
@@ -242,7 +245,8 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
         if (ok) tc_commit(B(ACC_FULL));
       }
     }
-  } else {
+  } else if (warp < ACC_WARP) {
+    // ---------------- element-wise warps 2..9 ----------------
     const int q4 = warp & 3;
     const int wsel = (warp - 2) >> 2;            // which of the two warps of this accumulator lane quarter
     const int r = q4 * 32 + lane;                // key row inside the tile = accumulator lane
@@ -309,12 +313,21 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
         if (!ok) break;
         if (++s == RING) { s = 0; ++n; }
       }
-      // dK (scaled) and dV of this key tile: tensor memory -> bf16 -> staged in the P^T buffer -> TMA stores
+    }
+  } else if (warp >= OUT_WARP0) {
+    // ---------------- output: dK (scaled) and dV of a finished key tile ----------------
+    // Own warps, so that the element-wise warps go on with the next key tile while the last
+    // products of this one drain: tensor memory -> bf16 -> shared memory -> TMA stores.
+    const int q4 = warp & 3;
+    const int r = q4 * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    bool ok = true;
+    for (int kt = 0; kt < nq; ++kt) {
       if (ok && !mbar_wait(B(ACC_FULL), done(kt), abort_flag, p.status, 51)) ok = false;
       if (ok) {
         tc_fence_after();
-        {
-          const int half = wsel;                       // the first warp of a lane quarter writes dK, the other dV
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
           const uint32_t tsrc = half == 0 ? tDK : tDV;
           const float mul = half == 0 ? p.scale : 1.0f;
 #pragma unroll
@@ -338,16 +351,16 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
         mbar_arrive(B(ACC_FREE));
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (ok && warp == 2 && lane == 0) {
+      asm volatile("bar.sync 1, 128;" ::: "memory");         // the four output warps (always reached)
+      if (ok && warp == OUT_WARP0 && lane == 0) {
         tma_store_2d(&mapDQKV, base + OFF_OUT, p.d + h * DH, seq_row0 + kt * BT);
         tma_store_2d(&mapDQKV, base + OFF_OUT + TILE, 2 * p.d + h * DH, seq_row0 + kt * BT);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
       }
-      asm volatile("bar.sync 1, 256;" ::: "memory");
+      asm volatile("bar.sync 1, 128;" ::: "memory");
     }
-    if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (warp == OUT_WARP0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
   T5_TEARDOWN()
 }
@@ -456,7 +469,8 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
         if (ok) tc_commit(B(ACC_FULL));
       }
     }
-  } else {
+  } else if (warp < ACC_WARP) {
+    // ---------------- element-wise warps 2..9 ----------------
     const int q4 = warp & 3;
     const int wsel = (warp - 2) >> 2;            // which of the two warps of this accumulator lane quarter
     const int r = q4 * 32 + lane;                // query row inside the tile
@@ -530,11 +544,20 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
         }
         if (!ok) break;
       }
+    }
+  } else if (warp >= OUT_WARP0) {
+    // ---------------- output: dQ (scaled) of a finished query tile (own warps, see the dK/dV kernel) ----------------
+    const int q4 = warp & 3;
+    const int r = q4 * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    bool ok = true;
+    for (int qi = 0; qi < nq; ++qi) {
+      const int i = nq - 1 - qi;
       if (ok && !mbar_wait(B(ACC_FULL), done(qi), abort_flag, p.status, 70)) ok = false;
       if (ok) {
         tc_fence_after();
-        {
-          const int c = wsel * 32;                     // each of the two warps of a lane quarter takes 32 of the 64 columns
+#pragma unroll
+        for (int c = 0; c < DH; c += 32) {
           float v[32];
           tc_ld32(tDQ + lane_off + (uint32_t)c, v);
           tc_wait_ld();
@@ -553,15 +576,15 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
         mbar_arrive(B(ACC_FREE));
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (ok && warp == 2 && lane == 0) {
+      asm volatile("bar.sync 1, 128;" ::: "memory");         // the four output warps (always reached)
+      if (ok && warp == OUT_WARP0 && lane == 0) {
         tma_store_2d(&mapDQKV, base + OFF_OUT, h * DH, seq_row0 + i * BT);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
       }
-      asm volatile("bar.sync 1, 256;" ::: "memory");
+      asm volatile("bar.sync 1, 128;" ::: "memory");
     }
-    if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (warp == OUT_WARP0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
   T5_TEARDOWN()
 }
