@@ -87,6 +87,7 @@ struct BwdParams {
   int T, H, d;
   float scale;             // 1/sqrt(dh)
   const float* lse;        // [nseq, H, T] natural log
+  int nitems;              // nseq * H (sequence, head) items, shared out over the CTAs
   const float* rowdot;     // [nseq, H, T]: D[row] = sum(dO * O), read by the dK/dV kernel
   float* rowdot_out;       // the same buffer, written by the dQ kernel (which runs first)
   int* status;
@@ -157,10 +158,10 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
                        const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dkv;
   T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, QD_EMPTY, QD_EMPTY + RING)
-  const int h = blockIdx.x, b = blockIdx.y;
   const int nq = p.T / BT;
-  const int seq_row0 = b * p.T;
-  const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+  // persistent: this CTA takes items blockIdx.x, blockIdx.x + gridDim.x, ... and every role walks the
+  // tiles of all of them in one flat loop, so loads for the next item are issued while this one ends
+  const int my_tiles = ((p.nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * nq;
   const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDV = tmem_base + 256u, tDK = tmem_base + 320u;
   const uint32_t tPT = tmem_base + 384u, tDST = tmem_base + 448u;     // P^T, dS^T: bf16, 64 columns each
 
@@ -168,9 +169,14 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     if (lane == 0) {
       bool ok = true;
       int s = 0, n = 0;                            // ring stage and how often it has been used
-      for (int kt = 0; kt < nq && ok; ++kt) {
-        const int kb = kt & 1;
-        if (!mbar_wait(B(KV_EMPTY + kb), freed(kt >> 1), abort_flag, p.status, 41)) { ok = false; break; }
+      for (int tk = 0; tk < my_tiles && ok; ++tk) {
+        const int item = (int)blockIdx.x + (tk / nq) * (int)gridDim.x, kt = tk % nq;
+        const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
+        const int seq_row0 = b * p.T;
+        const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+        (void)seq_row0; (void)stat0;
+        const int kb = tk & 1;
+        if (!mbar_wait(B(KV_EMPTY + kb), freed(tk >> 1), abort_flag, p.status, 41)) { ok = false; break; }
         mbar_expect_tx(B(KV_FULL + kb), 2 * TILE);
         tma_load_2d(base + OFF_KV + kb * 2 * TILE, &mapQKV, B(KV_FULL + kb), p.d + h * DH, seq_row0 + kt * BT);
         tma_load_2d(base + OFF_KV + kb * 2 * TILE + TILE, &mapQKV, B(KV_FULL + kb), 2 * p.d + h * DH, seq_row0 + kt * BT);
@@ -197,10 +203,15 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       int it = 0, s = 0, n = 0;
       const uint32_t lo_kv = desc_lo(base + OFF_KV), lo_qd = desc_lo(base + OFF_QD);
       constexpr uint32_t TILE16 = TILE >> 4;
-      for (int kt = 0; kt < nq && ok; ++kt) {
-        const int kb = kt & 1;
+      for (int tk = 0; tk < my_tiles && ok; ++tk) {
+        const int item = (int)blockIdx.x + (tk / nq) * (int)gridDim.x, kt = tk % nq;
+        const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
+        const int seq_row0 = b * p.T;
+        const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+        (void)seq_row0; (void)stat0;
+        const int kb = tk & 1;
         const uint32_t lo_k = lo_kv + (uint32_t)kb * 2u * TILE16, lo_v = lo_k + TILE16;
-        if (!mbar_wait(B(KV_FULL + kb), done(kt >> 1), abort_flag, p.status, 45)) { ok = false; break; }
+        if (!mbar_wait(B(KV_FULL + kb), done(tk >> 1), abort_flag, p.status, 45)) { ok = false; break; }
         for (int i = kt; i < nq && ok; ++i, ++it) {
           const uint32_t lo_q = lo_qd + (uint32_t)s * 2u * TILE16;
           if (!mbar_wait(B(QD_FULL + s), done(n), abort_flag, p.status, 43)) { ok = false; break; }
@@ -225,9 +236,14 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       int it = 0, s = 0, n = 0;
       const uint32_t lo_qd = desc_lo(base + OFF_QD);
       constexpr uint32_t TILE16 = TILE >> 4;
-      for (int kt = 0; kt < nq && ok; ++kt) {
+      for (int tk = 0; tk < my_tiles && ok; ++tk) {
+        const int item = (int)blockIdx.x + (tk / nq) * (int)gridDim.x, kt = tk % nq;
+        const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
+        const int seq_row0 = b * p.T;
+        const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+        (void)seq_row0; (void)stat0;
         // the accumulators of the previous key tile must have been read
-        if (!mbar_wait(B(ACC_FREE), freed(kt), abort_flag, p.status, 46)) { ok = false; break; }
+        if (!mbar_wait(B(ACC_FREE), freed(tk), abort_flag, p.status, 46)) { ok = false; break; }
         for (int i = kt; i < nq && ok; ++i, ++it) {
           const uint32_t lo_q = lo_qd + (uint32_t)s * 2u * TILE16, lo_do = lo_q + TILE16;
           if (!mbar_wait(B(QD_FULL + s), done(n), abort_flag, p.status, 43)) { ok = false; break; }
@@ -254,7 +270,12 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     const float scale_log2 = p.scale * LOG2E;
     bool ok = true;
     int it = 0, s = 0, n = 0;
-    for (int kt = 0; kt < nq; ++kt) {
+    for (int tk = 0; tk < my_tiles; ++tk) {
+      const int item = (int)blockIdx.x + (tk / nq) * (int)gridDim.x, kt = tk % nq;
+      const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
+      const int seq_row0 = b * p.T;
+      const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+      (void)seq_row0; (void)stat0;
       for (int i = kt; i < nq && ok; ++i, ++it) {
         const float* Ls = reinterpret_cast<const float*>(base_ptr + OFF_STAT + s * 1024);
         const float* Ds = Ls + 128;
@@ -322,8 +343,13 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     const int r = q4 * 32 + lane;
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     bool ok = true;
-    for (int kt = 0; kt < nq; ++kt) {
-      if (ok && !mbar_wait(B(ACC_FULL), done(kt), abort_flag, p.status, 51)) ok = false;
+    for (int tk = 0; tk < my_tiles; ++tk) {
+      const int item = (int)blockIdx.x + (tk / nq) * (int)gridDim.x, kt = tk % nq;
+      const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
+      const int seq_row0 = b * p.T;
+      const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+      (void)seq_row0; (void)stat0;
+      if (ok && !mbar_wait(B(ACC_FULL), done(tk), abort_flag, p.status, 51)) ok = false;
       if (ok) {
         tc_fence_after();
 #pragma unroll
@@ -386,10 +412,10 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
                       const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dq;
   T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, KV_EMPTY, KV_EMPTY + RING)
-  const int h = blockIdx.x, b = blockIdx.y;
   const int nq = p.T / BT;
-  const int seq_row0 = b * p.T;
-  const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+  // persistent: this CTA takes items blockIdx.x, blockIdx.x + gridDim.x, ... and every role walks the
+  // tiles of all of them in one flat loop, so loads for the next item are issued while this one ends
+  const int my_tiles = ((p.nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * nq;
   const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDQ = tmem_base + 256u;
   const uint32_t tDS = tmem_base + 320u;                               // dS: bf16, 64 columns
 
@@ -398,9 +424,14 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
     if (lane == 0) {
       bool ok = true;
       int s = 0, n = 0;
-      for (int qi = 0; qi < nq && ok; ++qi) {
-        const int i = nq - 1 - qi, qb = qi & 1;
-        if (!mbar_wait(B(QO_EMPTY + qb), freed(qi >> 1), abort_flag, p.status, 61)) { ok = false; break; }
+      for (int tq = 0; tq < my_tiles && ok; ++tq) {
+        const int item = (int)blockIdx.x + (tq / nq) * (int)gridDim.x, qi = tq % nq;
+        const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
+        const int seq_row0 = b * p.T;
+        const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+        (void)seq_row0; (void)stat0;
+        const int i = nq - 1 - qi, qb = tq & 1;
+        if (!mbar_wait(B(QO_EMPTY + qb), freed(tq >> 1), abort_flag, p.status, 61)) { ok = false; break; }
         mbar_expect_tx(B(QO_FULL + qb), 3 * TILE);
         tma_load_2d(base + OFF_QO + qb * 3 * TILE, &mapQKV, B(QO_FULL + qb), h * DH, seq_row0 + i * BT);
         tma_load_2d(base + OFF_QO + qb * 3 * TILE + TILE, &mapDO, B(QO_FULL + qb), h * DH, seq_row0 + i * BT);
@@ -421,11 +452,16 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       int it = 0, s = 0, n = 0;
       const uint32_t lo_qo = desc_lo(base + OFF_QO), lo_kv = desc_lo(base + OFF_KV);
       constexpr uint32_t TILE16 = TILE >> 4;
-      for (int qi = 0; qi < nq && ok; ++qi) {
+      for (int tq = 0; tq < my_tiles && ok; ++tq) {
+        const int item = (int)blockIdx.x + (tq / nq) * (int)gridDim.x, qi = tq % nq;
+        const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
+        const int seq_row0 = b * p.T;
+        const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+        (void)seq_row0; (void)stat0;
         const int steps = nq - qi;               // key tiles 0 .. i, i = nq-1-qi
-        const int qb = qi & 1;
+        const int qb = tq & 1;
         const uint32_t lo_q = lo_qo + (uint32_t)qb * 3u * TILE16, lo_do = lo_q + TILE16;
-        if (!mbar_wait(B(QO_FULL + qb), done(qi >> 1), abort_flag, p.status, 65)) { ok = false; break; }
+        if (!mbar_wait(B(QO_FULL + qb), done(tq >> 1), abort_flag, p.status, 65)) { ok = false; break; }
         for (int st = 0; st < steps && ok; ++st, ++it) {
           const uint32_t lo_k = lo_kv + (uint32_t)s * 2u * TILE16;
           if (!mbar_wait(B(KV_FULL + s), done(n), abort_flag, p.status, 63)) { ok = false; break; }
@@ -450,9 +486,14 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       int it = 0, s = 0, n = 0;
       const uint32_t lo_kv = desc_lo(base + OFF_KV);
       constexpr uint32_t TILE16 = TILE >> 4;
-      for (int qi = 0; qi < nq && ok; ++qi) {
+      for (int tq = 0; tq < my_tiles && ok; ++tq) {
+        const int item = (int)blockIdx.x + (tq / nq) * (int)gridDim.x, qi = tq % nq;
+        const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
+        const int seq_row0 = b * p.T;
+        const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+        (void)seq_row0; (void)stat0;
         const int steps = nq - qi;
-        if (!mbar_wait(B(ACC_FREE), freed(qi), abort_flag, p.status, 66)) { ok = false; break; }
+        if (!mbar_wait(B(ACC_FREE), freed(tq), abort_flag, p.status, 66)) { ok = false; break; }
         for (int st = 0; st < steps && ok; ++st, ++it) {
           const uint32_t lo_k = lo_kv + (uint32_t)s * 2u * TILE16;
           if (!mbar_wait(B(KV_FULL + s), done(n), abort_flag, p.status, 63)) { ok = false; break; }
@@ -478,15 +519,20 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
     const float scale_log2 = p.scale * LOG2E;
     bool ok = true;
     int it = 0;
-    for (int qi = 0; qi < nq; ++qi) {
+    for (int tq = 0; tq < my_tiles; ++tq) {
+      const int item = (int)blockIdx.x + (tq / nq) * (int)gridDim.x, qi = tq % nq;
+      const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
+      const int seq_row0 = b * p.T;
+      const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+      (void)seq_row0; (void)stat0;
       const int i = nq - 1 - qi;
       const float L2 = p.lse[stat0 + (size_t)i * BT + r] * LOG2E;
       // D[row] = sum(dO * O) from the staged tiles: both have the same swizzle, so 16-byte chunk j of
       // one row holds the same eight columns in both
       float Dr = 0.f;
       {
-        const int qb = qi & 1;
-        if (!mbar_wait(B(QO_FULL + qb), done(qi >> 1), abort_flag, p.status, 71)) ok = false;
+        const int qb = tq & 1;
+        if (!mbar_wait(B(QO_FULL + qb), done(tq >> 1), abort_flag, p.status, 71)) ok = false;
         if (ok) {
           const uint8_t* dorow = base_ptr + OFF_QO + qb * 3 * TILE + TILE + r * 128;
           const uint8_t* orow = dorow + TILE;
@@ -551,9 +597,14 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
     const int r = q4 * 32 + lane;
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     bool ok = true;
-    for (int qi = 0; qi < nq; ++qi) {
+    for (int tq = 0; tq < my_tiles; ++tq) {
+      const int item = (int)blockIdx.x + (tq / nq) * (int)gridDim.x, qi = tq % nq;
+      const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
+      const int seq_row0 = b * p.T;
+      const size_t stat0 = ((size_t)b * p.H + h) * p.T;
+      (void)seq_row0; (void)stat0;
       const int i = nq - 1 - qi;
-      if (ok && !mbar_wait(B(ACC_FULL), done(qi), abort_flag, p.status, 70)) ok = false;
+      if (ok && !mbar_wait(B(ACC_FULL), done(tq), abort_flag, p.status, 70)) ok = false;
       if (ok) {
         tc_fence_after();
 #pragma unroll
@@ -594,6 +645,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 int* g_status = nullptr;
+int g_num_sms = 0;
 __device__ int g_t5b_status[4];
 
 bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols) {
@@ -614,6 +666,10 @@ bool init_once() {
       q != cudaDriverEntryPointSuccess)
     return false;
   if (cudaGetSymbolAddress((void**)&g_status, g_t5b_status) != cudaSuccess) return false;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_num_sms < 1)
+    return false;
   if (cudaMemset(g_status, 0, sizeof(int) * 4) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(attn_bwd_dkv_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dkv::SMEM) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(attn_bwd_dq_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dq::SMEM) != cudaSuccess) return false;
@@ -635,7 +691,8 @@ cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, c
   BwdParams p;
   p.T = T; p.H = H; p.d = d; p.scale = 1.0f / sqrtf((float)DH); p.lse = lse; p.rowdot = rowdot; p.rowdot_out = rowdot;
   p.status = status ? status : g_status;
-  dim3 grid(H, nseq);
+  p.nitems = nseq * H;
+  dim3 grid((unsigned)(p.nitems < g_num_sms ? p.nitems : g_num_sms));     // one persistent CTA per SM
   // dQ first: it leaves D[row] = sum(dO * O) in `rowdot` for the dK/dV kernel
   attn_bwd_dq_t5_kernel<<<grid, NTHREADS, dq::SMEM, st>>>(mQKV, mDO, mO, mDQKV, p);
   attn_bwd_dkv_t5_kernel<<<grid, NTHREADS, dkv::SMEM, st>>>(mQKV, mDO, mDQKV, p);
