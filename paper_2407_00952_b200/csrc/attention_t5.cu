@@ -1,8 +1,8 @@
 // Causal multi-head attention forward on the 5th-generation tensor cores (tcgen05 + TMEM + TMA),
 // bf16, head width 64, sequence length a multiple of 128.
 //
-// One CTA per (sequence, head): it walks the 128-row query tiles of that head one after another
-// (set-up cost is paid once per head, K/V tiles are re-read from L2); two CTAs fit on an SM so that
+// Persistent CTAs, two per SM; each takes (sequence, head) items in turn and walks the 128-row query
+// tiles of an item one after another (K/V tiles are re-read from L2); with two CTAs on an SM
 // the softmax of one overlaps the products of the other.  Per 128-row key tile:
 //   S  = Q K^T      tcgen05.mma M128 N128 K16 x4, both operands K-major from TMA-swizzled tiles
 //   softmax         one thread per query row reads S from tensor memory (twice: row max, then
@@ -49,6 +49,7 @@ __device__ __forceinline__ float ex2(float x) {
 
 struct T5Params {
   int T, H, d;
+  int nitems;              // nseq * H (sequence, head) items, shared out over the CTAs
   float scale_log2;
   float* lse;
   int* status;
@@ -69,9 +70,14 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + OFF_BAR + 8 * N_BARS + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int h = blockIdx.x, b = blockIdx.y;
   const int nq = p.T / BQ;
-  const int seq_row0 = b * p.T;
+  // persistent: this CTA takes the (sequence, head) items blockIdx.x, blockIdx.x + gridDim.x, ... and
+  // every role walks the query tiles of all of them in one flat sequence tq = 0 .. my_tiles - 1, so
+  // the loads of the next item are issued while the current one ends
+  const int my_tiles = ((p.nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * nq;
+  auto item_of = [&](int tq) { return (int)blockIdx.x + (tq / nq) * (int)gridDim.x; };
+  auto head_of = [&](int tq) { return item_of(tq) % p.H; };
+  auto row0_of = [&](int tq) { return (item_of(tq) / p.H) * p.T; };
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < N_BARS; ++i) mbar_init(B(i), (i == S_FREE || i == P_READY || i == O_FREE) ? 128 : 1);
@@ -95,24 +101,25 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
     if (lane == 0) {
       bool ok = true;
       int it = 0;                                   // running step index of the K loads issued
-      auto load_K = [&](int step, int j) -> bool {
+      auto load_K = [&](int step, int j, int h, int seq_row0) -> bool {
         const int s = step & 1;
         if (!mbar_wait(B(K_EMPTY + s), (((uint32_t)(step >> 1)) & 1u) ^ 1u, abort_flag, p.status, 21)) return false;
         mbar_expect_tx(B(K_FULL + s), TILE);
         tma_load_2d(base + OFF_K + s * TILE, &mapQKV, B(K_FULL + s), p.d + h * DH, seq_row0 + j * BKV);
         return true;
       };
-      for (int iq = 0; iq < nq && ok; ++iq) {
-        const int qt = nq - 1 - iq;
+      for (int tq = 0; tq < my_tiles && ok; ++tq) {
+        const int qt = nq - 1 - tq % nq;
+        const int h = head_of(tq), seq_row0 = row0_of(tq);
         // Q of this query tile (the buffer is free once the previous tile's last S product is done)
-        if (!mbar_wait(B(Q_EMPTY), ((uint32_t)iq & 1u) ^ 1u, abort_flag, p.status, 20)) { ok = false; break; }
+        if (!mbar_wait(B(Q_EMPTY), ((uint32_t)tq & 1u) ^ 1u, abort_flag, p.status, 20)) { ok = false; break; }
         mbar_expect_tx(B(Q_FULL), TILE);
         tma_load_2d(base + OFF_Q, &mapQKV, B(Q_FULL), h * DH, seq_row0 + qt * BQ);
-        if (iq == 0) ok = load_K(0, 0);              // K runs one step ahead of V
+        if (tq == 0) ok = load_K(0, 0, h, seq_row0);   // K runs one step ahead of V
         for (int j = 0; j <= qt && ok; ++j, ++it) {
-          // next step's K: the next key tile, or key tile 0 of the next query tile
-          if (j < qt) ok = load_K(it + 1, j + 1);
-          else if (iq + 1 < nq) ok = load_K(it + 1, 0);
+          // next step's K: the next key tile, or key tile 0 of the next query tile (maybe of the next item)
+          if (j < qt) ok = load_K(it + 1, j + 1, h, seq_row0);
+          else if (tq + 1 < my_tiles) ok = load_K(it + 1, 0, head_of(tq + 1), row0_of(tq + 1));
           if (!ok) break;
           if (!mbar_wait(B(V_EMPTY), ((uint32_t)it & 1u) ^ 1u, abort_flag, p.status, 22)) { ok = false; break; }
           mbar_expect_tx(B(V_FULL), TILE);
@@ -127,9 +134,9 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
       const uint32_t lo_q = desc_lo(base + OFF_Q), lo_k0 = desc_lo(base + OFF_K), lo_v = desc_lo(base + OFF_V);
       constexpr uint32_t TILE16 = TILE >> 4;
       // S of step `step`; first_of_q: wait for the query tile iq; last_of_q: release the Q buffer
-      auto issue_S = [&](int step, int iq, bool first_of_q, bool last_of_q) -> bool {
+      auto issue_S = [&](int step, int tq, bool first_of_q, bool last_of_q) -> bool {
         const int s = step & 1;
-        if (first_of_q && !mbar_wait(B(Q_FULL), (uint32_t)iq & 1u, abort_flag, p.status, 25)) return false;
+        if (first_of_q && !mbar_wait(B(Q_FULL), (uint32_t)tq & 1u, abort_flag, p.status, 25)) return false;
         if (!mbar_wait(B(K_FULL + s), (uint32_t)(step >> 1) & 1u, abort_flag, p.status, 23)) return false;
         if (!mbar_wait(B(S_FREE), ((uint32_t)step & 1u) ^ 1u, abort_flag, p.status, 24)) return false;
         tc_fence_after();
@@ -145,12 +152,12 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
       };
       int it = 0;
       ok = issue_S(0, 0, true, nq - 1 == 0);
-      for (int iq = 0; iq < nq && ok; ++iq) {
-        const int qt = nq - 1 - iq;
+      for (int tq = 0; tq < my_tiles && ok; ++tq) {
+        const int qt = nq - 1 - tq % nq;
         for (int j = 0; j <= qt && ok; ++j, ++it) {
           // next step's S overlaps this step's softmax
-          if (j < qt) ok = issue_S(it + 1, iq, false, j + 1 == qt);
-          else if (iq + 1 < nq) ok = issue_S(it + 1, iq + 1, true, qt - 1 == 0);
+          if (j < qt) ok = issue_S(it + 1, tq, false, j + 1 == qt);
+          else if (tq + 1 < my_tiles) ok = issue_S(it + 1, tq + 1, true, nq - 1 - (tq + 1) % nq == 0);
           if (!ok) break;
           if (!mbar_wait(B(P_READY), (uint32_t)it & 1u, abort_flag, p.status, 26)) { ok = false; break; }
           if (!mbar_wait(B(V_FULL), (uint32_t)it & 1u, abort_flag, p.status, 27)) { ok = false; break; }
@@ -173,8 +180,9 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     bool ok = true;
     int it = 0;
-    for (int iq = 0; iq < nq; ++iq) {
-      const int qt = nq - 1 - iq;
+    for (int tq = 0; tq < my_tiles; ++tq) {
+      const int qt = nq - 1 - tq % nq;
+      const int h = head_of(tq), seq_row0 = row0_of(tq), b = seq_row0 / p.T;
       float o_acc[DH];
 #pragma unroll
       for (int i = 0; i < DH; ++i) o_acc[i] = 0.f;
@@ -303,6 +311,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 int* g_status = nullptr;      // device word for expired waits when the caller gives none
+int g_num_sms = 0;
 __device__ int g_t5_status[4];
 
 bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
@@ -323,6 +332,10 @@ bool init_once() {
       q != cudaDriverEntryPointSuccess)
     return false;
   if (cudaGetSymbolAddress((void**)&g_status, g_t5_status) != cudaSuccess) return false;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_num_sms < 1)
+    return false;
   if (cudaMemset(g_status, 0, sizeof(int) * 4) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(attn_fwd_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T5_SMEM) != cudaSuccess) return false;
   g_encode = (EncodeTiledFn)fn;
@@ -345,7 +358,8 @@ cudaError_t attention_fwd_t5(const void* qkv, int nseq, int T, int H, int d, voi
   T5Params p;
   p.T = T; p.H = H; p.d = d; p.scale_log2 = LOG2E / sqrtf((float)DH); p.lse = lse;
   p.status = status ? status : g_status;
-  dim3 grid(H, nseq);
+  p.nitems = nseq * H;
+  dim3 grid((unsigned)(p.nitems < 2 * g_num_sms ? p.nitems : 2 * g_num_sms));    // two persistent CTAs per SM
   attn_fwd_t5_kernel<<<grid, T5_THREADS, T5_SMEM, st>>>(mQKV, mO, p);
   return cudaGetLastError();
 }
