@@ -340,6 +340,104 @@ __global__ void ce_kernel(T* __restrict__ logits, int64_t ld, const int32_t* __r
   }
 }
 
+// bf16 rows with a 16-byte aligned stride: the same two passes with fewer instructions per element
+// (the arithmetic of this kernel weighs as much as its memory traffic: about 15 instructions and 2.1
+// exponentials per element in ce_kernel).  Row maximum on packed bf16 pairs, exponentials as
+// ex2(fma(z, log2 e, -max log2 e)), no per-element test for the label or the pad columns: the vectors
+// that hold only valid columns take the fast loop, the last few go element by element, and the
+// label's entry is corrected by one thread afterwards.
+__device__ __forceinline__ float ce_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__global__ void __launch_bounds__(256)
+ce_bf16_kernel(bf16* __restrict__ logits, int64_t ld, const int32_t* __restrict__ labels, int V,
+               float* __restrict__ row_loss, const int* __restrict__ n_valid) {
+  __shared__ float sh_m[32], sh_s[32];
+  __shared__ float sh_lse, sh_zy;
+  const float L = 1.4426950408889634f;
+  const int row = blockIdx.x;
+  bf16* z = logits + (size_t)row * ld;
+  uint4* zv = reinterpret_cast<uint4*>(z);
+  const int y = labels[row];
+  const bool valid = y >= 0 && y < V;
+  const int nfull = V >> 3, nvec = (int)(ld >> 3);
+  float mx = -INFINITY, sm = 0.f;
+  for (int i = threadIdx.x; i < nfull; i += blockDim.x) {
+    const uint4 raw = zv[i];
+    const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+    const uint32_t* w = reinterpret_cast<const uint32_t*>(&raw);
+    const __nv_bfloat162 m2 = __hmax2(__hmax2(h2[0], h2[1]), __hmax2(h2[2], h2[3]));
+    const float nm = fmaxf(mx, fmaxf(__low2float(m2), __high2float(m2)));
+    const float nml = -nm * L;
+    float acc = 0.f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      acc += ce_ex2(fmaf(__uint_as_float(w[k] << 16), L, nml)) + ce_ex2(fmaf(__uint_as_float(w[k] & 0xffff0000u), L, nml));
+    sm = sm * ce_ex2(fmaf(mx, L, nml)) + acc;      // mx = -inf the first time: the factor is 0
+    mx = nm;
+  }
+  for (int c = 8 * nfull + threadIdx.x; c < V; c += blockDim.x) {
+    const float zc = __bfloat162float(z[c]);
+    const float nm = fmaxf(mx, zc);
+    sm = sm * __expf(mx - nm) + __expf(zc - nm);
+    mx = nm;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    float om = __shfl_xor_sync(0xffffffffu, mx, o), os = __shfl_xor_sync(0xffffffffu, sm, o);
+    float nm = fmaxf(mx, om);
+    float a = (mx == -INFINITY) ? 0.f : sm * __expf(mx - nm);
+    float b = (om == -INFINITY) ? 0.f : os * __expf(om - nm);
+    sm = a + b; mx = nm;
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  if (lane == 0) { sh_m[warp] = mx; sh_s[warp] = sm; }
+  __syncthreads();
+  if (warp == 0) {
+    float m2 = lane < nw ? sh_m[lane] : -INFINITY, s2 = lane < nw ? sh_s[lane] : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      float om = __shfl_xor_sync(0xffffffffu, m2, o), os = __shfl_xor_sync(0xffffffffu, s2, o);
+      float nm = fmaxf(m2, om);
+      float a = (m2 == -INFINITY) ? 0.f : s2 * __expf(m2 - nm);
+      float b = (om == -INFINITY) ? 0.f : os * __expf(om - nm);
+      s2 = a + b; m2 = nm;
+    }
+    if (lane == 0) {
+      const float lse = m2 + logf(s2);
+      const float zy = valid ? __bfloat162float(z[y]) : 0.f;
+      sh_lse = lse; sh_zy = zy;
+      row_loss[row] = valid ? lse - zy : 0.f;
+    }
+  }
+  __syncthreads();
+  const float lse = sh_lse;
+  const int nv = *n_valid;
+  const float inv = (valid && nv > 0) ? 1.0f / (float)nv : 0.f;
+  const float nl = -lse * L;
+  for (int i = threadIdx.x; i < nfull; i += blockDim.x) {
+    const uint4 raw = zv[i];
+    const uint32_t* w = reinterpret_cast<const uint32_t*>(&raw);
+    uint4 out;
+    uint32_t* o = reinterpret_cast<uint32_t*>(&out);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float p0 = ce_ex2(fmaf(__uint_as_float(w[k] << 16), L, nl)) * inv;
+      const float p1 = ce_ex2(fmaf(__uint_as_float(w[k] & 0xffff0000u), L, nl)) * inv;
+      __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+      o[k] = *reinterpret_cast<uint32_t*>(&pb);
+    }
+    zv[i] = out;
+  }
+  for (int c = 8 * nfull + threadIdx.x; c < 8 * nvec; c += blockDim.x)    // last valid columns, then the pad
+    z[c] = __float2bfloat16_rn(c < V ? __expf(__bfloat162float(z[c]) - lse) * inv : 0.f);
+  __syncthreads();
+  if (threadIdx.x == 0 && valid)                     // d/dz_y = (p_y - 1) / n_valid
+    z[y] = __float2bfloat16_rn((__expf(sh_zy - lse) - 1.0f) * inv);
+}
+
 __global__ void loss_reduce_kernel(const float* __restrict__ row_loss, int M, const int* __restrict__ n_valid,
                                    float* __restrict__ loss) {
   __shared__ double sh[32];
@@ -359,7 +457,9 @@ __global__ void loss_reduce_kernel(const float* __restrict__ row_loss, int M, co
 cudaError_t cross_entropy(int dt, void* logits, int64_t ld, const int32_t* labels, int M, int V, float* row_loss,
                           int* n_valid, float* loss, int normalizer_override, cudaStream_t st) {
   count_valid_kernel<<<1, 1024, 0, st>>>(labels, M, n_valid, normalizer_override);
-  if (dt == DT_BF16) ce_kernel<bf16><<<M, 256, 0, st>>>((bf16*)logits, ld, labels, V, row_loss, n_valid);
+  if (dt == DT_BF16 && ld % 8 == 0 && (reinterpret_cast<uintptr_t>(logits) & 15u) == 0)
+    ce_bf16_kernel<<<M, 256, 0, st>>>((bf16*)logits, ld, labels, V, row_loss, n_valid);
+  else if (dt == DT_BF16) ce_kernel<bf16><<<M, 256, 0, st>>>((bf16*)logits, ld, labels, V, row_loss, n_valid);
   else ce_kernel<float><<<M, 256, 0, st>>>((float*)logits, ld, labels, V, row_loss, n_valid);
   loss_reduce_kernel<<<1, 1024, 0, st>>>(row_loss, M, n_valid, loss);
   return cudaGetLastError();
