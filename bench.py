@@ -309,8 +309,8 @@ def run_gpu(args, w):
                 # DRAM bytes of one launch from the committed ncu capture of the CTA-pair kernel
                 # (profiles/gemm_tc_pair_kernel_qkv_m32768.md): the QKV + LoRA forward launch of this
                 # workload, whose algorithmic bytes are 275 MB.  Null for any other workload.
-                "traffic": 236582400 if w.index == 3 else None,
-                "traffic_launch": "QKV+LoRA forward, M 32768 K 1024(+64) N 3072: 81.3 MB read + 155.3 MB written; "
+                "traffic": 236960000 if w.index == 3 else None,
+                "traffic_launch": "QKV+LoRA forward, M 32768 K 1024(+64) N 3072: 81.1 MB read + 155.9 MB written; "
                                   "algorithmic 275 MB" if w.index == 3 else None,
                 "launches": n_launch, "avg_launch_us": round(t_ms * 1e3 / max(1, n_launch), 2),
                 "by_class": by_class, "share_of_step": round(t_ms / ms, 4)}
