@@ -392,6 +392,14 @@ __device__ __forceinline__ void load_bias_chunk(const TcParams& p, int n, uint4*
 // chunk, so that the 32 independent element chains can be interleaved by the instruction scheduler
 // (with a test inside the loop each element is a basic block of its own and runs serially).
 // Columns past N carry garbage that the TMA store clips.
+// A warp barrier between runs of independent arithmetic.  The epilogue's element loops are long runs
+// of instructions that never wait for each other, and two warps issuing such runs on one scheduler
+// keep the single threads that feed the tensor pipe (TMA producer, MMA issuer) off it: in a
+// stand-alone loop, bursts of four products took 574-620 cycles instead of 512 next to two warps of
+// plain fp32 chains per scheduler, and 512 again with this barrier after every 32 of their
+// instructions.
+__device__ __forceinline__ void epi_yield() { __syncwarp(); }
+
 __device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, const uint4* bcur, const uint4* rpre, int n,
                                                bool tanh_form, uint32_t stage, int& buf, const CUtensorMap* mapY,
                                                const CUtensorMap* mapZ, int m_warp0, int lane) {
@@ -401,6 +409,7 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, cons
       const bf16* bp = reinterpret_cast<const bf16*>(&bcur[j]);
 #pragma unroll
       for (int i = 0; i < 8; ++i) v[8 * j + i] += __bfloat162float(bp[i]);
+      if (j & 1) epi_yield();
     }
   }
   uint32_t packed[16];
@@ -413,9 +422,13 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, cons
       zr[2 * i] = __low2float(z2);
       zr[2 * i + 1] = __high2float(z2);
     }
+    epi_yield();
     if (tanh_form) {
 #pragma unroll
-      for (int i = 0; i < 32; i += 2) { v[i] = zr[i]; v[i + 1] = zr[i + 1]; gelu_tanh_pair(v[i], v[i + 1]); }
+      for (int i = 0; i < 32; i += 2) {
+        v[i] = zr[i]; v[i + 1] = zr[i + 1]; gelu_tanh_pair(v[i], v[i + 1]);
+        if ((i & 6) == 6) epi_yield();
+      }
     } else {
 #pragma unroll
       for (int i = 0; i < 32; ++i) v[i] = gelu_f(zr[i], false);
@@ -428,6 +441,7 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, cons
       const bf16* rp = reinterpret_cast<const bf16*>(&rpre[j]);
 #pragma unroll
       for (int i = 0; i < 8; ++i) v[8 * j + i] += __bfloat162float(rp[i]);
+      if (j & 1) epi_yield();
     }
   } else if (p.epi == EPI_MUL_GELUGRAD) {
     if (tanh_form) {
@@ -435,7 +449,10 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, cons
       for (int j = 0; j < 4; ++j) {
         const uint32_t* rw = reinterpret_cast<const uint32_t*>(&rpre[j]);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) mul_gelu_grad_tanh_pair(v[8 * j + 2 * i], v[8 * j + 2 * i + 1], rw[i]);
+        for (int i = 0; i < 4; ++i) {
+          mul_gelu_grad_tanh_pair(v[8 * j + 2 * i], v[8 * j + 2 * i + 1], rw[i]);
+          if (i & 1) epi_yield();
+        }
       }
     } else {
 #pragma unroll
@@ -451,6 +468,7 @@ __device__ __forceinline__ void epilogue_chunk(const TcParams& p, float* v, cons
     __nv_bfloat162 y2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
     packed[i] = *reinterpret_cast<uint32_t*>(&y2);
   }
+  epi_yield();
   stage_and_store(stage + (uint32_t)buf * 2048u, mapY, packed, lane, n, m_warp0);
   buf ^= 1;
 }
