@@ -41,14 +41,17 @@ template <int BN> struct Cfg {
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (196608 / STAGE_BYTES) > 8 ? 8 : (196608 / STAGE_BYTES);
+  // BN 64 is the HBM-bound rank-r down projection: two CTAs per SM (three stages each) keep every
+  // SM streaming when the tiles do not fill whole waves of one CTA per SM
+  static constexpr int CTAS_PER_SM = BN == 64 ? 2 : 1;
+  static constexpr int STAGES = BN == 64 ? 3 : ((196608 / STAGE_BYTES) > 8 ? 8 : (196608 / STAGE_BYTES));
   static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
   static constexpr uint32_t IDESC = make_idesc(BM, BN);
 };
 
 template <int BN>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(NUM_THREADS, Cfg<BN>::CTAS_PER_SM)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
                const __grid_constant__ CUtensorMap mapXe, const __grid_constant__ CUtensorMap mapWe,
                const __grid_constant__ CUtensorMap mapY, const __grid_constant__ CUtensorMap mapZ, TcParams p) {
@@ -496,7 +499,8 @@ cudaError_t launch(const GemmArgs& a, int* status, cudaStream_t st) {
   if (!prepare(a, status, BN, &mX, &mW, &mXe, &mWe, &mY, &mZ, &p)) return cudaErrorInvalidValue;
   p.tiles_m = a.M / BM; p.tiles_n = (a.N + BN - 1) / BN;
   const int tiles = p.tiles_m * p.tiles_n;
-  const int grid = tiles < g_num_sms ? tiles : g_num_sms;
+  const int slots = g_num_sms * C::CTAS_PER_SM;
+  const int grid = tiles < slots ? tiles : slots;
   gemm_tc_kernel<BN><<<grid, NUM_THREADS, C::SMEM_BYTES, st>>>(mX, mW, mXe, mWe, mY, mZ, p);
   return cudaGetLastError();
 }
