@@ -5,13 +5,15 @@
 // tiles of an item one after another (K/V tiles are re-read from L2); with two CTAs on an SM
 // the softmax of one overlaps the products of the other.  Per 128-row key tile:
 //   S  = Q K^T      tcgen05.mma M128 N128 K16 x4, both operands K-major from TMA-swizzled tiles
-//   softmax         one thread per query row reads S from tensor memory (twice: row max, then
-//                   exponentials), keeps the running max / sum, writes P (bf16) back to tensor memory
+//   softmax         two threads per query row read their halves of S from tensor memory (twice:
+//                   row max, then exponentials), keep the running max / sum, write P (bf16) back to
+//                   tensor memory
 //   O' = P V        tcgen05.mma M128 N64 K16 x8, P read from tensor memory; V is used as loaded
 //                   ([key, feature] rows, i.e. an MN-major operand), no transpose
-//   O  = O*corr+O'  in registers of the row's thread
-// Warp roles (192 threads): warp 0 TMA producer, warp 1 tensor-memory owner + MMA issuer,
-// warps 2..5 softmax (warp w owns accumulator lanes 32*(w%4)..+31).
+//   O  = O*corr+O'  in registers of the row's two threads (32 columns each)
+// Warp roles (320 threads): warp 0 TMA producer, warp 1 tensor-memory owner + MMA issuer,
+// warps 2..9 softmax: two threads per query row (warp w owns accumulator lanes 32*(w%4)..+31, warps
+// 2..5 the first half of the score and output columns, warps 6..9 the second).
 // All mbarrier waits are bounded (see tc_common.cuh); on expiry a code is left in `status`.
 #include "tc_common.cuh"
 
@@ -24,9 +26,11 @@ constexpr int DH = 64;
 constexpr int BQ = 128;                   // query rows per tile
 constexpr int BKV = 128;                  // key rows per step
 constexpr int TILE = BQ * DH * 2;         // 16 KB: one [128 x 64] bf16 tile
-constexpr int T5_THREADS = 192;
-constexpr int OFF_Q = 0, OFF_K = TILE, OFF_V = 3 * TILE, OFF_P = 4 * TILE /* staging of the output tile */, OFF_BAR = 5 * TILE;
-constexpr int T5_SMEM = 5 * TILE + 256 + 1024;     // tiles + barriers + alignment slack
+constexpr int T5_THREADS = 320;           // TMA warp, MMA warp, eight softmax warps (two threads per row)
+constexpr int SM_THREADS = 256;
+constexpr int OFF_Q = 0, OFF_K = TILE, OFF_V = 3 * TILE, OFF_P = 4 * TILE /* staging of the output tile */, OFF_BAR = 5 * TILE,
+              OFF_X = 5 * TILE + 256 /* half-row maxima and sums exchanged by the two threads of a row: 4 KB */;
+constexpr int T5_SMEM = 5 * TILE + 256 + 4096 + 1024;     // tiles + barriers + exchange + alignment slack
 constexpr int TMEM_COLS = 256;            // S at columns [0,128), O' at [128,192), P (bf16) at [192,256)
 constexpr uint32_t IDESC_S = make_idesc(BQ, BKV);
 constexpr uint32_t IDESC_PV = make_idesc(BQ, DH) | (1u << 16);   // B operand MN-major
@@ -35,7 +39,7 @@ constexpr float LN2 = 0.6931471805599453f;
 
 // barrier slots
 enum { Q_FULL = 0, Q_EMPTY = 1, K_FULL = 2 /*+stage*/, K_EMPTY = 4 /*+stage*/, V_FULL = 6, V_EMPTY = 7,
-       S_FULL = 8, S_FREE = 9, P_READY = 10, O_FULL = 11, O_FREE = 12, N_BARS = 13 };
+       S_FULL = 8, S_FREE = 9, P_READY = 10, O_FULL = 11, O_FREE = 12, X_MAX = 13, X_SUM = 14, N_BARS = 15 };
 
 // Operand descriptors are passed to the products as their address-carrying lower halves (desc_lo);
 // the upper half is the same constant for the K-major tiles (Q, K, P) and for V, which is used as
@@ -80,7 +84,8 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
   auto row0_of = [&](int tq) { return (item_of(tq) / p.H) * p.T; };
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < N_BARS; ++i) mbar_init(B(i), (i == S_FREE || i == P_READY || i == O_FREE) ? 128 : 1);
+    for (int i = 0; i < N_BARS; ++i)
+      mbar_init(B(i), (i == S_FREE || i == P_READY || i == O_FREE || i == X_MAX || i == X_SUM) ? SM_THREADS : 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -174,19 +179,26 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
       }
     }
   } else {
-    // ---------------- softmax / output: one thread per query row ----------------
+    // ---------------- softmax / output: two threads per query row ----------------
+    // Warps 2..5 take score columns [0, 64) and output columns [0, 32) of their lane quarter's rows,
+    // warps 6..9 the other halves.  The two threads of a row exchange their half-row maxima through
+    // shared memory once per step (barrier X_MAX) and their partial row sums once per query tile
+    // (barrier X_SUM); everything else they do on their own halves.
     const int q = warp & 3;
+    const int hf = (warp - 2) >> 2;              // which half of the columns
     const int r = q * 32 + lane;                 // row inside the tile = accumulator lane
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+    float* xmax = reinterpret_cast<float*>(base_ptr + OFF_X);          // [2 steps][2 halves][128 rows]
+    float* xsum = xmax + 2 * 2 * BQ;                                   // [2 tiles][2 halves][128 rows]
     bool ok = true;
     int it = 0;
     for (int tq = 0; tq < my_tiles; ++tq) {
       const int qt = nq - 1 - tq % nq;
       const int h = head_of(tq), seq_row0 = row0_of(tq), b = seq_row0 / p.T;
-      float o_acc[DH];
+      float o_acc[DH / 2];
 #pragma unroll
-      for (int i = 0; i < DH; ++i) o_acc[i] = 0.f;
-      float m_run = -INFINITY, l_run = 0.f;
+      for (int i = 0; i < DH / 2; ++i) o_acc[i] = 0.f;
+      float m_run = -INFINITY, l_run = 0.f;      // l_run: this thread's half of the row sum
       for (int j = 0; j <= qt && ok; ++j, ++it) {
         if (!mbar_wait(B(S_FULL), (uint32_t)it & 1u, abort_flag, p.status, 29)) { ok = false; break; }
         tc_fence_after();
@@ -194,10 +206,11 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         // On the diagonal tile only columns <= r count; whole 32-column chunks beyond the row are
         // skipped (their probabilities are zero), the chunk that holds the diagonal is masked.
         const int c_last = diag ? (r & ~31) : (BKV - 32);       // last chunk with a live column
-        // pass 1: row maximum of the raw scores (the scale is positive)
+        const int c_lo = hf * (BKV / 2), c_hi = c_lo + BKV / 2;
+        // pass 1: maximum of the raw scores of this half row (the scale is positive)
         float mx = -INFINITY;
 #pragma unroll 1
-        for (int c = 0; c <= c_last; c += 32) {
+        for (int c = c_lo; c < c_hi && c <= c_last; c += 32) {
           float v[32];
           tc_ld32(tS + lane_off + (uint32_t)c, v);
           tc_wait_ld();
@@ -213,12 +226,17 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
           }
           mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
         }
+        float* xm = xmax + (it & 1) * 2 * BQ;
+        xm[hf * BQ + r] = mx;
+        mbar_arrive(B(X_MAX));
+        if (!mbar_wait(B(X_MAX), (uint32_t)it & 1u, abort_flag, p.status, 31)) { ok = false; break; }
+        mx = fmaxf(mx, xm[(hf ^ 1) * BQ + r]);
         const float m_new = fmaxf(m_run, mx * p.scale_log2);   // finite: column 0 is never masked
         const float corr = ex2(m_run - m_new);
-        // pass 2: exponentials, row sum, P to shared memory
+        // pass 2: exponentials, partial row sum, P back to tensor memory
         float psum = 0.f;
 #pragma unroll 1
-        for (int c = 0; c < BKV; c += 32) {
+        for (int c = c_lo; c < c_hi; c += 32) {
           uint32_t pk[16];
           if (c <= c_last) {
             float v[32];
@@ -247,48 +265,55 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         mbar_arrive(B(P_READY));                     // P complete in tensor memory
         l_run = l_run * corr + psum;
         m_run = m_new;
-        // O = O * corr + O'
+        // O = O * corr + O' on this thread's 32 output columns
         if (!mbar_wait(B(O_FULL), (uint32_t)it & 1u, abort_flag, p.status, 30)) { ok = false; break; }
         tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < DH; c += 32) {
+        {
           float v[32];
-          tc_ld32(tO + lane_off + (uint32_t)c, v);
+          tc_ld32(tO + lane_off + (uint32_t)(hf * (DH / 2)), v);
           tc_wait_ld();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) o_acc[c + i] = o_acc[c + i] * corr + v[i];
+          for (int i = 0; i < 32; ++i) o_acc[i] = o_acc[i] * corr + v[i];
         }
         tc_fence_before();
         mbar_arrive(B(O_FREE));                      // O' may be overwritten
       }
-      // normalise, stage the [128 x 64] output tile in the P buffer (free: its last product is
-      // done), one TMA store per query tile
+      // row sum = the two partial sums; normalise, stage this thread's half of the output row in the
+      // staging tile, one TMA store per query tile
+      float l_tot = l_run;
       if (ok) {
-        const float inv = 1.0f / l_run;
+        float* xs = xsum + (tq & 1) * 2 * BQ;
+        xs[hf * BQ + r] = l_run;
+        mbar_arrive(B(X_SUM));
+        if (!mbar_wait(B(X_SUM), (uint32_t)tq & 1u, abort_flag, p.status, 32)) ok = false;
+        else l_tot += xs[(hf ^ 1) * BQ + r];
+      }
+      if (ok) {
+        const float inv = 1.0f / l_tot;
         const uint32_t orow = base + OFF_P + (uint32_t)r * 128u;
 #pragma unroll
-        for (uint32_t jj = 0; jj < 8; ++jj) {
+        for (uint32_t jj = 0; jj < 4; ++jj) {
           uint32_t w[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             __nv_bfloat162 ob = __floats2bfloat162_rn(o_acc[8 * jj + 2 * i] * inv, o_acc[8 * jj + 2 * i + 1] * inv);
             w[i] = *reinterpret_cast<uint32_t*>(&ob);
           }
-          const uint32_t chunk = jj ^ ((uint32_t)r & 7u);
+          const uint32_t chunk = (jj + 4u * (uint32_t)hf) ^ ((uint32_t)r & 7u);
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(orow + (chunk << 4)), "r"(w[0]), "r"(w[1]),
                        "r"(w[2]), "r"(w[3]) : "memory");
         }
-        p.lse[((size_t)b * p.H + h) * p.T + (size_t)qt * BQ + r] = (m_run + log2f(l_run)) * LN2;
+        if (hf == 0) p.lse[((size_t)b * p.H + h) * p.T + (size_t)qt * BQ + r] = (m_run + log2f(l_tot)) * LN2;
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      asm volatile("bar.sync 1, 128;" ::: "memory");         // the four softmax warps (always reached)
+      asm volatile("bar.sync 1, 256;" ::: "memory");         // the eight softmax warps (always reached)
       if (ok && warp == 2 && lane == 0) {
         asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                      ::"l"(&mapO), "r"(base + OFF_P), "r"(h * DH), "r"(seq_row0 + qt * BQ) : "memory");
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging reusable for the next P
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging reusable for the next tile
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");
     }
     if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
