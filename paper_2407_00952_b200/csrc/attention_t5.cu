@@ -10,7 +10,9 @@
 //                   tensor memory
 //   O' = P V        tcgen05.mma M128 N64 K16 x8, P read from tensor memory; V is used as loaded
 //                   ([key, feature] rows, i.e. an MN-major operand), no transpose
-//   O  = O*corr+O'  in registers of the row's two threads (32 columns each)
+//   O += P V        accumulates in tensor memory over the key tiles of a query tile; before a step's
+//                   product the row's two threads rescale their 32 columns of O in place by the
+//                   factor the new running maximum implies
 // Warp roles (320 threads): warp 0 TMA producer, warp 1 tensor-memory owner + MMA issuer,
 // warps 2..9 softmax: two threads per query row (warp w owns accumulator lanes 32*(w%4)..+31, warps
 // 2..5 the first half of the score and output columns, warps 6..9 the second).
@@ -166,15 +168,16 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
           if (!ok) break;
           if (!mbar_wait(B(P_READY), (uint32_t)it & 1u, abort_flag, p.status, 26)) { ok = false; break; }
           if (!mbar_wait(B(V_FULL), (uint32_t)it & 1u, abort_flag, p.status, 27)) { ok = false; break; }
-          if (!mbar_wait(B(O_FREE), ((uint32_t)it & 1u) ^ 1u, abort_flag, p.status, 28)) { ok = false; break; }
+          // the first product of a query tile overwrites O: the previous tile's O must have been read
+          if (j == 0 && !mbar_wait(B(O_FREE), ((uint32_t)tq & 1u) ^ 1u, abort_flag, p.status, 28)) { ok = false; break; }
           tc_fence_after();
           // P is read from tensor memory (16 keys = 8 columns per product);
           // V advances 16 key rows = 2048 bytes = 128 units per product
 #pragma unroll
           for (int k = 0; k < BKV / UMMA_K; ++k)
-            tc_mma_ts_lo(tO, tP + (uint32_t)(8 * k), lo_v + (uint32_t)(128 * k), IDESC_PV, k != 0 ? 1u : 0u);
+            tc_mma_ts_lo(tO, tP + (uint32_t)(8 * k), lo_v + (uint32_t)(128 * k), IDESC_PV, (j | k) != 0 ? 1u : 0u);
           tc_commit(B(V_EMPTY));      // V (and P) reusable
-          tc_commit(B(O_FULL));       // O' complete
+          tc_commit(B(O_FULL));       // this step's contribution is in O
         }
       }
     }
@@ -195,9 +198,6 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
     for (int tq = 0; tq < my_tiles; ++tq) {
       const int qt = nq - 1 - tq % nq;
       const int h = head_of(tq), seq_row0 = row0_of(tq), b = seq_row0 / p.T;
-      float o_acc[DH / 2];
-#pragma unroll
-      for (int i = 0; i < DH / 2; ++i) o_acc[i] = 0.f;
       float m_run = -INFINITY, l_run = 0.f;      // l_run: this thread's half of the row sum
       for (int j = 0; j <= qt && ok; ++j, ++it) {
         if (!mbar_wait(B(S_FULL), (uint32_t)it & 1u, abort_flag, p.status, 29)) { ok = false; break; }
@@ -233,6 +233,21 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         mx = fmaxf(mx, xm[(hf ^ 1) * BQ + r]);
         const float m_new = fmaxf(m_run, mx * p.scale_log2);   // finite: column 0 is never masked
         const float corr = ex2(m_run - m_new);
+        // O stays in tensor memory and the products accumulate onto it; when the running maximum
+        // moves, this thread's 32 columns of it are rescaled in place before this step's product
+        // (which cannot start before P_READY below).  The previous step's product is long done.
+        if (j > 0) {
+          if (!mbar_wait(B(O_FULL), (uint32_t)(it - 1) & 1u, abort_flag, p.status, 30)) { ok = false; break; }
+          tc_fence_after();
+          float v[32];
+          tc_ld32(tO + lane_off + (uint32_t)(hf * (DH / 2)), v);
+          tc_wait_ld();
+          uint32_t w[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(v[i] * corr);
+          tc_st16(tO + lane_off + (uint32_t)(hf * (DH / 2)), w);
+          tc_st16(tO + lane_off + (uint32_t)(hf * (DH / 2) + 16), w + 16);
+        }
         // pass 2: exponentials, partial row sum, P back to tensor memory
         float psum = 0.f;
 #pragma unroll 1
@@ -265,18 +280,6 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         mbar_arrive(B(P_READY));                     // P complete in tensor memory
         l_run = l_run * corr + psum;
         m_run = m_new;
-        // O = O * corr + O' on this thread's 32 output columns
-        if (!mbar_wait(B(O_FULL), (uint32_t)it & 1u, abort_flag, p.status, 30)) { ok = false; break; }
-        tc_fence_after();
-        {
-          float v[32];
-          tc_ld32(tO + lane_off + (uint32_t)(hf * (DH / 2)), v);
-          tc_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o_acc[i] = o_acc[i] * corr + v[i];
-        }
-        tc_fence_before();
-        mbar_arrive(B(O_FREE));                      // O' may be overwritten
       }
       // row sum = the two partial sums; normalise, stage this thread's half of the output row in the
       // staging tile, one TMA store per query tile
@@ -288,7 +291,15 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         if (!mbar_wait(B(X_SUM), (uint32_t)tq & 1u, abort_flag, p.status, 32)) ok = false;
         else l_tot += xs[(hf ^ 1) * BQ + r];
       }
+      // the tile's last product
+      if (ok && !mbar_wait(B(O_FULL), (uint32_t)(it - 1) & 1u, abort_flag, p.status, 30)) ok = false;
       if (ok) {
+        tc_fence_after();
+        float o_acc[DH / 2];
+        tc_ld32(tO + lane_off + (uint32_t)(hf * (DH / 2)), o_acc);
+        tc_wait_ld();
+        tc_fence_before();
+        mbar_arrive(B(O_FREE));                      // O may be overwritten by the next query tile
         const float inv = 1.0f / l_tot;
         const uint32_t orow = base + OFF_P + (uint32_t)r * 128u;
 #pragma unroll
