@@ -1,17 +1,18 @@
 // Causal multi-head attention forward on the 5th-generation tensor cores (tcgen05 + TMEM + TMA),
-// bf16, head width 64, sequence length a multiple of 128.
+// bf16, head width 64 or 128, sequence length a multiple of 128.
 //
-// Persistent CTAs, two per SM; each takes (sequence, head) items in turn and walks the 128-row query
+// Persistent CTAs (two per SM at head width 64, one at 128, where every operand tile is two
+// 64-feature blocks and O takes 128 tensor-memory columns); each takes (sequence, head) items in turn and walks the 128-row query
 // tiles of an item one after another (K/V tiles are re-read from L2); with two CTAs on an SM
 // the softmax of one overlaps the products of the other.  Per 128-row key tile:
-//   S  = Q K^T      tcgen05.mma M128 N128 K16 x4, both operands K-major from TMA-swizzled tiles
+//   S  = Q K^T      tcgen05.mma M128 N128 K16 x4 per 64 features, both operands K-major from TMA-swizzled tiles
 //   softmax         two threads per query row read their halves of S from tensor memory (twice:
 //                   row max, then exponentials), keep the running max / sum, write P (bf16) back to
 //                   tensor memory
-//   O' = P V        tcgen05.mma M128 N64 K16 x8, P read from tensor memory; V is used as loaded
+//   O' = P V        tcgen05.mma M128 N64 K16 x8 per 64 output features, P read from tensor memory; V is used as loaded
 //                   ([key, feature] rows, i.e. an MN-major operand), no transpose
 //   O += P V        accumulates in tensor memory over the key tiles of a query tile; before a step's
-//                   product the row's two threads rescale their 32 columns of O in place by the
+//                   product the row's two threads rescale their halves of the columns of O in place by the
 //                   factor the new running maximum implies
 // Warp roles (320 threads): warp 0 TMA producer, warp 1 tensor-memory owner + MMA issuer,
 // warps 2..9 softmax: two threads per query row (warp w owns accumulator lanes 32*(w%4)..+31, warps
@@ -24,18 +25,24 @@ namespace {
 
 using namespace tc;
 
-constexpr int DH = 64;
 constexpr int BQ = 128;                   // query rows per tile
 constexpr int BKV = 128;                  // key rows per step
-constexpr int TILE = BQ * DH * 2;         // 16 KB: one [128 x 64] bf16 tile
+constexpr int TILE = BQ * 64 * 2;         // 16 KB: one [128 x 64] bf16 block; a head of width DH is DH / 64 blocks
 constexpr int T5_THREADS = 320;           // TMA warp, MMA warp, eight softmax warps (two threads per row)
 constexpr int SM_THREADS = 256;
-constexpr int OFF_Q = 0, OFF_K = TILE, OFF_V = 3 * TILE, OFF_P = 4 * TILE /* staging of the output tile */, OFF_BAR = 5 * TILE,
-              OFF_X = 5 * TILE + 256 /* half-row maxima and sums exchanged by the two threads of a row: 4 KB */;
-constexpr int T5_SMEM = 5 * TILE + 256 + 4096 + 1024;     // tiles + barriers + exchange + alignment slack
-constexpr int TMEM_COLS = 256;            // S at columns [0,128), O' at [128,192), P (bf16) at [192,256)
+// Head width 64: two CTAs per SM (83 KB, 256 tensor-memory columns each).  Head width 128: every
+// operand is two blocks, O takes 128 columns, one CTA per SM.
+template <int DH> struct FwdCfg {
+  static constexpr int NB = DH / 64;
+  static constexpr int OFF_Q = 0, OFF_K = NB * TILE, OFF_V = 3 * NB * TILE, OFF_P = 4 * NB * TILE /* output staging */,
+                       OFF_BAR = 5 * NB * TILE,
+                       OFF_X = OFF_BAR + 256 /* half-row maxima and sums exchanged by the two threads of a row: 4 KB */;
+  static constexpr int SMEM = 5 * NB * TILE + 256 + 4096 + 1024;     // tiles + barriers + exchange + alignment slack
+  static constexpr int TMEM_COLS = DH == 64 ? 256 : 512;             // S [0,128), O [128,128+DH), P (bf16) after it
+  static constexpr int CTAS_PER_SM = DH == 64 ? 2 : 1;
+};
 constexpr uint32_t IDESC_S = make_idesc(BQ, BKV);
-constexpr uint32_t IDESC_PV = make_idesc(BQ, DH) | (1u << 16);   // B operand MN-major
+constexpr uint32_t IDESC_PV = make_idesc(BQ, 64) | (1u << 16);   // one 64-column block of O; B operand MN-major
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
@@ -64,8 +71,12 @@ struct T5Params {
 // The CTA's work is a flat sequence of (query tile, key tile) steps: query tiles nq-1 .. 0, for
 // each the key tiles 0 .. qt.  `it` counts steps, `iq` counts query tiles; barrier parities derive
 // from these counters so that every role stays in lock step without sharing state.
-__global__ void __launch_bounds__(T5_THREADS, 2)
+template <int DH>
+__global__ void __launch_bounds__(T5_THREADS, FwdCfg<DH>::CTAS_PER_SM)
 attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapO, T5Params p) {
+  using C = FwdCfg<DH>;
+  constexpr int NB = C::NB, OFF_Q = C::OFF_Q, OFF_K = C::OFF_K, OFF_V = C::OFF_V, OFF_P = C::OFF_P, OFF_BAR = C::OFF_BAR,
+                OFF_X = C::OFF_X, TMEM_COLS = C::TMEM_COLS;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -101,7 +112,7 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tS = tmem_base, tO = tmem_base + 128u, tP = tmem_base + 192u;
+  const uint32_t tS = tmem_base, tO = tmem_base + 128u, tP = tmem_base + 128u + (uint32_t)DH;
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -111,8 +122,10 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
       auto load_K = [&](int step, int j, int h, int seq_row0) -> bool {
         const int s = step & 1;
         if (!mbar_wait(B(K_EMPTY + s), (((uint32_t)(step >> 1)) & 1u) ^ 1u, abort_flag, p.status, 21)) return false;
-        mbar_expect_tx(B(K_FULL + s), TILE);
-        tma_load_2d(base + OFF_K + s * TILE, &mapQKV, B(K_FULL + s), p.d + h * DH, seq_row0 + j * BKV);
+        mbar_expect_tx(B(K_FULL + s), NB * TILE);
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb)
+          tma_load_2d(base + OFF_K + (s * NB + nb) * TILE, &mapQKV, B(K_FULL + s), p.d + h * DH + 64 * nb, seq_row0 + j * BKV);
         return true;
       };
       for (int tq = 0; tq < my_tiles && ok; ++tq) {
@@ -120,8 +133,10 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         const int h = head_of(tq), seq_row0 = row0_of(tq);
         // Q of this query tile (the buffer is free once the previous tile's last S product is done)
         if (!mbar_wait(B(Q_EMPTY), ((uint32_t)tq & 1u) ^ 1u, abort_flag, p.status, 20)) { ok = false; break; }
-        mbar_expect_tx(B(Q_FULL), TILE);
-        tma_load_2d(base + OFF_Q, &mapQKV, B(Q_FULL), h * DH, seq_row0 + qt * BQ);
+        mbar_expect_tx(B(Q_FULL), NB * TILE);
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb)
+          tma_load_2d(base + OFF_Q + nb * TILE, &mapQKV, B(Q_FULL), h * DH + 64 * nb, seq_row0 + qt * BQ);
         if (tq == 0) ok = load_K(0, 0, h, seq_row0);   // K runs one step ahead of V
         for (int j = 0; j <= qt && ok; ++j, ++it) {
           // next step's K: the next key tile, or key tile 0 of the next query tile (maybe of the next item)
@@ -129,8 +144,10 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
           else if (tq + 1 < my_tiles) ok = load_K(it + 1, 0, head_of(tq + 1), row0_of(tq + 1));
           if (!ok) break;
           if (!mbar_wait(B(V_EMPTY), ((uint32_t)it & 1u) ^ 1u, abort_flag, p.status, 22)) { ok = false; break; }
-          mbar_expect_tx(B(V_FULL), TILE);
-          tma_load_2d(base + OFF_V, &mapQKV, B(V_FULL), 2 * p.d + h * DH, seq_row0 + j * BKV);
+          mbar_expect_tx(B(V_FULL), NB * TILE);
+#pragma unroll
+          for (int nb = 0; nb < NB; ++nb)
+            tma_load_2d(base + OFF_V + nb * TILE, &mapQKV, B(V_FULL), 2 * p.d + h * DH + 64 * nb, seq_row0 + j * BKV);
         }
       }
     }
@@ -147,11 +164,15 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         if (!mbar_wait(B(K_FULL + s), (uint32_t)(step >> 1) & 1u, abort_flag, p.status, 23)) return false;
         if (!mbar_wait(B(S_FREE), ((uint32_t)step & 1u) ^ 1u, abort_flag, p.status, 24)) return false;
         tc_fence_after();
-        const uint32_t lo_k = lo_k0 + (uint32_t)s * TILE16;
-        tc_mma_lo(tS, lo_q, lo_k, IDESC_S, 0u);              // 16 elements along K = +32 bytes = +2 units
-        tc_mma_lo_acc(tS, lo_q + 2, lo_k + 2, IDESC_S);
-        tc_mma_lo_acc(tS, lo_q + 4, lo_k + 4, IDESC_S);
-        tc_mma_lo_acc(tS, lo_q + 6, lo_k + 6, IDESC_S);
+        const uint32_t lo_k = lo_k0 + (uint32_t)(s * NB) * TILE16;
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {                    // 64 features per block; 16 elements = +32 bytes = +2 units
+          const uint32_t a = lo_q + (uint32_t)nb * TILE16, bq = lo_k + (uint32_t)nb * TILE16;
+          tc_mma_lo(tS, a, bq, IDESC_S, nb != 0 ? 1u : 0u);
+          tc_mma_lo_acc(tS, a + 2, bq + 2, IDESC_S);
+          tc_mma_lo_acc(tS, a + 4, bq + 4, IDESC_S);
+          tc_mma_lo_acc(tS, a + 6, bq + 6, IDESC_S);
+        }
         tc_commit(B(K_EMPTY + s));
         if (last_of_q) tc_commit(B(Q_EMPTY));
         tc_commit(B(S_FULL));
@@ -174,8 +195,11 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
           // P is read from tensor memory (16 keys = 8 columns per product);
           // V advances 16 key rows = 2048 bytes = 128 units per product
 #pragma unroll
-          for (int k = 0; k < BKV / UMMA_K; ++k)
-            tc_mma_ts_lo(tO, tP + (uint32_t)(8 * k), lo_v + (uint32_t)(128 * k), IDESC_PV, (j | k) != 0 ? 1u : 0u);
+          for (int nb = 0; nb < NB; ++nb)                    // one 64-column block of O per block of V
+#pragma unroll
+            for (int k = 0; k < BKV / UMMA_K; ++k)
+              tc_mma_ts_lo(tO + (uint32_t)(64 * nb), tP + (uint32_t)(8 * k), lo_v + (uint32_t)nb * TILE16 + (uint32_t)(128 * k),
+                           IDESC_PV, (j | k) != 0 ? 1u : 0u);
           tc_commit(B(V_EMPTY));      // V (and P) reusable
           tc_commit(B(O_FULL));       // this step's contribution is in O
         }
@@ -239,14 +263,17 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         if (j > 0) {
           if (!mbar_wait(B(O_FULL), (uint32_t)(it - 1) & 1u, abort_flag, p.status, 30)) { ok = false; break; }
           tc_fence_after();
-          float v[32];
-          tc_ld32(tO + lane_off + (uint32_t)(hf * (DH / 2)), v);
-          tc_wait_ld();
-          uint32_t w[32];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(v[i] * corr);
-          tc_st16(tO + lane_off + (uint32_t)(hf * (DH / 2)), w);
-          tc_st16(tO + lane_off + (uint32_t)(hf * (DH / 2) + 16), w + 16);
+          for (int oc = 0; oc < DH / 2; oc += 32) {
+            float v[32];
+            tc_ld32(tO + lane_off + (uint32_t)(hf * (DH / 2) + oc), v);
+            tc_wait_ld();
+            uint32_t w[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(v[i] * corr);
+            tc_st16(tO + lane_off + (uint32_t)(hf * (DH / 2) + oc), w);
+            tc_st16(tO + lane_off + (uint32_t)(hf * (DH / 2) + oc + 16), w + 16);
+          }
         }
         // pass 2: exponentials, partial row sum, P back to tensor memory
         float psum = 0.f;
@@ -296,21 +323,23 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
       if (ok) {
         tc_fence_after();
         float o_acc[DH / 2];
-        tc_ld32(tO + lane_off + (uint32_t)(hf * (DH / 2)), o_acc);
+#pragma unroll
+        for (int oc = 0; oc < DH / 2; oc += 32) tc_ld32(tO + lane_off + (uint32_t)(hf * (DH / 2) + oc), o_acc + oc);
         tc_wait_ld();
         tc_fence_before();
         mbar_arrive(B(O_FREE));                      // O may be overwritten by the next query tile
         const float inv = 1.0f / l_tot;
-        const uint32_t orow = base + OFF_P + (uint32_t)r * 128u;
 #pragma unroll
-        for (uint32_t jj = 0; jj < 4; ++jj) {
+        for (uint32_t jj = 0; jj < DH / 16; ++jj) {  // this thread's DH/2 columns as 16-byte chunks of 8
           uint32_t w[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             __nv_bfloat162 ob = __floats2bfloat162_rn(o_acc[8 * jj + 2 * i] * inv, o_acc[8 * jj + 2 * i + 1] * inv);
             w[i] = *reinterpret_cast<uint32_t*>(&ob);
           }
-          const uint32_t chunk = (jj + 4u * (uint32_t)hf) ^ ((uint32_t)r & 7u);
+          const uint32_t gc = (uint32_t)(hf * (DH / 2)) + 8u * jj;          // first column of the chunk in the head
+          const uint32_t orow = base + OFF_P + (gc >> 6) * TILE + (uint32_t)r * 128u;
+          const uint32_t chunk = ((gc & 63u) >> 3) ^ ((uint32_t)r & 7u);
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(orow + (chunk << 4)), "r"(w[0]), "r"(w[1]),
                        "r"(w[2]), "r"(w[3]) : "memory");
         }
@@ -319,8 +348,10 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("bar.sync 1, 256;" ::: "memory");         // the eight softmax warps (always reached)
       if (ok && warp == 2 && lane == 0) {
-        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                     ::"l"(&mapO), "r"(base + OFF_P), "r"(h * DH), "r"(seq_row0 + qt * BQ) : "memory");
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb)
+          asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                       ::"l"(&mapO), "r"(base + OFF_P + nb * TILE), "r"(h * DH + 64 * nb), "r"(seq_row0 + qt * BQ) : "memory");
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging reusable for the next tile
       }
@@ -373,7 +404,8 @@ bool init_once() {
       cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_num_sms < 1)
     return false;
   if (cudaMemset(g_status, 0, sizeof(int) * 4) != cudaSuccess) return false;
-  if (cudaFuncSetAttribute(attn_fwd_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T5_SMEM) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(attn_fwd_t5_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<64>::SMEM) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(attn_fwd_t5_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128>::SMEM) != cudaSuccess) return false;
   g_encode = (EncodeTiledFn)fn;
   return true;
 }
@@ -381,22 +413,33 @@ bool init_once() {
 }  // namespace
 
 bool attention_t5_supported(int dt, int T, int H, int d) {
-  return dt == DT_BF16 && H > 0 && d % H == 0 && d / H == DH && T >= BQ && T % BQ == 0;
+  return dt == DT_BF16 && H > 0 && d % H == 0 && d / H == 64 && T >= BQ && T % BQ == 0;
+}
+
+// The forward kernel also exists for heads of width 128 (the backward kernels do not).
+bool attention_fwd_t5_supported(int dt, int T, int H, int d) {
+  return dt == DT_BF16 && H > 0 && d % H == 0 && (d / H == 64 || d / H == 128) && T >= BQ && T % BQ == 0;
 }
 
 cudaError_t attention_fwd_t5(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, int* status,
                              cudaStream_t st) {
-  if (!attention_t5_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
+  if (!attention_fwd_t5_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
   if (!init_once()) return cudaErrorInitializationError;
   CUtensorMap mQKV, mO;
   if (!make_map(&mQKV, qkv, (uint64_t)nseq * T, (uint64_t)3 * d, BQ)) return cudaErrorInvalidValue;
   if (!make_map(&mO, o, (uint64_t)nseq * T, (uint64_t)d, BQ)) return cudaErrorInvalidValue;
+  const int dh = d / H;
   T5Params p;
-  p.T = T; p.H = H; p.d = d; p.scale_log2 = LOG2E / sqrtf((float)DH); p.lse = lse;
+  p.T = T; p.H = H; p.d = d; p.scale_log2 = LOG2E / sqrtf((float)dh); p.lse = lse;
   p.status = status ? status : g_status;
   p.nitems = nseq * H;
-  dim3 grid((unsigned)(p.nitems < 2 * g_num_sms ? p.nitems : 2 * g_num_sms));    // two persistent CTAs per SM
-  attn_fwd_t5_kernel<<<grid, T5_THREADS, T5_SMEM, st>>>(mQKV, mO, p);
+  if (dh == 64) {
+    const int cap = FwdCfg<64>::CTAS_PER_SM * g_num_sms;                         // persistent CTAs
+    attn_fwd_t5_kernel<64><<<p.nitems < cap ? p.nitems : cap, T5_THREADS, FwdCfg<64>::SMEM, st>>>(mQKV, mO, p);
+  } else {
+    const int cap = FwdCfg<128>::CTAS_PER_SM * g_num_sms;
+    attn_fwd_t5_kernel<128><<<p.nitems < cap ? p.nitems : cap, T5_THREADS, FwdCfg<128>::SMEM, st>>>(mQKV, mO, p);
+  }
   return cudaGetLastError();
 }
 

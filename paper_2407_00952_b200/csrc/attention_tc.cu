@@ -440,7 +440,7 @@ static bool prefer_mma_sync() {
 
 cudaError_t attention_fwd_tc(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, cudaStream_t st) {
   if (!attention_tc_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
-  if (attention_t5_supported(DT_BF16, T, H, d) && !prefer_mma_sync())
+  if (attention_fwd_t5_supported(DT_BF16, T, H, d) && !prefer_mma_sync())
     return attention_fwd_t5(qkv, nseq, T, H, d, o, lse, nullptr, st);
   return d / H == 64 ? launch_fwd<64>(qkv, nseq, T, H, d, o, lse, st) : launch_fwd<128>(qkv, nseq, T, H, d, o, lse, st);
 }
