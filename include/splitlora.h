@@ -172,6 +172,15 @@ int splitlora_aggregate(splitlora_ctx* ctx, const int64_t* sample_counts);
 int splitlora_round(splitlora_ctx* ctx, const int32_t* tokens, const int32_t* labels,
                     const int64_t* sample_counts, float* loss_out);
 
+/* One full t of Algorithm 1 like splitlora_round, with the two tensors that cross the cut handed off
+ * compressed (format: see splitlora_handoff_quantize): S after the client forward and dL/dS after the
+ * server step are each replaced by codes + scales, and the receiving side continues from the restored
+ * values.  codes: device, [2][M, d] bytes (S first, then dL/dS), 16-byte aligned; scales: device,
+ * [2][M] fp32; both caller-owned and left holding what the links would carry (M = K*b*T tokens).
+ * Everything else (tokens, labels, sample_counts, loss_out_host, errors) as splitlora_round. */
+int splitlora_round_compressed(splitlora_ctx* ctx, const int32_t* tokens, const int32_t* labels,
+                               const int64_t* sample_counts, uint8_t* codes, float* scales,
+                               float* loss_out_host);
 /* Same round with HOST tokens and labels: copies them to the device on the stream first.  This is
  * the end-to-end call (host in, host loss out). */
 int splitlora_round_host(splitlora_ctx* ctx, const int32_t* tokens_host, const int32_t* labels_host,
@@ -252,6 +261,24 @@ int splitlora_lora_linear_bwd(int dtype, int use_tensor_cores, const void* x, co
 int splitlora_linear(int dtype, int use_tensor_cores, const void* x, const void* W, const void* bias,
                      int epilogue, const void* r, void* z, int gelu_tanh, int M, int n_in, int n_out,
                      void* y, int* status_word, void* stream);
+/* Compressed cut-layer hand-off.  The tensors that cross the cut (S in step a2 and dL/dS in step a4
+ * of Sec. III-B) are what the paper's links carry; Sec. V (efficiency) names quantisation as the way
+ * to shrink that exchange and fixes no format.  Format of this library: per token (row of d values)
+ * one fp32 scale and d 8-bit E4M3 codes (4 exponent bits with bias 7, 3 mantissa bits, subnormals,
+ * no infinities, largest finite value 448, code 0x7F / 0xFF = NaN, never produced):
+ *   absmax = max |x[m,:]|, code[m,c] = E4M3(x[m,c] * (448 / absmax)), scales[m] = absmax / 448,
+ * nearest value with ties to the even code, all in fp32; a row of zeros has scale 0 and codes 0.
+ * _dequantize writes value(code[m,c]) * scales[m], rounded once to `dtype`.
+ * x, y: device, [M, d] row-major in `dtype` (0 fp32, 1 bf16), 16-byte aligned; codes: device, [M, d]
+ * bytes, 16-byte aligned; scales: device, [M] fp32; d a multiple of 8 (bf16) or 4 (fp32).  All
+ * buffers are the caller's; nothing is allocated; work is enqueued on `stream`.  Bytes per token
+ * handed off: d + 4 instead of 2 d (bf16) or 4 d (fp32).
+ * Errors: SPLITLORA_ERR_ARG (null pointer, M < 1, d not a multiple of the vector width, dtype),
+ * SPLITLORA_ERR_ALIGN, SPLITLORA_ERR_CUDA (launch failure). */
+int splitlora_handoff_quantize(int dtype, const void* x, int64_t M, int d, uint8_t* codes, float* scales,
+                               void* stream);
+int splitlora_handoff_dequantize(int dtype, const uint8_t* codes, const float* scales, int64_t M, int d,
+                                 void* y, void* stream);
 /* out [cols, rows] = in [rows, cols]^T in `dtype` (for building Wt). */
 int splitlora_transpose(int dtype, const void* in, int rows, int cols, void* out, void* stream);
 

@@ -31,7 +31,8 @@ EXPORTS = [
     "splitlora_transpose", "splitlora_aggregate_buffers", "splitlora_attention_fwd", "splitlora_attention_bwd",
     "splitlora_attention_bwd_static", "splitlora_linear", "splitlora_set_loss_normalizer",
     "splitlora_set_deferred_server_update", "splitlora_server_update", "splitlora_adapter_buffer",
-    "splitlora_adapters_changed", "splitlora_aggregate_partial",
+    "splitlora_adapters_changed", "splitlora_aggregate_partial", "splitlora_handoff_quantize",
+    "splitlora_handoff_dequantize", "splitlora_round_compressed",
 ]
 
 
@@ -204,6 +205,14 @@ class SplitLoRA:
                                              C.byref(loss) if want_loss else None))
         return loss.value if want_loss else None
 
+    def round_compressed(self, tokens, labels, counts, codes, scales, want_loss: bool = True):
+        """codes uint8 [2, M, d], scales fp32 [2, M]: what crosses the cut (S, then dL/dS)."""
+        arr = (C.c_int64 * len(counts))(*[int(x) for x in counts])
+        loss = C.c_float(0.0)
+        self._check(self.lib.splitlora_round_compressed(self.ctx, _ptr(tokens), _ptr(labels), arr, _ptr(codes),
+                                                        _ptr(scales), C.byref(loss) if want_loss else None))
+        return loss.value if want_loss else None
+
     def round_host(self, tokens_host: torch.Tensor, labels_host: torch.Tensor, counts, want_loss: bool = True):
         """tokens / labels are (pinned) HOST int32 tensors; the copies happen inside the call."""
         assert not tokens_host.is_cuda and tokens_host.dtype == torch.int32 and tokens_host.is_contiguous()
@@ -338,6 +347,28 @@ def linear(x, W, bias=None, epilogue=EPI_BIAS, r=None, y=None, z=None, gelu_tanh
                              _ptr(z), 1 if gelu_tanh else 0, M, n_in, n_out, _ptr(y), _ptr(_status_words[dev]),
                              _stream_ptr()), "linear")
     return (y, z) if epilogue == EPI_BIAS_GELU else y
+
+
+def handoff_quantize(x: torch.Tensor, codes: Optional[torch.Tensor] = None, scales: Optional[torch.Tensor] = None):
+    """x [M, d] -> (codes uint8 [M, d], scales fp32 [M]) (splitlora_handoff_quantize)."""
+    lib = load()
+    M, d = x.shape
+    if codes is None:
+        codes = torch.empty(M, d, dtype=torch.uint8, device="cuda")
+    if scales is None:
+        scales = torch.empty(M, dtype=torch.float32, device="cuda")
+    _rc(lib.splitlora_handoff_quantize(_dt(x), _ptr(x), C.c_int64(M), d, _ptr(codes), _ptr(scales), _stream_ptr()),
+        "handoff_quantize")
+    return codes, scales
+
+
+def handoff_dequantize(codes: torch.Tensor, scales: torch.Tensor, out: torch.Tensor) -> torch.Tensor:
+    """(codes [M, d], scales [M]) -> out [M, d] in out's dtype (splitlora_handoff_dequantize)."""
+    lib = load()
+    M, d = codes.shape
+    _rc(lib.splitlora_handoff_dequantize(_dt(out), _ptr(codes), _ptr(scales), C.c_int64(M), d, _ptr(out), _stream_ptr()),
+        "handoff_dequantize")
+    return out
 
 
 def transpose(t: torch.Tensor) -> torch.Tensor:

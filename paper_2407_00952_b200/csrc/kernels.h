@@ -151,5 +151,9 @@ struct AdapterCopyArgs {
 cudaError_t refresh_adapter_copies(const AdapterCopyArgs& a, cudaStream_t st);
 
 cudaError_t transpose(int dt, const void* in, int rows, int cols, void* out, int64_t ldo, cudaStream_t st);
+// compressed hand-off (handoff.cu): rows of d values <-> d E4M3 codes + one fp32 scale
+cudaError_t handoff_quantize(int dt, const void* x, int64_t M, int d, uint8_t* codes, float* scales, cudaStream_t st);
+cudaError_t handoff_dequantize(int dt, const uint8_t* codes, const float* scales, int64_t M, int d, void* y,
+                               cudaStream_t st);
 
 }  // namespace sl

@@ -158,6 +158,21 @@ int splitlora_transpose(int dtype, const void* in, int rows, int cols, void* out
   return transpose(dtype, in, rows, cols, out, rows, (cudaStream_t)stream) == cudaSuccess ? SPLITLORA_OK : SPLITLORA_ERR_CUDA;
 }
 
+int splitlora_handoff_quantize(int dtype, const void* x, int64_t M, int d, uint8_t* codes, float* scales, void* stream) {
+  const int n = dtype == DT_BF16 ? 8 : 4;
+  if (!x || !codes || !scales || M < 1 || d < n || d % n != 0 || (dtype != DT_F32 && dtype != DT_BF16)) return SPLITLORA_ERR_ARG;
+  if (!aligned16(x) || !aligned16(codes)) return SPLITLORA_ERR_ALIGN;
+  return handoff_quantize(dtype, x, M, d, codes, scales, (cudaStream_t)stream) == cudaSuccess ? SPLITLORA_OK : SPLITLORA_ERR_CUDA;
+}
+
+int splitlora_handoff_dequantize(int dtype, const uint8_t* codes, const float* scales, int64_t M, int d, void* y,
+                                 void* stream) {
+  const int n = dtype == DT_BF16 ? 8 : 4;
+  if (!y || !codes || !scales || M < 1 || d < n || d % n != 0 || (dtype != DT_F32 && dtype != DT_BF16)) return SPLITLORA_ERR_ARG;
+  if (!aligned16(y) || !aligned16(codes)) return SPLITLORA_ERR_ALIGN;
+  return handoff_dequantize(dtype, codes, scales, M, d, y, (cudaStream_t)stream) == cudaSuccess ? SPLITLORA_OK : SPLITLORA_ERR_CUDA;
+}
+
 int splitlora_aggregate_buffers(float* params, int K, int64_t P, const double* weights, void* stream) {
   if (!params || !weights || K < 1 || K > AGG_MAX_CLIENTS || P < 4 || P % 4 != 0) return SPLITLORA_ERR_ARG;
   if (!aligned16(params)) return SPLITLORA_ERR_ALIGN;

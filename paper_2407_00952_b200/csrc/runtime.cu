@@ -896,6 +896,40 @@ int splitlora_round(splitlora_ctx* c, const int32_t* tokens, const int32_t* labe
   return SPLITLORA_OK;
 }
 
+int splitlora_round_compressed(splitlora_ctx* c, const int32_t* tokens, const int32_t* labels, const int64_t* counts,
+                               uint8_t* codes, float* scales, float* loss_out) {
+  int rc = check_ready(c);
+  if (rc) return rc;
+  if (!counts || !codes || !scales) return fail(c, SPLITLORA_ERR_ARG, "null pointer");
+  const int n = c->dt == DT_BF16 ? 8 : 4;
+  if (c->d % n != 0) return fail(c, SPLITLORA_ERR_ARG, "d_model is not a multiple of the codec's vector width");
+  if (!aligned16(codes)) return fail(c, SPLITLORA_ERR_ALIGN, "codes not 16-byte aligned");
+  const size_t Md = (size_t)c->M * (size_t)c->d;
+  // what crosses the cut is codes + scales; the receiving side restores into the buffer it reads
+  auto cross = [&](void* buf, uint8_t* q, float* sc) -> int {
+    Scope s(c, "handoff_codec", 2);
+    CK(c, handoff_quantize(c->dt, buf, c->M, c->d, q, sc, c->st));
+    CK(c, handoff_dequantize(c->dt, q, sc, c->M, c->d, buf, c->st));
+    return SPLITLORA_OK;
+  };
+  if ((rc = splitlora_client_fwd(c, tokens, c->S))) return rc;
+  if ((rc = cross(c->S, codes, scales))) return rc;
+  if ((rc = splitlora_server_step(c, c->S, labels, c->dS, nullptr))) return rc;
+  if ((rc = cross(c->dS, codes + Md, scales + c->M))) return rc;
+  if ((rc = splitlora_client_bwd(c, c->dS))) return rc;
+  c->round_index++;
+  if (c->round_index % c->cfg.agg_interval == 0)
+    if ((rc = splitlora_aggregate(c, counts))) return rc;
+  if (loss_out) {
+    CK(c, cudaMemcpyAsync(loss_out, c->loss_dev, 4, cudaMemcpyDeviceToHost, c->st));
+    CK(c, cudaStreamSynchronize(c->st));
+    int code = 0;
+    CK(c, cudaMemcpy(&code, c->status, 4, cudaMemcpyDeviceToHost));
+    if (code) return fail(c, SPLITLORA_ERR_TIMEOUT, "a bounded device wait expired (code " + std::to_string(code) + ")");
+  }
+  return SPLITLORA_OK;
+}
+
 int splitlora_round_host(splitlora_ctx* c, const int32_t* tokens_host, const int32_t* labels_host,
                          const int64_t* counts, float* loss_out) {
   int rc = check_ready(c);

@@ -154,10 +154,53 @@ def bench_split(config: int, cut: int, agg_interval: int, n_clients: int, steps:
             "aggregation_bytes_per_client": 2 * per_client, "aggregations_per_round": round(1.0 / agg_interval, 3)}
 
 
+def bench_handoff(config: int, steps: int):
+    """Compressed cut-layer hand-off (E4M3 codes + one scale per token): the two codec kernels against
+    the HBM roofline on the workload's [M, d] hand-off tensor (algorithmic bytes: the tensor once in,
+    the codes once out, and the reverse), and whole rounds with and without compression with the bytes
+    that cross the cut per round."""
+    from . import runner, synth
+    hbm, _, src = _peaks()
+    w = synth.WORKLOADS[config]
+    M, d = w.tokens_per_round, w.d_model
+    es = 2 if w.dtype == "bf16" else 4
+    dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    nset = max(2, -(-2 * L2_BYTES // (M * d * es)))           # rotate buffers so that nothing stays in L2
+    xs = [(torch.randn(M, d, device="cuda") * torch.exp(torch.randn(M, 1, device="cuda"))).to(dt) for _ in range(nset)]
+    cs = [torch.empty(M, d, dtype=torch.uint8, device="cuda") for _ in range(nset)]
+    sc = torch.empty(M, dtype=torch.float32, device="cuda")
+    q = _time(lambda i: B.handoff_quantize(xs[i % nset], cs[i % nset], sc), 20)
+    dq = _time(lambda i: B.handoff_dequantize(cs[i % nset], sc, xs[i % nset]), 20)
+    by = M * d * (es + 1) + M * 4
+    rows = [{"op": "handoff_quantize", "M": M, "d": d, "us": round(q * 1e3, 1), "GBps": round(by / q / 1e6, 1),
+             "frac_of_hbm": round(by / q / 1e6 / hbm, 3), "peak_source": src},
+            {"op": "handoff_dequantize", "M": M, "d": d, "us": round(dq * 1e3, 1), "GBps": round(by / dq / 1e6, 1),
+             "frac_of_hbm": round(by / dq / 1e6 / hbm, 3), "peak_source": src}]
+    del xs, cs
+    cads = [synth.make_adapters(w, range(w.cut)) for _ in range(w.n_clients)]
+    sads = synth.make_adapters(w, range(w.cut, w.n_layer))
+    eng = runner.make_engine(w, synth.iter_frozen(w), cads, sads, optimizer="adamw")
+    counts = synth.make_counts(w)
+    batches = []
+    for s in range(2):
+        t, l = synth.make_tokens(w, round_index=s)
+        batches.append((torch.from_numpy(t).cuda(), torch.from_numpy(l).cuda()))
+    codes = torch.empty(2, M, d, dtype=torch.uint8, device="cuda")
+    scales = torch.empty(2, M, dtype=torch.float32, device="cuda")
+    plain = _time(lambda i: eng.round(*batches[i % 2], counts, want_loss=False), steps)
+    comp = _time(lambda i: eng.round_compressed(*batches[i % 2], counts, codes, scales, want_loss=False), steps)
+    assert eng.device_status() == 0
+    rows.append({"op": "round", "config": config, "handoff": "native", "ms_per_round": round(plain, 3),
+                 "tokens_per_s": round(M / plain * 1e3, 1), "handoff_bytes_per_round": 2 * M * d * es + M * 4})
+    rows.append({"op": "round", "config": config, "handoff": "e4m3 + scale per token", "ms_per_round": round(comp, 3),
+                 "tokens_per_s": round(M / comp * 1e3, 1), "handoff_bytes_per_round": 2 * (M * d + M * 4) + M * 4})
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("what", choices=["linear", "linear-sweep", "epilogues", "aggregate", "aggregate-sweep", "attention",
-                                     "split-sweep"])
+                                     "split-sweep", "handoff"])
     ap.add_argument("--config", type=int, default=3)
     ap.add_argument("--M", type=int, default=32768)
     ap.add_argument("--n-in", type=int, default=1024)
@@ -199,6 +242,9 @@ def main():
             for lg in range(17, 27 if K == 32 else 29, 2):
                 print(json.dumps(bench_aggregate(K, 1 << lg)), flush=True)
         print(json.dumps(dict(bench_aggregate(8, 98304), note="GPT-2-medium-shaped client adapter set")))
+    elif a.what == "handoff":
+        for row in bench_handoff(a.config, 5):
+            print(json.dumps(row), flush=True)
     elif a.what == "split-sweep":
         from . import synth
         w = synth.WORKLOADS[a.config]
