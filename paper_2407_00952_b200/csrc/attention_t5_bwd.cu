@@ -75,9 +75,9 @@ __device__ __forceinline__ void mma_acc_half(uint32_t d_tmem, uint32_t a_tmem, u
 }
 // 4 products [128 x 64] = A[128 x 64] * (rows [64h, 64h + 64) of the K-major tile at blo)^T:
 // one half (64 columns) of a [128 x 128] score tile.  64 rows of 128 bytes = 512 descriptor units.
-__device__ __forceinline__ void mma_score_half(uint32_t d_tmem, uint32_t alo, uint32_t blo, int h) {
+__device__ __forceinline__ void mma_score_half(uint32_t d_tmem, uint32_t alo, uint32_t blo, int h, bool fresh = true) {
   const uint32_t b0 = blo + (uint32_t)(512 * h);
-  tc_mma_lo(d_tmem, alo, b0, IDESC_64KK, 0u);
+  tc_mma_lo(d_tmem, alo, b0, IDESC_64KK, fresh ? 0u : 1u);
   tc_mma_lo_acc(d_tmem, alo + 2, b0 + 2, IDESC_64KK);
   tc_mma_lo_acc(d_tmem, alo + 4, b0 + 4, IDESC_64KK);
   tc_mma_lo_acc(d_tmem, alo + 6, b0 + 6, IDESC_64KK);
@@ -398,26 +398,41 @@ namespace dq {
 enum { QO_FULL = 0 /*+buffer*/, QO_FULL1, QO_EMPTY /*+buffer*/, QO_EMPTY1, KV_FULL /*+s*/, KV_FULL1, KV_FULL2,
        KV_EMPTY /*+s*/, KV_EMPTY1, KV_EMPTY2, S_FULL /*+half*/, S_FULL1, S_FREE /*+half*/, S_FREE1,
        P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, N_BARS };
-// Q, dO and O of a query tile are double buffered (O only serves D[row] = sum(dO * O), which this
-// kernel computes for itself and leaves in global memory for the dK/dV kernel); K, V of a step go
-// through a ring of RING stages.
-constexpr int OFF_QO = 0 /* buffer qb: Q at +qb*3*TILE, then dO, then O */,
-              OFF_KV = 6 * TILE /* stage s: K at +s*2*TILE, V after it */,
-              OFF_OUT = 12 * TILE /* dQ staged for the TMA store */, OFF_BAR = 13 * TILE;
-constexpr int SMEM = OFF_BAR + 256 + 1024;
+// Head width 64: Q, dO and O of a query tile are double buffered (O only serves D[row] = sum(dO * O),
+// which the kernel then computes for itself and leaves in global memory for the dK/dV kernel); K, V
+// of a step go through a ring of three stages.  Head width 128: every operand is two 64-feature
+// blocks, so shared memory holds one Q / dO buffer and a ring of two K / V stages, and D[row] is read
+// from global memory (computed beforehand by a kernel of its own).
+template <int DHT> struct Cfg {
+  static constexpr int NB = DHT / 64;
+  static constexpr bool HAS_O = DHT == 64;
+  static constexpr int QOB = DHT == 64 ? 2 : 1;                 // Q / dO (/ O) buffers
+  static constexpr int RINGN = DHT == 64 ? 3 : 2;               // K / V stages
+  static constexpr int QO_TILES = (HAS_O ? 3 : 2) * NB;         // blocks per buffer: Q, then dO, then O
+  static constexpr int OFF_QO = 0;
+  static constexpr int OFF_KV = QOB * QO_TILES * TILE;          // stage s: K blocks at +s*2*NB*TILE, V blocks after them
+  static constexpr int OFF_OUT = OFF_KV + RINGN * 2 * NB * TILE;   // dQ staged for the TMA store
+  static constexpr int OFF_BAR = OFF_OUT + NB * TILE;
+  static constexpr int SMEM = OFF_BAR + 256 + 1024;
+};
 }  // namespace dq
 
+template <int DHT>
 __global__ void __launch_bounds__(NTHREADS, 1)
 attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
                       const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dq;
-  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, KV_EMPTY, KV_EMPTY + RING)
+  using C = Cfg<DHT>;
+  constexpr int NB = C::NB, QOB = C::QOB, RINGN = C::RINGN, QO_TILES = C::QO_TILES, OFF_QO = C::OFF_QO, OFF_KV = C::OFF_KV,
+                OFF_OUT = C::OFF_OUT, OFF_BAR = C::OFF_BAR;
+  constexpr bool HAS_O = C::HAS_O;
+  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, KV_EMPTY, KV_EMPTY + RINGN)
   const int nq = p.T / BT;
   // persistent: this CTA takes items blockIdx.x, blockIdx.x + gridDim.x, ... and every role walks the
   // tiles of all of them in one flat loop, so loads for the next item are issued while this one ends
   const int my_tiles = ((p.nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * nq;
-  const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDQ = tmem_base + 256u;
-  const uint32_t tDS = tmem_base + 320u;                               // dS: bf16, 64 columns
+  const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDQ = tmem_base + 256u;      // dQ: DHT columns
+  const uint32_t tDS = tmem_base + 256u + (uint32_t)DHT;               // dS: bf16, 64 columns
 
   // query tiles are walked from the last (most key tiles) to the first
   if (warp == 0) {
@@ -430,18 +445,26 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
         (void)seq_row0; (void)stat0;
-        const int i = nq - 1 - qi, qb = tq & 1;
-        if (!mbar_wait(B(QO_EMPTY + qb), freed(tq >> 1), abort_flag, p.status, 61)) { ok = false; break; }
-        mbar_expect_tx(B(QO_FULL + qb), 3 * TILE);
-        tma_load_2d(base + OFF_QO + qb * 3 * TILE, &mapQKV, B(QO_FULL + qb), h * DH, seq_row0 + i * BT);
-        tma_load_2d(base + OFF_QO + qb * 3 * TILE + TILE, &mapDO, B(QO_FULL + qb), h * DH, seq_row0 + i * BT);
-        tma_load_2d(base + OFF_QO + qb * 3 * TILE + 2 * TILE, &mapO, B(QO_FULL + qb), h * DH, seq_row0 + i * BT);
+        const int i = nq - 1 - qi, qb = tq % QOB;
+        if (!mbar_wait(B(QO_EMPTY + qb), freed(tq / QOB), abort_flag, p.status, 61)) { ok = false; break; }
+        mbar_expect_tx(B(QO_FULL + qb), QO_TILES * TILE);
+        const uint32_t qo = base + OFF_QO + qb * QO_TILES * TILE;
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+          tma_load_2d(qo + nb * TILE, &mapQKV, B(QO_FULL + qb), h * DHT + 64 * nb, seq_row0 + i * BT);
+          tma_load_2d(qo + (NB + nb) * TILE, &mapDO, B(QO_FULL + qb), h * DHT + 64 * nb, seq_row0 + i * BT);
+          if (HAS_O) tma_load_2d(qo + (2 * NB + nb) * TILE, &mapO, B(QO_FULL + qb), h * DHT + 64 * nb, seq_row0 + i * BT);
+        }
         for (int j = 0; j <= i; ++j) {
           if (!mbar_wait(B(KV_EMPTY + s), freed(n), abort_flag, p.status, 62)) { ok = false; break; }
-          mbar_expect_tx(B(KV_FULL + s), 2 * TILE);
-          tma_load_2d(base + OFF_KV + s * 2 * TILE, &mapQKV, B(KV_FULL + s), p.d + h * DH, seq_row0 + j * BT);
-          tma_load_2d(base + OFF_KV + s * 2 * TILE + TILE, &mapQKV, B(KV_FULL + s), 2 * p.d + h * DH, seq_row0 + j * BT);
-          if (++s == RING) { s = 0; ++n; }
+          mbar_expect_tx(B(KV_FULL + s), 2 * NB * TILE);
+          const uint32_t kv = base + OFF_KV + s * 2 * NB * TILE;
+#pragma unroll
+          for (int nb = 0; nb < NB; ++nb) {
+            tma_load_2d(kv + nb * TILE, &mapQKV, B(KV_FULL + s), p.d + h * DHT + 64 * nb, seq_row0 + j * BT);
+            tma_load_2d(kv + (NB + nb) * TILE, &mapQKV, B(KV_FULL + s), 2 * p.d + h * DHT + 64 * nb, seq_row0 + j * BT);
+          }
+          if (++s == RINGN) { s = 0; ++n; }
         }
       }
     }
@@ -459,22 +482,26 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
         (void)seq_row0; (void)stat0;
         const int steps = nq - qi;               // key tiles 0 .. i, i = nq-1-qi
-        const int qb = tq & 1;
-        const uint32_t lo_q = lo_qo + (uint32_t)qb * 3u * TILE16, lo_do = lo_q + TILE16;
-        if (!mbar_wait(B(QO_FULL + qb), done(tq >> 1), abort_flag, p.status, 65)) { ok = false; break; }
+        const int qb = tq % QOB;
+        const uint32_t lo_q = lo_qo + (uint32_t)(qb * QO_TILES) * TILE16, lo_do = lo_q + (uint32_t)NB * TILE16;
+        if (!mbar_wait(B(QO_FULL + qb), done(tq / QOB), abort_flag, p.status, 65)) { ok = false; break; }
         for (int st = 0; st < steps && ok; ++st, ++it) {
-          const uint32_t lo_k = lo_kv + (uint32_t)s * 2u * TILE16;
+          const uint32_t lo_k = lo_kv + (uint32_t)(s * 2 * NB) * TILE16;
           if (!mbar_wait(B(KV_FULL + s), done(n), abort_flag, p.status, 63)) { ok = false; break; }
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             if (!mbar_wait(B(S_FREE + hh), freed(it), abort_flag, p.status, 64)) { ok = false; break; }
             tc_fence_after();
-            mma_score_half(tS + 64u * hh, lo_q, lo_k, hh);
-            mma_score_half(tDP + 64u * hh, lo_do, lo_k + TILE16, hh);
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb)           // contraction over the head's features, 64 per block
+              mma_score_half(tS + 64u * hh, lo_q + (uint32_t)nb * TILE16, lo_k + (uint32_t)nb * TILE16, hh, nb == 0);
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb)
+              mma_score_half(tDP + 64u * hh, lo_do + (uint32_t)nb * TILE16, lo_k + (uint32_t)(NB + nb) * TILE16, hh, nb == 0);
             tc_commit(B(S_FULL + hh));
           }
           if (ok) tc_commit(B(KV_EMPTY + s));        // second arrival comes from the accumulating thread
-          if (++s == RING) { s = 0; ++n; }
+          if (++s == RINGN) { s = 0; ++n; }
         }
         if (ok) tc_commit(B(QO_EMPTY + qb));         // Q, dO are read by these products only
       }
@@ -495,17 +522,19 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
         const int steps = nq - qi;
         if (!mbar_wait(B(ACC_FREE), freed(tq), abort_flag, p.status, 66)) { ok = false; break; }
         for (int st = 0; st < steps && ok; ++st, ++it) {
-          const uint32_t lo_k = lo_kv + (uint32_t)s * 2u * TILE16;
+          const uint32_t lo_k = lo_kv + (uint32_t)(s * 2 * NB) * TILE16;
           if (!mbar_wait(B(KV_FULL + s), done(n), abort_flag, p.status, 63)) { ok = false; break; }
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             if (!mbar_wait(B(P_READY + hh), done(it), abort_flag, p.status, 67)) { ok = false; break; }
             tc_fence_after();
-            mma_acc_half(tDQ, tDS, lo_k, hh, st == 0 && hh == 0);
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb)           // one 64-column block of dQ per block of K
+              mma_acc_half(tDQ + 64u * nb, tDS, lo_k + (uint32_t)nb * TILE16, hh, st == 0 && hh == 0);
             tc_commit(B(P_FREE + hh));
           }
           if (ok) tc_commit(B(KV_EMPTY + s));
-          if (++s == RING) { s = 0; ++n; }
+          if (++s == RINGN) { s = 0; ++n; }
         }
         if (ok) tc_commit(B(ACC_FULL));
       }
@@ -530,9 +559,11 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       // D[row] = sum(dO * O) from the staged tiles: both have the same swizzle, so 16-byte chunk j of
       // one row holds the same eight columns in both
       float Dr = 0.f;
-      {
-        const int qb = tq & 1;
-        if (!mbar_wait(B(QO_FULL + qb), done(tq >> 1), abort_flag, p.status, 71)) ok = false;
+      if (!HAS_O) {
+        Dr = p.rowdot[stat0 + (size_t)i * BT + r];
+      } else {
+        const int qb = tq % QOB;
+        if (!mbar_wait(B(QO_FULL + qb), done(tq / QOB), abort_flag, p.status, 71)) ok = false;
         if (ok) {
           const uint8_t* dorow = base_ptr + OFF_QO + qb * 3 * TILE + TILE + r * 128;
           const uint8_t* orow = dorow + TILE;
@@ -608,7 +639,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       if (ok) {
         tc_fence_after();
 #pragma unroll
-        for (int c = 0; c < DH; c += 32) {
+        for (int c = 0; c < DHT; c += 32) {
           float v[32];
           tc_ld32(tDQ + lane_off + (uint32_t)c, v);
           tc_wait_ld();
@@ -620,7 +651,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
               __nv_bfloat162 ob = __floats2bfloat162_rn(v[8 * jj + 2 * e] * p.scale, v[8 * jj + 2 * e + 1] * p.scale);
               w[e] = *reinterpret_cast<uint32_t*>(&ob);
             }
-            st_row_chunk(base + OFF_OUT, r, (uint32_t)(c >> 3) + jj, w);
+            st_row_chunk(base + OFF_OUT + (uint32_t)(c >> 6) * TILE, r, (uint32_t)((c & 63) >> 3) + jj, w);
           }
         }
         tc_fence_before();
@@ -629,7 +660,8 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("bar.sync 1, 128;" ::: "memory");         // the four output warps (always reached)
       if (ok && warp == OUT_WARP0 && lane == 0) {
-        tma_store_2d(&mapDQKV, base + OFF_OUT, h * DH, seq_row0 + i * BT);
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) tma_store_2d(&mapDQKV, base + OFF_OUT + nb * TILE, h * DHT + 64 * nb, seq_row0 + i * BT);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
       }
@@ -672,7 +704,8 @@ bool init_once() {
     return false;
   if (cudaMemset(g_status, 0, sizeof(int) * 4) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(attn_bwd_dkv_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dkv::SMEM) != cudaSuccess) return false;
-  if (cudaFuncSetAttribute(attn_bwd_dq_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dq::SMEM) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(attn_bwd_dq_t5_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, dq::Cfg<64>::SMEM) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(attn_bwd_dq_t5_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, dq::Cfg<128>::SMEM) != cudaSuccess) return false;
   g_encode = (EncodeTiledFn)fn;
   return true;
 }
@@ -694,8 +727,32 @@ cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, c
   p.nitems = nseq * H;
   dim3 grid((unsigned)(p.nitems < g_num_sms ? p.nitems : g_num_sms));     // one persistent CTA per SM
   // dQ first: it leaves D[row] = sum(dO * O) in `rowdot` for the dK/dV kernel
-  attn_bwd_dq_t5_kernel<<<grid, NTHREADS, dq::SMEM, st>>>(mQKV, mDO, mO, mDQKV, p);
+  attn_bwd_dq_t5_kernel<64><<<grid, NTHREADS, dq::Cfg<64>::SMEM, st>>>(mQKV, mDO, mO, mDQKV, p);
   attn_bwd_dkv_t5_kernel<<<grid, NTHREADS, dkv::SMEM, st>>>(mQKV, mDO, mDQKV, p);
+  return cudaGetLastError();
+}
+
+// dQ alone for heads of width 128 (D[row] = sum(dO * O) must already be in `rowdot`; dK and dV of that
+// width are computed elsewhere).
+bool attention_bwd_dq_t5_128_supported(int dt, int T, int H, int d) {
+  return dt == DT_BF16 && H > 0 && d % H == 0 && d / H == 128 && T >= BT && T % BT == 0;
+}
+
+cudaError_t attention_bwd_dq_t5_128(const void* qkv, const float* lse, const void* d_o, const float* rowdot, int nseq,
+                                    int T, int H, int d, void* dqkv, int* status, cudaStream_t st) {
+  if (!attention_bwd_dq_t5_128_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
+  if (!init_once()) return cudaErrorInitializationError;
+  CUtensorMap mQKV, mDO, mDQKV;
+  const uint64_t rows = (uint64_t)nseq * T;
+  if (!make_map(&mQKV, qkv, rows, (uint64_t)3 * d) || !make_map(&mDO, d_o, rows, (uint64_t)d) ||
+      !make_map(&mDQKV, dqkv, rows, (uint64_t)3 * d))
+    return cudaErrorInvalidValue;
+  BwdParams p;
+  p.T = T; p.H = H; p.d = d; p.scale = 1.0f / sqrtf(128.0f); p.lse = lse; p.rowdot = rowdot; p.rowdot_out = nullptr;
+  p.status = status ? status : g_status;
+  p.nitems = nseq * H;
+  dim3 grid((unsigned)(p.nitems < g_num_sms ? p.nitems : g_num_sms));
+  attn_bwd_dq_t5_kernel<128><<<grid, NTHREADS, dq::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDO /* unused */, mDQKV, p);
   return cudaGetLastError();
 }
 
