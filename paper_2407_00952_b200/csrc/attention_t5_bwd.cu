@@ -1,5 +1,8 @@
 // Causal multi-head attention backward on the 5th-generation tensor cores (tcgen05 + TMEM + TMA),
-// bf16, head width 64, sequence length a multiple of 128.  Two kernels, no atomics, bit-reproducible:
+// bf16, head width 64 or 128, sequence length a multiple of 128.  Two kernels, no atomics,
+// bit-reproducible (product counts below are for head width 64; at 128 every operand tile is two
+// 64-feature blocks, the contractions over features take twice the products and dQ, dK, dV are two
+// 64-column blocks each):
 //
 //   attn_bwd_dkv_t5_kernel   one CTA per (sequence, head); for each 128-row key tile it walks the
 //       query tiles i >= key tile and keeps dK, dV as fp32 accumulators in tensor memory:
@@ -14,7 +17,8 @@
 //         S = Q K^T, dP = dO V^T,  dS = P (dP - D[row]),  dQ += dS K   (K as loaded: MN-major)
 //
 // D[row] = sum(dO * O) is computed by the dQ kernel from its staged dO and O tiles and left in global
-// memory for the dK/dV kernel, which runs second.  Warp roles (480 threads): warp 0 TMA producer,
+// memory for the dK/dV kernel, which runs second (head width 128: shared memory has no room for O,
+// both kernels read D from global memory, where a small kernel has put it beforehand).  Warp roles (480 threads): warp 0 TMA producer,
 // warp 1 tensor-memory owner + issuer of the score products, warp 10 issuer of the accumulating
 // products, warps 2..9 element-wise work (thread = accumulator lane, two warps per lane quarter),
 // warps 11..14 output of the finished accumulators.
@@ -33,7 +37,6 @@ constexpr int NTHREADS = 480;             // TMA warp, two MMA-issuing warps (1 
 constexpr int OUT_WARP0 = 11;             // warps 11..14 move finished accumulators to global memory
 constexpr int OUT_THREADS = 128;
 constexpr int ACC_WARP = 10;              // issues the products that accumulate dK, dV / dQ
-constexpr int RING = 3;                   // stages of the per-step operand ring (Q/dO, resp. K/V)
 constexpr int EW_THREADS = 256;           // two warps per accumulator lane quarter, 64 columns each
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t IDESC_64KK = make_idesc(BT, DH);                   // [128 x 64] products, both operands K-major
@@ -66,12 +69,17 @@ __device__ __forceinline__ void st_row_chunk(uint32_t tile, int r, uint32_t jj, 
 // over a 128-row tile.  A (P^T, dS^T or dS, bf16) lives in tensor memory at a_tmem: 128 contraction
 // elements = 64 columns, so half h starts 32 columns in and each product advances 8 columns.  B is an
 // MN-major tile used as loaded (lower descriptor half blo); 16 of its rows = 2048 bytes = 128 units.
+// With SPREAD the 64 columns of A are not side by side: each 32-column chunk of the fp32 tile they
+// were computed from holds 16 of them in its first half, so half h starts 64 columns in and the
+// third product hops to the next chunk.
+template <bool SPREAD = false>
 __device__ __forceinline__ void mma_acc_half(uint32_t d_tmem, uint32_t a_tmem, uint32_t blo, int h, bool fresh) {
-  const uint32_t a0 = a_tmem + (uint32_t)(32 * h), b0 = blo + (uint32_t)(512 * h);
+  const uint32_t a0 = a_tmem + (uint32_t)((SPREAD ? 64 : 32) * h), b0 = blo + (uint32_t)(512 * h);
+  constexpr uint32_t HOP = SPREAD ? 32u : 16u;
   tc_mma_ts_lo(d_tmem, a0, b0, IDESC_64MN, fresh ? 0u : 1u);
   tc_mma_ts_lo(d_tmem, a0 + 8, b0 + 128, IDESC_64MN, 1u);
-  tc_mma_ts_lo(d_tmem, a0 + 16, b0 + 256, IDESC_64MN, 1u);
-  tc_mma_ts_lo(d_tmem, a0 + 24, b0 + 384, IDESC_64MN, 1u);
+  tc_mma_ts_lo(d_tmem, a0 + HOP, b0 + 256, IDESC_64MN, 1u);
+  tc_mma_ts_lo(d_tmem, a0 + HOP + 8, b0 + 384, IDESC_64MN, 1u);
 }
 // 4 products [128 x 64] = A[128 x 64] * (rows [64h, 64h + 64) of the K-major tile at blo)^T:
 // one half (64 columns) of a [128 x 128] score tile.  64 rows of 128 bytes = 512 descriptor units.
@@ -143,27 +151,57 @@ namespace dkv {
 enum { KV_FULL = 0 /*+buffer*/, KV_FULL1, KV_EMPTY /*+buffer*/, KV_EMPTY1, QD_FULL /*+s*/, QD_FULL1, QD_FULL2,
        QD_EMPTY /*+s*/, QD_EMPTY1, QD_EMPTY2, S_FULL /*+half*/, S_FULL1, S_FREE /*+half*/, S_FREE1,
        P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, N_BARS };
-// K, V of a key tile are double buffered (the next key tile's arrive during this one's last steps);
-// Q, dO and the row statistics of a step go through a ring of RING stages.
-constexpr int OFF_KV = 0 /* buffer kb: K at +kb*2*TILE, V after it */,
-              OFF_QD = 4 * TILE /* stage s: Q at +s*2*TILE, dO after it */,
-              OFF_OUT = 10 * TILE /* dK, dV staged for the TMA stores */,
-              OFF_STAT = 12 * TILE /* stage s: lse at +s*1024, D at +512 */,
-              OFF_BAR = 12 * TILE + RING * 1024;
-constexpr int SMEM = OFF_BAR + 256 + 1024;
+// Head width 64: K, V of a key tile are double buffered (the next key tile's arrive during this
+// one's last steps); Q, dO and the row statistics of a step go through a ring of three stages; P^T
+// and dS^T have tensor-memory columns of their own.
+// Head width 128: every operand is two 64-feature blocks and dK, dV take 128 columns each, which
+// fills tensor memory next to S^T and dP^T.  P^T and dS^T are then written over the S^T and dP^T
+// columns they were computed from (each thread over the first half of its own 32-column chunk), and
+// a half of S^T / dP^T is only recomputed once the accumulating products that read it have
+// finished.  Shared memory holds one K / V buffer, two Q / dO stages and a two-block staging area
+// through which dK and then dV leave.
+template <int DHT> struct Cfg {
+  static constexpr int NB = DHT / 64;
+  static constexpr bool ALIAS = DHT == 128;
+  static constexpr int KVB = DHT == 64 ? 2 : 1;
+  static constexpr int RINGN = DHT == 64 ? 3 : 2;
+  static constexpr int OFF_KV = 0;                                  // buffer kb: K blocks at +kb*2*NB*TILE, V blocks after them
+  static constexpr int OFF_QD = KVB * 2 * NB * TILE;                // stage s: Q blocks at +s*2*NB*TILE, dO blocks after them
+  static constexpr int OFF_OUT = OFF_QD + RINGN * 2 * NB * TILE;    // two blocks staged for the TMA stores
+  static constexpr int OFF_STAT = OFF_OUT + 2 * TILE;               // stage s: lse at +s*1024, D at +512
+  static constexpr int OFF_BAR = OFF_STAT + RINGN * 1024;
+  static constexpr int USED = OFF_BAR + 256;
+  static constexpr int SMEM = DHT == 64 ? USED + 1024 : 232448;     // width 128 takes all a CTA can have
+};
 }  // namespace dkv
 
+template <int DHT>
 __global__ void __launch_bounds__(NTHREADS, 1)
 attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
                        const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dkv;
-  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, QD_EMPTY, QD_EMPTY + RING)
+  using C = Cfg<DHT>;
+  constexpr int NB = C::NB, KVB = C::KVB, RINGN = C::RINGN, OFF_KV = C::OFF_KV, OFF_QD = C::OFF_QD, OFF_OUT = C::OFF_OUT,
+                OFF_STAT = C::OFF_STAT, OFF_BAR = C::OFF_BAR;
+  constexpr bool ALIAS = C::ALIAS;
+  {
+    // the tiles start at the next 1024-byte boundary of the dynamic shared memory: leave, with a
+    // code, if what is left after that does not hold them (nothing has been set up yet)
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw0 = smem_u32(smem_raw);
+    if ((((raw0 + 1023u) & ~1023u) - raw0) + (uint32_t)C::USED > (uint32_t)C::SMEM) {
+      if (threadIdx.x == 0) atomicExch(p.status, 90);
+      return;
+    }
+  }
+  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, QD_EMPTY, QD_EMPTY + RINGN)
   const int nq = p.T / BT;
   // persistent: this CTA takes items blockIdx.x, blockIdx.x + gridDim.x, ... and every role walks the
   // tiles of all of them in one flat loop, so loads for the next item are issued while this one ends
   const int my_tiles = ((p.nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * nq;
-  const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDV = tmem_base + 256u, tDK = tmem_base + 320u;
-  const uint32_t tPT = tmem_base + 384u, tDST = tmem_base + 448u;     // P^T, dS^T: bf16, 64 columns each
+  const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDV = tmem_base + 256u, tDK = tmem_base + 256u + (uint32_t)DHT;
+  // P^T, dS^T (bf16): 64 columns each after dK, or on top of S^T and dP^T
+  const uint32_t tPT = ALIAS ? tS : tmem_base + 384u, tDST = ALIAS ? tDP : tmem_base + 448u;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -175,19 +213,27 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
         (void)seq_row0; (void)stat0;
-        const int kb = tk & 1;
-        if (!mbar_wait(B(KV_EMPTY + kb), freed(tk >> 1), abort_flag, p.status, 41)) { ok = false; break; }
-        mbar_expect_tx(B(KV_FULL + kb), 2 * TILE);
-        tma_load_2d(base + OFF_KV + kb * 2 * TILE, &mapQKV, B(KV_FULL + kb), p.d + h * DH, seq_row0 + kt * BT);
-        tma_load_2d(base + OFF_KV + kb * 2 * TILE + TILE, &mapQKV, B(KV_FULL + kb), 2 * p.d + h * DH, seq_row0 + kt * BT);
+        const int kb = tk % KVB;
+        if (!mbar_wait(B(KV_EMPTY + kb), freed(tk / KVB), abort_flag, p.status, 41)) { ok = false; break; }
+        mbar_expect_tx(B(KV_FULL + kb), 2 * NB * TILE);
+        const uint32_t kv = base + OFF_KV + kb * 2 * NB * TILE;
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+          tma_load_2d(kv + nb * TILE, &mapQKV, B(KV_FULL + kb), p.d + h * DHT + 64 * nb, seq_row0 + kt * BT);
+          tma_load_2d(kv + (NB + nb) * TILE, &mapQKV, B(KV_FULL + kb), 2 * p.d + h * DHT + 64 * nb, seq_row0 + kt * BT);
+        }
         for (int i = kt; i < nq; ++i) {
           if (!mbar_wait(B(QD_EMPTY + s), freed(n), abort_flag, p.status, 42)) { ok = false; break; }
-          mbar_expect_tx(B(QD_FULL + s), 2 * TILE + 1024);
-          tma_load_2d(base + OFF_QD + s * 2 * TILE, &mapQKV, B(QD_FULL + s), h * DH, seq_row0 + i * BT);
-          tma_load_2d(base + OFF_QD + s * 2 * TILE + TILE, &mapDO, B(QD_FULL + s), h * DH, seq_row0 + i * BT);
+          mbar_expect_tx(B(QD_FULL + s), 2 * NB * TILE + 1024);
+          const uint32_t qd = base + OFF_QD + s * 2 * NB * TILE;
+#pragma unroll
+          for (int nb = 0; nb < NB; ++nb) {
+            tma_load_2d(qd + nb * TILE, &mapQKV, B(QD_FULL + s), h * DHT + 64 * nb, seq_row0 + i * BT);
+            tma_load_2d(qd + (NB + nb) * TILE, &mapDO, B(QD_FULL + s), h * DHT + 64 * nb, seq_row0 + i * BT);
+          }
           bulk_load(base + OFF_STAT + s * 1024, p.lse + stat0 + (size_t)i * BT, 512, B(QD_FULL + s));
           bulk_load(base + OFF_STAT + s * 1024 + 512, p.rowdot + stat0 + (size_t)i * BT, 512, B(QD_FULL + s));
-          if (++s == RING) { s = 0; ++n; }
+          if (++s == RINGN) { s = 0; ++n; }
         }
       }
     }
@@ -209,22 +255,28 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
         (void)seq_row0; (void)stat0;
-        const int kb = tk & 1;
-        const uint32_t lo_k = lo_kv + (uint32_t)kb * 2u * TILE16, lo_v = lo_k + TILE16;
-        if (!mbar_wait(B(KV_FULL + kb), done(tk >> 1), abort_flag, p.status, 45)) { ok = false; break; }
+        const int kb = tk % KVB;
+        const uint32_t lo_k = lo_kv + (uint32_t)(kb * 2 * NB) * TILE16, lo_v = lo_k + (uint32_t)NB * TILE16;
+        if (!mbar_wait(B(KV_FULL + kb), done(tk / KVB), abort_flag, p.status, 45)) { ok = false; break; }
         for (int i = kt; i < nq && ok; ++i, ++it) {
-          const uint32_t lo_q = lo_qd + (uint32_t)s * 2u * TILE16;
+          const uint32_t lo_q = lo_qd + (uint32_t)(s * 2 * NB) * TILE16, lo_do = lo_q + (uint32_t)NB * TILE16;
           if (!mbar_wait(B(QD_FULL + s), done(n), abort_flag, p.status, 43)) { ok = false; break; }
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
-            if (!mbar_wait(B(S_FREE + hh), freed(it), abort_flag, p.status, 44)) { ok = false; break; }
+            // the half's columns are free once read (own P^T columns) or, where P^T and dS^T lie on
+            // top of them, once the accumulating products of the previous step have used those
+            if (!mbar_wait(B((ALIAS ? P_FREE : S_FREE) + hh), freed(it), abort_flag, p.status, 44)) { ok = false; break; }
             tc_fence_after();
-            mma_score_half(tS + 64u * hh, lo_k, lo_q, hh);
-            mma_score_half(tDP + 64u * hh, lo_v, lo_q + TILE16, hh);
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb)           // contraction over the head's features, 64 per block
+              mma_score_half(tS + 64u * hh, lo_k + (uint32_t)nb * TILE16, lo_q + (uint32_t)nb * TILE16, hh, nb == 0);
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb)
+              mma_score_half(tDP + 64u * hh, lo_v + (uint32_t)nb * TILE16, lo_do + (uint32_t)nb * TILE16, hh, nb == 0);
             tc_commit(B(S_FULL + hh));
           }
           if (ok) tc_commit(B(QD_EMPTY + s));        // second arrival comes from the accumulating thread
-          if (++s == RING) { s = 0; ++n; }
+          if (++s == RINGN) { s = 0; ++n; }
         }
         if (ok) tc_commit(B(KV_EMPTY + kb));         // K, V are read by these products only
       }
@@ -245,18 +297,22 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
         // the accumulators of the previous key tile must have been read
         if (!mbar_wait(B(ACC_FREE), freed(tk), abort_flag, p.status, 46)) { ok = false; break; }
         for (int i = kt; i < nq && ok; ++i, ++it) {
-          const uint32_t lo_q = lo_qd + (uint32_t)s * 2u * TILE16, lo_do = lo_q + TILE16;
+          const uint32_t lo_q = lo_qd + (uint32_t)(s * 2 * NB) * TILE16, lo_do = lo_q + (uint32_t)NB * TILE16;
           if (!mbar_wait(B(QD_FULL + s), done(n), abort_flag, p.status, 43)) { ok = false; break; }
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             if (!mbar_wait(B(P_READY + hh), done(it), abort_flag, p.status, 47)) { ok = false; break; }
             tc_fence_after();
-            mma_acc_half(tDV, tPT, lo_do, hh, i == kt && hh == 0);
-            mma_acc_half(tDK, tDST, lo_q, hh, i == kt && hh == 0);
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb)           // one 64-column block of dV per block of dO
+              mma_acc_half<ALIAS>(tDV + 64u * nb, tPT, lo_do + (uint32_t)nb * TILE16, hh, i == kt && hh == 0);
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb)
+              mma_acc_half<ALIAS>(tDK + 64u * nb, tDST, lo_q + (uint32_t)nb * TILE16, hh, i == kt && hh == 0);
             tc_commit(B(P_FREE + hh));
           }
           if (ok) tc_commit(B(QD_EMPTY + s));
-          if (++s == RING) { s = 0; ++n; }
+          if (++s == RINGN) { s = 0; ++n; }
         }
         if (ok) tc_commit(B(ACC_FULL));
       }
@@ -289,7 +345,8 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
         for (int hh = 0; hh < 2; ++hh) {
           const int c = hh * 64 + wsel * 32;
           if (!mbar_wait(B(S_FULL + hh), done(it), abort_flag, p.status, 49)) { ok = false; break; }
-          if (!mbar_wait(B(P_FREE + hh), freed(it), abort_flag, p.status, 50)) { ok = false; break; }
+          // (with P^T on top of S^T, S_FULL already implies that the previous step's products are done)
+          if (!ALIAS && !mbar_wait(B(P_FREE + hh), freed(it), abort_flag, p.status, 50)) { ok = false; break; }
           tc_fence_after();
           uint32_t pk[16], dk[16];
           if (c >= c_first) {
@@ -324,15 +381,17 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
 #pragma unroll
             for (int e = 0; e < 16; ++e) { pk[e] = 0u; dk[e] = 0u; }
           }
-          tc_st16(tPT + lane_off + (uint32_t)(c >> 1), pk);      // 32 bf16 = 16 columns
-          tc_st16(tDST + lane_off + (uint32_t)(c >> 1), dk);
+          // 32 bf16 = 16 columns: packed side by side, or over the first half of the chunk just read
+          const uint32_t pcol = ALIAS ? (uint32_t)c : (uint32_t)(c >> 1);
+          tc_st16(tPT + lane_off + pcol, pk);
+          tc_st16(tDST + lane_off + pcol, dk);
           tc_wait_st();
           tc_fence_before();
-          mbar_arrive(B(S_FREE + hh));                 // this half of S^T, dP^T may be overwritten
+          if (!ALIAS) mbar_arrive(B(S_FREE + hh));     // this half of S^T, dP^T may be overwritten
           mbar_arrive(B(P_READY + hh));                // this half of P^T, dS^T is complete
         }
         if (!ok) break;
-        if (++s == RING) { s = 0; ++n; }
+        if (++s == RINGN) { s = 0; ++n; }
       }
     }
   } else if (warp >= OUT_WARP0) {
@@ -350,14 +409,16 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       const size_t stat0 = ((size_t)b * p.H + h) * p.T;
       (void)seq_row0; (void)stat0;
       if (ok && !mbar_wait(B(ACC_FULL), done(tk), abort_flag, p.status, 51)) ok = false;
-      if (ok) {
-        tc_fence_after();
+      if (ok) tc_fence_after();
+      // dK (scaled), then dV, in 64-column blocks through the two staging tiles; two blocks per store
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const uint32_t tsrc = half == 0 ? tDK : tDV;
-          const float mul = half == 0 ? p.scale : 1.0f;
+      for (int blk = 0; blk < 2 * NB; ++blk) {
+        const int which = blk / NB, nb = blk % NB, slot = blk & 1;
+        if (ok) {
+          const uint32_t tsrc = (which == 0 ? tDK : tDV) + (uint32_t)(64 * nb);
+          const float mul = which == 0 ? p.scale : 1.0f;
 #pragma unroll
-          for (int c = 0; c < DH; c += 32) {
+          for (int c = 0; c < 64; c += 32) {
             float v[32];
             tc_ld32(tsrc + lane_off + (uint32_t)c, v);
             tc_wait_ld();
@@ -369,22 +430,27 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
                 __nv_bfloat162 ob = __floats2bfloat162_rn(v[8 * jj + 2 * e] * mul, v[8 * jj + 2 * e + 1] * mul);
                 w[e] = *reinterpret_cast<uint32_t*>(&ob);
               }
-              st_row_chunk(base + OFF_OUT + half * TILE, r, (uint32_t)(c >> 3) + jj, w);
+              st_row_chunk(base + OFF_OUT + slot * TILE, r, (uint32_t)(c >> 3) + jj, w);
             }
           }
+          if (blk == 2 * NB - 1) {
+            tc_fence_before();
+            mbar_arrive(B(ACC_FREE));
+          }
         }
-        tc_fence_before();
-        mbar_arrive(B(ACC_FREE));
+        if (slot == 1) {
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          asm volatile("bar.sync 1, 128;" ::: "memory");         // the four output warps (always reached)
+          if (ok && warp == OUT_WARP0 && lane == 0) {
+            const int pw = (blk - 1) / NB, pnb = (blk - 1) % NB;
+            tma_store_2d(&mapDQKV, base + OFF_OUT, (pw + 1) * p.d + h * DHT + 64 * pnb, seq_row0 + kt * BT);
+            tma_store_2d(&mapDQKV, base + OFF_OUT + TILE, (which + 1) * p.d + h * DHT + 64 * nb, seq_row0 + kt * BT);
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          }
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      asm volatile("bar.sync 1, 128;" ::: "memory");         // the four output warps (always reached)
-      if (ok && warp == OUT_WARP0 && lane == 0) {
-        tma_store_2d(&mapDQKV, base + OFF_OUT, p.d + h * DH, seq_row0 + kt * BT);
-        tma_store_2d(&mapDQKV, base + OFF_OUT + TILE, 2 * p.d + h * DH, seq_row0 + kt * BT);
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-      }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
     }
     if (warp == OUT_WARP0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
@@ -703,7 +769,8 @@ bool init_once() {
       cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_num_sms < 1)
     return false;
   if (cudaMemset(g_status, 0, sizeof(int) * 4) != cudaSuccess) return false;
-  if (cudaFuncSetAttribute(attn_bwd_dkv_t5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dkv::SMEM) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(attn_bwd_dkv_t5_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, dkv::Cfg<64>::SMEM) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(attn_bwd_dkv_t5_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, dkv::Cfg<128>::SMEM) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(attn_bwd_dq_t5_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, dq::Cfg<64>::SMEM) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(attn_bwd_dq_t5_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, dq::Cfg<128>::SMEM) != cudaSuccess) return false;
   g_encode = (EncodeTiledFn)fn;
@@ -728,19 +795,18 @@ cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, c
   dim3 grid((unsigned)(p.nitems < g_num_sms ? p.nitems : g_num_sms));     // one persistent CTA per SM
   // dQ first: it leaves D[row] = sum(dO * O) in `rowdot` for the dK/dV kernel
   attn_bwd_dq_t5_kernel<64><<<grid, NTHREADS, dq::Cfg<64>::SMEM, st>>>(mQKV, mDO, mO, mDQKV, p);
-  attn_bwd_dkv_t5_kernel<<<grid, NTHREADS, dkv::SMEM, st>>>(mQKV, mDO, mDQKV, p);
+  attn_bwd_dkv_t5_kernel<64><<<grid, NTHREADS, dkv::Cfg<64>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
   return cudaGetLastError();
 }
 
-// dQ alone for heads of width 128 (D[row] = sum(dO * O) must already be in `rowdot`; dK and dV of that
-// width are computed elsewhere).
-bool attention_bwd_dq_t5_128_supported(int dt, int T, int H, int d) {
+// Heads of width 128: D[row] = sum(dO * O) must already be in `rowdot` (both kernels read it).
+bool attention_bwd_t5_128_supported(int dt, int T, int H, int d) {
   return dt == DT_BF16 && H > 0 && d % H == 0 && d / H == 128 && T >= BT && T % BT == 0;
 }
 
-cudaError_t attention_bwd_dq_t5_128(const void* qkv, const float* lse, const void* d_o, const float* rowdot, int nseq,
+cudaError_t attention_bwd_t5_128(const void* qkv, const float* lse, const void* d_o, const float* rowdot, int nseq,
                                     int T, int H, int d, void* dqkv, int* status, cudaStream_t st) {
-  if (!attention_bwd_dq_t5_128_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
+  if (!attention_bwd_t5_128_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
   if (!init_once()) return cudaErrorInitializationError;
   CUtensorMap mQKV, mDO, mDQKV;
   const uint64_t rows = (uint64_t)nseq * T;
@@ -753,6 +819,7 @@ cudaError_t attention_bwd_dq_t5_128(const void* qkv, const float* lse, const voi
   p.nitems = nseq * H;
   dim3 grid((unsigned)(p.nitems < g_num_sms ? p.nitems : g_num_sms));
   attn_bwd_dq_t5_kernel<128><<<grid, NTHREADS, dq::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDO /* unused */, mDQKV, p);
+  attn_bwd_dkv_t5_kernel<128><<<grid, NTHREADS, dkv::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
   return cudaGetLastError();
 }
 

@@ -420,13 +420,10 @@ cudaError_t launch_bwd(const void* qkv, const void* o, const float* lse, const v
   attn_rowdot_tc_kernel<DH><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>((const bf16*)o, (const bf16*)d_o, nseq, T, H, d, rowdot);
   dim3 grid(T / BT, H, nseq);
   const float scale = 1.0f / sqrtf((float)DH);
-  if (DH == 128 && attention_bwd_dq_t5_128_supported(DT_BF16, T, H, d) && !prefer_mma_sync()) {
-    // dQ on the tcgen05 kernel (it reads D[row] from `rowdot`, written just above)
-    cudaError_t e = attention_bwd_dq_t5_128(qkv, lse, d_o, rowdot, nseq, T, H, d, dqkv, nullptr, st);
-    if (e != cudaSuccess) return e;
-  } else {
-    attn_bwd_dq_tc_kernel<DH><<<grid, NT, Sizes<DH>::DQ, st>>>((const bf16*)qkv, (const bf16*)d_o, lse, rowdot, (bf16*)dqkv, T, H, d, scale);
-  }
+  if (DH == 128 && attention_bwd_t5_128_supported(DT_BF16, T, H, d) && !prefer_mma_sync())
+    // dQ, dK, dV on the tcgen05 kernels (they read D[row] from `rowdot`, written just above)
+    return attention_bwd_t5_128(qkv, lse, d_o, rowdot, nseq, T, H, d, dqkv, nullptr, st);
+  attn_bwd_dq_tc_kernel<DH><<<grid, NT, Sizes<DH>::DQ, st>>>((const bf16*)qkv, (const bf16*)d_o, lse, rowdot, (bf16*)dqkv, T, H, d, scale);
   attn_bwd_dkv_tc_kernel<DH><<<grid, NT, Sizes<DH>::DKV, st>>>((const bf16*)qkv, (const bf16*)d_o, lse, rowdot, (bf16*)dqkv, T, H, d, scale);
   return cudaGetLastError();
 }

@@ -94,8 +94,8 @@ cudaError_t attention_bwd_simt(int dt, const void* qkv, const void* o, const flo
 // code of an expired bounded wait (nullptr: a word inside the library).
 bool attention_t5_supported(int dt, int T, int H, int d);
 bool attention_fwd_t5_supported(int dt, int T, int H, int d);
-bool attention_bwd_dq_t5_128_supported(int dt, int T, int H, int d);
-cudaError_t attention_bwd_dq_t5_128(const void* qkv, const float* lse, const void* d_o, const float* rowdot, int nseq,
+bool attention_bwd_t5_128_supported(int dt, int T, int H, int d);
+cudaError_t attention_bwd_t5_128(const void* qkv, const float* lse, const void* d_o, const float* rowdot, int nseq,
                                     int T, int H, int d, void* dqkv, int* status, cudaStream_t st);
 cudaError_t attention_fwd_t5(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, int* status,
                              cudaStream_t st);

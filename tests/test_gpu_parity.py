@@ -250,12 +250,15 @@ def test_lora_linear_fp32():
                                                 (1, 512, 2, 128, True), (3, 40, 4, 96, False),
                                                 (2, 192, 2, 256, True), (1, 1024, 1, 128, True),
                                                 (3, 128, 2, 128, True), (2, 384, 4, 256, True),
-                                                (40, 128, 8, 512, True), (37, 256, 5, 320, True)])
+                                                (40, 128, 8, 512, True), (37, 256, 5, 320, True),
+                                                (3, 128, 2, 256, True), (2, 384, 3, 384, True),
+                                                (20, 256, 8, 1024, True)])
 def test_attention_bf16(nseq, T, Hh, d, use_tc):
     """Causal attention forward/backward: tensor-core kernels (head width 64 and 128) and the plain kernels
-    (any head width, ragged length) against the oracle.  The last four cases exercise the persistent
-    tcgen05 kernels: a single query tile, an odd number of tiles (ring and double-buffer parities), and
-    more (sequence, head) items than resident CTAs, so that a CTA walks several items (320 and 185)."""
+    (any head width, ragged length) against the oracle.  Cases 7-10 exercise the persistent tcgen05
+    kernels at head width 64: a single query tile, an odd number of tiles (ring and double-buffer
+    parities), and more (sequence, head) items than resident CTAs, so that a CTA walks several items
+    (320 and 185); the last three do the same at head width 128 (160 items in the last)."""
     torch.manual_seed(T + d)
     qkv = torch.randn(nseq * T, 3 * d, device="cuda").bfloat16()
     do = torch.randn(nseq * T, d, device="cuda").bfloat16()
