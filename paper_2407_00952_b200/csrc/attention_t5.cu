@@ -88,11 +88,16 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nq = p.T / BQ;
-  // persistent: this CTA takes the (sequence, head) items blockIdx.x, blockIdx.x + gridDim.x, ... and
-  // every role walks the query tiles of all of them in one flat sequence tq = 0 .. my_tiles - 1, so
-  // the loads of the next item are issued while the current one ends
-  const int my_tiles = ((p.nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * nq;
-  auto item_of = [&](int tq) { return (int)blockIdx.x + (tq / nq) * (int)gridDim.x; };
+  // persistent: the work units are (query tile, item) pairs, item = (sequence, head), ordered by
+  // falling cost (the last query tile of every item first: it has the most key tiles); this CTA
+  // takes units blockIdx.x, blockIdx.x + gridDim.x, ..., so every CTA gets the same mix of long and
+  // short tiles.  Every role walks its units in one flat sequence tq = 0 .. my_tiles - 1, so the loads
+  // of the next unit are issued while the current one ends.
+  const int n_units = p.nitems * nq;
+  const int my_tiles = (int)blockIdx.x < n_units ? (n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  auto unit_of = [&](int tq) { return (int)blockIdx.x + tq * (int)gridDim.x; };
+  auto qt_of = [&](int tq) { return nq - 1 - unit_of(tq) / p.nitems; };
+  auto item_of = [&](int tq) { return unit_of(tq) % p.nitems; };
   auto head_of = [&](int tq) { return item_of(tq) % p.H; };
   auto row0_of = [&](int tq) { return (item_of(tq) / p.H) * p.T; };
 
@@ -129,7 +134,7 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         return true;
       };
       for (int tq = 0; tq < my_tiles && ok; ++tq) {
-        const int qt = nq - 1 - tq % nq;
+        const int qt = qt_of(tq);
         const int h = head_of(tq), seq_row0 = row0_of(tq);
         // Q of this query tile (the buffer is free once the previous tile's last S product is done)
         if (!mbar_wait(B(Q_EMPTY), ((uint32_t)tq & 1u) ^ 1u, abort_flag, p.status, 20)) { ok = false; break; }
@@ -179,13 +184,13 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
         return true;
       };
       int it = 0;
-      ok = issue_S(0, 0, true, nq - 1 == 0);
+      ok = issue_S(0, 0, true, qt_of(0) == 0);
       for (int tq = 0; tq < my_tiles && ok; ++tq) {
-        const int qt = nq - 1 - tq % nq;
+        const int qt = qt_of(tq);
         for (int j = 0; j <= qt && ok; ++j, ++it) {
           // next step's S overlaps this step's softmax
           if (j < qt) ok = issue_S(it + 1, tq, false, j + 1 == qt);
-          else if (tq + 1 < my_tiles) ok = issue_S(it + 1, tq + 1, true, nq - 1 - (tq + 1) % nq == 0);
+          else if (tq + 1 < my_tiles) ok = issue_S(it + 1, tq + 1, true, qt_of(tq + 1) == 0);
           if (!ok) break;
           if (!mbar_wait(B(P_READY), (uint32_t)it & 1u, abort_flag, p.status, 26)) { ok = false; break; }
           if (!mbar_wait(B(V_FULL), (uint32_t)it & 1u, abort_flag, p.status, 27)) { ok = false; break; }
@@ -220,7 +225,7 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
     bool ok = true;
     int it = 0;
     for (int tq = 0; tq < my_tiles; ++tq) {
-      const int qt = nq - 1 - tq % nq;
+      const int qt = qt_of(tq);
       const int h = head_of(tq), seq_row0 = row0_of(tq), b = seq_row0 / p.T;
       float m_run = -INFINITY, l_run = 0.f;      // l_run: this thread's half of the row sum
       for (int j = 0; j <= qt && ok; ++j, ++it) {

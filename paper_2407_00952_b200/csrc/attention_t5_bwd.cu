@@ -196,9 +196,11 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
   }
   T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, QD_EMPTY, QD_EMPTY + RINGN)
   const int nq = p.T / BT;
-  // persistent: this CTA takes items blockIdx.x, blockIdx.x + gridDim.x, ... and every role walks the
-  // tiles of all of them in one flat loop, so loads for the next item are issued while this one ends
-  const int my_tiles = ((p.nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * nq;
+  // persistent: the work units are (tile, item) pairs, item = (sequence, head), ordered by falling
+  // cost (the tile with the most steps of every item first); this CTA takes units blockIdx.x,
+  // blockIdx.x + gridDim.x, ..., so every CTA gets the same mix of long and short tiles, and every role
+  // walks its units in one flat loop, so loads for the next unit are issued while this one ends
+  const int my_tiles = (p.nitems * nq - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
   const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDV = tmem_base + 256u, tDK = tmem_base + 256u + (uint32_t)DHT;
   // P^T, dS^T (bf16): 64 columns each after dK, or on top of S^T and dP^T
   const uint32_t tPT = ALIAS ? tS : tmem_base + 384u, tDST = ALIAS ? tDP : tmem_base + 448u;
@@ -208,7 +210,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       bool ok = true;
       int s = 0, n = 0;                            // ring stage and how often it has been used
       for (int tk = 0; tk < my_tiles && ok; ++tk) {
-        const int item = (int)blockIdx.x + (tk / nq) * (int)gridDim.x, kt = tk % nq;
+        const int u = (int)blockIdx.x + tk * (int)gridDim.x, item = u % p.nitems, kt = u / p.nitems;
         const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -250,7 +252,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       const uint32_t lo_kv = desc_lo(base + OFF_KV), lo_qd = desc_lo(base + OFF_QD);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int tk = 0; tk < my_tiles && ok; ++tk) {
-        const int item = (int)blockIdx.x + (tk / nq) * (int)gridDim.x, kt = tk % nq;
+        const int u = (int)blockIdx.x + tk * (int)gridDim.x, item = u % p.nitems, kt = u / p.nitems;
         const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -289,7 +291,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       const uint32_t lo_qd = desc_lo(base + OFF_QD);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int tk = 0; tk < my_tiles && ok; ++tk) {
-        const int item = (int)blockIdx.x + (tk / nq) * (int)gridDim.x, kt = tk % nq;
+        const int u = (int)blockIdx.x + tk * (int)gridDim.x, item = u % p.nitems, kt = u / p.nitems;
         const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -327,7 +329,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     bool ok = true;
     int it = 0, s = 0, n = 0;
     for (int tk = 0; tk < my_tiles; ++tk) {
-      const int item = (int)blockIdx.x + (tk / nq) * (int)gridDim.x, kt = tk % nq;
+      const int u = (int)blockIdx.x + tk * (int)gridDim.x, item = u % p.nitems, kt = u / p.nitems;
       const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
       const int seq_row0 = b * p.T;
       const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -403,7 +405,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     bool ok = true;
     for (int tk = 0; tk < my_tiles; ++tk) {
-      const int item = (int)blockIdx.x + (tk / nq) * (int)gridDim.x, kt = tk % nq;
+      const int u = (int)blockIdx.x + tk * (int)gridDim.x, item = u % p.nitems, kt = u / p.nitems;
       const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
       const int seq_row0 = b * p.T;
       const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -494,9 +496,11 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
   constexpr bool HAS_O = C::HAS_O;
   T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, KV_EMPTY, KV_EMPTY + RINGN)
   const int nq = p.T / BT;
-  // persistent: this CTA takes items blockIdx.x, blockIdx.x + gridDim.x, ... and every role walks the
-  // tiles of all of them in one flat loop, so loads for the next item are issued while this one ends
-  const int my_tiles = ((p.nitems - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * nq;
+  // persistent: the work units are (tile, item) pairs, item = (sequence, head), ordered by falling
+  // cost (the tile with the most steps of every item first); this CTA takes units blockIdx.x,
+  // blockIdx.x + gridDim.x, ..., so every CTA gets the same mix of long and short tiles, and every role
+  // walks its units in one flat loop, so loads for the next unit are issued while this one ends
+  const int my_tiles = (p.nitems * nq - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
   const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDQ = tmem_base + 256u;      // dQ: DHT columns
   const uint32_t tDS = tmem_base + 256u + (uint32_t)DHT;               // dS: bf16, 64 columns
 
@@ -506,7 +510,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       bool ok = true;
       int s = 0, n = 0;
       for (int tq = 0; tq < my_tiles && ok; ++tq) {
-        const int item = (int)blockIdx.x + (tq / nq) * (int)gridDim.x, qi = tq % nq;
+        const int u = (int)blockIdx.x + tq * (int)gridDim.x, item = u % p.nitems, qi = u / p.nitems;
         const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -542,7 +546,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       const uint32_t lo_qo = desc_lo(base + OFF_QO), lo_kv = desc_lo(base + OFF_KV);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int tq = 0; tq < my_tiles && ok; ++tq) {
-        const int item = (int)blockIdx.x + (tq / nq) * (int)gridDim.x, qi = tq % nq;
+        const int u = (int)blockIdx.x + tq * (int)gridDim.x, item = u % p.nitems, qi = u / p.nitems;
         const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -580,7 +584,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       const uint32_t lo_kv = desc_lo(base + OFF_KV);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int tq = 0; tq < my_tiles && ok; ++tq) {
-        const int item = (int)blockIdx.x + (tq / nq) * (int)gridDim.x, qi = tq % nq;
+        const int u = (int)blockIdx.x + tq * (int)gridDim.x, item = u % p.nitems, qi = u / p.nitems;
         const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -615,7 +619,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
     bool ok = true;
     int it = 0;
     for (int tq = 0; tq < my_tiles; ++tq) {
-      const int item = (int)blockIdx.x + (tq / nq) * (int)gridDim.x, qi = tq % nq;
+      const int u = (int)blockIdx.x + tq * (int)gridDim.x, item = u % p.nitems, qi = u / p.nitems;
       const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
       const int seq_row0 = b * p.T;
       const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -695,7 +699,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     bool ok = true;
     for (int tq = 0; tq < my_tiles; ++tq) {
-      const int item = (int)blockIdx.x + (tq / nq) * (int)gridDim.x, qi = tq % nq;
+      const int u = (int)blockIdx.x + tq * (int)gridDim.x, item = u % p.nitems, qi = u / p.nitems;
       const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
       const int seq_row0 = b * p.T;
       const size_t stat0 = ((size_t)b * p.H + h) * p.T;

@@ -113,16 +113,16 @@ def bench_aggregate(K, P, iters=50):
             "frac_of_hbm": round(gbs / hbm, 3), "peak_source": src}
 
 
-def bench_attention(nseq, T, heads, iters=10):
+def bench_attention(nseq, T, heads, iters=10, head_dim=64):
     _, tflops, src = _peaks()
-    d = heads * 64
+    d = heads * head_dim
     qkv = torch.randn(nseq * T, 3 * d, device="cuda").bfloat16()
     do = torch.randn(nseq * T, d, device="cuda").bfloat16()
     o, lse = B.attention_fwd(qkv, nseq, T, heads, True)
     f = _time(lambda i: B.attention_fwd(qkv, nseq, T, heads, True), iters)
     b = _time(lambda i: B.attention_bwd(qkv, o, lse, do, nseq, T, heads, True), iters)
-    fl = 2.0 * nseq * heads * T * T * 64            # causal: half of 4 T^2 dh
-    return {"op": "attention", "nseq": nseq, "T": T, "heads": heads, "fwd_us": round(f * 1e3, 1),
+    fl = 2.0 * nseq * heads * T * T * head_dim      # causal: half of 4 T^2 dh
+    return {"op": "attention", "nseq": nseq, "T": T, "heads": heads, "head_dim": head_dim, "fwd_us": round(f * 1e3, 1),
             "fwd_tflops": round(fl / f / 1e9, 1), "bwd_us": round(b * 1e3, 1),
             "bwd_tflops_algorithmic": round(2.5 * fl / b / 1e9, 1), "peak_source": src}
 
@@ -212,6 +212,7 @@ def main():
     ap.add_argument("--nseq", type=int, default=64)
     ap.add_argument("--T", type=int, default=512)
     ap.add_argument("--heads", type=int, default=16)
+    ap.add_argument("--head-dim", type=int, default=64)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--no-backward", action="store_true")
     ap.add_argument("--quick", action="store_true")
@@ -255,7 +256,7 @@ def main():
                 print(json.dumps(bench_split(a.config, cut, I, w.n_clients, 5)), flush=True)
         print(json.dumps(dict(bench_split(a.config, w.cut, 1, 1, 5), note="one client: centralised baseline")), flush=True)
     else:
-        print(json.dumps(bench_attention(a.nseq, a.T, a.heads, a.iters)))
+        print(json.dumps(bench_attention(a.nseq, a.T, a.heads, a.iters, a.head_dim)))
 
 
 if __name__ == "__main__":
