@@ -4,7 +4,7 @@
 // 64-feature blocks, the contractions over features take twice the products and dQ, dK, dV are two
 // 64-column blocks each):
 //
-//   attn_bwd_dkv_t5_kernel   one CTA per (sequence, head); for each 128-row key tile it walks the
+//   attn_bwd_dkv_t5_kernel   persistent CTAs; for each 128-row key tile of a (sequence, head) it walks the
 //       query tiles i >= key tile and keeps dK, dV as fp32 accumulators in tensor memory:
 //         S^T = K Q^T, dP^T = V dO^T                (M128 N128 K16 x4 each, operands K-major)
 //         P^T = exp(S^T/sqrt(dh) - lse[q]),  dS^T = P^T (dP^T - D[q])      (one thread per key row; the
@@ -12,7 +12,7 @@
 //         dV += P^T dO,  dK += dS^T Q               (M128 N64 K16 x8 each; left operand read from
 //                                                    tensor memory, dO and Q used as loaded:
 //                                                    MN-major right operands)
-//   attn_bwd_dq_t5_kernel    one CTA per (sequence, head); for each 128-row query tile it walks the
+//   attn_bwd_dq_t5_kernel    persistent CTAs; for each 128-row query tile of a (sequence, head) it walks the
 //       key tiles j <= query tile and keeps dQ in tensor memory:
 //         S = Q K^T, dP = dO V^T,  dS = P (dP - D[row]),  dQ += dS K   (K as loaded: MN-major)
 //
