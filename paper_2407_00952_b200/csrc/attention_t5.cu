@@ -2,9 +2,10 @@
 // bf16, head width 64 or 128, sequence length a multiple of 128.
 //
 // Persistent CTAs (two per SM at head width 64, one at 128, where every operand tile is two
-// 64-feature blocks and O takes 128 tensor-memory columns); each takes (sequence, head) items in turn and walks the 128-row query
-// tiles of an item one after another (K/V tiles are re-read from L2); with two CTAs on an SM
-// the softmax of one overlaps the products of the other.  Per 128-row key tile:
+// 64-feature blocks and O takes 128 tensor-memory columns).  The work units are 128-row query tiles
+// of (sequence, head) items, longest first, dealt round-robin to the CTAs (K/V tiles are re-read
+// from L2); with two CTAs on an SM the softmax of one overlaps the products of the other.
+// Per 128-row key tile:
 //   S  = Q K^T      tcgen05.mma M128 N128 K16 x4 per 64 features, both operands K-major from TMA-swizzled tiles
 //   softmax         two threads per query row read their halves of S from tensor memory (twice:
 //                   row max, then exponentials), keep the running max / sum, write P (bf16) back to
