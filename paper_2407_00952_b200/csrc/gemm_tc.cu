@@ -37,25 +37,27 @@ constexpr int NUM_THREADS = 320;
 // ------------------------------------------------------------------------------------------
 // one CTA per tile
 // ------------------------------------------------------------------------------------------
-template <int BN> struct Cfg {
+template <int BN, bool DEEP = false> struct Cfg {
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   // BN 64 is the HBM-bound rank-r down projection: two CTAs per SM (three stages each) keep every
-  // SM streaming when the tiles do not fill whole waves of one CTA per SM
-  static constexpr int CTAS_PER_SM = BN == 64 ? 2 : 1;
-  static constexpr int STAGES = BN == 64 ? 3 : ((196608 / STAGE_BYTES) > 8 ? 8 : (196608 / STAGE_BYTES));
+  // SM streaming when the tiles do not fill whole waves of one CTA per SM.  DEEP is for the case
+  // with fewer tiles than SMs (few tokens, wide rows): then a CTA has an SM to itself and what
+  // limits it is the bytes it keeps in flight, so it takes an eight-stage ring.
+  static constexpr int CTAS_PER_SM = (BN == 64 && !DEEP) ? 2 : 1;
+  static constexpr int STAGES = BN == 64 ? (DEEP ? 8 : 3) : ((196608 / STAGE_BYTES) > 8 ? 8 : (196608 / STAGE_BYTES));
   static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
   static constexpr uint32_t IDESC = make_idesc(BM, BN);
 };
 
-template <int BN>
-__global__ void __launch_bounds__(NUM_THREADS, Cfg<BN>::CTAS_PER_SM)
+template <int BN, bool DEEP = false>
+__global__ void __launch_bounds__(NUM_THREADS, Cfg<BN, DEEP>::CTAS_PER_SM)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
                const __grid_constant__ CUtensorMap mapXe, const __grid_constant__ CUtensorMap mapWe,
                const __grid_constant__ CUtensorMap mapY, const __grid_constant__ CUtensorMap mapZ, TcParams p) {
-  using C = Cfg<BN>;
+  using C = Cfg<BN, DEEP>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -485,12 +487,13 @@ bool prepare(const GemmArgs& a, int* status, int w_box_rows, CUtensorMap* mX, CU
   return true;
 }
 
-template <int BN>
+template <int BN, bool DEEP = false>
 cudaError_t launch(const GemmArgs& a, int* status, cudaStream_t st) {
-  using C = Cfg<BN>;
+  using C = Cfg<BN, DEEP>;
+  if (BN == 64 && !DEEP && (a.M / BM) * ((a.N + BN - 1) / BN) <= g_num_sms) return launch<64, true>(a, status, st);
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -501,7 +504,7 @@ cudaError_t launch(const GemmArgs& a, int* status, cudaStream_t st) {
   const int tiles = p.tiles_m * p.tiles_n;
   const int slots = g_num_sms * C::CTAS_PER_SM;
   const int grid = tiles < slots ? tiles : slots;
-  gemm_tc_kernel<BN><<<grid, NUM_THREADS, C::SMEM_BYTES, st>>>(mX, mW, mXe, mWe, mY, mZ, p);
+  gemm_tc_kernel<BN, DEEP><<<grid, NUM_THREADS, C::SMEM_BYTES, st>>>(mX, mW, mXe, mWe, mY, mZ, p);
   return cudaGetLastError();
 }
 
