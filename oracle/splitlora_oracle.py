@@ -604,6 +604,36 @@ def aggregate_clients(state: OracleState, counts, store_fp32: bool = True):
                 ca[key][name] = avg.copy()
 
 
+def aggregate_ranks(client_mats: Sequence[np.ndarray], counts, rank_axis: int) -> np.ndarray:
+    """Clients whose adapters have different ranks r_i (Sec. V, heterogeneous configuration: the
+    paper names per-client ranks as a direction and gives no rule for averaging them).  Reading
+    taken: every matrix is padded with zeros along its rank axis (0 for A [r_i, in], 1 for
+    B [out, r_i]) to the largest rank, and Eq. 8-9 is applied to the padded matrices: rank
+    component j of the result is sum_i w_i P_i[j], a client without component j adding nothing.
+    Returns the padded average."""
+    r_max = max(np.asarray(p).shape[rank_axis] for p in client_mats)
+    padded = []
+    for p in client_mats:
+        p = np.asarray(p, dtype=F64)
+        widths = [(0, 0), (0, 0)]
+        widths[rank_axis] = (0, r_max - p.shape[rank_axis])
+        padded.append(np.pad(p, widths))
+    return aggregate(padded, counts)
+
+
+def aggregate_clients_ranks(state: OracleState, counts, store_fp32: bool = True):
+    """Stage b with per-client ranks: the padded average (aggregate_ranks) goes back to every
+    client cut to that client's own rank (its leading r_i components)."""
+    for key in list(state.client_adapters[0].keys()):
+        for name, axis in (("A", 0), ("B", 1)):
+            avg = aggregate_ranks([ca[key][name] for ca in state.client_adapters], counts, axis)
+            if store_fp32:
+                avg = avg.astype(np.float32).astype(F64)
+            for ca in state.client_adapters:
+                r_i = ca[key][name].shape[axis]
+                ca[key][name] = (avg[:r_i, :] if axis == 0 else avg[:, :r_i]).copy()
+
+
 def split_round(cfg: OracleConfig, params, state: OracleState, tokens, labels, counts):
     """One iteration t of Algorithm 1.  Returns (loss, info) where info holds S, dS and the
     gradients so that tests can compare intermediate quantities."""
