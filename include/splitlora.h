@@ -166,6 +166,16 @@ int splitlora_client_bwd(splitlora_ctx* ctx, const void* act_grad_in);
  * all zero.  Every client A and B becomes sum_i (|D_i|/|D|) P_i, written back to all K clients. */
 int splitlora_aggregate(splitlora_ctx* ctx, const int64_t* sample_counts);
 
+/* Clients with different adapter ranks (Sec. V, heterogeneous configuration: named as a direction,
+ * no rule given).  ranks: HOST int32[K], 1 <= ranks[i] <= lora_r, or NULL to return to one rank for
+ * all.  Every client stays stored at lora_r; rank components >= ranks[i] of client i (rows of A,
+ * columns of B, and their optimizer moments) are set to zero now and stay zero: their gradients are
+ * exactly zero.  The scaling stays alpha / lora_r for every client.  Aggregation applies Eq. 8-9 to
+ * these zero-padded matrices (a client without a component adds nothing to it) and each client keeps
+ * its own leading ranks[i] components of the average.  Call after the adapters have been set.
+ * Errors: SPLITLORA_ERR_ARG (rank out of range), SPLITLORA_ERR_WORKSPACE. */
+int splitlora_set_client_ranks(splitlora_ctx* ctx, const int32_t* ranks);
+
 /* One iteration t of Algorithm 1: client_fwd, server_step, client_bwd (through internal hand-off
  * buffers) and, when t % agg_interval == 0, aggregate.  tokens, labels DEVICE [K, b, T] int32;
  * sample_counts HOST; loss_out HOST or NULL. */

@@ -32,7 +32,7 @@ EXPORTS = [
     "splitlora_attention_bwd_static", "splitlora_linear", "splitlora_set_loss_normalizer",
     "splitlora_set_deferred_server_update", "splitlora_server_update", "splitlora_adapter_buffer",
     "splitlora_adapters_changed", "splitlora_aggregate_partial", "splitlora_handoff_quantize",
-    "splitlora_handoff_dequantize", "splitlora_round_compressed",
+    "splitlora_handoff_dequantize", "splitlora_round_compressed", "splitlora_set_client_ranks",
 ]
 
 
@@ -204,6 +204,14 @@ class SplitLoRA:
         self._check(self.lib.splitlora_round(self.ctx, _ptr(tokens), _ptr(labels), arr,
                                              C.byref(loss) if want_loss else None))
         return loss.value if want_loss else None
+
+    def set_client_ranks(self, ranks):
+        """Per-client adapter ranks (None: one rank for all); see splitlora_set_client_ranks."""
+        if ranks is None:
+            self._check(self.lib.splitlora_set_client_ranks(self.ctx, None))
+            return
+        arr = (C.c_int32 * len(ranks))(*[int(x) for x in ranks])
+        self._check(self.lib.splitlora_set_client_ranks(self.ctx, arr))
 
     def round_compressed(self, tokens, labels, counts, codes, scales, want_loss: bool = True):
         """codes uint8 [2, M, d], scales fp32 [2, M]: what crosses the cut (S, then dL/dS)."""

@@ -529,6 +529,29 @@ __global__ void __launch_bounds__(256) aggregate_kernel(float* __restrict__ para
   }
 }
 
+// Clients with different adapter ranks (Sec. V, heterogeneous configuration): every client is stored
+// at the configured rank r with the components it does not have equal to zero.  The arena of client
+// i is a sequence of (A [r, d], B [d, r]) pairs; this kernel zeroes rank components >= rank[i]
+// (rows of A, columns of B), e.g. after the average of Eq. 8-9 has been written back to everyone.
+struct ClientRanks { int r[AGG_MAX_CLIENTS]; };
+__global__ void rank_mask_kernel(float* __restrict__ p, int64_t n, int64_t P, int r, int d, ClientRanks ranks) {
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= n) return;
+  const int client = (int)(e / P);
+  const int64_t off = (e % P) % (2 * (int64_t)r * d);
+  const int j = off < (int64_t)r * d ? (int)(off / d) : (int)((off - (int64_t)r * d) % r);
+  if (j >= ranks.r[client]) p[e] = 0.f;
+}
+
+cudaError_t rank_mask(float* params, int K, int64_t P, int r, int d, const int* ranks_host, cudaStream_t st) {
+  if (K < 1 || K > AGG_MAX_CLIENTS || P < 1 || r < 1 || d < 1 || P % (2 * (int64_t)r * d) != 0) return cudaErrorInvalidValue;
+  ClientRanks ranks;
+  for (int k = 0; k < AGG_MAX_CLIENTS; ++k) ranks.r[k] = k < K ? ranks_host[k] : r;
+  const int64_t n = (int64_t)K * P;
+  rank_mask_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(params, n, P, r, d, ranks);
+  return cudaGetLastError();
+}
+
 cudaError_t aggregate(float* params, int K, int64_t P, const float* w_host, cudaStream_t st) {
   if (K < 1 || K > AGG_MAX_CLIENTS || P % 4 != 0) return cudaErrorInvalidValue;
   AggWeights w;

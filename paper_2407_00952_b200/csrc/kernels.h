@@ -133,6 +133,8 @@ cudaError_t optimizer_step(float* p, const float* g, float* m, float* v, int64_t
 
 // Eq. 8-9 and the write-back: every row of params [K, P] becomes sum_i w[i] params[i, :].
 static const int AGG_MAX_CLIENTS = 64;
+// zero rank components >= ranks_host[i] in client i's arena of (A [r, d], B [d, r]) pairs (P floats per client)
+cudaError_t rank_mask(float* params, int K, int64_t P, int r, int d, const int* ranks_host, cudaStream_t st);
 cudaError_t aggregate(float* params, int K, int64_t P, const float* w_host, cudaStream_t st);
 
 // Compute copies of the adapters of one layer (G groups), built from fp32 masters.

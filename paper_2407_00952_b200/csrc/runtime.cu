@@ -97,6 +97,7 @@ struct splitlora_ctx {
   // sharding over devices: global loss normaliser (0: local count) and server update left to the caller
   int64_t loss_normalizer = 0;
   bool defer_server_update = false;
+  std::vector<int> client_rank;             // per-client adapter rank (empty: every client has lora_r)
   int64_t round_index = 0, server_steps = 0, client_steps = 0;
   int64_t launches = 0;
   // profiling
@@ -822,8 +823,26 @@ static int aggregate_with_total(splitlora_ctx* c, const int64_t* counts, double 
   if (!(total > 0.0)) return fail(c, SPLITLORA_ERR_COUNTS, "all sample counts are zero");
   float w[AGG_MAX_CLIENTS];
   for (int i = 0; i < c->K; ++i) w[i] = (float)((double)counts[i] / total);
-  { Scope s(c, "aggregate", 1);
-    CK(c, aggregate(c->cp, c->K, c->Pc, w, c->st)); }
+  { Scope s(c, "aggregate", c->client_rank.empty() ? 1 : 2);
+    CK(c, aggregate(c->cp, c->K, c->Pc, w, c->st));
+    // clients of lower rank keep only their own components of the (zero-padded) average
+    if (!c->client_rank.empty()) CK(c, rank_mask(c->cp, c->K, c->Pc, c->r, c->d, c->client_rank.data(), c->st)); }
+  c->client_copies_dirty = true;
+  return SPLITLORA_OK;
+}
+
+int splitlora_set_client_ranks(splitlora_ctx* c, const int32_t* ranks) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
+  if (!ranks) { c->client_rank.clear(); return SPLITLORA_OK; }
+  for (int i = 0; i < c->K; ++i)
+    if (ranks[i] < 1 || ranks[i] > c->r) return fail(c, SPLITLORA_ERR_ARG, "client rank outside [1, lora_r]");
+  c->client_rank.assign(ranks, ranks + c->K);
+  // parameters and both moments: what a client does not have is zero from here on (its gradient is
+  // exactly zero, so the updates keep it there)
+  float* arenas[3] = {c->cp, c->cm, c->cv};
+  for (float* a : arenas) CK(c, rank_mask(a, c->K, c->Pc, c->r, c->d, c->client_rank.data(), c->st));
+  c->launches += 3;
   c->client_copies_dirty = true;
   return SPLITLORA_OK;
 }

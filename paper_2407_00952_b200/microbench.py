@@ -197,10 +197,37 @@ def bench_handoff(config: int, steps: int):
     return rows
 
 
+def bench_ranks(config: int, steps: int):
+    """Per-client adapter ranks (zero-padded storage): whole rounds with one rank for all and with a
+    mix of ranks, and the aggregation step (weighted mean + write-back, plus the rank mask) alone."""
+    from . import runner, synth
+    w = synth.WORKLOADS[config]
+    cads = [synth.make_adapters(w, range(w.cut), nonzero_b=True, salt=i + 1) for i in range(w.n_clients)]
+    sads = synth.make_adapters(w, range(w.cut, w.n_layer))
+    eng = runner.make_engine(w, synth.iter_frozen(w), cads, sads, optimizer="adamw")
+    counts = synth.make_counts(w)
+    batches = []
+    for s in range(2):
+        t, l = synth.make_tokens(w, round_index=s)
+        batches.append((torch.from_numpy(t).cuda(), torch.from_numpy(l).cuda()))
+    M = w.tokens_per_round
+    rows = []
+    mix = [max(1, w.lora_r >> (i % 3)) for i in range(w.n_clients)]
+    for name, ranks in (("one rank", None), ("mixed ranks", mix)):
+        eng.set_client_ranks(ranks)
+        ms = _time(lambda i: eng.round(*batches[i % 2], counts, want_loss=False), steps)
+        agg = _time(lambda i: eng.aggregate(counts), 50)
+        rows.append({"op": "round", "config": config, "ranks": name, "client_ranks": ranks or [w.lora_r] * w.n_clients,
+                     "ms_per_round": round(ms, 3), "tokens_per_s": round(M / ms * 1e3, 1),
+                     "aggregate_us": round(agg * 1e3, 2)})
+    assert eng.device_status() == 0
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("what", choices=["linear", "linear-sweep", "epilogues", "aggregate", "aggregate-sweep", "attention",
-                                     "split-sweep", "handoff"])
+                                     "split-sweep", "handoff", "ranks"])
     ap.add_argument("--config", type=int, default=3)
     ap.add_argument("--M", type=int, default=32768)
     ap.add_argument("--n-in", type=int, default=1024)
@@ -243,6 +270,9 @@ def main():
             for lg in range(17, 27 if K == 32 else 29, 2):
                 print(json.dumps(bench_aggregate(K, 1 << lg)), flush=True)
         print(json.dumps(dict(bench_aggregate(8, 98304), note="GPT-2-medium-shaped client adapter set")))
+    elif a.what == "ranks":
+        for row in bench_ranks(a.config, 5):
+            print(json.dumps(row), flush=True)
     elif a.what == "handoff":
         for row in bench_handoff(a.config, 5):
             print(json.dumps(row), flush=True)
