@@ -213,7 +213,7 @@ def bench_ranks(config: int, steps: int):
     M = w.tokens_per_round
     rows = []
     mix = [max(1, w.lora_r >> (i % 3)) for i in range(w.n_clients)]
-    for name, ranks in (("one rank", None), ("mixed ranks", mix)):
+    for name, ranks in (("one rank", None), ("mixed ranks", mix), ("one rank, measured again", None)):
         eng.set_client_ranks(ranks)
         ms = _time(lambda i: eng.round(*batches[i % 2], counts, want_loss=False), steps)
         agg = _time(lambda i: eng.aggregate(counts), 50)
