@@ -274,6 +274,33 @@ def test_attention_bf16(nseq, T, Hh, d, use_tc):
         assert H.rel_err(got[:, j * d:(j + 1) * d], ref.reshape(-1, d)) <= TOL_BF16
 
 
+@pytest.mark.parametrize("Hh,d", [(2, 128), (2, 256)])
+def test_attention_bf16_peaked_scores(Hh, d):
+    """Scores with a standard deviation of about 6 and a drift along the keys: the row maximum keeps
+    moving from key tile to key tile (the running rescale of O and of the row sum does real work),
+    most probabilities underflow, a few carry the row."""
+    nseq, T = 2, 512
+    g = torch.Generator(device="cpu").manual_seed(d)
+    dh = d // Hh
+    qkv = torch.randn(nseq * T, 3 * d, generator=g)
+    qkv[:, :2 * d] *= (6.0 * dh ** 0.5) ** 0.5 / dh ** 0.25          # q.k / sqrt(dh) ~ N(0, 36)
+    ramp = torch.linspace(0.0, 3.0, T).repeat(nseq)[:, None]         # later keys score higher
+    qkv[:, d:2 * d] += ramp * torch.sign(qkv[:, :d].mean(dim=0, keepdim=True))
+    qkv = qkv.bfloat16().cuda()
+    do = torch.randn(nseq * T, d, generator=g).bfloat16().cuda()
+    o, lse = B.attention_fwd(qkv, nseq, T, Hh, True)
+    dqkv = B.attention_bwd(qkv, o, lse, do, nseq, T, Hh, True)
+    q64 = H.tnp(qkv)
+    q, k, v = (q64[:, i * d:(i + 1) * d].reshape(nseq, T, d) for i in range(3))
+    o_ref, probs = O.causal_attention_fwd(q, k, v, Hh)
+    dq, dk, dv = O.causal_attention_bwd(H.tnp(do).reshape(nseq, T, d), q, k, v, probs, Hh)
+    assert float(probs.max(axis=-1).mean()) > 0.5                    # peaked indeed
+    assert H.rel_err(H.tnp(o), o_ref.reshape(-1, d)) <= TOL_BF16
+    got = H.tnp(dqkv)
+    for j, ref in enumerate((dq, dk, dv)):
+        assert H.rel_err(got[:, j * d:(j + 1) * d], ref.reshape(-1, d)) <= TOL_BF16, j
+
+
 def test_checkpoint_resume_and_determinism():
     """Two contexts fed the same state produce bit-identical results; state copied out of one
     context and into a fresh one continues identically (adapters, moments, counters)."""
