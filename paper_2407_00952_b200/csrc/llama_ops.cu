@@ -85,15 +85,23 @@ __global__ void __launch_bounds__(NORM_THREADS) rms_bwd_kernel(const T* __restri
   const float rs = rstd[blockIdx.x];
   float s2 = 0.f;
   if constexpr (NV > 0) {
-    Vec16<T> xv[NV], dv[NV];
+    // everything the row needs is requested before the reduction (the residual too), so that the
+    // block waits for memory once
+    Vec16<T> xv[NV], dv[NV], gv[NV], rv[NV];
 #pragma unroll
     for (int k = 0; k < NV; ++k) {
       const int v = k * NORM_THREADS + threadIdx.x;
       if (v < nvec) {
-        Vec16<T> gv;
-        xv[k].load(x + off + (size_t)v * N); dv[k].load(dy + off + (size_t)v * N); gv.load(g + (size_t)v * N);
+        xv[k].load(x + off + (size_t)v * N); dv[k].load(dy + off + (size_t)v * N); gv[k].load(g + (size_t)v * N);
+        if (resid) rv[k].load(resid + off + (size_t)v * N);
+      }
+    }
 #pragma unroll
-        for (int i = 0; i < N; ++i) s2 += dv[k].get(i) * gv.get(i) * xv[k].get(i) * rs;
+    for (int k = 0; k < NV; ++k) {
+      const int v = k * NORM_THREADS + threadIdx.x;
+      if (v < nvec) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) s2 += dv[k].get(i) * gv[k].get(i) * xv[k].get(i) * rs;
       }
     }
     const float m2 = block_sum_128(s2, sh) / d;
@@ -101,13 +109,11 @@ __global__ void __launch_bounds__(NORM_THREADS) rms_bwd_kernel(const T* __restri
     for (int k = 0; k < NV; ++k) {
       const int v = k * NORM_THREADS + threadIdx.x;
       if (v < nvec) {
-        Vec16<T> gv, rv, o;
-        gv.load(g + (size_t)v * N);
-        if (resid) rv.load(resid + off + (size_t)v * N);
+        Vec16<T> o;
 #pragma unroll
         for (int i = 0; i < N; ++i) {
-          float val = (dv[k].get(i) * gv.get(i) - xv[k].get(i) * rs * m2) * rs;
-          if (resid) val += rv.get(i);
+          float val = (dv[k].get(i) * gv[k].get(i) - xv[k].get(i) * rs * m2) * rs;
+          if (resid) val += rv[k].get(i);
           o.set(i, val);
         }
         o.store(dx + off + (size_t)v * N);
