@@ -172,16 +172,21 @@ __global__ void __launch_bounds__(256) ln_bwd_reg_kernel(const T* __restrict__ d
   if (row >= M) return;
   const size_t off = (size_t)row * d;
   const float mu = mean[row], rs = rstd[row];
-  Vec16<T> xv[NV], dv[NV];
+  // everything the row needs is requested before the reduction (gain and residual too), so that the
+  // warp waits for memory once
+  Vec16<T> xv[NV], dv[NV], gv[NV], rv[NV];
 #pragma unroll
-  for (int k = 0; k < NV; ++k) { xv[k].load(x + off + (k * 32 + lane) * N); dv[k].load(dy + off + (k * 32 + lane) * N); }
+  for (int k = 0; k < NV; ++k) {
+    const int c = (k * 32 + lane) * N;
+    xv[k].load(x + off + c); dv[k].load(dy + off + c); gv[k].load(g + c);
+    if (resid) rv[k].load(resid + off + c);
+  }
   float s1 = 0.f, s2 = 0.f;
 #pragma unroll
   for (int k = 0; k < NV; ++k) {
-    Vec16<T> gv; gv.load(g + (k * 32 + lane) * N);
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-      float dxh = dv[k].get(i) * gv.get(i);
+      float dxh = dv[k].get(i) * gv[k].get(i);
       s1 += dxh;
       s2 += dxh * (xv[k].get(i) - mu) * rs;
     }
@@ -190,14 +195,12 @@ __global__ void __launch_bounds__(256) ln_bwd_reg_kernel(const T* __restrict__ d
 #pragma unroll
   for (int k = 0; k < NV; ++k) {
     const int c = (k * 32 + lane) * N;
-    Vec16<T> gv, rv, o;
-    gv.load(g + c);
-    if (resid) rv.load(resid + off + c);
+    Vec16<T> o;
 #pragma unroll
     for (int i = 0; i < N; ++i) {
       float xh = (xv[k].get(i) - mu) * rs;
-      float v = (dv[k].get(i) * gv.get(i) - m1 - xh * m2) * rs;
-      if (resid) v += rv.get(i);
+      float v = (dv[k].get(i) * gv[k].get(i) - m1 - xh * m2) * rs;
+      if (resid) v += rv[k].get(i);
       o.set(i, v);
     }
     o.store(dx + off + c);
