@@ -4,7 +4,7 @@
 // once per 4 weight columns.  A block is 64 column threads (one 16-byte vector each) x 4 row lanes
 // over a chunk of LG_ROWS rows, four blocks per SM so that enough loads are in flight; the row
 // lanes are summed through shared memory, chunk partials go to scratch and a second kernel adds
-// them in a fixed order (no float atomics, so the result does not depend on scheduling).
+// them in chunk order (no float atomics, so the result does not depend on scheduling).
 #include "common.cuh"
 #include "kernels.h"
 
@@ -15,7 +15,6 @@ constexpr int LG_ROWS = 128;   // rows per chunk; group sizes must be multiples 
 constexpr int LG_CT = 64;      // column threads per block
 constexpr int LG_RL = 4;       // row lanes per block
 constexpr int RJ = 4;          // weight columns per block
-constexpr int RED_LANES = 8;   // chunk lanes of the second kernel
 
 // four consecutive weights of one row
 template <typename T> __device__ __forceinline__ void load4(const T* p, float* w);
@@ -104,9 +103,31 @@ lora_grad_partial_kernel(const T* __restrict__ Z, int64_t ldz, int zcol0, int C,
   }
 }
 
-// 32 outputs per block (threadIdx.x), RED_LANES chunk lanes (threadIdx.y) combined in lane order.
-__global__ void __launch_bounds__(32 * RED_LANES)
+// Many outputs (wide models): one output per thread; the chunk partials of a group are added in chunk order (adjacent threads
+// read adjacent floats of every partial, so the reads coalesce; no shared memory, no barrier).
+constexpr int RED_THREADS = 256;
+__global__ void __launch_bounds__(RED_THREADS)
 lora_grad_reduce_kernel(const float* __restrict__ partial, int r, int R, int C, int chunks_per_group, float scale,
+                        float* __restrict__ out, int64_t out_group_stride, int64_t out_target_stride,
+                        int64_t out_sj, int64_t out_sc) {
+  const int idx = blockIdx.x * RED_THREADS + threadIdx.x;   // over R*C
+  const int g = blockIdx.y;
+  if (idx >= R * C) return;
+  const size_t rc = (size_t)R * C;
+  const float* p = partial + (size_t)g * chunks_per_group * rc + idx;
+  float s = 0.f;
+#pragma unroll 4
+  for (int k = 0; k < chunks_per_group; ++k) s += p[(size_t)k * rc];
+  const int j = idx / C, c = idx % C;
+  out[(size_t)g * out_group_stride + (size_t)(j / r) * out_target_stride + (size_t)(j % r) * out_sj +
+      (size_t)c * out_sc] = scale * s;
+}
+
+// Few outputs, many chunks (narrow models, long groups): 32 outputs per block (threadIdx.x) and
+// RED_LANES chunk lanes (threadIdx.y), each adding every RED_LANES-th partial, combined in lane order.
+constexpr int RED_LANES = 8;
+__global__ void __launch_bounds__(32 * RED_LANES)
+lora_grad_reduce_lanes_kernel(const float* __restrict__ partial, int r, int R, int C, int chunks_per_group, float scale,
                         float* __restrict__ out, int64_t out_group_stride, int64_t out_target_stride,
                         int64_t out_sj, int64_t out_sc) {
   __shared__ float red[RED_LANES][32];
@@ -127,6 +148,18 @@ lora_grad_reduce_kernel(const float* __restrict__ partial, int r, int R, int C, 
     const int j = idx / C, c = idx % C;
     out[(size_t)g * out_group_stride + (size_t)(j / r) * out_target_stride + (size_t)(j % r) * out_sj +
         (size_t)c * out_sc] = scale * t;
+  }
+}
+
+// picks the second kernel by the number of outputs (both add in a fixed order)
+void launch_reduce(const float* partial, int r, int R, int C, int cpg, int groups, float scale, float* out,
+                   int64_t out_group_stride, int64_t out_target_stride, int64_t out_sj, int64_t out_sc, cudaStream_t st) {
+  if ((int64_t)R * C >= 32768) {
+    dim3 g2((R * C + RED_THREADS - 1) / RED_THREADS, groups), b2(RED_THREADS);
+    lora_grad_reduce_kernel<<<g2, b2, 0, st>>>(partial, r, R, C, cpg, scale, out, out_group_stride, out_target_stride, out_sj, out_sc);
+  } else {
+    dim3 g2((R * C + 31) / 32, groups), b2(32, RED_LANES);
+    lora_grad_reduce_lanes_kernel<<<g2, b2, 0, st>>>(partial, r, R, C, cpg, scale, out, out_group_stride, out_target_stride, out_sj, out_sc);
   }
 }
 
@@ -166,9 +199,8 @@ cudaError_t lora_grad(int dt, const void* Z, int64_t ldz, int zcol0, int C, cons
         cudaError_t e = lora_grad_tc_partial(Z, ldz, zcol0, C, Wt, ldwt, wcol0 + t0 * rp, r, rp, ntw, M, rows_per_group,
                                              partial, status, &cpg, st);
         if (e != cudaSuccess) return e;
-        dim3 g2((Rw * C + 31) / 32, groups), b2(32, RED_LANES);
-        lora_grad_reduce_kernel<<<g2, b2, 0, st>>>(partial, r, Rw, C, cpg, scale, out + (size_t)t0 * out_target_stride,
-                                                   out_group_stride, out_target_stride, out_sj, out_sc);
+        launch_reduce(partial, r, Rw, C, cpg, groups, scale, out + (size_t)t0 * out_target_stride, out_group_stride,
+                      out_target_stride, out_sj, out_sc, st);
       }
       return cudaGetLastError();
     }
@@ -190,9 +222,8 @@ cudaError_t lora_grad(int dt, const void* Z, int64_t ldz, int zcol0, int C, cons
   dim3 grid((cvec + LG_CT - 1) / LG_CT, chunks, (R + RJ - 1) / RJ);
   if (dt == DT_BF16) launch_partial<bf16>(grid, st, vec4, Z, ldz, zcol0, C, Wt, ldwt, wcol0, r, rp, R, M, partial);
   else launch_partial<float>(grid, st, vec4, Z, ldz, zcol0, C, Wt, ldwt, wcol0, r, rp, R, M, partial);
-  dim3 g2((R * C + 31) / 32, groups), b2(32, RED_LANES);
-  lora_grad_reduce_kernel<<<g2, b2, 0, st>>>(partial, r, R, C, chunks_per_group, scale, out, out_group_stride,
-                                             out_target_stride, out_sj, out_sc);
+  launch_reduce(partial, r, R, C, chunks_per_group, groups, scale, out, out_group_stride, out_target_stride, out_sj,
+                out_sc, st);
   return cudaGetLastError();
 }
 
