@@ -71,3 +71,33 @@ def oracle_three_calls(w, frozen, cads, sads, tokens, labels, optimizer="sgd", *
     loss, dS, sg = O.server_fwd_bwd(cfg, params, s64, S, labels)
     cg = O.client_bwd_grads(cfg, params, c64, dS, caches)
     return cfg, params, c64, s64, S, dS, loss, sg, cg
+
+
+# ---- parity cases whose q / k adapter gradients are looser than the general bf16 bound --------------
+# The three bf16 cases below have random labels and random non-zero B, and their q / k adapter gradients
+# come out of the attention backward, whose row term sum_j P_ij dP_ij is taken from the STORED (bf16)
+# attention output.  tests/test_storage_noise.py computes, on the CPU, what bf16 storage alone does to
+# these gradients in otherwise exact arithmetic, and fixes the rule: a case keeps the general 2e-2 when
+# that noise, with a margin of 1.4 for a different rounding realisation, stays inside it; otherwise its
+# q / k bound is QK_BOUND, which must cover the noise with the same margin.
+TOL_BF16 = 2e-2
+QK_BOUND = 4e-2
+NOISE_MARGIN = 1.4
+
+
+def qk_case(name):
+    """(workload, per-client ranks or None, bound for the q / k adapter gradients or None for the general one)"""
+    if name == "federated_small":
+        return (synth.scaled(synth.WORKLOADS[2], n_layer=2, cut=2, n_clients=2, batch_per_client=2, seq=256,
+                             max_seq=256), None, QK_BOUND)
+    if name == "llama_full_width":
+        return (synth.scaled(synth.WORKLOADS[5], n_layer=2, cut=1, vocab=4096, n_clients=2, batch_per_client=1,
+                             seq=256, max_seq=256), None, QK_BOUND)
+    if name == "ranks_medium":
+        return (synth.scaled(synth.WORKLOADS[3], n_layer=3, cut=2, n_clients=3, batch_per_client=2, seq=128,
+                             max_seq=128), (2, 4, 1), None)
+    raise KeyError(name)
+
+
+def cut_to_rank(ad, r):
+    return {k: {"A": v["A"][:r].copy(), "B": v["B"][:, :r].copy()} for k, v in ad.items()}

@@ -12,8 +12,7 @@ from paper_2407_00952_b200 import runner, synth
 pytestmark = pytest.mark.gpu
 
 
-def _cut(ad, r):
-    return {k: {"A": v["A"][:r].copy(), "B": v["B"][:, :r].copy()} for k, v in ad.items()}
+_cut = H.cut_to_rank
 
 
 def _check_round(w, ranks, tol, optimizer, tol_qk=None):
@@ -104,8 +103,8 @@ def test_ranks_tiny_fp32_adamw_second_round_keeps_zeros():
 
 
 def test_ranks_bf16_medium_shaped():
-    w = synth.scaled(synth.WORKLOADS[3], n_layer=3, cut=2, n_clients=3, batch_per_client=2, seq=128, max_seq=128)
-    _check_round(w, (2, 4, 1), 2e-2, "sgd", tol_qk=4e-2)
+    w, ranks, qk_bound = H.qk_case("ranks_medium")      # storage noise leaves the general bound in reach here
+    _check_round(w, ranks, 2e-2, "sgd", tol_qk=qk_bound)
 
 
 def test_ranks_argument_errors_and_reset():

@@ -5,12 +5,14 @@ device-memory budget fixed at start, or a plug-in whose host application owns th
 them the library keeps the small per-row scratch of the attention backward in a fixed internal
 array.  This test drives that entry point through the C ABI twice in a row, with different shapes
 so that the second call finds the first call's leftovers in the shared array, and requires the
-same gradients as the ordinary entry point (which takes caller scratch); it also checks that a
-problem larger than the internal array is refused.  It is collected last on purpose.
+same gradients as the ordinary entry point (which takes caller scratch) and as the CPU reference;
+it also checks that a problem larger than the internal array is refused.  It is collected last on purpose.
 """
+import numpy as np
 import pytest
 import torch
 
+from oracle import splitlora_oracle as O
 from paper_2407_00952_b200 import binding as B
 
 pytestmark = pytest.mark.gpu
@@ -44,6 +46,16 @@ def test_static_scratch_matches_caller_scratch_twice():
         assert torch.isfinite(got).all()
         assert _rel(got, want) <= (TOL_BF16 if dtype == torch.bfloat16 else 1e-4)
         assert torch.equal(got, want)       # same kernels, same order of operations
+        # and against the CPU reference of the attention gradients itself
+        q64 = qkv.float().cpu().numpy().astype(np.float64)
+        q, k, v = (q64[:, j * d:(j + 1) * d].reshape(nseq, T, d) for j in range(3))
+        _, probs = O.causal_attention_fwd(q, k, v, heads)
+        ref = O.causal_attention_bwd(d_o.float().cpu().numpy().astype(np.float64).reshape(nseq, T, d), q, k, v,
+                                     probs, heads)
+        got64 = got.float().cpu().numpy().astype(np.float64)
+        for j in range(3):
+            err = np.abs(got64[:, j * d:(j + 1) * d] - ref[j].reshape(-1, d)).max() / np.abs(ref[j]).max()
+            assert err <= (TOL_BF16 if dtype == torch.bfloat16 else 1e-4), (nseq, T, j, err)
 
 
 def test_static_scratch_rejects_oversize():
