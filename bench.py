@@ -2,6 +2,7 @@
 """Benchmark of the split-LoRA round: training tokens/s on the GPT-2-medium-shaped workload.
 
   python bench.py --gpus 1 --steps 10 --warmup 3            # the CUDA library
+  python bench.py --gpus 4 --scaling strong                 # starts its own 4 ranks (or run it under torchrun)
   python bench.py --impl reference --steps 2 --warmup 1     # the CPU oracle on a bounded sample
 
 A step is one full round of Algorithm 1 (client forward, server step, client backward and the
@@ -36,6 +37,32 @@ def load_peaks():
         return dict(hbm_gbs=p["hbm_gbs"], tflops_burst=p["bf16_tflops"], tflops_sustained=p["bf16_tflops_sustained"],
                     source="measured")
     return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+def kernel_source_digest():
+    """Digest of the sources of the linear-layer kernel, to tell whether counters taken earlier still apply."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("gemm_tc.cu", "tc_common.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_2407_00952_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def load_traffic(w):
+    """DRAM bytes of one launch of the dominant kernel, from the record written beside its ncu summary
+    (profiles/gemm_tc_pair_kernel_traffic.txt: key = value lines).  None when there is no record for this
+    workload or when the kernel's sources have changed since the counters were taken."""
+    path = os.path.join(ROOT, "profiles", "gemm_tc_pair_kernel_traffic.txt")
+    if not os.path.exists(path):
+        return None, None
+    rec = {}
+    for line in open(path):
+        if "=" in line and not line.lstrip().startswith("#"):
+            k, v = line.split("=", 1)
+            rec[k.strip()] = v.strip()
+    if rec.get("workload") != f"cfg{w.index}" or rec.get("kernel_source_digest") != kernel_source_digest():
+        return None, None
+    return int(rec["dram_bytes_per_launch"]), rec.get("launch")
 
 
 def workload_description(w):
@@ -161,7 +188,7 @@ def run_reference(args, w):
         return
     tps, sec, threads, ws = time_oracle_rounds(w, args.steps, args.warmup)
     line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": args.scaling,
             "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": workload_description(w),
             "cpu_baseline": {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample_text(ws)},
             "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -181,16 +208,25 @@ def run_gpu(args, w):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    cads = [synth.make_adapters(w, range(w.cut)) for _ in range(w.n_clients)]
-    sads = synth.make_adapters(w, range(w.cut, w.n_layer))
-    eng = runner.make_engine(w, synth.iter_frozen(w), cads, sads, optimizer="adamw")   # uploaded as drawn
-    counts = synth.make_counts(w)
+    # Clients over ranks.  weak: every rank owns all K clients of the workload (a K*world-client job);
+    # strong: the workload's K clients are spread over the ranks (K / world each, contiguous blocks).
+    from paper_2407_00952_b200 import parallel
+    strong = args.scaling == "strong"
+    if strong and world > w.n_clients:
+        raise SystemExit(f"strong scaling needs at least one client per rank ({w.n_clients} clients, {world} ranks)")
+    mine = parallel.shard_clients(w.n_clients, world, rank) if strong else list(range(w.n_clients))
+    all_counts = synth.make_counts(w)
+    wl = synth.scaled(w, n_clients=len(mine))
+    counts = all_counts[mine]
+    cads = [synth.make_adapters(wl, range(wl.cut)) for _ in mine]
+    sads = synth.make_adapters(wl, range(wl.cut, wl.n_layer))
+    eng = runner.make_engine(wl, synth.iter_frozen(wl), cads, sads, optimizer="adamw")   # uploaded as drawn
     nbatch = 4
     host_tok, host_lab, dev_tok, dev_lab = [], [], [], []
     for s in range(nbatch):
-        t, l = synth.make_tokens(w, round_index=1000 * rank + s)
-        host_tok.append(torch.from_numpy(t).pin_memory())
-        host_lab.append(torch.from_numpy(l).pin_memory())
+        t, l = synth.make_tokens(w, round_index=s if strong else 1000 * rank + s)
+        host_tok.append(torch.from_numpy(np.ascontiguousarray(t[mine])).pin_memory())
+        host_lab.append(torch.from_numpy(np.ascontiguousarray(l[mine])).pin_memory())
         dev_tok.append(host_tok[-1].cuda())
         dev_lab.append(host_lab[-1].cuda())
     stream = torch.cuda.current_stream()
@@ -207,13 +243,11 @@ def run_gpu(args, w):
         def step_host(s):
             return eng.round_host(host_tok[s % nbatch], host_lab[s % nbatch], counts, want_loss=True)
     else:
-        # weak scaling: every rank owns K clients of a K*world-client job; the server adapter
-        # gradients and the aggregation sums are all-reduced (NCCL) inside the round
-        from paper_2407_00952_b200 import parallel
+        # the server adapter gradients and the aggregation sum are all-reduced (NCCL) inside the round
         sharded = parallel.ShardedRound(eng, agg_interval=w.agg_interval)
         S_buf, dS_buf = eng.new_activation_buffer(), eng.new_activation_buffer()
-        total_count = int(counts.sum()) * world
-        n_valid_global = w.tokens_per_round * world
+        total_count = int(all_counts.sum()) * (1 if strong else world)
+        n_valid_global = w.tokens_per_round * (1 if strong else world)
         stage_tok, stage_lab = torch.empty_like(dev_tok[0]), torch.empty_like(dev_lab[0])
 
         def step_dev(s):
@@ -287,16 +321,18 @@ def run_gpu(args, w):
             dist.destroy_process_group()
         return
 
-    tokens_total = w.tokens_per_round * args.steps * world
+    tokens_total = w.tokens_per_round * args.steps * (1 if strong else world)
+    w_local = wl                                   # what one rank runs: the per-launch figures below are its
     value = tokens_total / (ms * 1e-3)
     e2e_value = tokens_total / (ms_e2e * 1e-3)
     peaks = load_peaks()
-    fl = gemm_flops_per_round(w)
+    fl = gemm_flops_per_round(w_local)
     t_ms = sum(prof[k][1] for k in fl if k in prof)
     n_launch = sum(prof[k][0] for k in fl if k in prof)
     flops = sum(fl[k] for k in fl if k in prof) * args.steps
     achieved = flops / (t_ms * 1e-3) / 1e12 if t_ms > 0 else 0.0
     peak = peaks["tflops_sustained"]
+    traffic, traffic_launch = load_traffic(w)
     by_class = {k: {"launches": prof[k][0], "ms_total": round(prof[k][1], 3),
                     "tflops": round(fl[k] * args.steps / (prof[k][1] * 1e-3) / 1e12, 1)}
                 for k in fl if k in prof and prof[k][1] > 0}
@@ -306,12 +342,9 @@ def run_gpu(args, w):
                 "achieved": round(achieved, 1), "peak": peak, "unit": "TFLOP/s",
                 "frac": round(achieved / peak, 4) if peak else None,
                 "peak_source": f"{peaks['source']} sustained bf16 (kernel timed inside a long step)",
-                # DRAM bytes of one launch from the committed ncu capture of the CTA-pair kernel
-                # (profiles/gemm_tc_pair_kernel_qkv_m32768.md): the QKV + LoRA forward launch of this
-                # workload, whose algorithmic bytes are 275 MB.  Null for any other workload.
-                "traffic": 236960000 if w.index == 3 else None,
-                "traffic_launch": "QKV+LoRA forward, M 32768 K 1024(+64) N 3072: 81.1 MB read + 155.9 MB written; "
-                                  "algorithmic 275 MB" if w.index == 3 else None,
+                # DRAM bytes of one launch from the ncu capture recorded under profiles/ (None when the
+                # kernel has changed since, or for a workload without a capture)
+                "traffic": traffic, "traffic_launch": traffic_launch,
                 "launches": n_launch, "avg_launch_us": round(t_ms * 1e3 / max(1, n_launch), 2),
                 "by_class": by_class, "share_of_step": round(t_ms / ms, 4)}
     breakdown = {k: {"launches": v[0], "ms_per_step": round(v[1] / args.steps, 3)}
@@ -322,13 +355,19 @@ def run_gpu(args, w):
         tps, sec, threads, ws = time_oracle_rounds(w, 1, 0)
         cpu = {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample_text(ws, sec)}
 
-    M = w.tokens_per_round
+    M = w_local.tokens_per_round
+    if world == 1:
+        par = "1 GPU"
+    elif strong:
+        par = (f"strong: the workload's {w.n_clients} clients spread over {world} GPUs, NCCL all-reduce of the server "
+               f"adapter gradients and of one client's worth of aggregation sums")
+    else:
+        par = (f"weak: {w.n_clients} clients on each of {world} GPUs, NCCL all-reduce of the server adapter gradients "
+               f"and of one client's worth of aggregation sums")
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms / args.steps, "host_enqueue_ms_per_step": host_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms / args.steps, "host_enqueue_ms_per_step": host_ms / args.steps, "higher_is_better": True, "scaling": args.scaling, "vs_baseline": None,
             "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": dict(workload_description(w), parallelism="1 GPU" if world == 1 else
-                           f"clients sharded over {world} GPUs ({w.n_clients} each), NCCL all-reduce of server "
-                           f"adapter gradients and aggregation sums"),
+            "config": workload_description(w), "parallelism": par,
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 2 * M * 4, "d2h_bytes_per_step": 4,
                     "ms_per_step": ms_e2e / args.steps, "last_loss": losses[-1]},
@@ -346,7 +385,19 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=3, help="workload index (3 = GPT-2-medium-shaped, the headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="weak: every GPU runs the workload's K clients; strong: the K clients are spread over the GPUs")
     args = ap.parse_args()
+    if args.impl == "ours" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain command: launch one rank per GPU and let them run this file
+        import socket
+        sock = socket.socket()
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+        sock.close()
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
     if args.impl == "ours":
         args.warmup = max(args.warmup, 3)
     w = synth.WORKLOADS[args.config]

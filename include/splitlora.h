@@ -19,6 +19,9 @@
  *     unless they write to a HOST pointer (loss_out).
  *   - The library never allocates device memory in the calls below: all of its state lives in the
  *     caller-provided workspace (splitlora_workspace_bytes / splitlora_bind_workspace).
+ *   - A process may use several devices: per-device set-up (kernel attributes, SM count, status
+ *     words) is keyed by the device that is current when a call is made, so make the context's
+ *     device current before every call on that context.
  *   - Conventions: a linear layer stores W as [out, in]; a LoRA adapter is A [r, in], B [out, r]
  *     and the adapted layer computes  y = x W^T + bias + (alpha/r) (x A^T) B^T   (Sec. II-C).
  *     Activations are [K, b, T, d] = [clients, sequences per client, positions, width].
@@ -150,7 +153,8 @@ int splitlora_set_counters(splitlora_ctx* ctx, int64_t round_index, int64_t serv
 int splitlora_client_fwd(splitlora_ctx* ctx, const int32_t* tokens, void* act_out);
 
 /* Step a3/a4, Eq. 3-5.  act_in [K, b, T, d] is treated as the concatenation S^t; labels [K, b, T]
- * int32, negative = ignored position.  One forward/backward over the concatenated batch with the
+ * int32; a label outside [0, vocab) marks an ignored position (it adds nothing to the loss, to the
+ * gradients or to the count the mean is taken over).  One forward/backward over the concatenated batch with the
  * single server adapter set, loss = mean cross-entropy over valid positions, server adapters
  * updated with lr_server.  Writes dL/dS to act_grad_out [K, b, T, d] (context dtype).
  * loss_out is HOST and may be NULL; when given, the call synchronises the stream. */
@@ -201,8 +205,8 @@ int splitlora_round_host(splitlora_ctx* ctx, const int32_t* tokens_host, const i
  * concatenated batch (step a3), so a device can own a subset of the clients and the matching rows
  * of S^t.  Every device holds the same frozen weights and the same server adapters and runs the
  * three calls on its own clients; two sums over devices make the result equal to the one-device
- * round: the server adapter gradients before the server update, and the weighted adapter sums of
- * Eq. 8-9 at aggregation.  The library does no communication itself; the caller reduces the
+ * round: the server adapter gradients before the server update, and the weighted adapter sum of
+ * Eq. 8-9 (one client's worth of parameters) at aggregation.  The library does no communication itself; the caller reduces the
  * buffers below (e.g. with an NCCL all-reduce on the context stream). */
 
 /* Number of valid label positions of the WHOLE concatenated batch (all devices).  When > 0 it
@@ -218,15 +222,28 @@ int splitlora_server_update(splitlora_ctx* ctx);
  * the workspace is bound.  After writing parameters call splitlora_adapters_changed(side). */
 int splitlora_adapter_buffer(splitlora_ctx* ctx, int side, int kind, float** dev, int64_t* count);
 int splitlora_adapters_changed(splitlora_ctx* ctx, int side);
-/* Eq. 8-9 for the local clients of one device: every local client A and B becomes
- * sum_{i local} (|D_i| / total_count) P_i, total_count = |D| over ALL devices' clients.  Summing
- * the client parameter buffers over devices afterwards gives every client the global average. */
-int splitlora_aggregate_partial(splitlora_ctx* ctx, const int64_t* sample_counts, int64_t total_count);
+/* Eq. 8-9 with the clients spread over devices, in two halves around one sum over devices.
+ * _local_sum: sum_{i local} (|D_i| / total_count) P_i for every client A and B, total_count = |D| over
+ * ALL devices' clients; the result is left in a buffer of the workspace, *sum_dev (DEVICE pointer, HOST
+ * out) with *count fp32 elements (one client's adapter set; the same on every device however many
+ * clients each holds).  The caller adds these buffers up over devices in place (one all-reduce of
+ * *count floats), then calls _broadcast, which writes the buffer to every local client (the downlink b3)
+ * and, with per-client ranks, cuts each client back to its own rank afterwards.
+ * sample_counts: HOST int64 [local clients].  Errors: SPLITLORA_ERR_COUNTS, SPLITLORA_ERR_WORKSPACE. */
+int splitlora_aggregate_local_sum(splitlora_ctx* ctx, const int64_t* sample_counts, int64_t total_count,
+                                  float** sum_dev, int64_t* count);
+int splitlora_aggregate_broadcast(splitlora_ctx* ctx);
 
 /* Device loss of the last server_step (fp32 scalar, DEVICE pointer into the workspace). */
 int splitlora_loss_device(splitlora_ctx* ctx, const float** loss_dev);
 
 const char* splitlora_last_error(const splitlora_ctx* ctx);
+/* The stand-alone operators below that take no status word (attention, adapter gradients inside
+ * lora_linear_bwd without a workspace word) record an expired bounded wait in a word the library keeps
+ * per device.  This call synchronises the current device, copies that word to *code (HOST) and
+ * returns SPLITLORA_ERR_TIMEOUT when it is non-zero, else SPLITLORA_OK.  The kernels of a context
+ * report through splitlora_device_status instead. */
+int splitlora_library_status(int32_t* code);
 /* Reads the device status word (HOST out): 0, or the code left by a bounded wait that expired.
  * Synchronises the stream. */
 int splitlora_device_status(splitlora_ctx* ctx, int32_t* code);

@@ -31,8 +31,10 @@ EXPORTS = [
     "splitlora_transpose", "splitlora_aggregate_buffers", "splitlora_attention_fwd", "splitlora_attention_bwd",
     "splitlora_attention_bwd_static", "splitlora_linear", "splitlora_set_loss_normalizer",
     "splitlora_set_deferred_server_update", "splitlora_server_update", "splitlora_adapter_buffer",
-    "splitlora_adapters_changed", "splitlora_aggregate_partial", "splitlora_handoff_quantize",
+    "splitlora_adapters_changed", "splitlora_aggregate_local_sum", "splitlora_aggregate_broadcast",
+    "splitlora_handoff_quantize",
     "splitlora_handoff_dequantize", "splitlora_round_compressed", "splitlora_set_client_ranks",
+    "splitlora_library_status",
 ]
 
 
@@ -252,9 +254,17 @@ class SplitLoRA:
     def adapters_changed(self, side: int):
         self._check(self.lib.splitlora_adapters_changed(self.ctx, side))
 
-    def aggregate_partial(self, counts, total_count: int):
+    def aggregate_local_sum(self, counts, total_count: int) -> torch.Tensor:
+        """Weighted sum of the local clients' adapters (weights |D_i| / total_count): fp32 view [Pc] of the
+        workspace buffer that the caller all-reduces in place before aggregate_broadcast."""
         arr = (C.c_int64 * len(counts))(*[int(x) for x in counts])
-        self._check(self.lib.splitlora_aggregate_partial(self.ctx, arr, C.c_int64(total_count)))
+        ptr, n = C.c_void_p(0), C.c_int64(0)
+        self._check(self.lib.splitlora_aggregate_local_sum(self.ctx, arr, C.c_int64(total_count), C.byref(ptr), C.byref(n)))
+        off = ptr.value - self.workspace.data_ptr()
+        return self.workspace[off:off + 4 * n.value].view(torch.float32)
+
+    def aggregate_broadcast(self):
+        self._check(self.lib.splitlora_aggregate_broadcast(self.ctx))
 
     def loss_tensor(self) -> torch.Tensor:
         """fp32 view of the device loss scalar of the last server_step."""
@@ -412,6 +422,16 @@ def attention_bwd(qkv, o, lse, d_o, nseq, T, n_head, use_tensor_cores=True):
     _rc(lib.splitlora_attention_bwd(_dt(qkv), 1 if use_tensor_cores else 0, _ptr(qkv), _ptr(o), _ptr(lse), _ptr(d_o),
                                     nseq, T, n_head, d, _ptr(dqkv), _ptr(rowdot), _stream_ptr()), "attention_bwd")
     return dqkv
+
+
+def library_status() -> int:
+    """Status word of the stand-alone operators on the current device (0 = no bounded wait expired);
+    synchronises the device."""
+    code = C.c_int32(0)
+    rc = load().splitlora_library_status(C.byref(code))
+    if rc not in (0, -7):
+        raise SplitLoraError(rc, "library_status")
+    return code.value
 
 
 STATIC_ATTENTION_ROWS = 1 << 20

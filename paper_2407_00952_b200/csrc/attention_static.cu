@@ -53,7 +53,7 @@ extern "C" int splitlora_attention_bwd_static(int dtype, int use_tc, const void*
   // kernel of this same call, so nothing has to be cleared between calls.
   cudaError_t e;
   if (use_tc && attention_tc_supported(dtype, T, n_head, d_model))
-    e = attention_bwd_tc(qkv, o, lse, d_o, nseq, T, n_head, d_model, dqkv, rowdot, (cudaStream_t)stream);
+    e = attention_bwd_tc(qkv, o, lse, d_o, nseq, T, n_head, d_model, dqkv, rowdot, nullptr, (cudaStream_t)stream);
   else
     e = attention_bwd_simt(dtype, qkv, o, lse, d_o, nseq, T, n_head, d_model, dqkv, rowdot, (cudaStream_t)stream);
   return e == cudaSuccess ? SPLITLORA_OK : SPLITLORA_ERR_CUDA;

@@ -19,6 +19,7 @@
 // warps 2..9 softmax: two threads per query row (warp w owns accumulator lanes 32*(w%4)..+31, warps
 // 2..5 the first half of the score and output columns, warps 6..9 the second).
 // All mbarrier waits are bounded (see tc_common.cuh); on expiry a code is left in `status`.
+#include "host_common.h"
 #include "tc_common.cuh"
 
 namespace sl {
@@ -379,40 +380,21 @@ attn_fwd_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_cons
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn g_encode = nullptr;
-int* g_status = nullptr;      // device word for expired waits when the caller gives none
-int g_num_sms = 0;
-__device__ int g_t5_status[4];
+PerDeviceOnce g_once;
 
 bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
-  cuuint32_t box[2] = {64, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return cached_map_2d(m, ptr, rows, cols, cols, 64, box_rows, CU_TENSOR_MAP_SWIZZLE_128B,
+                       CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
 
-bool init_once() {
-  if (g_encode) return true;
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult q;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
-      q != cudaDriverEntryPointSuccess)
-    return false;
-  if (cudaGetSymbolAddress((void**)&g_status, g_t5_status) != cudaSuccess) return false;
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_num_sms < 1)
-    return false;
-  if (cudaMemset(g_status, 0, sizeof(int) * 4) != cudaSuccess) return false;
+// kernel attributes are per device: set them the first time each device launches
+bool init_device() {
+  const int dev = current_device();
+  if (dev < 0 || !tensor_map_encoder()) return false;
+  if (!g_once.needed(dev)) return true;
   if (cudaFuncSetAttribute(attn_fwd_t5_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<64>::SMEM) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(attn_fwd_t5_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128>::SMEM) != cudaSuccess) return false;
-  g_encode = (EncodeTiledFn)fn;
+  g_once.done(dev);
   return true;
 }
 
@@ -430,20 +412,23 @@ bool attention_fwd_t5_supported(int dt, int T, int H, int d) {
 cudaError_t attention_fwd_t5(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, int* status,
                              cudaStream_t st) {
   if (!attention_fwd_t5_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
-  if (!init_once()) return cudaErrorInitializationError;
+  if (!init_device()) return cudaErrorInitializationError;
+  const int sms = num_sms();
+  if (!status) status = library_status_word();
+  if (!status || sms < 1) return cudaErrorInitializationError;
   CUtensorMap mQKV, mO;
   if (!make_map(&mQKV, qkv, (uint64_t)nseq * T, (uint64_t)3 * d, BQ)) return cudaErrorInvalidValue;
   if (!make_map(&mO, o, (uint64_t)nseq * T, (uint64_t)d, BQ)) return cudaErrorInvalidValue;
   const int dh = d / H;
   T5Params p;
   p.T = T; p.H = H; p.d = d; p.scale_log2 = LOG2E / sqrtf((float)dh); p.lse = lse;
-  p.status = status ? status : g_status;
+  p.status = status;
   p.nitems = nseq * H;
   if (dh == 64) {
-    const int cap = FwdCfg<64>::CTAS_PER_SM * g_num_sms;                         // persistent CTAs
+    const int cap = FwdCfg<64>::CTAS_PER_SM * sms;                         // persistent CTAs
     attn_fwd_t5_kernel<64><<<p.nitems < cap ? p.nitems : cap, T5_THREADS, FwdCfg<64>::SMEM, st>>>(mQKV, mO, p);
   } else {
-    const int cap = FwdCfg<128>::CTAS_PER_SM * g_num_sms;
+    const int cap = FwdCfg<128>::CTAS_PER_SM * sms;
     attn_fwd_t5_kernel<128><<<p.nitems < cap ? p.nitems : cap, T5_THREADS, FwdCfg<128>::SMEM, st>>>(mQKV, mO, p);
   }
   return cudaGetLastError();

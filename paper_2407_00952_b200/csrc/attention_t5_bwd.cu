@@ -23,6 +23,7 @@
 // products, warps 2..9 element-wise work (thread = accumulator lane, two warps per lane quarter),
 // warps 11..14 output of the finished accumulators.
 // All mbarrier waits are bounded (tc_common.cuh); on expiry a code is left in `status`.
+#include "host_common.h"
 #include "tc_common.cuh"
 
 namespace sl {
@@ -742,42 +743,23 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
   T5_TEARDOWN()
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn g_encode = nullptr;
-int* g_status = nullptr;
-int g_num_sms = 0;
-__device__ int g_t5b_status[4];
+PerDeviceOnce g_once;
 
 bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols) {
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)BT};
-  cuuint32_t estr[2] = {1, 1};
-  return g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return cached_map_2d(m, ptr, rows, cols, cols, 64, (uint32_t)BT, CU_TENSOR_MAP_SWIZZLE_128B,
+                       CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
 
-bool init_once() {
-  if (g_encode) return true;
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult q;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
-      q != cudaDriverEntryPointSuccess)
-    return false;
-  if (cudaGetSymbolAddress((void**)&g_status, g_t5b_status) != cudaSuccess) return false;
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_num_sms < 1)
-    return false;
-  if (cudaMemset(g_status, 0, sizeof(int) * 4) != cudaSuccess) return false;
+// kernel attributes are per device: set them the first time each device launches
+bool init_device() {
+  const int dev = current_device();
+  if (dev < 0 || !tensor_map_encoder()) return false;
+  if (!g_once.needed(dev)) return true;
   if (cudaFuncSetAttribute(attn_bwd_dkv_t5_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, dkv::Cfg<64>::SMEM) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(attn_bwd_dkv_t5_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, dkv::Cfg<128>::SMEM) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(attn_bwd_dq_t5_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, dq::Cfg<64>::SMEM) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(attn_bwd_dq_t5_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, dq::Cfg<128>::SMEM) != cudaSuccess) return false;
-  g_encode = (EncodeTiledFn)fn;
+  g_once.done(dev);
   return true;
 }
 
@@ -786,7 +768,10 @@ bool init_once() {
 cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq, int T, int H,
                              int d, void* dqkv, float* rowdot, int* status, cudaStream_t st) {
   if (!attention_t5_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
-  if (!init_once()) return cudaErrorInitializationError;
+  if (!init_device()) return cudaErrorInitializationError;
+  const int sms = num_sms();
+  if (!status) status = library_status_word();
+  if (!status || sms < 1) return cudaErrorInitializationError;
   CUtensorMap mQKV, mDO, mO, mDQKV;
   const uint64_t rows = (uint64_t)nseq * T;
   if (!make_map(&mQKV, qkv, rows, (uint64_t)3 * d) || !make_map(&mDO, d_o, rows, (uint64_t)d) ||
@@ -794,9 +779,9 @@ cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, c
     return cudaErrorInvalidValue;
   BwdParams p;
   p.T = T; p.H = H; p.d = d; p.scale = 1.0f / sqrtf((float)DH); p.lse = lse; p.rowdot = rowdot; p.rowdot_out = rowdot;
-  p.status = status ? status : g_status;
+  p.status = status;
   p.nitems = nseq * H;
-  dim3 grid((unsigned)(p.nitems < g_num_sms ? p.nitems : g_num_sms));     // one persistent CTA per SM
+  dim3 grid((unsigned)(p.nitems < sms ? p.nitems : sms));     // one persistent CTA per SM
   // dQ first: it leaves D[row] = sum(dO * O) in `rowdot` for the dK/dV kernel
   attn_bwd_dq_t5_kernel<64><<<grid, NTHREADS, dq::Cfg<64>::SMEM, st>>>(mQKV, mDO, mO, mDQKV, p);
   attn_bwd_dkv_t5_kernel<64><<<grid, NTHREADS, dkv::Cfg<64>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
@@ -811,7 +796,10 @@ bool attention_bwd_t5_128_supported(int dt, int T, int H, int d) {
 cudaError_t attention_bwd_t5_128(const void* qkv, const float* lse, const void* d_o, const float* rowdot, int nseq,
                                     int T, int H, int d, void* dqkv, int* status, cudaStream_t st) {
   if (!attention_bwd_t5_128_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
-  if (!init_once()) return cudaErrorInitializationError;
+  if (!init_device()) return cudaErrorInitializationError;
+  const int sms = num_sms();
+  if (!status) status = library_status_word();
+  if (!status || sms < 1) return cudaErrorInitializationError;
   CUtensorMap mQKV, mDO, mDQKV;
   const uint64_t rows = (uint64_t)nseq * T;
   if (!make_map(&mQKV, qkv, rows, (uint64_t)3 * d) || !make_map(&mDO, d_o, rows, (uint64_t)d) ||
@@ -819,9 +807,9 @@ cudaError_t attention_bwd_t5_128(const void* qkv, const float* lse, const void* 
     return cudaErrorInvalidValue;
   BwdParams p;
   p.T = T; p.H = H; p.d = d; p.scale = 1.0f / sqrtf(128.0f); p.lse = lse; p.rowdot = rowdot; p.rowdot_out = nullptr;
-  p.status = status ? status : g_status;
+  p.status = status;
   p.nitems = nseq * H;
-  dim3 grid((unsigned)(p.nitems < g_num_sms ? p.nitems : g_num_sms));
+  dim3 grid((unsigned)(p.nitems < sms ? p.nitems : sms));
   attn_bwd_dq_t5_kernel<128><<<grid, NTHREADS, dq::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDO /* unused */, mDQKV, p);
   attn_bwd_dkv_t5_kernel<128><<<grid, NTHREADS, dkv::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
   return cudaGetLastError();

@@ -6,13 +6,12 @@
 //   backward: rowdot = sum(dO*O); a dQ kernel per query tile (loops over key tiles) and a dK/dV
 //             kernel per key tile (loops over query tiles).  No atomics: results are bit-reproducible.
 // Products use mma.sync m16n8k16 with ldmatrix-fed fragments from XOR-swizzled shared tiles.
-#include <cstdlib>
 
 #include "common.cuh"
+#include "host_common.h"
 #include "kernels.h"
 
 namespace sl {
-static bool prefer_mma_sync();   // environment switch, defined with the dispatchers below
 namespace {
 
 constexpr int BT = 64;            // rows of a query tile and of a key tile
@@ -393,11 +392,12 @@ __global__ void __launch_bounds__(NT) attn_bwd_dkv_tc_kernel(const bf16* __restr
 
 template <int DH>
 cudaError_t launch_fwd(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, cudaStream_t st) {
-  static bool attr = false;
-  if (!attr) {
+  static PerDeviceOnce once;                    // one per instantiation; attributes are per device
+  const int dev = current_device();
+  if (once.needed(dev)) {
     cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, Sizes<DH>::FWD);
     if (e != cudaSuccess) return e;
-    attr = true;
+    once.done(dev);
   }
   dim3 grid(T / BT, H, nseq);
   attn_fwd_tc_kernel<DH><<<grid, NT, Sizes<DH>::FWD, st>>>((const bf16*)qkv, (bf16*)o, lse, T, H, d,
@@ -407,22 +407,23 @@ cudaError_t launch_fwd(const void* qkv, int nseq, int T, int H, int d, void* o, 
 
 template <int DH>
 cudaError_t launch_bwd(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq, int T, int H, int d,
-                       void* dqkv, float* rowdot, cudaStream_t st) {
-  static bool attr = false;
-  if (!attr) {
+                       void* dqkv, float* rowdot, int* status, cudaStream_t st) {
+  static PerDeviceOnce once;
+  const int dev = current_device();
+  if (once.needed(dev)) {
     cudaError_t e = cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, Sizes<DH>::DQ);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_bwd_dkv_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, Sizes<DH>::DKV);
     if (e != cudaSuccess) return e;
-    attr = true;
+    once.done(dev);
   }
   int64_t threads = (int64_t)nseq * T * H * (DH / 8);
   attn_rowdot_tc_kernel<DH><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>((const bf16*)o, (const bf16*)d_o, nseq, T, H, d, rowdot);
   dim3 grid(T / BT, H, nseq);
   const float scale = 1.0f / sqrtf((float)DH);
-  if (DH == 128 && attention_bwd_t5_128_supported(DT_BF16, T, H, d) && !prefer_mma_sync())
+  if (DH == 128 && attention_bwd_t5_128_supported(DT_BF16, T, H, d))
     // dQ, dK, dV on the tcgen05 kernels (they read D[row] from `rowdot`, written just above)
-    return attention_bwd_t5_128(qkv, lse, d_o, rowdot, nseq, T, H, d, dqkv, nullptr, st);
+    return attention_bwd_t5_128(qkv, lse, d_o, rowdot, nseq, T, H, d, dqkv, status, st);
   attn_bwd_dq_tc_kernel<DH><<<grid, NT, Sizes<DH>::DQ, st>>>((const bf16*)qkv, (const bf16*)d_o, lse, rowdot, (bf16*)dqkv, T, H, d, scale);
   attn_bwd_dkv_tc_kernel<DH><<<grid, NT, Sizes<DH>::DKV, st>>>((const bf16*)qkv, (const bf16*)d_o, lse, rowdot, (bf16*)dqkv, T, H, d, scale);
   return cudaGetLastError();
@@ -434,28 +435,22 @@ bool attention_tc_supported(int dt, int T, int H, int d) {
   return dt == DT_BF16 && H > 0 && d % H == 0 && (d / H == 64 || d / H == 128) && T >= BT && T % BT == 0;
 }
 
-// SPLITLORA_ATTENTION_MMA_SYNC=1 keeps the mma.sync kernels even where the tcgen05 ones apply
-// (debugging aid / second opinion).
-static bool prefer_mma_sync() {
-  static int v = -1;
-  if (v < 0) { const char* e = std::getenv("SPLITLORA_ATTENTION_MMA_SYNC"); v = (e && e[0] == '1') ? 1 : 0; }
-  return v == 1;
-}
-
-cudaError_t attention_fwd_tc(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, cudaStream_t st) {
+// status: device word that receives a code when a bounded wait inside the tcgen05 kernels expires
+// (nullptr: the library's own word, see library_status_word).
+cudaError_t attention_fwd_tc(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, int* status,
+                             cudaStream_t st) {
   if (!attention_tc_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
-  if (attention_fwd_t5_supported(DT_BF16, T, H, d) && !prefer_mma_sync())
-    return attention_fwd_t5(qkv, nseq, T, H, d, o, lse, nullptr, st);
+  if (attention_fwd_t5_supported(DT_BF16, T, H, d)) return attention_fwd_t5(qkv, nseq, T, H, d, o, lse, status, st);
   return d / H == 64 ? launch_fwd<64>(qkv, nseq, T, H, d, o, lse, st) : launch_fwd<128>(qkv, nseq, T, H, d, o, lse, st);
 }
 
 cudaError_t attention_bwd_tc(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq, int T, int H,
-                             int d, void* dqkv, float* rowdot, cudaStream_t st) {
+                             int d, void* dqkv, float* rowdot, int* status, cudaStream_t st) {
   if (!attention_tc_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
-  if (attention_t5_supported(DT_BF16, T, H, d) && !prefer_mma_sync())
-    return attention_bwd_t5(qkv, o, lse, d_o, nseq, T, H, d, dqkv, rowdot, nullptr, st);
-  return d / H == 64 ? launch_bwd<64>(qkv, o, lse, d_o, nseq, T, H, d, dqkv, rowdot, st)
-                     : launch_bwd<128>(qkv, o, lse, d_o, nseq, T, H, d, dqkv, rowdot, st);
+  if (attention_t5_supported(DT_BF16, T, H, d))
+    return attention_bwd_t5(qkv, o, lse, d_o, nseq, T, H, d, dqkv, rowdot, status, st);
+  return d / H == 64 ? launch_bwd<64>(qkv, o, lse, d_o, nseq, T, H, d, dqkv, rowdot, status, st)
+                     : launch_bwd<128>(qkv, o, lse, d_o, nseq, T, H, d, dqkv, rowdot, status, st);
 }
 
 }  // namespace sl

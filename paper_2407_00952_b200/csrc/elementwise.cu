@@ -247,7 +247,7 @@ cudaError_t layernorm_bwd(int dt, const void* dy, const void* x, const void* g, 
 // cross-entropy: one block per row.  Pass 1: online max / sum of exp; pass 2: overwrite the row
 // with (softmax - onehot) / n_valid.  Pad columns [V, ld) are written as zero.
 // ------------------------------------------------------------------------------------------
-__global__ void count_valid_kernel(const int32_t* __restrict__ labels, int M, int* __restrict__ n_valid,
+__global__ void count_valid_kernel(const int32_t* __restrict__ labels, int M, int V, int* __restrict__ n_valid,
                                    int normalizer_override) {
   if (normalizer_override > 0) {       // the batch is one shard of a larger one: use the global count
     if (threadIdx.x == 0) *n_valid = normalizer_override;
@@ -255,7 +255,7 @@ __global__ void count_valid_kernel(const int32_t* __restrict__ labels, int M, in
   }
   __shared__ int sh[32];
   int c = 0;
-  for (int i = threadIdx.x; i < M; i += blockDim.x) c += labels[i] >= 0 ? 1 : 0;
+  for (int i = threadIdx.x; i < M; i += blockDim.x) c += (labels[i] >= 0 && labels[i] < V) ? 1 : 0;   // the predicate of the row kernels
   for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
   if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = c;
   __syncthreads();
@@ -459,7 +459,7 @@ __global__ void loss_reduce_kernel(const float* __restrict__ row_loss, int M, co
 
 cudaError_t cross_entropy(int dt, void* logits, int64_t ld, const int32_t* labels, int M, int V, float* row_loss,
                           int* n_valid, float* loss, int normalizer_override, cudaStream_t st) {
-  count_valid_kernel<<<1, 1024, 0, st>>>(labels, M, n_valid, normalizer_override);
+  count_valid_kernel<<<1, 1024, 0, st>>>(labels, M, V, n_valid, normalizer_override);
   if (dt == DT_BF16 && ld % 8 == 0 && (reinterpret_cast<uintptr_t>(logits) & 15u) == 0)
     ce_bf16_kernel<<<M, 256, 0, st>>>((bf16*)logits, ld, labels, V, row_loss, n_valid);
   else if (dt == DT_BF16) ce_kernel<bf16><<<M, 256, 0, st>>>((bf16*)logits, ld, labels, V, row_loss, n_valid);
@@ -532,6 +532,33 @@ __global__ void __launch_bounds__(256) aggregate_kernel(float* __restrict__ para
   }
 }
 
+// The two halves of the same step for clients spread over several devices: the weighted sum of the
+// local clients' rows goes to `sum` [P] (which the caller then adds up over devices), and `sum` is
+// afterwards written to every local client's row (the downlink of step b3).
+__global__ void __launch_bounds__(256) weighted_sum_kernel(const float* __restrict__ params, int K, int64_t P4,
+                                                           AggWeights w, float* __restrict__ sum) {
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < P4; i += stride) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k = 0; k < K; ++k) {
+      float4 v = __ldcs(reinterpret_cast<const float4*>(params) + (size_t)k * P4 + i);
+      acc.x = fmaf(w.w[k], v.x, acc.x);
+      acc.y = fmaf(w.w[k], v.y, acc.y);
+      acc.z = fmaf(w.w[k], v.z, acc.z);
+      acc.w = fmaf(w.w[k], v.w, acc.w);
+    }
+    reinterpret_cast<float4*>(sum)[i] = acc;
+  }
+}
+__global__ void __launch_bounds__(256) broadcast_rows_kernel(const float* __restrict__ sum, int K, int64_t P4,
+                                                             float* __restrict__ params) {
+  int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < P4; i += stride) {
+    const float4 v = reinterpret_cast<const float4*>(sum)[i];
+    for (int k = 0; k < K; ++k) __stcs(reinterpret_cast<float4*>(params) + (size_t)k * P4 + i, v);
+  }
+}
+
 // Clients with different adapter ranks (Sec. V, heterogeneous configuration): every client is stored
 // at the configured rank r with the components it does not have equal to zero.  The arena of client
 // i is a sequence of (A [r, d], B [d, r]) pairs; this kernel zeroes rank components >= rank[i]
@@ -565,6 +592,27 @@ cudaError_t aggregate(float* params, int K, int64_t P, const float* w_host, cuda
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   aggregate_kernel<<<(unsigned)blocks, 256, 0, st>>>(params, K, P4, w);
+  return cudaGetLastError();
+}
+
+static unsigned agg_blocks(int64_t P4) {
+  int64_t blocks = (P4 + 255) / 256;
+  const int64_t cap = 148 * 8;
+  if (blocks > cap) blocks = cap;
+  return (unsigned)(blocks < 1 ? 1 : blocks);
+}
+
+cudaError_t aggregate_local_sum(const float* params, int K, int64_t P, const float* w_host, float* sum, cudaStream_t st) {
+  if (K < 1 || K > AGG_MAX_CLIENTS || P % 4 != 0) return cudaErrorInvalidValue;
+  AggWeights w;
+  for (int k = 0; k < AGG_MAX_CLIENTS; ++k) w.w[k] = k < K ? w_host[k] : 0.f;
+  weighted_sum_kernel<<<agg_blocks(P / 4), 256, 0, st>>>(params, K, P / 4, w, sum);
+  return cudaGetLastError();
+}
+
+cudaError_t aggregate_broadcast(const float* sum, int K, int64_t P, float* params, cudaStream_t st) {
+  if (K < 1 || K > AGG_MAX_CLIENTS || P % 4 != 0) return cudaErrorInvalidValue;
+  broadcast_rows_kernel<<<agg_blocks(P / 4), 256, 0, st>>>(sum, K, P / 4, params);
   return cudaGetLastError();
 }
 

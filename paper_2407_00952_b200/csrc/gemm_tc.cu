@@ -23,8 +23,7 @@
 // two warps of a lane quarter take one half of the tile's columns each).
 // Every wait on an mbarrier is bounded: when it expires the kernel records a code in `status`,
 // stops issuing work, waits briefly for copies in flight, frees its tensor memory and returns.
-#include <cstdlib>
-
+#include "host_common.h"
 #include "tc_common.cuh"
 
 namespace sl {
@@ -409,35 +408,24 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_const
 }
 
 // ---- host side -----------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn g_encode = nullptr;
-int g_num_sms = 0;
-int g_max_pairs = 0;      // CTA pairs that can be resident at once (0: pair kernel unavailable)
+// CTA pairs that can be resident at once, per device (0: pair kernel unavailable there)
+int g_max_pairs[MAX_DEVICES] = {};
+PerDeviceOnce g_pair_once;
 
 // 2-D bf16 tensor [rows, cols] with leading dimension ld (elements); box = 64 columns x box_rows rows.
 bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {ld * 2};
-  cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  return cached_map_2d(m, ptr, rows, cols, ld, (uint32_t)BK, box_rows, CU_TENSOR_MAP_SWIZZLE_128B,
+                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
 // Output map: bf16 [rows, cols], box = 32 columns x 32 rows, 64-byte swizzle (the epilogue's staging layout).
 bool make_out_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld) {
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {ld * 2};
-  cuuint32_t box[2] = {32, 32};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  return cached_map_2d(m, ptr, rows, cols, ld, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE);
+}
+
+int max_pairs() {
+  const int dev = current_device();
+  return dev < 0 ? 0 : g_max_pairs[dev];
 }
 
 int pick_bn(const GemmArgs& a) {
@@ -448,7 +436,7 @@ int pick_bn(const GemmArgs& a) {
 }
 
 bool pair_ok(const GemmArgs& a) {
-  if (g_max_pairs < 1 || a.k_gap_len > 0) return false;
+  if (max_pairs() < 1 || a.k_gap_len > 0) return false;
   if (a.M % (2 * BM) != 0 || a.N < 256) return false;
   if (a.rows_per_group > 0 && a.rows_per_group % (2 * BM) != 0) return false;
   return true;
@@ -490,19 +478,21 @@ bool prepare(const GemmArgs& a, int* status, int w_box_rows, CUtensorMap* mX, CU
 template <int BN, bool DEEP = false>
 cudaError_t launch(const GemmArgs& a, int* status, cudaStream_t st) {
   using C = Cfg<BN, DEEP>;
-  if (BN == 64 && !DEEP && (a.M / BM) * ((a.N + BN - 1) / BN) <= g_num_sms) return launch<64, true>(a, status, st);
-  static bool attr_set = false;
-  if (!attr_set) {
+  const int sms = num_sms();
+  if (BN == 64 && !DEEP && (a.M / BM) * ((a.N + BN - 1) / BN) <= sms) return launch<64, true>(a, status, st);
+  static PerDeviceOnce once;                    // one per instantiation; attributes are per device
+  const int dev = current_device();
+  if (once.needed(dev)) {
     cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    once.done(dev);
   }
   CUtensorMap mX, mW, mXe, mWe, mY, mZ;
   TcParams p;
   if (!prepare(a, status, BN, &mX, &mW, &mXe, &mWe, &mY, &mZ, &p)) return cudaErrorInvalidValue;
   p.tiles_m = a.M / BM; p.tiles_n = (a.N + BN - 1) / BN;
   const int tiles = p.tiles_m * p.tiles_n;
-  const int slots = g_num_sms * C::CTAS_PER_SM;
+  const int slots = sms * C::CTAS_PER_SM;
   const int grid = tiles < slots ? tiles : slots;
   gemm_tc_kernel<BN, DEEP><<<grid, NUM_THREADS, C::SMEM_BYTES, st>>>(mX, mW, mXe, mWe, mY, mZ, p);
   return cudaGetLastError();
@@ -515,7 +505,7 @@ cudaError_t launch_pair(const GemmArgs& a, int* status, cudaStream_t st) {
   if (!prepare(a, status, BN / 2, &mX, &mW, &mXe, &mWe, &mY, &mZ, &p)) return cudaErrorInvalidValue;
   p.tiles_m = a.M / (2 * BM); p.tiles_n = (a.N + BN - 1) / BN;
   const int tiles = p.tiles_m * p.tiles_n;
-  const int pairs = tiles < g_max_pairs ? tiles : g_max_pairs;
+  const int pairs = tiles < max_pairs() ? tiles : max_pairs();
   const bool need_r = a.epi == EPI_BIAS_RESID || a.epi == EPI_MUL_GELUGRAD;
   if (need_r) {
     if (!make_map(&mR, a.R, a.M, a.N, a.ldr, BM)) return cudaErrorInvalidValue;
@@ -530,39 +520,32 @@ cudaError_t launch_pair(const GemmArgs& a, int* status, cudaStream_t st) {
 }  // namespace
 
 int gemm_tc_init() {
-  if (g_encode) return 0;
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult q;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
-      q != cudaDriverEntryPointSuccess)
-    return -1;
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return -1;
-  if (cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_num_sms < 1) return -1;
-  // how many CTA pairs fit on the device at once (the pair kernel is persistent: one wave)
-  g_max_pairs = 0;
-  const char* off = std::getenv("SPLITLORA_NO_CTA_PAIRS");     // debugging aid: force the single-CTA kernel
-  if (!(off && off[0] == '1') &&
-      cudaFuncSetAttribute(gemm_tc_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<false>::SMEM_BYTES) == cudaSuccess &&
+  if (!tensor_map_encoder()) return -1;
+  const int dev = current_device(), sms = num_sms();
+  if (dev < 0 || sms < 1) return -1;
+  if (!g_pair_once.needed(dev)) return 0;
+  // how many CTA pairs fit on this device at once (the pair kernel is persistent: one wave)
+  g_max_pairs[dev] = 0;
+  if (cudaFuncSetAttribute(gemm_tc_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<false>::SMEM_BYTES) == cudaSuccess &&
       cudaFuncSetAttribute(gemm_tc_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<true>::SMEM_BYTES) == cudaSuccess) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(g_num_sms & ~1); cfg.blockDim = dim3(NUM_THREADS); cfg.dynamicSmemBytes = PairCfg<true>::SMEM_BYTES;
+    cfg.gridDim = dim3(sms & ~1); cfg.blockDim = dim3(NUM_THREADS); cfg.dynamicSmemBytes = PairCfg<true>::SMEM_BYTES;
     cudaLaunchAttribute at;
     at.id = cudaLaunchAttributeClusterDimension;
     at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
     cfg.attrs = &at; cfg.numAttrs = 1;
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_pair_kernel<true>, &cfg) == cudaSuccess && n > 0)
-      g_max_pairs = n < g_num_sms / 2 ? n : g_num_sms / 2;
+      g_max_pairs[dev] = n < sms / 2 ? n : sms / 2;
     cudaGetLastError();
   }
-  g_encode = (EncodeTiledFn)fn;
+  g_pair_once.done(dev);
   return 0;
 }
 
 bool gemm_tc_supported(const GemmArgs& a) {
   auto al16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
-  if (!g_encode || a.dtype != DT_BF16) return false;
+  if (!tensor_map_encoder() || a.dtype != DT_BF16) return false;
   if (a.M < BM || a.M % BM != 0 || a.K < BK || a.K % BK != 0 || a.N < 8 || a.N % 8 != 0) return false;
   if (a.rows_per_group > 0 && (a.rows_per_group % BM != 0 || a.M % a.rows_per_group != 0)) return false;
   if (a.ldx % 8 || a.ldw % 8 || a.ldy % 8) return false;

@@ -102,9 +102,10 @@ cudaError_t attention_fwd_t5(const void* qkv, int nseq, int T, int H, int d, voi
 cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq, int T, int H,
                              int d, void* dqkv, float* rowdot, int* status, cudaStream_t st);
 bool attention_tc_supported(int dt, int T, int H, int d);
-cudaError_t attention_fwd_tc(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, cudaStream_t st);
+cudaError_t attention_fwd_tc(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, int* status,
+                             cudaStream_t st);
 cudaError_t attention_bwd_tc(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq,
-                             int T, int H, int d, void* dqkv, float* rowdot, cudaStream_t st);
+                             int T, int H, int d, void* dqkv, float* rowdot, int* status, cudaStream_t st);
 
 // Adapter gradients: for nt targets of rank r (weight columns wcol0 + t*rp + jj of Wt),
 //   out[g][t][jj][c] = scale * sum_{m in group g} Wt[m, wcol0 + t*rp + jj] * Z[m, zcol0 + c],  c < C,
@@ -136,6 +137,10 @@ static const int AGG_MAX_CLIENTS = 64;
 // zero rank components >= ranks_host[i] in client i's arena of (A [r, d], B [d, r]) pairs (P floats per client)
 cudaError_t rank_mask(float* params, int K, int64_t P, int r, int d, const int* ranks_host, cudaStream_t st);
 cudaError_t aggregate(float* params, int K, int64_t P, const float* w_host, cudaStream_t st);
+// The same step in two halves, for clients spread over devices: sum [P] = sum_i w[i] params[i, :], and
+// (after the caller has added the sums of all devices) every row of params [K, P] = sum.
+cudaError_t aggregate_local_sum(const float* params, int K, int64_t P, const float* w_host, float* sum, cudaStream_t st);
+cudaError_t aggregate_broadcast(const float* sum, int K, int64_t P, float* params, cudaStream_t st);
 
 // Compute copies of the adapters of one layer (G groups), built from fp32 masters.
 // Target t of group g has A_t [r, d_in] at A + g*a_gs + t*a_ts and B_t [d_out, r] at B + g*b_gs + t*b_ts.

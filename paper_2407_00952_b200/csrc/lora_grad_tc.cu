@@ -12,6 +12,7 @@
 
 #include "common.cuh"
 #include "kernels.h"
+#include "host_common.h"
 #include "tc_common.cuh"
 
 namespace sl {
@@ -151,32 +152,21 @@ lora_grad_tc_kernel(const __grid_constant__ CUtensorMap mapZ, const __grid_const
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn g_encode = nullptr;
+PerDeviceOnce g_once;
 
 // bf16 [rows, cols] with leading dimension ld; box = 64 columns x 64 rows, 128-byte swizzle
 bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld) {
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {ld * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)LT_K};
-  cuuint32_t estr[2] = {1, 1};
-  return g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return cached_map_2d(m, ptr, rows, cols, ld, 64, (uint32_t)LT_K, CU_TENSOR_MAP_SWIZZLE_128B,
+                       CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
 
-bool init_once() {
-  if (g_encode) return true;
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult q;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
-      q != cudaDriverEntryPointSuccess)
-    return false;
+bool init_device() {
+  const int dev = current_device();
+  if (dev < 0 || !tensor_map_encoder()) return false;
+  if (!g_once.needed(dev)) return true;
   if (cudaFuncSetAttribute(lora_grad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LT_SMEM) != cudaSuccess)
     return false;
-  g_encode = (EncodeTiledFn)fn;
+  g_once.done(dev);
   return true;
 }
 
@@ -199,7 +189,9 @@ bool lora_grad_tc_supported(int dt, const void* Z, int64_t ldz, int zcol0, int C
 cudaError_t lora_grad_tc_partial(const void* Z, int64_t ldz, int zcol0, int C, const void* Wt, int64_t ldwt, int wcol0,
                                  int r, int rp, int nt, int M, int rows_per_group, float* partial, int* status,
                                  int* chunks_per_group, cudaStream_t st) {
-  if (!init_once()) return cudaErrorNotSupported;
+  if (!init_device()) return cudaErrorNotSupported;
+  if (!status) status = library_status_word();
+  if (!status) return cudaErrorNotSupported;
   const int rpg = rows_per_group > 0 ? rows_per_group : M;
   const int groups = M / rpg;
   const int ctiles = (C + LT_C - 1) / LT_C;

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include "../../include/splitlora.h"
+#include "host_common.h"
 #include "kernels.h"
 
 using namespace sl;
@@ -153,6 +154,15 @@ int splitlora_lora_linear_bwd(int dtype, int use_tc, const void* x, const void* 
   return SPLITLORA_OK;
 }
 
+int splitlora_library_status(int32_t* code) {
+  if (!code) return SPLITLORA_ERR_ARG;
+  int* word = library_status_word();
+  if (!word) return SPLITLORA_ERR_CUDA;
+  if (cudaDeviceSynchronize() != cudaSuccess) return SPLITLORA_ERR_CUDA;
+  if (cudaMemcpy(code, word, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SPLITLORA_ERR_CUDA;
+  return *code ? SPLITLORA_ERR_TIMEOUT : SPLITLORA_OK;
+}
+
 int splitlora_transpose(int dtype, const void* in, int rows, int cols, void* out, void* stream) {
   if (!in || !out || rows < 1 || cols < 1 || (dtype != DT_F32 && dtype != DT_BF16)) return SPLITLORA_ERR_ARG;
   return transpose(dtype, in, rows, cols, out, rows, (cudaStream_t)stream) == cudaSuccess ? SPLITLORA_OK : SPLITLORA_ERR_CUDA;
@@ -183,11 +193,12 @@ int splitlora_aggregate_buffers(float* params, int K, int64_t P, const double* w
 
 int splitlora_attention_fwd(int dtype, int use_tc, const void* qkv, int nseq, int T, int n_head, int d_model, void* o,
                             float* lse, void* stream) {
-  if (!qkv || !o || !lse || nseq < 1 || T < 1 || n_head < 1 || d_model % n_head != 0 || d_model / n_head > 128)
+  if (!qkv || !o || !lse || nseq < 1 || T < 1 || n_head < 1 || d_model % n_head != 0 || d_model / n_head > 128 ||
+      (dtype != DT_F32 && dtype != DT_BF16))
     return SPLITLORA_ERR_ARG;
   cudaError_t e;
   if (use_tc && attention_tc_supported(dtype, T, n_head, d_model))
-    e = attention_fwd_tc(qkv, nseq, T, n_head, d_model, o, lse, (cudaStream_t)stream);
+    e = attention_fwd_tc(qkv, nseq, T, n_head, d_model, o, lse, nullptr, (cudaStream_t)stream);
   else
     e = attention_fwd_simt(dtype, qkv, nseq, T, n_head, d_model, o, lse, (cudaStream_t)stream);
   return e == cudaSuccess ? SPLITLORA_OK : SPLITLORA_ERR_CUDA;
@@ -196,11 +207,11 @@ int splitlora_attention_fwd(int dtype, int use_tc, const void* qkv, int nseq, in
 int splitlora_attention_bwd(int dtype, int use_tc, const void* qkv, const void* o, const float* lse, const void* d_o,
                             int nseq, int T, int n_head, int d_model, void* dqkv, float* rowdot, void* stream) {
   if (!qkv || !o || !lse || !d_o || !dqkv || !rowdot || nseq < 1 || T < 1 || n_head < 1 || d_model % n_head != 0 ||
-      d_model / n_head > 128)
+      d_model / n_head > 128 || (dtype != DT_F32 && dtype != DT_BF16))
     return SPLITLORA_ERR_ARG;
   cudaError_t e;
   if (use_tc && attention_tc_supported(dtype, T, n_head, d_model))
-    e = attention_bwd_tc(qkv, o, lse, d_o, nseq, T, n_head, d_model, dqkv, rowdot, (cudaStream_t)stream);
+    e = attention_bwd_tc(qkv, o, lse, d_o, nseq, T, n_head, d_model, dqkv, rowdot, nullptr, (cudaStream_t)stream);
   else
     e = attention_bwd_simt(dtype, qkv, o, lse, d_o, nseq, T, n_head, d_model, dqkv, rowdot, (cudaStream_t)stream);
   return e == cudaSuccess ? SPLITLORA_OK : SPLITLORA_ERR_CUDA;

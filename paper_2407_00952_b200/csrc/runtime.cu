@@ -83,6 +83,7 @@ struct splitlora_ctx {
   int64_t per_layer = 0, Pc = 0, Ps = 0;     // floats per layer, per client set, server set
   float *cp = nullptr, *cg = nullptr, *cm = nullptr, *cv = nullptr;   // client params/grads/moments [K, Pc]
   float *sp = nullptr, *sg = nullptr, *sm = nullptr, *sv = nullptr;   // server [Ps]
+  float* agg_sum = nullptr;   // [Pc]: weighted sum of the local clients' adapters (clients spread over devices)
   void *emb = nullptr, *u2 = nullptr, *act = nullptr, *xf = nullptr, *logits = nullptr;
   float *meanf = nullptr, *rstdf = nullptr, *row_loss = nullptr, *rowdot = nullptr, *loss_dev = nullptr,
         *grad_scratch = nullptr;
@@ -196,6 +197,7 @@ size_t plan(splitlora_ctx* c, char* ws) {
   c->cm = (float*)a.take((size_t)c->K * c->Pc * 4); c->cv = (float*)a.take((size_t)c->K * c->Pc * 4);
   c->sp = (float*)a.take((size_t)c->Ps * 4); c->sg = (float*)a.take((size_t)c->Ps * 4);
   c->sm = (float*)a.take((size_t)c->Ps * 4); c->sv = (float*)a.take((size_t)c->Ps * 4);
+  c->agg_sum = (float*)a.take((size_t)c->Pc * 4);
   c->fl.resize(c->L);
   c->lb.resize(c->L);
   for (int l = 0; l < c->L; ++l) {
@@ -351,7 +353,7 @@ cudaError_t block_forward(splitlora_ctx* c, int l, const void* x_in, void* x_out
   }
   { Scope s(c, "attention_fwd", 1);
     if (c->tc && attention_tc_supported(c->dt, c->cfg.seq, c->cfg.n_head, d))
-      e = attention_fwd_tc(b.qkv, c->nseq, c->cfg.seq, c->cfg.n_head, d, b.o, b.lse, c->st);
+      e = attention_fwd_tc(b.qkv, c->nseq, c->cfg.seq, c->cfg.n_head, d, b.o, b.lse, c->status, c->st);
     else
       e = attention_fwd_simt(c->dt, b.qkv, c->nseq, c->cfg.seq, c->cfg.n_head, d, b.o, b.lse, c->st);
     if (e) return e; }
@@ -431,7 +433,8 @@ cudaError_t block_backward(splitlora_ctx* c, int l, const void* dy, void* dx) {
     if ((e = linear(c, c->has_o ? "lora_linear_bwd" : "linear_bwd", a))) return e; }
   { Scope s(c, "attention_bwd", c->tc && attention_t5_supported(c->dt, c->cfg.seq, c->cfg.n_head, d) ? 2 : 3);
     if (c->tc && attention_tc_supported(c->dt, c->cfg.seq, c->cfg.n_head, d))
-      e = attention_bwd_tc(b.qkv, b.o, b.lse, c->g_do, c->nseq, c->cfg.seq, c->cfg.n_head, d, c->g_dqkv, c->rowdot, c->st);
+      e = attention_bwd_tc(b.qkv, b.o, b.lse, c->g_do, c->nseq, c->cfg.seq, c->cfg.n_head, d, c->g_dqkv, c->rowdot, c->status,
+                           c->st);
     else
       e = attention_bwd_simt(c->dt, b.qkv, b.o, b.lse, c->g_do, c->nseq, c->cfg.seq, c->cfg.n_head, d, c->g_dqkv, c->rowdot, c->st);
     if (e) return e; }
@@ -807,7 +810,8 @@ int splitlora_client_bwd(splitlora_ctx* c, const void* act_grad_in) {
   return SPLITLORA_OK;
 }
 
-static int aggregate_with_total(splitlora_ctx* c, const int64_t* counts, double total_override) {
+// w_i = |D_i| / total, total = the local sum or, when the clients are spread over devices, |D| of all of them
+static int aggregation_weights(splitlora_ctx* c, const int64_t* counts, double total_override, float* w) {
   if (!c) return SPLITLORA_ERR_ARG;
   if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
   if (!counts) return fail(c, SPLITLORA_ERR_ARG, "null counts");
@@ -821,13 +825,7 @@ static int aggregate_with_total(splitlora_ctx* c, const int64_t* counts, double 
     total = total_override;
   }
   if (!(total > 0.0)) return fail(c, SPLITLORA_ERR_COUNTS, "all sample counts are zero");
-  float w[AGG_MAX_CLIENTS];
   for (int i = 0; i < c->K; ++i) w[i] = (float)((double)counts[i] / total);
-  { Scope s(c, "aggregate", c->client_rank.empty() ? 1 : 2);
-    CK(c, aggregate(c->cp, c->K, c->Pc, w, c->st));
-    // clients of lower rank keep only their own components of the (zero-padded) average
-    if (!c->client_rank.empty()) CK(c, rank_mask(c->cp, c->K, c->Pc, c->r, c->d, c->client_rank.data(), c->st)); }
-  c->client_copies_dirty = true;
   return SPLITLORA_OK;
 }
 
@@ -847,13 +845,42 @@ int splitlora_set_client_ranks(splitlora_ctx* c, const int32_t* ranks) {
   return SPLITLORA_OK;
 }
 
-int splitlora_aggregate(splitlora_ctx* c, const int64_t* counts) { return aggregate_with_total(c, counts, 0.0); }
+int splitlora_aggregate(splitlora_ctx* c, const int64_t* counts) {
+  float w[AGG_MAX_CLIENTS];
+  int rc = aggregation_weights(c, counts, 0.0, w);
+  if (rc) return rc;
+  { Scope s(c, "aggregate", c->client_rank.empty() ? 1 : 2);
+    CK(c, aggregate(c->cp, c->K, c->Pc, w, c->st));
+    // clients of lower rank keep only their own components of the (zero-padded) average
+    if (!c->client_rank.empty()) CK(c, rank_mask(c->cp, c->K, c->Pc, c->r, c->d, c->client_rank.data(), c->st)); }
+  c->client_copies_dirty = true;
+  return SPLITLORA_OK;
+}
 
 // ---- hooks for sharding the clients over several devices --------------------------------------
 
-int splitlora_aggregate_partial(splitlora_ctx* c, const int64_t* counts, int64_t total_count) {
+int splitlora_aggregate_local_sum(splitlora_ctx* c, const int64_t* counts, int64_t total_count, float** sum_dev,
+                                  int64_t* count) {
+  if (!c || !sum_dev || !count) return SPLITLORA_ERR_ARG;
   if (total_count <= 0) return fail(c, SPLITLORA_ERR_COUNTS, "total_count must be positive");
-  return aggregate_with_total(c, counts, (double)total_count);
+  float w[AGG_MAX_CLIENTS];
+  int rc = aggregation_weights(c, counts, (double)total_count, w);
+  if (rc) return rc;
+  { Scope s(c, "aggregate", 1);
+    CK(c, aggregate_local_sum(c->cp, c->K, c->Pc, w, c->agg_sum, c->st)); }
+  *sum_dev = c->agg_sum; *count = c->Pc;
+  return SPLITLORA_OK;
+}
+
+int splitlora_aggregate_broadcast(splitlora_ctx* c) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
+  { Scope s(c, "aggregate", c->client_rank.empty() ? 1 : 2);
+    CK(c, aggregate_broadcast(c->agg_sum, c->K, c->Pc, c->cp, c->st));
+    // the mask comes after the sum over devices: the sum holds every client's components
+    if (!c->client_rank.empty()) CK(c, rank_mask(c->cp, c->K, c->Pc, c->r, c->d, c->client_rank.data(), c->st)); }
+  c->client_copies_dirty = true;
+  return SPLITLORA_OK;
 }
 
 int splitlora_set_loss_normalizer(splitlora_ctx* c, int64_t n_valid_global) {

@@ -7,7 +7,8 @@ calls of the round on its own clients.  Two sums over ranks make the result equa
 single-device round:
 
   1. the server adapter gradients (and the loss) after the server backward, before Eq. 4-5;
-  2. the weighted client adapter sums of Eq. 8-9 at aggregation.
+  2. the weighted client adapter sum of Eq. 8-9 at aggregation: one client's worth of parameters per
+     rank, so ranks may hold different numbers of clients.
 
 This module only orders the calls and the collectives (torch.distributed: NCCL on GPUs, gloo in
 the CPU tests); all arithmetic happens inside the engine.  `engine` is a binding.SplitLoRA or any
@@ -60,8 +61,7 @@ class ShardedRound:
         eng.client_bwd(dS)                                          # step a5
         self.round_index += 1
         if self.round_index % self.agg_interval == 0:               # stage b
-            eng.aggregate_partial(local_counts, int(total_count))
-            params = eng.adapter_buffer(SIDE_CLIENT, KIND_PARAMS)
-            self._sum(params)
-            eng.adapters_changed(SIDE_CLIENT)
+            part = eng.aggregate_local_sum(local_counts, int(total_count))   # [Pc], whatever K_local is
+            self._sum(part)
+            eng.aggregate_broadcast()                                        # downlink b3 to the local clients
         return loss

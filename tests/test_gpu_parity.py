@@ -270,6 +270,7 @@ def test_attention_bf16(nseq, T, Hh, d, use_tc):
     got = H.tnp(dqkv)
     for j, ref in enumerate((dq, dk, dv)):
         assert H.rel_err(got[:, j * d:(j + 1) * d], ref.reshape(-1, d)) <= TOL_BF16
+    assert B.library_status() == 0          # no bounded wait of the stand-alone kernels expired
 
 
 @pytest.mark.parametrize("Hh,d", [(2, 128), (2, 256)])
@@ -297,6 +298,25 @@ def test_attention_bf16_peaked_scores(Hh, d):
     got = H.tnp(dqkv)
     for j, ref in enumerate((dq, dk, dv)):
         assert H.rel_err(got[:, j * d:(j + 1) * d], ref.reshape(-1, d)) <= TOL_BF16, j
+
+
+def test_out_of_range_labels_are_ignored():
+    """A label outside [0, vocab) is an ignored position for the loss, the gradients and the normaliser
+    alike: the round equals the oracle's with those positions marked -1."""
+    w = synth.WORKLOADS[1]
+    frozen, cads, sads, tokens, labels = H.build_case(w)
+    gpu_labels, ref_labels = labels.copy(), labels.copy()
+    gpu_labels[0, 1, 5:40] = w.vocab + 3
+    gpu_labels[1, 2, :7] = -5
+    ref_labels[0, 1, 5:40] = -1
+    ref_labels[1, 2, :7] = -1
+    eng, S, dS, loss = H.run_three_calls(w, frozen, cads, sads, tokens, gpu_labels)
+    _, _, _, _, S_ref, dS_ref, loss_ref, sg, _ = H.oracle_three_calls(w, frozen, cads, sads, tokens, ref_labels)
+    assert abs(loss - loss_ref) <= TOL_LOSS * abs(loss_ref)
+    assert H.rel_err(H.tnp(dS), dS_ref) <= TOL_FP32
+    for (l, t), (dA, dB) in sg.items():
+        gA, gB = eng.get_adapter_grad(B.SIDE_SERVER, 0, l, B.TARGET_BITS[t])
+        assert H.rel_err(H.tnp(gA), dA) <= TOL_FP32 and H.rel_err(H.tnp(gB), dB) <= TOL_FP32
 
 
 def test_checkpoint_resume_and_determinism():

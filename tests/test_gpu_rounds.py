@@ -165,8 +165,10 @@ def test_adamw_kernel_on_identical_inputs(step):
         mA, vA, mB, vB = (H.tnp(x) for x in eng.get_opt_state(side, i, l, bit))
         for part, (m_got, v_got) in enumerate(((mA, vA), (mB, vB))):
             b = before[key]
-            p_ref, m_ref, v_ref = O.adamw_update(b["p"][part], g[part], b["m"][part], b["v"][part], step, w.lr,
-                                                 0.9, 0.999, 1e-8, 0.01)
+            # the hyper-parameters as the configuration struct holds them (fp32 fields)
+            lr, b1, b2, eps, wd = (float(np.float32(x)) for x in (w.lr, 0.9, 0.999, 1e-8, 0.01))
+            p_ref, m_ref, v_ref = O.adamw_update(b["p"][part], g[part], b["m"][part], b["v"][part], step, lr,
+                                                 b1, b2, eps, wd)
             assert H.rel_err(m_got, m_ref) <= 1e-6, (key, part)
             assert H.rel_err(v_got, v_ref) <= 1e-6, (key, part)
             if step == 1:   # -lr * g / (|g| + eps): the quotient is decided by rounding where g is ~ eps

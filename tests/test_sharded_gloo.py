@@ -1,5 +1,5 @@
 """Clients sharded over two ranks (gloo, CPU): the orchestration in paper_2407_00952_b200.parallel
-(order of the calls, the two sums over ranks, the global loss normaliser, partial aggregation)
+(order of the calls, the two sums over ranks, the global loss normaliser, the aggregation in two halves around one sum)
 must reproduce the single-process round.  The engine on each rank is a stand-in with the same
 methods as the CUDA binding, backed by the CPU oracle, so this runs without a GPU."""
 import os
@@ -15,9 +15,10 @@ from oracle import splitlora_oracle as O
 from paper_2407_00952_b200 import parallel, synth
 
 
-def _workload():
+def _workload(n_clients=4):
+    counts = (300, 500, 200, 1000)[:n_clients]
     return synth.scaled(synth.WORKLOADS[1], n_layer=3, cut=1, d_model=32, n_head=2, d_ff=64, vocab=96, max_seq=16,
-                        seq=16, batch_per_client=2, n_clients=4, lora_r=2, lora_alpha=4.0, counts=(300, 500, 200, 1000),
+                        seq=16, batch_per_client=2, n_clients=n_clients, lora_r=2, lora_alpha=4.0, counts=counts,
                         agg_interval=1, lr=1e-2)
 
 
@@ -51,7 +52,7 @@ class OracleEngine:
         n_s = sum(server_adapters[k][n].size for k in self.skeys for n in ("A", "B"))
         n_c = sum(client_adapters[0][k][n].size for k in self.ckeys for n in ("A", "B"))
         self.sgrad = torch.zeros(n_s, dtype=torch.float64)
-        self.cparams = torch.zeros(len(client_adapters), n_c, dtype=torch.float64)
+        self.csum = torch.zeros(n_c, dtype=torch.float64)     # one client's worth, whatever the local client count
         self.loss_t = torch.zeros(1, dtype=torch.float64)
         self.norm, self.deferred = 0, False
 
@@ -74,7 +75,8 @@ class OracleEngine:
         assert self.deferred
 
     def adapter_buffer(self, side, kind):
-        return self.sgrad if side == parallel.SIDE_SERVER else self.cparams
+        assert side == parallel.SIDE_SERVER
+        return self.sgrad
 
     def server_update(self):
         grads, off, flat = {}, 0, self.sgrad.numpy()
@@ -94,27 +96,29 @@ class OracleEngine:
             O.apply_update(self.cfg, self.state.client_adapters[i], self.state.client_opt[i], g, self.cfg.lr_client,
                            self.state.client_steps)
 
-    def aggregate_partial(self, counts, total):
+    def aggregate_local_sum(self, counts, total):
         row = []
         for k in self.ckeys:
             for n in ("A", "B"):
                 acc = sum((counts[i] / total) * ca[k][n] for i, ca in enumerate(self.state.client_adapters))
                 row.append(acc.ravel())
-        self.cparams[:] = torch.from_numpy(np.concatenate(row))
+        self.csum[:] = torch.from_numpy(np.concatenate(row))
+        return self.csum
 
-    def adapters_changed(self, side):
-        for i, ca in enumerate(self.state.client_adapters):
-            off, flat = 0, self.cparams[i].numpy()
+    def aggregate_broadcast(self):
+        flat = self.csum.numpy()
+        for ca in self.state.client_adapters:
+            off = 0
             for k in self.ckeys:
                 for n in ("A", "B"):
                     ca[k][n] = flat[off:off + ca[k][n].size].reshape(ca[k][n].shape).copy()
                     off += ca[k][n].size
 
 
-def _worker(rank, world, port, out):
+def _worker(rank, world, port, out, n_clients):
     os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
     dist.init_process_group("gloo", rank=rank, world_size=world)
-    w = _workload()
+    w = _workload(n_clients)
     params, cads, sads, tokens, labels = _case(w)
     mine = parallel.shard_clients(w.n_clients, world, rank)
     counts = synth.make_counts(w)
@@ -148,22 +152,26 @@ def test_shard_clients_partition():
 
 
 @pytest.mark.timeout(300)
-def test_two_rank_round_equals_single_process():
+@pytest.mark.parametrize("n_clients", [4, 3])
+def test_two_rank_round_equals_single_process(n_clients):
+    """Four clients over two ranks, and three (rank 0 holds two clients, rank 1 one): the messages have the
+    same size on both ranks either way, because the aggregation exchanges one client's worth of sums."""
     world = 2
     ctx = mp.get_context("spawn")
     out = ctx.Manager().dict()
     port = _free_port()
-    procs = [ctx.Process(target=_worker, args=(r, world, port, out)) for r in range(world)]
+    procs = [ctx.Process(target=_worker, args=(r, world, port, out, n_clients)) for r in range(world)]
     for p in procs:
         p.start()
     for p in procs:
         p.join(240)
         assert p.exitcode == 0
-    # single-process reference: all four clients in one oracle state
-    w = _workload()
+    # single-process reference: all clients in one oracle state
+    w = _workload(n_clients)
     params, cads, sads, tokens, labels = _case(w)
     st = O.OracleState(client_adapters=cads, server_adapters=sads)
     ref_losses = [O.split_round(_cfg(w, w.n_clients), params, st, tokens, labels, synth.make_counts(w))[0] for _ in range(2)]
+    assert sorted(i for r in range(world) for i in out[r]["mine"]) == list(range(n_clients))
     for r in range(world):
         # round 1 agrees to rounding; round 2 sees client adapters that the single-process oracle
         # stored as fp32 after aggregation (6e-8 relative), hence the looser bounds below
@@ -179,4 +187,4 @@ def test_two_rank_round_equals_single_process():
                     assert np.allclose(out[r]["clients"][li][k][n], ad[n], rtol=1e-6, atol=1e-9)
     # every client on every rank holds the same aggregated adapters
     a0 = out[0]["clients"][0][(0, "q")]["A"]
-    assert np.array_equal(a0, out[1]["clients"][1][(0, "q")]["A"])
+    assert np.array_equal(a0, out[1]["clients"][-1][(0, "q")]["A"])

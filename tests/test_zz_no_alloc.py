@@ -58,6 +58,9 @@ def test_static_scratch_matches_caller_scratch_twice():
             assert err <= (TOL_BF16 if dtype == torch.bfloat16 else 1e-4), (nseq, T, j, err)
 
 
+    assert B.library_status() == 0
+
+
 def test_static_scratch_rejects_oversize():
     heads, d, T = 2, 128, 64
     nseq = B.STATIC_ATTENTION_ROWS // (T * heads) + 1
