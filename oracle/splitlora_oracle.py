@@ -657,6 +657,119 @@ def split_round(cfg: OracleConfig, params, state: OracleState, tokens, labels, c
     return loss, dict(S=S, dS=dS, server_grads=sgrads, client_grads=cgrads, aggregated=aggregated)
 
 
+# --------------------------------------------------------------------------
+# clients cut at different depths (Sec. V, heterogeneous configuration)
+# --------------------------------------------------------------------------
+# The paper names the joint choice of cut layers and ranks per client as a direction and gives no rule.
+# Reading taken here: client i runs blocks 1..c_i with its own adapters and hands off s_i at depth c_i;
+# the server holds adapters on blocks c_min+1..L (c_min = min_i c_i) and takes client i's activations in
+# at block c_i+1, so that at block l its batch is the concatenation of everything that has entered so
+# far; there is still ONE loss (the mean over all valid positions of all clients) and one server update
+# per round; dL/ds_i is handed back at depth c_i; Eq. 8-9 is applied per block to the clients that hold
+# that block, w_i = |D_i| / sum over those holders.  With all c_i equal this is Algorithm 1 unchanged.
+def client_fwd_cuts(cfg: OracleConfig, params, client_adapters: Sequence[dict], tokens, cuts):
+    """Step a1 with per-client depth: returns [s_i] (each [b, T, d], rounded once to bf16 in bf16 configs)
+    and the per-client caches."""
+    outs, caches = [], []
+    for i in range(tokens.shape[0]):
+        x = embed(cfg, params, tokens[i])
+        cl = []
+        for l in range(cuts[i]):
+            x, c = block_fwd(cfg, params, l, client_adapters[i], x)
+            cl.append(c)
+        outs.append(round_to_bf16(x) if cfg.bf16_handoff else x)
+        caches.append(cl)
+    return outs, caches
+
+
+def server_fwd_bwd_cuts(cfg: OracleConfig, params, server_adapters: dict, S_list, labels, cuts):
+    """Step a3 with per-client depth.  S_list[i] [b, T, d] enters at block cuts[i] (0-based index of the
+    first server block it passes); labels [K, b, T].  Returns loss, [dL/ds_i] and the server gradients for
+    blocks min(cuts)..L-1."""
+    K = len(S_list)
+    b, T, d = S_list[0].shape
+    order = []                        # clients in the order they entered; rows of x follow this order
+    x = np.zeros((0, T, d), dtype=F64)
+    caches, entered_at = {}, {}
+    for l in range(min(cuts), cfg.n_layer + 1):
+        new = [i for i in range(K) if cuts[i] == l]
+        if new:
+            x = np.concatenate([x] + [S_list[i] for i in new], axis=0)
+            order += new
+        entered_at[l] = list(new)
+        if l < cfg.n_layer:
+            x, caches[l] = block_fwd(cfg, params, l, server_adapters, x)
+    assert sorted(order) == list(range(K))
+    if cfg.arch == "llama":
+        xf, lnf = rmsnorm_fwd(x.reshape(-1, d), params["lnf.g"], cfg.norm_eps)
+    else:
+        xf, lnf = layernorm_fwd(x.reshape(-1, d), params["lnf.g"], params["lnf.b"], cfg.norm_eps)
+    head = params.get("head.w", params["wte"])
+    z = xf @ head.T
+    lab = np.concatenate([labels[i].reshape(-1) for i in order])
+    loss, dz = cross_entropy_fwd_bwd(z, lab)
+    dxf = dz @ head
+    dx = (rmsnorm_bwd(dxf, lnf) if cfg.arch == "llama" else layernorm_bwd(dxf, lnf)).reshape(-1, T, d)
+    grads, dS = {}, [None] * K
+    for l in range(cfg.n_layer, min(cuts) - 1, -1):
+        if l < cfg.n_layer:
+            dx, g = block_bwd(cfg, params, l, server_adapters, dx, caches[l])
+            grads.update(g)
+        n_new = len(entered_at[l])
+        if n_new:                     # the last n_new * b sequences entered here: their gradient goes back
+            keep = dx.shape[0] - n_new * b
+            for j, i in enumerate(entered_at[l]):
+                g_i = dx[keep + j * b: keep + (j + 1) * b]
+                dS[i] = round_to_bf16(g_i) if cfg.bf16_handoff else g_i
+            dx = dx[:keep]
+            order = order[:len(order) - n_new]
+    return loss, dS, grads
+
+
+def client_bwd_grads_cuts(cfg: OracleConfig, params, client_adapters: Sequence[dict], dS_list, caches, cuts):
+    """Step a5 with per-client depth."""
+    all_grads = []
+    for i, dx in enumerate(dS_list):
+        grads = {}
+        for l in range(cuts[i] - 1, -1, -1):
+            dx, g = block_bwd(cfg, params, l, client_adapters[i], dx, caches[i][l])
+            grads.update(g)
+        all_grads.append(grads)
+    return all_grads
+
+
+def aggregate_clients_cuts(state: OracleState, counts, cuts, store_fp32: bool = True):
+    """Stage b with per-client depth: Eq. 8-9 per block over the clients that hold the block."""
+    for l in range(max(cuts)):
+        holders = [i for i in range(len(cuts)) if cuts[i] > l]
+        for key in [k for k in state.client_adapters[holders[0]].keys() if k[0] == l]:
+            for name in ("A", "B"):
+                avg = aggregate([state.client_adapters[i][key][name] for i in holders], [counts[i] for i in holders])
+                if store_fp32:
+                    avg = avg.astype(np.float32).astype(F64)
+                for i in holders:
+                    state.client_adapters[i][key][name] = avg.copy()
+
+
+def split_round_cuts(cfg: OracleConfig, params, state: OracleState, tokens, labels, counts, cuts):
+    """One iteration t of Algorithm 1 with client i cut after block cuts[i] (see the reading above).
+    state.client_adapters[i] holds blocks 0..cuts[i]-1, state.server_adapters blocks min(cuts)..L-1."""
+    state.round_index += 1
+    S_list, caches = client_fwd_cuts(cfg, params, state.client_adapters, tokens, cuts)
+    loss, dS_list, sgrads = server_fwd_bwd_cuts(cfg, params, state.server_adapters, S_list, labels, cuts)
+    state.server_steps += 1
+    apply_update(cfg, state.server_adapters, state.server_opt, sgrads, cfg.lr_server, state.server_steps)
+    cgrads = client_bwd_grads_cuts(cfg, params, state.client_adapters, dS_list, caches, cuts)
+    state.client_steps += 1
+    for i, g in enumerate(cgrads):
+        apply_update(cfg, state.client_adapters[i], state.client_opt[i], g, cfg.lr_client, state.client_steps)
+    aggregated = False
+    if state.round_index % cfg.agg_interval == 0:
+        aggregate_clients_cuts(state, counts, cuts)
+        aggregated = True
+    return loss, dict(S=S_list, dS=dS_list, server_grads=sgrads, client_grads=cgrads, aggregated=aggregated)
+
+
 def trainable_parameter_count(cfg: OracleConfig, n_blocks: int) -> int:
     """Number of LoRA parameters on n_blocks blocks: per block and target r*d (A) + d*r (B)."""
     return n_blocks * len(cfg.targets) * 2 * cfg.lora_r * cfg.d_model
