@@ -95,6 +95,10 @@ typedef struct {
                                 0 = plain FMA kernels (a second opinion for debugging)      */
   int32_t arch;              /* SPLITLORA_ARCH_*                                            */
   float   rope_theta;        /* base of the rotary frequencies (ARCH_LLAMA only), e.g. 1e4  */
+  int32_t cut_min;           /* 0: every client is cut at `cut`.  Else 1 <= cut_min <= cut: clients
+                                may be cut at different depths in [cut_min, cut] (see
+                                splitlora_set_client_cuts); client adapters are stored for blocks
+                                0..cut-1 and the server has adapters on blocks cut_min..n_layer-1 */
 } splitlora_config;
 
 /* ---- context ------------------------------------------------------------------------------ */
@@ -126,7 +130,8 @@ int splitlora_bind_workspace(splitlora_ctx* ctx, void* dev, size_t bytes);
 int splitlora_bind_frozen(splitlora_ctx* ctx, const char* name, const void* dev, size_t bytes);
 
 /* Adapter access (fp32).  side: SPLITLORA_SIDE_*; client: 0..K-1 (ignored for the server);
- * layer: block index (0..cut-1 for clients, cut..n_layer-1 for the server); target: one
+ * layer: block index (0..cut-1 for clients, cut..n_layer-1 for the server; with cut_min > 0 the
+ * server's blocks start at cut_min); target: one
  * SPLITLORA_TARGET_* bit.  A [r, d], B [d, r] device buffers; copied in / out on the stream.
  * Either pointer may be NULL to skip that matrix. */
 int splitlora_set_adapter(splitlora_ctx* ctx, int side, int client, int layer, uint32_t target,
@@ -179,6 +184,20 @@ int splitlora_aggregate(splitlora_ctx* ctx, const int64_t* sample_counts);
  * its own leading ranks[i] components of the average.  Call after the adapters have been set.
  * Errors: SPLITLORA_ERR_ARG (rank out of range), SPLITLORA_ERR_WORKSPACE. */
 int splitlora_set_client_ranks(splitlora_ctx* ctx, const int32_t* ranks);
+
+/* Clients cut at different depths (Sec. V, heterogeneous configuration: the joint choice of cut layers
+ * and ranks per client is named as a direction, no rule is given).  cuts: HOST int32[K] with
+ * cut_min <= cuts[i] <= cut, non-decreasing in i (order the clients by depth), or NULL to return to one
+ * cut for all.  Client i then runs blocks 0..cuts[i]-1 with its own adapters and hands off at that
+ * depth (row block i of the hand-off buffers is s_i, resp. dL/ds_i, at depth cuts[i]); the server
+ * takes client i's rows in at block cuts[i], so the batch of a server block is the clients that have
+ * handed off by then, with the server adapters of blocks cut_min..n_layer-1; there is still one loss
+ * (mean over all valid positions of all clients) and one server update per round.  Aggregation
+ * applies Eq. 8-9 per block to the clients that hold the block, w_i = |D_i| / sum over those holders;
+ * a block held by one client is left as it is.  Adapter access for a client is limited to its own
+ * blocks.  Needs a configuration with cut_min > 0.  Not available together with clients spread over
+ * devices.  Errors: SPLITLORA_ERR_ARG (range, order), SPLITLORA_ERR_WORKSPACE. */
+int splitlora_set_client_cuts(splitlora_ctx* ctx, const int32_t* cuts);
 
 /* One iteration t of Algorithm 1: client_fwd, server_step, client_bwd (through internal hand-off
  * buffers) and, when t % agg_interval == 0, aggregate.  tokens, labels DEVICE [K, b, T] int32;

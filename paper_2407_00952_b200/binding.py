@@ -34,7 +34,7 @@ EXPORTS = [
     "splitlora_adapters_changed", "splitlora_aggregate_local_sum", "splitlora_aggregate_broadcast",
     "splitlora_handoff_quantize",
     "splitlora_handoff_dequantize", "splitlora_round_compressed", "splitlora_set_client_ranks",
-    "splitlora_library_status",
+    "splitlora_library_status", "splitlora_set_client_cuts",
 ]
 
 
@@ -53,7 +53,7 @@ class Config(C.Structure):
         ("lr_client", C.c_float), ("lr_server", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
         ("adam_eps", C.c_float), ("weight_decay", C.c_float), ("agg_interval", C.c_int32),
         ("norm_eps", C.c_float), ("gelu_tanh", C.c_int32), ("use_tensor_cores", C.c_int32),
-        ("arch", C.c_int32), ("rope_theta", C.c_float),
+        ("arch", C.c_int32), ("rope_theta", C.c_float), ("cut_min", C.c_int32),
     ]
 
 
@@ -83,7 +83,7 @@ def config_from_workload(w, optimizer: str = "adamw", use_tensor_cores: bool = T
         beta2=0.999, adam_eps=1e-8, weight_decay=0.01, agg_interval=w.agg_interval, norm_eps=1e-5, gelu_tanh=1,
         use_tensor_cores=1 if use_tensor_cores else 0,
         arch=ARCH_LLAMA if getattr(w, "arch", "gpt") == "llama" else ARCH_GPT,
-        rope_theta=float(getattr(w, "rope_theta", 10000.0)))
+        rope_theta=float(getattr(w, "rope_theta", 10000.0)), cut_min=0)
     for k, v in over.items():
         setattr(cfg, k, v)
     return cfg
@@ -214,6 +214,14 @@ class SplitLoRA:
             return
         arr = (C.c_int32 * len(ranks))(*[int(x) for x in ranks])
         self._check(self.lib.splitlora_set_client_ranks(self.ctx, arr))
+
+    def set_client_cuts(self, cuts):
+        """Per-client cut depths, non-decreasing (None: one cut for all); see splitlora_set_client_cuts."""
+        if cuts is None:
+            self._check(self.lib.splitlora_set_client_cuts(self.ctx, None))
+            return
+        arr = (C.c_int32 * len(cuts))(*[int(x) for x in cuts])
+        self._check(self.lib.splitlora_set_client_cuts(self.ctx, arr))
 
     def round_compressed(self, tokens, labels, counts, codes, scales, want_loss: bool = True):
         """codes uint8 [2, M, d], scales fp32 [2, M]: what crosses the cut (S, then dL/dS)."""

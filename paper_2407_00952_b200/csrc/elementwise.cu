@@ -516,19 +516,20 @@ cudaError_t optimizer_step(float* p, const float* g, float* m, float* v, int64_t
 // ------------------------------------------------------------------------------------------
 struct AggWeights { float w[AGG_MAX_CLIENTS]; };
 
-__global__ void __launch_bounds__(256) aggregate_kernel(float* __restrict__ params, int K, int64_t P4,
+__global__ void __launch_bounds__(256) aggregate_kernel(float* __restrict__ params, int K, int64_t P4, int64_t S4,
                                                         AggWeights w) {
+  // P4: float4s averaged per client, S4: float4s between two clients' rows (S4 >= P4)
   int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < P4; i += stride) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int k = 0; k < K; ++k) {
-      float4 v = __ldcs(reinterpret_cast<const float4*>(params) + (size_t)k * P4 + i);
+      float4 v = __ldcs(reinterpret_cast<const float4*>(params) + (size_t)k * S4 + i);
       acc.x = fmaf(w.w[k], v.x, acc.x);
       acc.y = fmaf(w.w[k], v.y, acc.y);
       acc.z = fmaf(w.w[k], v.z, acc.z);
       acc.w = fmaf(w.w[k], v.w, acc.w);
     }
-    for (int k = 0; k < K; ++k) __stcs(reinterpret_cast<float4*>(params) + (size_t)k * P4 + i, acc);
+    for (int k = 0; k < K; ++k) __stcs(reinterpret_cast<float4*>(params) + (size_t)k * S4 + i, acc);
   }
 }
 
@@ -582,8 +583,9 @@ cudaError_t rank_mask(float* params, int K, int64_t P, int r, int d, const int* 
   return cudaGetLastError();
 }
 
-cudaError_t aggregate(float* params, int K, int64_t P, const float* w_host, cudaStream_t st) {
-  if (K < 1 || K > AGG_MAX_CLIENTS || P % 4 != 0) return cudaErrorInvalidValue;
+cudaError_t aggregate(float* params, int K, int64_t P, const float* w_host, cudaStream_t st, int64_t row_stride) {
+  if (row_stride == 0) row_stride = P;
+  if (K < 1 || K > AGG_MAX_CLIENTS || P % 4 != 0 || row_stride % 4 != 0 || row_stride < P) return cudaErrorInvalidValue;
   AggWeights w;
   for (int k = 0; k < AGG_MAX_CLIENTS; ++k) w.w[k] = k < K ? w_host[k] : 0.f;
   int64_t P4 = P / 4;
@@ -591,7 +593,7 @@ cudaError_t aggregate(float* params, int K, int64_t P, const float* w_host, cuda
   const int64_t cap = 148 * 8;      // a few resident blocks per SM, grid-stride beyond that
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  aggregate_kernel<<<(unsigned)blocks, 256, 0, st>>>(params, K, P4, w);
+  aggregate_kernel<<<(unsigned)blocks, 256, 0, st>>>(params, K, P4, row_stride / 4, w);
   return cudaGetLastError();
 }
 

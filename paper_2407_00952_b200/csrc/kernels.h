@@ -136,7 +136,8 @@ cudaError_t optimizer_step(float* p, const float* g, float* m, float* v, int64_t
 static const int AGG_MAX_CLIENTS = 64;
 // zero rank components >= ranks_host[i] in client i's arena of (A [r, d], B [d, r]) pairs (P floats per client)
 cudaError_t rank_mask(float* params, int K, int64_t P, int r, int d, const int* ranks_host, cudaStream_t st);
-cudaError_t aggregate(float* params, int K, int64_t P, const float* w_host, cudaStream_t st);
+// row_stride: floats between two clients' rows (0: P), so that a column range of a wider arena can be averaged
+cudaError_t aggregate(float* params, int K, int64_t P, const float* w_host, cudaStream_t st, int64_t row_stride = 0);
 // The same step in two halves, for clients spread over devices: sum [P] = sum_i w[i] params[i, :], and
 // (after the caller has added the sums of all devices) every row of params [K, P] = sum.
 cudaError_t aggregate_local_sum(const float* params, int K, int64_t P, const float* w_host, float* sum, cudaStream_t st);

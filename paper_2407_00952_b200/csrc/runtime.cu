@@ -31,11 +31,22 @@ struct LayerBuf {
   void *u = nullptr, *hcat = nullptr, *qkv = nullptr, *o = nullptr, *x_mid = nullptr, *z = nullptr,
        *x_out = nullptr;
   float *mean1 = nullptr, *rstd1 = nullptr, *mean2 = nullptr, *rstd2 = nullptr, *lse = nullptr;
-  const void* x_in = nullptr;
-  // adapter compute copies of this layer (all groups stacked)
-  void *Acat = nullptr, *AcatT = nullptr, *Bext = nullptr, *BextT = nullptr;
-  // the same for an adapter on the attention output projection, and its down-projected input
-  void *AcatO = nullptr, *AcatOT = nullptr, *BextO = nullptr, *BextOT = nullptr, *hcat_o = nullptr;
+  const void* x_in = nullptr;     // base (row 0) of the buffer the block read its input from
+  void* hcat_o = nullptr;         // down-projected input of an adapter on the attention output projection
+  // Adapter compute copies of this layer: `cl` holds one set per client, stacked (blocks the clients
+  // run), `sv` the server's single set (blocks the server runs).  A block between the shallowest and the
+  // deepest client cut is run by both sides and has both.
+  struct Copies {
+    void *Acat = nullptr, *AcatT = nullptr, *Bext = nullptr, *BextT = nullptr;
+    void *AcatO = nullptr, *AcatOT = nullptr, *BextO = nullptr, *BextOT = nullptr;   // output projection
+  } cl, sv;
+};
+
+// The rows one call of a block works on: `rows` consecutive token rows from row0, which belong to the
+// clients client0, client0 + 1, ... (client side: each with its own adapters) or to the server's batch.
+struct Span {
+  int row0 = 0, rows = 0, client0 = 0, n_clients = 0;
+  bool client = false;
 };
 
 struct ProfRec { int cls; cudaEvent_t a, b; };
@@ -60,6 +71,8 @@ struct splitlora_ctx {
   std::string err;
   int dt = 0; size_t es = 4;
   int M = 0, nseq = 0, d = 0, F = 0, V = 0, Vpad = 0, L = 0, cut = 0, K = 0, rows_per_client = 0;
+  int cmin = 0;               // first block with server adapters (= cut unless clients are cut at different depths)
+  std::vector<int> client_cut;   // per-client cut, non-decreasing (empty: every client is cut at `cut`)
   int r = 0, rp = 0, ext = 0, ke = 0, n_targets = 0;
   int nq = 0;                 // adapted slices of the fused qkv projection (targets 0..nq-1)
   bool has_o = false;         // adapter on the attention output projection (target index nq)
@@ -131,6 +144,7 @@ int validate(const splitlora_config* c, std::string* why) {
   // cut == n_layer puts every block on the clients (the server keeps the final norm and the head):
   // the federated-LoRA baseline of Sec. IV as a degenerate case of the same round
   if (c->n_layer < 1 || c->cut < 1 || c->cut > c->n_layer) return bad("need 1 <= cut <= n_layer");
+  if (c->cut_min < 0 || c->cut_min > c->cut) return bad("need 0 <= cut_min <= cut");
   if (c->d_model < 8 || c->n_head < 1 || c->d_model % c->n_head != 0) return bad("d_model must be a multiple of n_head");
   if (c->d_model % 8 != 0 || c->d_ff % 8 != 0) return bad("d_model and d_ff must be multiples of 8");
   if (c->d_model / c->n_head > 128) return bad("head width above 128");
@@ -178,8 +192,9 @@ void derive(splitlora_ctx* c) {
   c->Fz = c->llama ? 2 * g.d_ff : g.d_ff;
   c->scale = g.lora_alpha / (float)g.lora_r;
   c->per_layer = (int64_t)c->n_targets * 2 * c->r * c->d;
+  c->cmin = g.cut_min > 0 ? g.cut_min : g.cut;
   c->Pc = c->per_layer * c->cut;
-  c->Ps = c->per_layer * (c->L - c->cut);
+  c->Ps = c->per_layer * (c->L - c->cmin);
   c->tc = (g.dtype == SPLITLORA_DTYPE_BF16) && g.use_tensor_cores != 0;
 }
 
@@ -205,14 +220,18 @@ size_t plan(splitlora_ctx* c, char* ws) {
     f.qkvwT = a.take(3 * d * d * es); f.projwT = a.take(d * d * es);
     f.fc1wT = a.take(Fz * d * es); f.fc2wT = a.take(d * F * es);
     LayerBuf& b = c->lb[l];
-    const size_t G = l < c->cut ? c->K : 1;
-    b.Acat = a.take(G * ext * d * es); b.AcatT = a.take(G * d * ext * es);
-    b.Bext = a.take(G * 3 * d * ext * es); b.BextT = a.take(G * ext * 3 * d * es);
-    if (c->has_o) {
-      b.AcatO = a.take(G * ext_o * d * es); b.AcatOT = a.take(G * d * ext_o * es);
-      b.BextO = a.take(G * d * ext_o * es); b.BextOT = a.take(G * ext_o * d * es);
-      b.hcat_o = a.take(M * ext_o * es);
+    for (int side = 0; side < 2; ++side) {
+      if (side == 0 ? l >= c->cut : l < c->cmin) continue;
+      const size_t G = side == 0 ? c->K : 1;
+      LayerBuf::Copies& k = side == 0 ? b.cl : b.sv;
+      k.Acat = a.take(G * ext * d * es); k.AcatT = a.take(G * d * ext * es);
+      k.Bext = a.take(G * 3 * d * ext * es); k.BextT = a.take(G * ext * 3 * d * es);
+      if (c->has_o) {
+        k.AcatO = a.take(G * ext_o * d * es); k.AcatOT = a.take(G * d * ext_o * es);
+        k.BextO = a.take(G * d * ext_o * es); k.BextOT = a.take(G * ext_o * d * es);
+      }
     }
+    if (c->has_o) b.hcat_o = a.take(M * ext_o * es);
     b.u = a.take(M * d * es); b.hcat = a.take(M * ext * es); b.qkv = a.take(M * 3 * d * es);
     b.o = a.take(M * d * es); b.x_mid = a.take(M * d * es); b.z = a.take(M * Fz * es);
     b.x_out = a.take(M * d * es);
@@ -287,14 +306,15 @@ cudaError_t refresh_side(splitlora_ctx* c, bool client) {
   a.r = c->r; a.rp = c->rp; a.d_in = c->d; a.d_out = c->d;
   a.scale = c->scale;
   a.G = client ? c->K : 1;
-  const int l0 = client ? 0 : c->cut, l1 = client ? c->cut : c->L;
+  const int l0 = client ? 0 : c->cmin, l1 = client ? c->cut : c->L;
   for (int l = l0; l < l1; ++l) {
     const float* base = (client ? c->cp : c->sp) + (size_t)(l - l0) * c->per_layer;
+    const LayerBuf::Copies& k = client ? c->lb[l].cl : c->lb[l].sv;
     {  // the adapted slices of the fused qkv projection
       a.A = base; a.B = a.A + (size_t)c->r * c->d;
       a.n_targets = c->nq; a.n_out = 3 * c->d; a.ext = c->ext;
       for (int t = 0; t < 4; ++t) a.slice_off[t] = c->slice_idx[t] * c->d;
-      a.Acat = c->lb[l].Acat; a.AcatT = c->lb[l].AcatT; a.Bext = c->lb[l].Bext; a.BextT = c->lb[l].BextT;
+      a.Acat = k.Acat; a.AcatT = k.AcatT; a.Bext = k.Bext; a.BextT = k.BextT;
       Scope s(c, "adapter_copies", 1);
       cudaError_t e = refresh_adapter_copies(a, c->st);
       if (e != cudaSuccess) return e;
@@ -303,7 +323,7 @@ cudaError_t refresh_side(splitlora_ctx* c, bool client) {
       a.A = base + (size_t)c->nq * 2 * c->r * c->d; a.B = a.A + (size_t)c->r * c->d;
       a.n_targets = 1; a.n_out = c->d; a.ext = c->ext_o;
       for (int t = 0; t < 4; ++t) a.slice_off[t] = 0;
-      a.Acat = c->lb[l].AcatO; a.AcatT = c->lb[l].AcatOT; a.Bext = c->lb[l].BextO; a.BextT = c->lb[l].BextOT;
+      a.Acat = k.AcatO; a.AcatT = k.AcatOT; a.Bext = k.BextO; a.BextT = k.BextOT;
       Scope s(c, "adapter_copies", 1);
       cudaError_t e = refresh_adapter_copies(a, c->st);
       if (e != cudaSuccess) return e;
@@ -312,138 +332,195 @@ cudaError_t refresh_side(splitlora_ctx* c, bool client) {
   return cudaSuccess;
 }
 
-// LayerNorm or RMSNorm, by architecture (mean is unused by RMSNorm)
-cudaError_t norm_forward(splitlora_ctx* c, const void* x, const void* g, const void* b, void* y, float* mean, float* rstd) {
+// LayerNorm or RMSNorm over M rows, by architecture (mean is unused by RMSNorm)
+cudaError_t norm_forward(splitlora_ctx* c, int M, const void* x, const void* g, const void* b, void* y, float* mean,
+                         float* rstd) {
   Scope s(c, "layernorm_fwd", 1);
-  if (c->llama) return rmsnorm_fwd(c->dt, x, g, y, rstd, c->M, c->d, c->cfg.norm_eps, c->st);
-  return layernorm_fwd(c->dt, x, g, b, y, mean, rstd, c->M, c->d, c->cfg.norm_eps, c->st);
+  if (c->llama) return rmsnorm_fwd(c->dt, x, g, y, rstd, M, c->d, c->cfg.norm_eps, c->st);
+  return layernorm_fwd(c->dt, x, g, b, y, mean, rstd, M, c->d, c->cfg.norm_eps, c->st);
 }
-cudaError_t norm_backward(splitlora_ctx* c, const void* dy, const void* x, const void* g, const float* mean,
+cudaError_t norm_backward(splitlora_ctx* c, int M, const void* dy, const void* x, const void* g, const float* mean,
                           const float* rstd, const void* resid, void* dx) {
   Scope s(c, "layernorm_bwd", 1);
-  if (c->llama) return rmsnorm_bwd(c->dt, dy, x, g, rstd, resid, dx, c->M, c->d, c->st);
-  return layernorm_bwd(c->dt, dy, x, g, mean, rstd, resid, dx, c->M, c->d, c->st);
+  if (c->llama) return rmsnorm_bwd(c->dt, dy, x, g, rstd, resid, dx, M, c->d, c->st);
+  return layernorm_bwd(c->dt, dy, x, g, mean, rstd, resid, dx, M, c->d, c->st);
+}
+
+// Spans of a block.  Clients are ordered by non-decreasing cut, so the clients that run block l
+// themselves are a suffix {i : cut_i > l} and the server's batch at block l is the prefix {i : cut_i <= l}.
+int cut_of(const splitlora_ctx* c, int i) { return c->client_cut.empty() ? c->cut : c->client_cut[i]; }
+bool uniform_cut(const splitlora_ctx* c) { return c->client_cut.empty(); }
+int first_client_above(const splitlora_ctx* c, int l) {       // first client with cut > l (K if none)
+  int i = 0;
+  while (i < c->K && cut_of(c, i) <= l) ++i;
+  return i;
+}
+Span client_span(const splitlora_ctx* c, int l) {
+  Span sp;
+  sp.client = true; sp.client0 = first_client_above(c, l); sp.n_clients = c->K - sp.client0;
+  sp.row0 = sp.client0 * c->rows_per_client; sp.rows = sp.n_clients * c->rows_per_client;
+  return sp;
+}
+Span server_span(const splitlora_ctx* c, int l) {
+  Span sp;
+  sp.client = false; sp.client0 = 0; sp.n_clients = first_client_above(c, l);
+  sp.row0 = 0; sp.rows = sp.n_clients * c->rows_per_client;
+  return sp;
+}
+// rows [client_a, client_b) of src -> the same rows of dst ([M, d] buffers): a hand-off of those clients
+cudaError_t copy_client_rows(splitlora_ctx* c, const void* src, void* dst, int client_a, int client_b) {
+  if (client_b <= client_a) return cudaSuccess;
+  const size_t off = (size_t)client_a * c->rows_per_client * c->d * c->es;
+  const size_t n = (size_t)(client_b - client_a) * c->rows_per_client * c->d * c->es;
+  return cudaMemcpyAsync((char*)dst + off, (const char*)src + off, n, cudaMemcpyDeviceToDevice, c->st);
 }
 
 // ---- one block -----------------------------------------------------------------------------
-cudaError_t block_forward(splitlora_ctx* c, int l, const void* x_in, void* x_out) {
-  const bool client = l < c->cut;
-  const int M = c->M, d = c->d, F = c->F, ext = c->ext;
+// x_in, x_out: bases (row 0) of [M, d] buffers; the block reads and writes the rows of `sp`.
+cudaError_t block_forward(splitlora_ctx* c, int l, const Span& sp, const void* x_in, void* x_out) {
+  const bool client = sp.client;
+  const int M = sp.rows, d = c->d, F = c->F, ext = c->ext, T = c->cfg.seq, H = c->cfg.n_head;
+  if (M == 0) return cudaSuccess;
   const int rpg = client ? c->rows_per_client : 0;
-  const bool grouped = client && c->K > 1;
+  const bool grouped = client && sp.n_clients > 1;
+  const size_t es = c->es;
   const FrozenLayer& f = c->fl[l];
   LayerBuf& b = c->lb[l];
+  const LayerBuf::Copies& k = client ? b.cl : b.sv;
+  auto at = [&](const void* p, size_t ld) { return (void*)((char*)p + (size_t)sp.row0 * ld * es); };        // activations
+  auto atf = [&](float* p) { return p + sp.row0; };                                                           // per-row fp32
+  auto grp = [&](const void* p, size_t elems) { return (const void*)((const char*)p + (size_t)(client ? sp.client0 : 0) * elems * es); };
+  float* lse = b.lse + (size_t)(sp.row0 / T) * H * T;
   b.x_in = x_in;
+  const void* xin = at(x_in, d);
+  void* u = at(b.u, d); void* hcat = at(b.hcat, ext); void* qkv = at(b.qkv, 3 * d); void* o = at(b.o, d);
+  void* x_mid = at(b.x_mid, d); void* z = at(b.z, c->Fz); void* xout = at(x_out, d);
   cudaError_t e;
-  if ((e = norm_forward(c, x_in, f.ln1g, f.ln1b, b.u, b.mean1, b.rstd1))) return e;
+  if ((e = norm_forward(c, M, xin, f.ln1g, f.ln1b, u, atf(b.mean1), atf(b.rstd1)))) return e;
   {  // h = u A_g^T for every target of the layer, one padded block of `ext` columns
-    GemmArgs a = base_args(c, b.u, d, b.Acat, d, b.hcat, ext, M, ext, d);
+    GemmArgs a = base_args(c, u, d, grp(k.Acat, (size_t)ext * d), d, hcat, ext, M, ext, d);
     a.rows_per_group = rpg; a.w_grouped = grouped;
     if ((e = linear(c, "lora_down_fwd", a))) return e;
   }
   {  // qkv = u Wqkv^T + b + hcat Bext_g^T   (the LoRA linear of Sec. II-C, grouped by client)
-    GemmArgs a = base_args(c, b.u, d, f.qkvw, d, b.qkv, 3 * d, M, 3 * d, d);
+    GemmArgs a = base_args(c, u, d, f.qkvw, d, qkv, 3 * d, M, 3 * d, d);
     a.bias = f.qkvb; a.rows_per_group = rpg;
-    a.Xe = b.hcat; a.ldxe = ext; a.We = b.Bext; a.ldwe = ext; a.Ke = c->ke; a.we_grouped = grouped;
+    a.Xe = hcat; a.ldxe = ext; a.We = grp(k.Bext, (size_t)3 * d * ext); a.ldwe = ext; a.Ke = c->ke; a.we_grouped = grouped;
     if ((e = linear(c, "lora_linear_fwd", a))) return e;
   }
   if (c->llama) {
     Scope s(c, "rope", 1);
-    if ((e = rope_inplace(c->dt, b.qkv, c->rope_table, M, c->cfg.seq, c->cfg.n_head, d, 1.0f, c->st))) return e;
+    if ((e = rope_inplace(c->dt, qkv, c->rope_table, M, T, H, d, 1.0f, c->st))) return e;
   }
   { Scope s(c, "attention_fwd", 1);
-    if (c->tc && attention_tc_supported(c->dt, c->cfg.seq, c->cfg.n_head, d))
-      e = attention_fwd_tc(b.qkv, c->nseq, c->cfg.seq, c->cfg.n_head, d, b.o, b.lse, c->status, c->st);
+    if (c->tc && attention_tc_supported(c->dt, T, H, d))
+      e = attention_fwd_tc(qkv, M / T, T, H, d, o, lse, c->status, c->st);
     else
-      e = attention_fwd_simt(c->dt, b.qkv, c->nseq, c->cfg.seq, c->cfg.n_head, d, b.o, b.lse, c->st);
+      e = attention_fwd_simt(c->dt, qkv, M / T, T, H, d, o, lse, c->st);
     if (e) return e; }
+  void* hcat_o = c->has_o ? at(b.hcat_o, c->ext_o) : nullptr;
   if (c->has_o) {  // h_o = o A_o,g^T
-    GemmArgs a = base_args(c, b.o, d, b.AcatO, d, b.hcat_o, c->ext_o, M, c->ext_o, d);
+    GemmArgs a = base_args(c, o, d, grp(k.AcatO, (size_t)c->ext_o * d), d, hcat_o, c->ext_o, M, c->ext_o, d);
     a.rows_per_group = rpg; a.w_grouped = grouped;
     if ((e = linear(c, "lora_down_fwd", a))) return e;
   }
-  { GemmArgs a = base_args(c, b.o, d, f.projw, d, b.x_mid, d, M, d, d);
-    a.bias = f.projb; a.epi = EPI_BIAS_RESID; a.R = x_in; a.ldr = d;
+  { GemmArgs a = base_args(c, o, d, f.projw, d, x_mid, d, M, d, d);
+    a.bias = f.projb; a.epi = EPI_BIAS_RESID; a.R = xin; a.ldr = d;
     if (c->has_o) {
       a.rows_per_group = rpg;
-      a.Xe = b.hcat_o; a.ldxe = c->ext_o; a.We = b.BextO; a.ldwe = c->ext_o; a.Ke = c->rp; a.we_grouped = grouped;
+      a.Xe = hcat_o; a.ldxe = c->ext_o; a.We = grp(k.BextO, (size_t)d * c->ext_o); a.ldwe = c->ext_o; a.Ke = c->rp;
+      a.we_grouped = grouped;
     }
     if ((e = linear(c, c->has_o ? "lora_linear_fwd" : "linear_fwd", a))) return e; }
-  if ((e = norm_forward(c, b.x_mid, f.ln2g, f.ln2b, c->u2, b.mean2, b.rstd2))) return e;
+  if ((e = norm_forward(c, M, x_mid, f.ln2g, f.ln2b, c->u2, atf(b.mean2), atf(b.rstd2)))) return e;
   if (c->llama) {
-    { GemmArgs a = base_args(c, c->u2, d, f.fc1w, d, b.z, 2 * F, M, 2 * F, d);     // (gate | up)
+    { GemmArgs a = base_args(c, c->u2, d, f.fc1w, d, z, 2 * F, M, 2 * F, d);     // (gate | up)
       if ((e = linear(c, "linear_fwd", a))) return e; }
     { Scope s(c, "swiglu_fwd", 1);
-      if ((e = swiglu_fwd(c->dt, b.z, c->act, M, F, c->st))) return e; }
+      if ((e = swiglu_fwd(c->dt, z, c->act, M, F, c->st))) return e; }
   } else {
     GemmArgs a = base_args(c, c->u2, d, f.fc1w, d, c->act, F, M, F, d);
-    a.bias = f.fc1b; a.epi = EPI_BIAS_GELU; a.Z = b.z; a.ldz = F;
+    a.bias = f.fc1b; a.epi = EPI_BIAS_GELU; a.Z = z; a.ldz = F;
     if ((e = linear(c, "linear_fwd", a))) return e;
   }
-  { GemmArgs a = base_args(c, c->act, F, f.fc2w, F, x_out, d, M, d, F);
-    a.bias = f.fc2b; a.epi = EPI_BIAS_RESID; a.R = b.x_mid; a.ldr = d;
+  { GemmArgs a = base_args(c, c->act, F, f.fc2w, F, xout, d, M, d, F);
+    a.bias = f.fc2b; a.epi = EPI_BIAS_RESID; a.R = x_mid; a.ldr = d;
     if ((e = linear(c, "linear_fwd", a))) return e; }
   return cudaSuccess;
 }
 
-// dy: gradient w.r.t. the block output.  dx: gradient w.r.t. the block input, or nullptr when it is
-// not needed (first client block: the embedding below it is frozen).
-cudaError_t block_backward(splitlora_ctx* c, int l, const void* dy, void* dx) {
-  const bool client = l < c->cut;
-  const int M = c->M, d = c->d, F = c->F, ext = c->ext;
+// dy: gradient w.r.t. the block output; dx: gradient w.r.t. the block input, or nullptr when it is not
+// needed (first client block: the embedding below it is frozen).  Both are bases of [M, d] buffers; the
+// rows of `sp` are read and written.
+cudaError_t block_backward(splitlora_ctx* c, int l, const Span& sp, const void* dy_base, void* dx_base) {
+  const bool client = sp.client;
+  const int M = sp.rows, d = c->d, F = c->F, ext = c->ext, T = c->cfg.seq, H = c->cfg.n_head;
+  if (M == 0) return cudaSuccess;
   const int rpg = client ? c->rows_per_client : 0;
-  const bool grouped = client && c->K > 1;
+  const bool grouped = client && sp.n_clients > 1;
+  const size_t es = c->es;
   const FrozenLayer& f = c->fl[l];
   LayerBuf& b = c->lb[l];
+  const LayerBuf::Copies& k = client ? b.cl : b.sv;
+  auto at = [&](const void* p, size_t ld) { return (void*)((char*)p + (size_t)sp.row0 * ld * es); };
+  auto atf = [&](float* p) { return p + sp.row0; };
+  auto grp = [&](const void* p, size_t elems) { return (const void*)((const char*)p + (size_t)(client ? sp.client0 : 0) * elems * es); };
+  const float* lse = b.lse + (size_t)(sp.row0 / T) * H * T;
+  const void* dy = at(dy_base, d);
+  void* dx = dx_base ? at(dx_base, d) : nullptr;
+  const void* u = at(b.u, d); const void* hcat = at(b.hcat, ext); const void* qkv = at(b.qkv, 3 * d);
+  const void* o = at(b.o, d); const void* x_mid = at(b.x_mid, d); const void* z = at(b.z, c->Fz);
   cudaError_t e;
   const int Fz = c->Fz;
-  float* gbase = client ? c->cg + (size_t)l * c->per_layer : c->sg + (size_t)(l - c->cut) * c->per_layer;
+  float* gbase = client ? c->cg + (size_t)sp.client0 * c->Pc + (size_t)l * c->per_layer
+                        : c->sg + (size_t)(l - c->cmin) * c->per_layer;
   const int64_t gstride = client ? c->Pc : 0;
   if (c->llama) {
     { GemmArgs a = base_args(c, dy, d, f.fc2wT, d, c->act, F, M, F, d);               // d act
       if ((e = linear(c, "linear_bwd", a))) return e; }
     { Scope s(c, "swiglu_bwd", 1);
-      if ((e = swiglu_bwd(c->dt, c->act, b.z, c->g_dz, M, F, c->st))) return e; }
+      if ((e = swiglu_bwd(c->dt, c->act, z, c->g_dz, M, F, c->st))) return e; }
   } else {
     GemmArgs a = base_args(c, dy, d, f.fc2wT, d, c->g_dz, F, M, F, d);
-    a.epi = EPI_MUL_GELUGRAD; a.R = b.z; a.ldr = F;
+    a.epi = EPI_MUL_GELUGRAD; a.R = z; a.ldr = F;
     if ((e = linear(c, "linear_bwd", a))) return e;
   }
   { GemmArgs a = base_args(c, c->g_dz, Fz, f.fc1wT, Fz, c->g_du2, d, M, d, Fz);
     if ((e = linear(c, "linear_bwd", a))) return e; }
-  if ((e = norm_backward(c, c->g_du2, b.x_mid, f.ln2g, b.mean2, b.rstd2, dy, c->g_dxmid))) return e;
+  if ((e = norm_backward(c, M, c->g_du2, x_mid, f.ln2g, atf(b.mean2), atf(b.rstd2), dy, c->g_dxmid))) return e;
   if (c->has_o) {
     // dh_o = (alpha/r) dx_mid B_o,g ;  G_A = dh_o^T o ;  G_B = (alpha/r) dx_mid^T h_o   (Eq. 4-7)
-    { GemmArgs a = base_args(c, c->g_dxmid, d, b.BextOT, d, c->g_dhcat_o, c->ext_o, M, c->ext_o, d);
+    const void* hcat_o = at(b.hcat_o, c->ext_o);
+    { GemmArgs a = base_args(c, c->g_dxmid, d, grp(k.BextOT, (size_t)c->ext_o * d), d, c->g_dhcat_o, c->ext_o, M, c->ext_o, d);
       a.rows_per_group = rpg; a.w_grouped = grouped;
       if ((e = linear(c, "lora_down_bwd", a))) return e; }
     float* gA = gbase + (size_t)c->nq * 2 * c->r * d;
     { Scope s(c, "lora_grad", 2);
-      if ((e = lora_grad(c->dt, b.o, d, 0, d, c->g_dhcat_o, c->ext_o, 0, c->r, c->rp, 1, M, rpg, 1.0f, gA, gstride, 0, d,
+      if ((e = lora_grad(c->dt, o, d, 0, d, c->g_dhcat_o, c->ext_o, 0, c->r, c->rp, 1, M, rpg, 1.0f, gA, gstride, 0, d,
                          1, c->grad_scratch, c->st, c->status, c->tc))) return e; }
     { Scope s(c, "lora_grad", 2);
-      if ((e = lora_grad(c->dt, c->g_dxmid, d, 0, d, b.hcat_o, c->ext_o, 0, c->r, c->rp, 1, M, rpg, c->scale,
+      if ((e = lora_grad(c->dt, c->g_dxmid, d, 0, d, hcat_o, c->ext_o, 0, c->r, c->rp, 1, M, rpg, c->scale,
                          gA + (size_t)c->r * d, gstride, 0, 1, c->r, c->grad_scratch, c->st, c->status, c->tc))) return e; }
   }
   { GemmArgs a = base_args(c, c->g_dxmid, d, f.projwT, d, c->g_do, d, M, d, d);
     if (c->has_o) {
       a.rows_per_group = rpg;
-      a.Xe = c->g_dhcat_o; a.ldxe = c->ext_o; a.We = b.AcatOT; a.ldwe = c->ext_o; a.Ke = c->rp; a.we_grouped = grouped;
+      a.Xe = c->g_dhcat_o; a.ldxe = c->ext_o; a.We = grp(k.AcatOT, (size_t)d * c->ext_o); a.ldwe = c->ext_o; a.Ke = c->rp;
+      a.we_grouped = grouped;
     }
     if ((e = linear(c, c->has_o ? "lora_linear_bwd" : "linear_bwd", a))) return e; }
-  { Scope s(c, "attention_bwd", c->tc && attention_t5_supported(c->dt, c->cfg.seq, c->cfg.n_head, d) ? 2 : 3);
-    if (c->tc && attention_tc_supported(c->dt, c->cfg.seq, c->cfg.n_head, d))
-      e = attention_bwd_tc(b.qkv, b.o, b.lse, c->g_do, c->nseq, c->cfg.seq, c->cfg.n_head, d, c->g_dqkv, c->rowdot, c->status,
-                           c->st);
+  { Scope s(c, "attention_bwd", c->tc && attention_t5_supported(c->dt, T, H, d) ? 2 : 3);
+    if (c->tc && attention_tc_supported(c->dt, T, H, d))
+      e = attention_bwd_tc(qkv, o, lse, c->g_do, M / T, T, H, d, c->g_dqkv, c->rowdot, c->status, c->st);
     else
-      e = attention_bwd_simt(c->dt, b.qkv, b.o, b.lse, c->g_do, c->nseq, c->cfg.seq, c->cfg.n_head, d, c->g_dqkv, c->rowdot, c->st);
+      e = attention_bwd_simt(c->dt, qkv, o, lse, c->g_do, M / T, T, H, d, c->g_dqkv, c->rowdot, c->st);
     if (e) return e; }
   if (c->llama) {  // the gradient of a rotation is the inverse rotation
     Scope s(c, "rope", 1);
-    if ((e = rope_inplace(c->dt, c->g_dqkv, c->rope_table, M, c->cfg.seq, c->cfg.n_head, d, -1.0f, c->st))) return e;
+    if ((e = rope_inplace(c->dt, c->g_dqkv, c->rope_table, M, T, H, d, -1.0f, c->st))) return e;
   }
   {  // dh = (alpha/r) dqkv B_g for every target (the scale lives in the compute copy)
-    GemmArgs a = base_args(c, c->g_dqkv, 3 * d, b.BextT, 3 * d, c->g_dhcat, ext, M, ext, 3 * d);
+    GemmArgs a = base_args(c, c->g_dqkv, 3 * d, grp(k.BextT, (size_t)ext * 3 * d), 3 * d, c->g_dhcat, ext, M, ext, 3 * d);
     a.rows_per_group = rpg; a.w_grouped = grouped;
     if (c->tc && c->nq < 3) {
       // only the adapted slices of dqkv contribute (the other rows of the compute copy are zero):
@@ -460,20 +537,20 @@ cudaError_t block_backward(splitlora_ctx* c, int l, const void* dy, void* dx) {
   }
   // G_A = dh^T u, G_B = (alpha/r) dy^T h, per group (Eq. 4-7)
   { Scope s(c, "lora_grad", 2);   // every qkv target's G_A in one pass over u
-    if ((e = lora_grad(c->dt, b.u, d, 0, d, c->g_dhcat, ext, 0, c->r, c->rp, c->nq, M, rpg, 1.0f, gbase,
+    if ((e = lora_grad(c->dt, u, d, 0, d, c->g_dhcat, ext, 0, c->r, c->rp, c->nq, M, rpg, 1.0f, gbase,
                        gstride, (int64_t)2 * c->r * d, d, 1, c->grad_scratch, c->st, c->status, c->tc))) return e; }
   for (int t = 0; t < c->nq; ++t) {
     float* gB = gbase + (size_t)t * 2 * c->r * d + (size_t)c->r * d;
     Scope s(c, "lora_grad", 2);
-    if ((e = lora_grad(c->dt, c->g_dqkv, 3 * d, c->slice_idx[t] * d, d, b.hcat, ext, t * c->rp, c->r, c->rp, 1, M,
+    if ((e = lora_grad(c->dt, c->g_dqkv, 3 * d, c->slice_idx[t] * d, d, hcat, ext, t * c->rp, c->r, c->rp, 1, M,
                        rpg, c->scale, gB, gstride, 0, 1, c->r, c->grad_scratch, c->st, c->status, c->tc))) return e;
   }
   if (dx) {
     GemmArgs a = base_args(c, c->g_dqkv, 3 * d, f.qkvwT, 3 * d, c->g_du, d, M, d, 3 * d);
     a.rows_per_group = rpg;
-    a.Xe = c->g_dhcat; a.ldxe = ext; a.We = b.AcatT; a.ldwe = ext; a.Ke = c->ke; a.we_grouped = grouped;
+    a.Xe = c->g_dhcat; a.ldxe = ext; a.We = grp(k.AcatT, (size_t)d * ext); a.ldwe = ext; a.Ke = c->ke; a.we_grouped = grouped;
     if ((e = linear(c, "lora_linear_bwd", a))) return e;
-    if ((e = norm_backward(c, c->g_du, b.x_in, f.ln1g, b.mean1, b.rstd1, c->g_dxmid, dx))) return e;
+    if ((e = norm_backward(c, M, c->g_du, at(b.x_in, d), f.ln1g, atf(b.mean1), atf(b.rstd1), c->g_dxmid, dx))) return e;
   }
   return cudaSuccess;
 }
@@ -504,12 +581,12 @@ float* adapter_ptr(splitlora_ctx* c, float* client_base, float* server_base, int
   for (int i = 0; i < c->n_targets; ++i) if (c->target_bit[i] == target) t = i;
   if (t < 0) { *rc = fail(c, SPLITLORA_ERR_ARG, "target is not an adapted slice"); return nullptr; }
   if (side == SPLITLORA_SIDE_CLIENT) {
-    if (client < 0 || client >= c->K || layer < 0 || layer >= c->cut) { *rc = fail(c, SPLITLORA_ERR_ARG, "client/layer out of range"); return nullptr; }
+    if (client < 0 || client >= c->K || layer < 0 || layer >= cut_of(c, client)) { *rc = fail(c, SPLITLORA_ERR_ARG, "client/layer out of range"); return nullptr; }
     return client_base + (size_t)client * c->Pc + (size_t)layer * c->per_layer + (size_t)t * 2 * c->r * c->d;
   }
   if (side == SPLITLORA_SIDE_SERVER) {
-    if (layer < c->cut || layer >= c->L) { *rc = fail(c, SPLITLORA_ERR_ARG, "layer out of range"); return nullptr; }
-    return server_base + (size_t)(layer - c->cut) * c->per_layer + (size_t)t * 2 * c->r * c->d;
+    if (layer < c->cmin || layer >= c->L) { *rc = fail(c, SPLITLORA_ERR_ARG, "layer out of range"); return nullptr; }
+    return server_base + (size_t)(layer - c->cmin) * c->per_layer + (size_t)t * 2 * c->r * c->d;
   }
   *rc = fail(c, SPLITLORA_ERR_ARG, "bad side");
   return nullptr;
@@ -574,15 +651,19 @@ int splitlora_bind_workspace(splitlora_ctx* c, void* dev, size_t bytes) {
   for (float* p : {c->cp, c->cg, c->cm, c->cv}) CK(c, cudaMemsetAsync(p, 0, (size_t)c->K * c->Pc * 4, c->st));
   for (float* p : {c->sp, c->sg, c->sm, c->sv}) CK(c, cudaMemsetAsync(p, 0, (size_t)c->Ps * 4, c->st));
   for (int l = 0; l < c->L; ++l) {
-    const size_t G = l < c->cut ? c->K : 1;
     const size_t es = c->es, d = c->d, ext = c->ext;
-    CK(c, cudaMemsetAsync(c->lb[l].Acat, 0, G * ext * d * es, c->st));
-    CK(c, cudaMemsetAsync(c->lb[l].AcatT, 0, G * ext * d * es, c->st));
-    CK(c, cudaMemsetAsync(c->lb[l].Bext, 0, G * 3 * d * ext * es, c->st));
-    CK(c, cudaMemsetAsync(c->lb[l].BextT, 0, G * 3 * d * ext * es, c->st));
-    if (c->has_o)
-      for (void* p : {c->lb[l].AcatO, c->lb[l].AcatOT, c->lb[l].BextO, c->lb[l].BextOT})
-        CK(c, cudaMemsetAsync(p, 0, G * (size_t)c->ext_o * d * es, c->st));
+    for (int side = 0; side < 2; ++side) {
+      if (side == 0 ? l >= c->cut : l < c->cmin) continue;
+      const size_t G = side == 0 ? c->K : 1;
+      const LayerBuf::Copies& k = side == 0 ? c->lb[l].cl : c->lb[l].sv;
+      CK(c, cudaMemsetAsync(k.Acat, 0, G * ext * d * es, c->st));
+      CK(c, cudaMemsetAsync(k.AcatT, 0, G * ext * d * es, c->st));
+      CK(c, cudaMemsetAsync(k.Bext, 0, G * 3 * d * ext * es, c->st));
+      CK(c, cudaMemsetAsync(k.BextT, 0, G * 3 * d * ext * es, c->st));
+      if (c->has_o)
+        for (void* p : {k.AcatO, k.AcatOT, k.BextO, k.BextOT})
+          CK(c, cudaMemsetAsync(p, 0, G * (size_t)c->ext_o * d * es, c->st));
+    }
   }
   if (c->llama) {  // (cos, sin) of t * theta^(-2j/dh), evaluated in double
     const int half = c->d / c->cfg.n_head / 2, T = c->cfg.seq;
@@ -599,6 +680,7 @@ int splitlora_bind_workspace(splitlora_ctx* c, void* dev, size_t bytes) {
   c->client_copies_dirty = c->server_copies_dirty = true;
   c->have_client_fwd = false;
   c->round_index = c->server_steps = c->client_steps = 0;
+  c->client_cut.clear();
   return SPLITLORA_OK;
 }
 
@@ -735,8 +817,13 @@ int splitlora_client_fwd(splitlora_ctx* c, const int32_t* tokens, void* act_out)
     CK(c, embed(c->dt, tokens, c->wte, c->wpe, c->emb, c->M, c->cfg.seq, c->d, c->V, c->st)); }
   const void* x = c->emb;
   for (int l = 0; l < c->cut; ++l) {
-    void* out = (l == c->cut - 1) ? act_out : c->lb[l].x_out;
-    CK(c, block_forward(c, l, x, out));
+    // clients whose last block this is hand their output off: written in place when that is everybody,
+    // else copied out of the block's output buffer (the others go on from there)
+    const Span sp = client_span(c, l);
+    const bool all_finish = first_client_above(c, l + 1) == c->K && sp.client0 == 0;
+    void* out = all_finish ? act_out : c->lb[l].x_out;
+    CK(c, block_forward(c, l, sp, x, out));
+    if (!all_finish) CK(c, copy_client_rows(c, out, act_out, sp.client0, first_client_above(c, l + 1)));
     x = out;
   }
   c->have_client_fwd = true;
@@ -751,30 +838,45 @@ int splitlora_server_step(splitlora_ctx* c, const void* act_in, const int32_t* l
   if (!aligned16(act_in) || !aligned16(labels) || !aligned16(act_grad_out)) return fail(c, SPLITLORA_ERR_ALIGN, "buffer not 16-byte aligned");
   if (c->server_copies_dirty) { CK(c, refresh_side(c, false)); c->server_copies_dirty = false; }
   const int M = c->M, d = c->d;
-  // forward over the concatenated batch S^t (Eq. 3)
+  // forward over the concatenated batch S^t (Eq. 3).  With clients cut at different depths the batch of
+  // block l is the prefix of clients that have handed off by then; a client's rows join the stream of the
+  // block below its entry point (a copy of its hand-off), so every block reads one contiguous buffer.
+  const bool uni = uniform_cut(c);
+  const int first = uni ? c->cut : c->cmin;        // first block the server runs
   const void* x = act_in;
-  for (int l = c->cut; l < c->L; ++l) {
-    CK(c, block_forward(c, l, x, c->lb[l].x_out));
+  for (int l = first; l < c->L; ++l) {
+    if (!uni) {
+      CK(c, copy_client_rows(c, act_in, c->lb[l - 1].x_out, first_client_above(c, l - 1), first_client_above(c, l)));
+      x = c->lb[l - 1].x_out;
+    }
+    CK(c, block_forward(c, l, server_span(c, l), x, c->lb[l].x_out));
     x = c->lb[l].x_out;
   }
-  CK(c, norm_forward(c, x, c->lnfg, c->lnfb, c->xf, c->meanf, c->rstdf));
+  if (!uni) {   // clients that hand off above the last block enter at the final norm
+    CK(c, copy_client_rows(c, act_in, c->lb[c->L - 1].x_out, first_client_above(c, c->L - 1), c->K));
+    x = c->lb[c->L - 1].x_out;
+  }
+  CK(c, norm_forward(c, M, x, c->lnfg, c->lnfb, c->xf, c->meanf, c->rstdf));
   { GemmArgs a = base_args(c, c->xf, d, c->headw, d, c->logits, c->Vpad, M, c->Vpad, d);
     a.w_rows = c->V;
     CK(c, linear(c, "head_fwd", a)); }
   { Scope s(c, "cross_entropy", 3);
     CK(c, cross_entropy(c->dt, c->logits, c->Vpad, labels, M, c->V, c->row_loss, c->n_valid, c->loss_dev,
                         (int)c->loss_normalizer, c->st)); }
-  // backward: head, final norm, blocks L-1 .. cut
+  // backward: head, final norm, blocks L-1 .. first
   { GemmArgs a = base_args(c, c->logits, c->Vpad, c->wteT, c->Vpad, c->g_a, d, M, d, c->Vpad);
     CK(c, linear(c, "head_bwd", a)); }
-  void* cur = (c->cut == c->L) ? act_grad_out : c->g_b;     // no server block: this is dL/dS already
-  CK(c, norm_backward(c, c->g_a, x, c->lnfg, c->meanf, c->rstdf, nullptr, cur));
+  void* cur = (uni && c->cut == c->L) ? act_grad_out : c->g_b;     // no server block: this is dL/dS already
+  CK(c, norm_backward(c, M, c->g_a, x, c->lnfg, c->meanf, c->rstdf, nullptr, cur));
   void* other = c->g_a;
-  for (int l = c->L - 1; l >= c->cut; --l) {
-    void* dst = (l == c->cut) ? act_grad_out : other;
-    CK(c, block_backward(c, l, cur, dst));
+  for (int l = c->L - 1; l >= first; --l) {
+    // rows of the clients that entered above block l hold their dL/ds_i now: hand them back
+    if (!uni) CK(c, copy_client_rows(c, cur, act_grad_out, first_client_above(c, l), first_client_above(c, l + 1)));
+    void* dst = (uni && l == first) ? act_grad_out : other;
+    CK(c, block_backward(c, l, server_span(c, l), cur, dst));
     other = cur; cur = dst;
   }
+  if (!uni) CK(c, copy_client_rows(c, cur, act_grad_out, 0, first_client_above(c, c->cmin)));
   // Eq. 4-5: server update
   if (!c->defer_server_update) {
     CK(c, run_optimizer(c, false));
@@ -796,12 +898,17 @@ int splitlora_client_bwd(splitlora_ctx* c, const void* act_grad_in) {
   if (!act_grad_in) return fail(c, SPLITLORA_ERR_ARG, "null pointer");
   if (!aligned16(act_grad_in)) return fail(c, SPLITLORA_ERR_ALIGN, "act_grad_in not 16-byte aligned");
   if (!c->have_client_fwd) return fail(c, SPLITLORA_ERR_STATE, "client_bwd needs a preceding client_fwd");
-  const void* cur = act_grad_in;
+  // With one cut for all, the hand-off gradient is read in place.  Otherwise each client's rows are copied
+  // into the stream of gradients where its deepest block begins.
+  const bool uni = uniform_cut(c);
   void* bufs[2] = {c->g_a, c->g_b};
+  const void* cur = uni ? act_grad_in : bufs[1];
   int which = 0;
   for (int l = c->cut - 1; l >= 0; --l) {
+    const Span sp = client_span(c, l);
+    if (!uni) CK(c, copy_client_rows(c, act_grad_in, (void*)cur, sp.client0, first_client_above(c, l + 1)));
     void* dst = (l == 0) ? nullptr : bufs[which];
-    CK(c, block_backward(c, l, cur, dst));
+    CK(c, block_backward(c, l, sp, cur, dst));
     cur = dst; which ^= 1;
   }
   CK(c, run_optimizer(c, true));   // Eq. 6-7, all K clients in one launch
@@ -849,11 +956,45 @@ int splitlora_aggregate(splitlora_ctx* c, const int64_t* counts) {
   float w[AGG_MAX_CLIENTS];
   int rc = aggregation_weights(c, counts, 0.0, w);
   if (rc) return rc;
-  { Scope s(c, "aggregate", c->client_rank.empty() ? 1 : 2);
+  if (uniform_cut(c)) {
+    Scope s(c, "aggregate", 1);
     CK(c, aggregate(c->cp, c->K, c->Pc, w, c->st));
-    // clients of lower rank keep only their own components of the (zero-padded) average
-    if (!c->client_rank.empty()) CK(c, rank_mask(c->cp, c->K, c->Pc, c->r, c->d, c->client_rank.data(), c->st)); }
+  } else {
+    // Eq. 8-9 per block over the clients that hold it (a suffix of the clients), weights renormalised
+    // over those holders; a block with a single holder stays as it is
+    for (int l = 0; l < c->cut; ++l) {
+      const int h0 = first_client_above(c, l), nh = c->K - h0;
+      if (nh < 2) continue;
+      double tot = 0.0;
+      for (int i = h0; i < c->K; ++i) tot += (double)counts[i];
+      if (!(tot > 0.0)) return fail(c, SPLITLORA_ERR_COUNTS, "all sample counts of a block's holders are zero");
+      float wl[AGG_MAX_CLIENTS];
+      for (int i = 0; i < nh; ++i) wl[i] = (float)((double)counts[h0 + i] / tot);
+      Scope s(c, "aggregate", 1);
+      CK(c, aggregate(c->cp + (size_t)h0 * c->Pc + (size_t)l * c->per_layer, nh, c->per_layer, wl, c->st, c->Pc));
+    }
+  }
+  // clients of lower rank keep only their own components of the (zero-padded) average
+  if (!c->client_rank.empty()) {
+    Scope s(c, "aggregate", 1);
+    CK(c, rank_mask(c->cp, c->K, c->Pc, c->r, c->d, c->client_rank.data(), c->st));
+  }
   c->client_copies_dirty = true;
+  return SPLITLORA_OK;
+}
+
+int splitlora_set_client_cuts(splitlora_ctx* c, const int32_t* cuts) {
+  if (!c) return SPLITLORA_ERR_ARG;
+  if (!c->ws) return fail(c, SPLITLORA_ERR_WORKSPACE, "no workspace bound");
+  if (!cuts) { c->client_cut.clear(); return SPLITLORA_OK; }
+  for (int i = 0; i < c->K; ++i) {
+    if (cuts[i] < c->cmin || cuts[i] > c->cut) return fail(c, SPLITLORA_ERR_ARG, "client cut outside [cut_min, cut]");
+    if (i > 0 && cuts[i] < cuts[i - 1]) return fail(c, SPLITLORA_ERR_ARG, "client cuts must be non-decreasing in the client index");
+  }
+  bool same = true;
+  for (int i = 0; i < c->K; ++i) same = same && cuts[i] == c->cut;
+  if (same) c->client_cut.clear(); else c->client_cut.assign(cuts, cuts + c->K);
+  c->have_client_fwd = false;
   return SPLITLORA_OK;
 }
 
@@ -863,6 +1004,7 @@ int splitlora_aggregate_local_sum(splitlora_ctx* c, const int64_t* counts, int64
                                   int64_t* count) {
   if (!c || !sum_dev || !count) return SPLITLORA_ERR_ARG;
   if (total_count <= 0) return fail(c, SPLITLORA_ERR_COUNTS, "total_count must be positive");
+  if (!uniform_cut(c)) return fail(c, SPLITLORA_ERR_UNSUPPORTED, "clients cut at different depths cannot be spread over devices");
   float w[AGG_MAX_CLIENTS];
   int rc = aggregation_weights(c, counts, (double)total_count, w);
   if (rc) return rc;

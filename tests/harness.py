@@ -85,8 +85,14 @@ QK_BOUND = 4e-2
 NOISE_MARGIN = 1.4
 
 
+CUTS_MEDIUM = (1, 3, 3)       # per-client cut depths of the "cuts_medium" case
+
+
 def qk_case(name):
     """(workload, per-client ranks or None, bound for the q / k adapter gradients or None for the general one)"""
+    if name == "cuts_medium":
+        return (synth.scaled(synth.WORKLOADS[3], n_layer=4, cut=3, n_clients=3, batch_per_client=2, seq=128,
+                             max_seq=128), None, QK_BOUND)
     if name == "federated_small":
         return (synth.scaled(synth.WORKLOADS[2], n_layer=2, cut=2, n_clients=2, batch_per_client=2, seq=256,
                              max_seq=256), None, QK_BOUND)

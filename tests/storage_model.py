@@ -142,48 +142,57 @@ def _block_bwd(cfg, params, l, adapters, dy, cache, st):
     return dx.reshape(nseq, T, d), grads
 
 
-def three_calls(cfg, params, client_adapters, server_adapters, tokens, labels, stored=True):
+def three_calls(cfg, params, client_adapters, server_adapters, tokens, labels, stored=True, cuts=None):
     """S, dS, loss, server gradients, per-client gradients; stored=False gives the exact model (it must then
-    agree with the oracle's own three calls, which the CPU tests check)."""
+    agree with the oracle's own three calls, which the CPU tests check).  cuts: per-client cut depths
+    (non-decreasing), None for cfg.cut everywhere; S and dS are stacked [K, b, T, d] either way, row block
+    i at client i's depth."""
     st = _st if stored else _ident
+    hand = O.round_to_bf16 if cfg.bf16_handoff else _ident
     K = tokens.shape[0]
-    outs, ccaches = [], []
+    cuts = [cfg.cut] * K if cuts is None else list(cuts)
+    S, ccaches = [], []
     for i in range(K):
         x = st(O.embed(cfg, params, tokens[i]))
         cl = []
-        for l in range(cfg.cut):
+        for l in range(cuts[i]):
             x, c = _block_fwd(cfg, params, l, client_adapters[i], x, st)
             cl.append(c)
-        outs.append(x)
+        S.append(hand(x))
         ccaches.append(cl)
-    S = O.round_to_bf16(np.stack(outs)) if cfg.bf16_handoff else np.stack(outs)
-    _, b, T, d = S.shape
-    x = S.reshape(K * b, T, d)
-    scaches = []
-    for l in range(cfg.cut, cfg.n_layer):
-        x, c = _block_fwd(cfg, params, l, server_adapters, x, st)
-        scaches.append(c)
+    b, T, d = S[0].shape
+    x = np.zeros((0, T, d))
+    order, entered, scaches = [], {}, {}
+    for l in range(min(cuts), cfg.n_layer + 1):
+        entered[l] = [i for i in range(K) if cuts[i] == l]
+        if entered[l]:
+            x = np.concatenate([x] + [S[i] for i in entered[l]], axis=0)
+            order += entered[l]
+        if l < cfg.n_layer:
+            x, scaches[l] = _block_fwd(cfg, params, l, server_adapters, x, st)
     if cfg.arch == "llama":
         xf, nf = O.rmsnorm_fwd(x.reshape(-1, d), params["lnf.g"], cfg.norm_eps)
     else:
         xf, nf = O.layernorm_fwd(x.reshape(-1, d), params["lnf.g"], params["lnf.b"], cfg.norm_eps)
     head = params.get("head.w", params["wte"])
     z = st(st(xf) @ head.T)
-    loss, dz = O.cross_entropy_fwd_bwd(z, labels.reshape(-1))
+    loss, dz = O.cross_entropy_fwd_bwd(z, np.concatenate([labels[i].reshape(-1) for i in order]))
     dxf = st(st(dz) @ head)
-    dx = st((O.rmsnorm_bwd if cfg.arch == "llama" else O.layernorm_bwd)(dxf, nf)).reshape(K * b, T, d)
-    sg = {}
-    for l in range(cfg.n_layer - 1, cfg.cut - 1, -1):
-        dx, g = _block_bwd(cfg, params, l, server_adapters, dx, scaches[l - cfg.cut], st)
-        sg.update(g)
-    dS = dx.reshape(K, b, T, d)
-    if cfg.bf16_handoff:
-        dS = O.round_to_bf16(dS)
+    dx = st((O.rmsnorm_bwd if cfg.arch == "llama" else O.layernorm_bwd)(dxf, nf)).reshape(-1, T, d)
+    sg, dS = {}, [None] * K
+    for l in range(cfg.n_layer, min(cuts) - 1, -1):
+        if l < cfg.n_layer:
+            dx, g = _block_bwd(cfg, params, l, server_adapters, dx, scaches[l], st)
+            sg.update(g)
+        keep = dx.shape[0] - len(entered[l]) * b
+        for j, i in enumerate(entered[l]):
+            dS[i] = hand(dx[keep + j * b: keep + (j + 1) * b])
+        dx = dx[:keep]
     cg = []
     for i in range(K):
         dx, grads = dS[i], {}
-        for l in range(cfg.cut - 1, -1, -1):
+        for l in range(cuts[i] - 1, -1, -1):
             dx, g = _block_bwd(cfg, params, l, client_adapters[i], dx, ccaches[i][l], st)
             grads.update(g)
         cg.append(grads)
-    return S, dS, loss, sg, cg
+    return np.stack(S), np.stack(dS), loss, sg, cg

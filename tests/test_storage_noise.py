@@ -21,8 +21,13 @@ from oracle import splitlora_oracle as O
 from paper_2407_00952_b200 import synth
 
 
-def _inputs(w, ranks):
+def _inputs(w, ranks, cuts=None):
     frozen, cads, sads, tokens, labels = H.build_case(w)
+    if cuts is not None:       # adapters as tests/test_gpu_cuts.py draws them: per client its own blocks
+        cads = [synth.make_adapters(w, range(cuts[i]), nonzero_b=True, salt=i + 1) for i in range(w.n_clients)]
+        sads = synth.make_adapters(w, range(min(cuts), w.n_layer), nonzero_b=True, salt=77)
+        labels = labels.copy()
+        labels[0, 0, :5] = -1
     c64 = [H.ads64(a) for a in cads]
     if ranks is not None:
         c64 = [H.cut_to_rank(c64[i], r) for i, r in enumerate(ranks)]
@@ -54,12 +59,31 @@ def test_exact_storage_model_is_the_oracle(arch):
                 assert H.rel_err(a, b) <= 1e-9, (i, key)
 
 
-@pytest.mark.parametrize("name", ["federated_small", "llama_full_width", "ranks_medium"])
+def test_exact_storage_model_with_client_cuts_is_the_oracle():
+    w = synth.scaled(synth.WORKLOADS[1], n_layer=4, cut=3, n_clients=3, counts=None)
+    cuts = [1, 2, 3]
+    cfg, params, c64, s64, tokens, labels = _inputs(w, None, cuts)
+    S, dS, loss, sg, cg = SM.three_calls(cfg, params, c64, s64, tokens, labels, stored=False, cuts=cuts)
+    S_ref, caches = O.client_fwd_cuts(cfg, params, c64, tokens, cuts)
+    loss_ref, dS_ref, sg_ref = O.server_fwd_bwd_cuts(cfg, params, s64, S_ref, labels, cuts)
+    cg_ref = O.client_bwd_grads_cuts(cfg, params, c64, dS_ref, caches, cuts)
+    assert H.rel_err(S, np.stack(S_ref)) <= 1e-12 and H.rel_err(dS, np.stack(dS_ref)) <= 1e-10
+    assert abs(loss - loss_ref) <= 1e-12
+    for key in sg_ref:
+        assert all(H.rel_err(a, b) <= 1e-9 for a, b in zip(sg[key], sg_ref[key])), key
+    for i in range(3):
+        assert set(cg[i]) == set(cg_ref[i])
+        for key in cg_ref[i]:
+            assert all(H.rel_err(a, b) <= 1e-9 for a, b in zip(cg[i][key], cg_ref[i][key])), (i, key)
+
+
+@pytest.mark.parametrize("name", ["federated_small", "llama_full_width", "ranks_medium", "cuts_medium"])
 def test_storage_noise_fixes_the_qk_bound(name):
     w, ranks, bound = H.qk_case(name)
-    cfg, params, c64, s64, tokens, labels = _inputs(w, ranks)
-    exact = SM.three_calls(cfg, params, c64, s64, tokens, labels, stored=False)
-    stored = SM.three_calls(cfg, params, c64, s64, tokens, labels, stored=True)
+    cuts = list(H.CUTS_MEDIUM) if name == "cuts_medium" else None
+    cfg, params, c64, s64, tokens, labels = _inputs(w, ranks, cuts)
+    exact = SM.three_calls(cfg, params, c64, s64, tokens, labels, stored=False, cuts=cuts)
+    stored = SM.three_calls(cfg, params, c64, s64, tokens, labels, stored=True, cuts=cuts)
     assert H.rel_err(stored[0], exact[0]) <= H.TOL_BF16            # S
     assert H.rel_err(stored[1], exact[1]) <= H.TOL_BF16            # dL/dS
     assert abs(stored[2] - exact[2]) <= 1e-3 * abs(exact[2])       # loss
