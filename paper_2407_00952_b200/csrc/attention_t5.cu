@@ -392,7 +392,6 @@ bool init_device() {
   const int dev = current_device();
   if (dev < 0 || !tensor_map_encoder()) return false;
   if (!g_once.needed(dev)) return true;
-  if (cudaFuncSetAttribute(attn_fwd_t5_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<64>::SMEM) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(attn_fwd_t5_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128>::SMEM) != cudaSuccess) return false;
   g_once.done(dev);
   return true;
@@ -412,6 +411,7 @@ bool attention_fwd_t5_supported(int dt, int T, int H, int d) {
 cudaError_t attention_fwd_t5(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, int* status,
                              cudaStream_t st) {
   if (!attention_fwd_t5_supported(DT_BF16, T, H, d)) return cudaErrorInvalidValue;
+  if (d / H == 64) return attention_fwd_t5_h64(qkv, nseq, T, H, d, o, lse, status, st);   // its own kernel
   if (!init_device()) return cudaErrorInitializationError;
   const int sms = num_sms();
   if (!status) status = library_status_word();
@@ -424,13 +424,8 @@ cudaError_t attention_fwd_t5(const void* qkv, int nseq, int T, int H, int d, voi
   p.T = T; p.H = H; p.d = d; p.scale_log2 = LOG2E / sqrtf((float)dh); p.lse = lse;
   p.status = status;
   p.nitems = nseq * H;
-  if (dh == 64) {
-    const int cap = FwdCfg<64>::CTAS_PER_SM * sms;                         // persistent CTAs
-    attn_fwd_t5_kernel<64><<<p.nitems < cap ? p.nitems : cap, T5_THREADS, FwdCfg<64>::SMEM, st>>>(mQKV, mO, p);
-  } else {
-    const int cap = FwdCfg<128>::CTAS_PER_SM * sms;
-    attn_fwd_t5_kernel<128><<<p.nitems < cap ? p.nitems : cap, T5_THREADS, FwdCfg<128>::SMEM, st>>>(mQKV, mO, p);
-  }
+  const int cap = FwdCfg<128>::CTAS_PER_SM * sms;                                  // persistent CTAs
+  attn_fwd_t5_kernel<128><<<p.nitems < cap ? p.nitems : cap, T5_THREADS, FwdCfg<128>::SMEM, st>>>(mQKV, mO, p);
   return cudaGetLastError();
 }
 

@@ -97,6 +97,9 @@ bool attention_fwd_t5_supported(int dt, int T, int H, int d);
 bool attention_bwd_t5_128_supported(int dt, int T, int H, int d);
 cudaError_t attention_bwd_t5_128(const void* qkv, const float* lse, const void* d_o, const float* rowdot, int nseq,
                                     int T, int H, int d, void* dqkv, int* status, cudaStream_t st);
+// head width 64: one softmax thread per row, half-steps of 64 keys (attention_t5_fwd64.cu)
+cudaError_t attention_fwd_t5_h64(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, int* status,
+                                 cudaStream_t st);
 cudaError_t attention_fwd_t5(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, int* status,
                              cudaStream_t st);
 cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, const void* d_o, int nseq, int T, int H,
