@@ -50,6 +50,17 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 struct F64Params {
   int T, H, d;
   int nitems;              // nseq * H (sequence, head) items, shared out over the CTAs
@@ -186,9 +197,42 @@ attn_fwd_t5_h64_kernel(const __grid_constant__ CUtensorMap mapQKV, F64Params p) 
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     bool ok = true;
     int it = 0;
+    // The output of a finished query tile is written one half-step late: its last product is still running
+    // when its last P has been handed over, so the thread first does the next tile's first half-step (whose
+    // scores are waiting already) and only then reads O, frees it and writes the row.
+    bool pend = false;
+    float pend_m = 0.f, pend_l = 1.f;
+    int pend_tq = 0;
+    auto finish_tile = [&](int tq_done, float m_fin, float l_fin, int it_after) -> bool {
+      // the tile's last product is half-step it_after - 1: its commit on its P buffer's barrier is the next
+      // phase this thread has not yet waited for there
+      if (!mbar_wait(B(P_FREE + ((it_after - 1) & 1)), (uint32_t)((it_after - 1) >> 1) & 1u, abort_flag, p.status, 30)) return false;
+      tc_fence_after();
+      float o_acc[DH];
+      tc_ld32(tO + lane_off, o_acc);
+      tc_ld32(tO + lane_off + 32u, o_acc + 32);
+      tc_wait_ld();
+      tc_fence_before();
+      mbar_arrive(B(O_FREE));                      // O may be overwritten by the next query tile
+      const int qt = qt_of(tq_done), h = head_of(tq_done), seq_row0 = row0_of(tq_done), b = seq_row0 / p.T;
+      const float inv = 1.0f / l_fin;
+      bf16* orow = p.o + (size_t)(seq_row0 + qt * BQ + r) * p.d + (size_t)h * DH;
+#pragma unroll
+      for (int jj = 0; jj < DH / 8; ++jj) {
+        uint4 w;
+        uint32_t* wp = reinterpret_cast<uint32_t*>(&w);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          __nv_bfloat162 ob = __floats2bfloat162_rn(o_acc[8 * jj + 2 * i] * inv, o_acc[8 * jj + 2 * i + 1] * inv);
+          wp[i] = *reinterpret_cast<uint32_t*>(&ob);
+        }
+        *reinterpret_cast<uint4*>(orow + 8 * jj) = w;
+      }
+      p.lse[((size_t)b * p.H + h) * p.T + (size_t)qt * BQ + r] = (m_fin + log2f(l_fin)) * LN2;
+      return true;
+    };
     for (int tq = 0; tq < my_tiles && ok; ++tq) {
       const int qt = qt_of(tq), nhs = 2 * (qt + 1);
-      const int h = head_of(tq), seq_row0 = row0_of(tq), b = seq_row0 / p.T;
       float m_run = -INFINITY;                   // running maximum of the scaled scores (log2 domain)
       float m_ref = -INFINITY;                   // the maximum the exponentials are taken against
       float l_run = 0.f;
@@ -214,12 +258,13 @@ attn_fwd_t5_h64_kernel(const __grid_constant__ CUtensorMap mapQKV, F64Params p) 
 #pragma unroll
             for (int i = 0; i < HK; ++i) v[i] = (i > lim) ? -INFINITY : v[i];
           }
-          float m4[4] = {v[0], v[1], v[2], v[3]};
+          float m4[4] = {max3(v[0], v[1], v[2]), max3(v[3], v[4], v[5]), max3(v[6], v[7], v[8]), max3(v[9], v[10], v[11])};
 #pragma unroll
-          for (int i = 4; i < HK; i += 4) {
-            m4[0] = fmaxf(m4[0], v[i]); m4[1] = fmaxf(m4[1], v[i + 1]);
-            m4[2] = fmaxf(m4[2], v[i + 2]); m4[3] = fmaxf(m4[3], v[i + 3]);
+          for (int i = 12; i < 60; i += 8) {     // three-input maxima, four chains
+            m4[0] = max3(m4[0], v[i], v[i + 1]); m4[1] = max3(m4[1], v[i + 2], v[i + 3]);
+            m4[2] = max3(m4[2], v[i + 4], v[i + 5]); m4[3] = max3(m4[3], v[i + 6], v[i + 7]);
           }
+          m4[0] = max3(m4[0], v[60], v[61]); m4[1] = max3(m4[1], v[62], v[63]);
           const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
           const float m_new = fmaxf(m_run, mx * p.scale_log2);   // finite: key 0 is visible to every row
           m_run = m_new;
@@ -249,13 +294,21 @@ attn_fwd_t5_h64_kernel(const __grid_constant__ CUtensorMap mapQKV, F64Params p) 
               if (need) m_ref = m_new;
             }
           }
+          // exponentials on pairs: one packed multiply-add and one packed add per two scores
+          const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(-m_ref, -m_ref);
+          uint64_t ps2 = pack2(0.f, 0.f);
 #pragma unroll
           for (int i = 0; i < HK; i += 2) {
-            const float p0 = ex2(fmaf(v[i], p.scale_log2, -m_ref)), p1 = ex2(fmaf(v[i + 1], p.scale_log2, -m_ref));
-            psum += p0 + p1;
+            float a0, a1;
+            unpack2(fma2(pack2(v[i], v[i + 1]), sc2, nm2), a0, a1);
+            const float p0 = ex2(a0), p1 = ex2(a1);
+            ps2 = add2(ps2, pack2(p0, p1));
             __nv_bfloat162 pb2 = __floats2bfloat162_rn(p0, p1);
             pk[i >> 1] = *reinterpret_cast<uint32_t*>(&pb2);
           }
+          float s0, s1;
+          unpack2(ps2, s0, s1);
+          psum = s0 + s1;
         } else {
 #pragma unroll
           for (int i = 0; i < HK / 2; ++i) pk[i] = 0u;
@@ -269,33 +322,14 @@ attn_fwd_t5_h64_kernel(const __grid_constant__ CUtensorMap mapQKV, F64Params p) 
         tc_fence_before();
         mbar_arrive(B(P_READY + sb));
         l_run += psum;
-      }
-      // the tile's last product, then normalise and write the row (64 bf16 = 128 bytes) straight to memory
-      if (ok && !mbar_wait(B(P_FREE + ((it - 1) & 1)), (uint32_t)((it - 1) >> 1) & 1u, abort_flag, p.status, 30)) ok = false;
-      if (ok) {
-        tc_fence_after();
-        float o_acc[DH];
-        tc_ld32(tO + lane_off, o_acc);
-        tc_ld32(tO + lane_off + 32u, o_acc + 32);
-        tc_wait_ld();
-        tc_fence_before();
-        mbar_arrive(B(O_FREE));                      // O may be overwritten by the next query tile
-        const float inv = 1.0f / l_run;
-        bf16* orow = p.o + (size_t)(seq_row0 + qt * BQ + r) * p.d + (size_t)h * DH;
-#pragma unroll
-        for (int jj = 0; jj < DH / 8; ++jj) {
-          uint4 w;
-          uint32_t* wp = reinterpret_cast<uint32_t*>(&w);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            __nv_bfloat162 ob = __floats2bfloat162_rn(o_acc[8 * jj + 2 * i] * inv, o_acc[8 * jj + 2 * i + 1] * inv);
-            wp[i] = *reinterpret_cast<uint32_t*>(&ob);
-          }
-          *reinterpret_cast<uint4*>(orow + 8 * jj) = w;
+        if (hs == 0 && pend) {                   // the previous tile's output (its products are done by now)
+          if (!finish_tile(pend_tq, pend_m, pend_l, it)) { ok = false; break; }
+          pend = false;
         }
-        p.lse[((size_t)b * p.H + h) * p.T + (size_t)qt * BQ + r] = (m_ref + log2f(l_run)) * LN2;
       }
+      pend = true; pend_m = m_ref; pend_l = l_run; pend_tq = tq;
     }
+    if (ok && pend) finish_tile(pend_tq, pend_m, pend_l, it);
   }
 
   // ---------------- teardown ----------------
