@@ -297,6 +297,14 @@ int splitlora_lora_linear_bwd(int dtype, int use_tensor_cores, const void* x, co
                               const float* A, const float* B, float alpha, int M, int n_in, int n_out,
                               int r, int G, void* dx, float* dA, float* dB,
                               void* workspace, size_t workspace_bytes, void* stream);
+/* The same backward in parts, so that they can be timed one by one: parts is a sum of 1 (the two rank-r
+ * projections h = x A_g^T and dh = (alpha/r) dy B_g, which the other parts read from the workspace),
+ * 2 (dx) and 4 (dA and dB).  Parts 2 and 4 need a preceding call with part 1 on the same workspace and
+ * operands.  parts = 7 is splitlora_lora_linear_bwd. */
+int splitlora_lora_linear_bwd_parts(int dtype, int use_tensor_cores, const void* x, const void* Wt, const void* dy,
+                                    const float* A, const float* B, float alpha, int M, int n_in, int n_out,
+                                    int r, int G, void* dx, float* dA, float* dB,
+                                    void* workspace, size_t workspace_bytes, void* stream, int parts);
 /* Frozen linear layer with a fused epilogue (the un-adapted projections of a block and their
  * backward products; W is frozen, so the backward is the same call on the transposed weight):
  *   epilogue 0: y = x W^T + bias                 1: z = x W^T + bias, y = gelu(z)

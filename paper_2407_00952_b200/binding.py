@@ -34,7 +34,7 @@ EXPORTS = [
     "splitlora_adapters_changed", "splitlora_aggregate_local_sum", "splitlora_aggregate_broadcast",
     "splitlora_handoff_quantize",
     "splitlora_handoff_dequantize", "splitlora_round_compressed", "splitlora_set_client_ranks",
-    "splitlora_library_status", "splitlora_set_client_cuts",
+    "splitlora_library_status", "splitlora_set_client_cuts", "splitlora_lora_linear_bwd_parts",
 ]
 
 
@@ -337,19 +337,24 @@ def lora_linear_fwd(x, W, bias, A, B, alpha, y=None, workspace=None, use_tensor_
     return y
 
 
-def lora_linear_bwd(x, Wt, dy, A, B, alpha, workspace=None, use_tensor_cores=True):
+def lora_linear_bwd(x, Wt, dy, A, B, alpha, workspace=None, use_tensor_cores=True, parts=7, out=None):
+    """parts: sum of 1 (rank-r projections), 2 (dx), 4 (dA, dB), see splitlora_lora_linear_bwd_parts;
+    out: (dx, dA, dB) buffers to reuse."""
     lib = load()
     M, n_in = x.shape
     n_out = dy.shape[1]
     G, r, _ = A.shape
-    dx = torch.empty(M, n_in, dtype=x.dtype, device="cuda")
-    dA = torch.empty(G, r, n_in, dtype=torch.float32, device="cuda")
-    dB = torch.empty(G, n_out, r, dtype=torch.float32, device="cuda")
+    if out is None:
+        out = (torch.empty(M, n_in, dtype=x.dtype, device="cuda"),
+               torch.empty(G, r, n_in, dtype=torch.float32, device="cuda"),
+               torch.empty(G, n_out, r, dtype=torch.float32, device="cuda"))
+    dx, dA, dB = out
     if workspace is None:
         workspace = lora_linear_workspace(_dt(x), M, n_in, n_out, r, G)
-    _rc(lib.splitlora_lora_linear_bwd(_dt(x), 1 if use_tensor_cores else 0, _ptr(x), _ptr(Wt), _ptr(dy), _ptr(A),
-                                      _ptr(B), C.c_float(alpha), M, n_in, n_out, r, G, _ptr(dx), _ptr(dA), _ptr(dB),
-                                      _ptr(workspace), C.c_size_t(workspace.numel()), _stream_ptr()), "lora_linear_bwd")
+    _rc(lib.splitlora_lora_linear_bwd_parts(_dt(x), 1 if use_tensor_cores else 0, _ptr(x), _ptr(Wt), _ptr(dy), _ptr(A),
+                                            _ptr(B), C.c_float(alpha), M, n_in, n_out, r, G, _ptr(dx), _ptr(dA), _ptr(dB),
+                                            _ptr(workspace), C.c_size_t(workspace.numel()), _stream_ptr(), int(parts)),
+        "lora_linear_bwd")
     return dx, dA, dB
 
 

@@ -116,8 +116,16 @@ int splitlora_lora_linear_fwd(int dtype, int use_tc, const void* x, const void* 
 int splitlora_lora_linear_bwd(int dtype, int use_tc, const void* x, const void* Wt, const void* dy, const float* A,
                               const float* B, float alpha, int M, int n_in, int n_out, int r, int G, void* dx,
                               float* dA, float* dB, void* workspace, size_t workspace_bytes, void* stream) {
+  return splitlora_lora_linear_bwd_parts(dtype, use_tc, x, Wt, dy, A, B, alpha, M, n_in, n_out, r, G, dx, dA, dB, workspace,
+                                         workspace_bytes, stream, 7);
+}
+
+int splitlora_lora_linear_bwd_parts(int dtype, int use_tc, const void* x, const void* Wt, const void* dy, const float* A,
+                                    const float* B, float alpha, int M, int n_in, int n_out, int r, int G, void* dx,
+                                    float* dA, float* dB, void* workspace, size_t workspace_bytes, void* stream, int parts) {
   int rc = check_linear(dtype, M, n_in, n_out, r, G);
   if (rc) return rc;
+  if (parts < 1 || parts > 7) return SPLITLORA_ERR_ARG;
   if (!x || !Wt || !dy || !A || !B || !dx || !dA || !dB || !workspace) return SPLITLORA_ERR_ARG;
   if (!aligned16(x) || !aligned16(Wt) || !aligned16(dy) || !aligned16(dx) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
     return SPLITLORA_ERR_ALIGN;
@@ -130,22 +138,27 @@ int splitlora_lora_linear_bwd(int dtype, int use_tc, const void* x, const void* 
   const int rpg = G > 1 ? M / G : 0;
   int* status = (int*)(ws + p.off_status);
   const float s = alpha / (float)r;
-  // h = x A_g^T (recomputed here; the training runtime keeps it from the forward pass)
-  GemmArgs h;
-  h.dtype = dtype; h.X = x; h.ldx = n_in; h.W = ws + p.off_acat; h.ldw = n_in; h.Y = ws + p.off_h; h.ldy = p.ext;
-  h.M = M; h.N = p.ext; h.K = n_in; h.rows_per_group = rpg; h.w_grouped = G > 1;
-  if (run_gemm(use_tc, h, status, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
-  // dh = s dy B_g
-  GemmArgs g;
-  g.dtype = dtype; g.X = dy; g.ldx = n_out; g.W = ws + p.off_bextT; g.ldw = n_out; g.Y = ws + p.off_dh; g.ldy = p.ext;
-  g.M = M; g.N = p.ext; g.K = n_out; g.rows_per_group = rpg; g.w_grouped = G > 1;
-  if (run_gemm(use_tc, g, status, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
-  // dx = dy W + dh A_g
-  GemmArgs a;
-  a.dtype = dtype; a.X = dy; a.ldx = n_out; a.W = Wt; a.ldw = n_out; a.Y = dx; a.ldy = n_in;
-  a.M = M; a.N = n_in; a.K = n_out; a.rows_per_group = rpg;
-  a.Xe = ws + p.off_dh; a.ldxe = p.ext; a.We = ws + p.off_acatT; a.ldwe = p.ext; a.Ke = p.rp; a.we_grouped = G > 1;
-  if (run_gemm(use_tc, a, status, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
+  if (parts & 1) {
+    // h = x A_g^T (recomputed here; the training runtime keeps it from the forward pass)
+    GemmArgs h;
+    h.dtype = dtype; h.X = x; h.ldx = n_in; h.W = ws + p.off_acat; h.ldw = n_in; h.Y = ws + p.off_h; h.ldy = p.ext;
+    h.M = M; h.N = p.ext; h.K = n_in; h.rows_per_group = rpg; h.w_grouped = G > 1;
+    if (run_gemm(use_tc, h, status, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
+    // dh = s dy B_g
+    GemmArgs g;
+    g.dtype = dtype; g.X = dy; g.ldx = n_out; g.W = ws + p.off_bextT; g.ldw = n_out; g.Y = ws + p.off_dh; g.ldy = p.ext;
+    g.M = M; g.N = p.ext; g.K = n_out; g.rows_per_group = rpg; g.w_grouped = G > 1;
+    if (run_gemm(use_tc, g, status, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
+  }
+  if (parts & 2) {
+    // dx = dy W + dh A_g
+    GemmArgs a;
+    a.dtype = dtype; a.X = dy; a.ldx = n_out; a.W = Wt; a.ldw = n_out; a.Y = dx; a.ldy = n_in;
+    a.M = M; a.N = n_in; a.K = n_out; a.rows_per_group = rpg;
+    a.Xe = ws + p.off_dh; a.ldxe = p.ext; a.We = ws + p.off_acatT; a.ldwe = p.ext; a.Ke = p.rp; a.we_grouped = G > 1;
+    if (run_gemm(use_tc, a, status, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
+  }
+  if (!(parts & 4)) return SPLITLORA_OK;
   float* scratch = (float*)(ws + p.off_scratch);
   if (lora_grad(dtype, x, n_in, 0, n_in, ws + p.off_dh, p.ext, 0, r, p.rp, 1, M, rpg, 1.0f, dA, (int64_t)r * n_in, 0, n_in, 1,
                 scratch, st, status, use_tc != 0) != cudaSuccess) return SPLITLORA_ERR_CUDA;

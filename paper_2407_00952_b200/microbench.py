@@ -43,7 +43,11 @@ def _time(fn, iters, warmup=3):
     return e0.elapsed_time(e1) / iters
 
 
-def bench_linear(M, n_in, n_out, r, G, iters=20, backward=True, tc=True):
+def bench_linear_shape(M, n_in, n_out, rs, Gs, iters=10, backward=True, tc=True):
+    """One (M, in, out) shape of the grouped LoRA linear for every rank in rs and group count in Gs.
+    Forward, and the backward in its parts: the rank-r projections, dx, and dA + dB, each timed by itself
+    (splitlora_lora_linear_bwd_parts).  Operands rotate over several buffer sets unless one set exceeds
+    twice the L2, so every launch reads from HBM.  Yields one dict per (r, G)."""
     hbm, tflops, src = _peaks()
     set_bytes = 2 * (M * n_in + M * n_out + n_in * n_out)
     nset = max(1, min(4, -(-2 * L2_BYTES // set_bytes)))
@@ -52,25 +56,45 @@ def bench_linear(M, n_in, n_out, r, G, iters=20, backward=True, tc=True):
     xs = [mk(M, n_in) for _ in range(nset)]
     dys = [mk(M, n_out, sc=n_out ** -0.5) for _ in range(nset)]
     ys = [torch.empty(M, n_out, device="cuda", dtype=torch.bfloat16) for _ in range(nset)]
+    dxs = [torch.empty(M, n_in, device="cuda", dtype=torch.bfloat16) for _ in range(nset)]
     W = mk(n_out, n_in, sc=n_in ** -0.5)
     Wt = B.transpose(W)
-    A = torch.randn(G, r, n_in, device="cuda", generator=g) * n_in ** -0.5
-    Bm = torch.randn(G, n_out, r, device="cuda", generator=g) * r ** -0.5
-    ws = B.lora_linear_workspace(B.DTYPE_BF16, M, n_in, n_out, r, G)
-    fwd = _time(lambda i: B.lora_linear_fwd(xs[i % nset], W, None, A, Bm, 16.0, y=ys[i % nset], workspace=ws,
-                                            use_tensor_cores=tc), iters)
-    flops = 2.0 * M * n_in * n_out + 2.0 * M * r * (n_in + n_out)
-    out = {"op": "lora_linear", "M": M, "n_in": n_in, "n_out": n_out, "r": r, "G": G,
-           "fwd_us": round(fwd * 1e3, 1), "fwd_tflops": round(flops / fwd / 1e9, 1),
-           "fwd_frac_of_bf16_peak": round(flops / fwd / 1e9 / tflops, 3), "peak_source": src + " burst"}
-    if backward:
-        bwd = _time(lambda i: B.lora_linear_bwd(xs[i % nset], Wt, dys[i % nset], A, Bm, 16.0, workspace=ws,
-                                                use_tensor_cores=tc), max(3, iters // 2))
-        # dx product + both rank-r products + the two skinny gradient reductions (no dW: W is frozen)
-        bflops = 2.0 * M * n_in * n_out + 4.0 * M * r * (n_in + n_out)
-        out.update({"bwd_us": round(bwd * 1e3, 1), "bwd_tflops": round(bflops / bwd / 1e9, 1),
-                    "bwd_frac_of_bf16_peak": round(bflops / bwd / 1e9 / tflops, 3)})
-    return out
+    for r in rs:
+        for G in Gs:
+            if M % G or (G > 1 and (M // G) % 128):
+                continue
+            A = torch.randn(G, r, n_in, device="cuda", generator=g) * n_in ** -0.5
+            Bm = torch.randn(G, n_out, r, device="cuda", generator=g) * r ** -0.5
+            ws = B.lora_linear_workspace(B.DTYPE_BF16, M, n_in, n_out, r, G)
+            fwd = _time(lambda i: B.lora_linear_fwd(xs[i % nset], W, None, A, Bm, 16.0, y=ys[i % nset], workspace=ws,
+                                                    use_tensor_cores=tc), iters)
+            flops = 2.0 * M * n_in * n_out + 2.0 * M * r * (n_in + n_out)
+            out = {"op": "lora_linear", "M": M, "n_in": n_in, "n_out": n_out, "r": r, "G": G, "buffer_sets": nset,
+                   "fwd_us": round(fwd * 1e3, 1), "fwd_tflops": round(flops / fwd / 1e9, 1),
+                   "fwd_frac_of_bf16_peak": round(flops / fwd / 1e9 / tflops, 3), "peak_source": src + " burst"}
+            if backward:
+                dA = torch.empty(G, r, n_in, dtype=torch.float32, device="cuda")
+                dB = torch.empty(G, n_out, r, dtype=torch.float32, device="cuda")
+                run = lambda parts: _time(lambda i: B.lora_linear_bwd(xs[i % nset], Wt, dys[i % nset], A, Bm, 16.0, workspace=ws,
+                                                                      use_tensor_cores=tc, parts=parts,
+                                                                      out=(dxs[i % nset], dA, dB)), iters)
+                t_down = run(1)                       # h = x A^T and dh = s dy B: skinny, HBM-bound
+                t_dx = run(1 | 2) - t_down            # dx = dy W + dh A on the tensor cores
+                t_g = run(1 | 4) - t_down             # dA = dh^T x, dB = s dy^T h: skinny reductions over the tokens
+                dx_flops = 2.0 * M * n_in * n_out + 2.0 * M * r * n_in
+                down_bytes = 2.0 * M * (n_in + n_out)               # x and dy read once
+                g_bytes = 2.0 * M * (n_in + n_out)                  # x and dy read once more
+                out.update({"down_us": round(t_down * 1e3, 1), "down_GBps": round(down_bytes / t_down / 1e6, 1),
+                            "down_frac_of_hbm": round(down_bytes / t_down / 1e6 / hbm, 3),
+                            "dx_us": round(t_dx * 1e3, 1), "dx_tflops": round(dx_flops / t_dx / 1e9, 1),
+                            "dx_frac_of_bf16_peak": round(dx_flops / t_dx / 1e9 / tflops, 3),
+                            "dAdB_us": round(t_g * 1e3, 1), "dAdB_GBps": round(g_bytes / t_g / 1e6, 1),
+                            "dAdB_frac_of_hbm": round(g_bytes / t_g / 1e6 / hbm, 3)})
+            yield out
+
+
+def bench_linear(M, n_in, n_out, r, G, iters=20, backward=True, tc=True):
+    return next(bench_linear_shape(M, n_in, n_out, [r], [G], iters, backward, tc))
 
 
 def bench_epilogues(M, d, F, iters=20):
@@ -257,9 +281,9 @@ def main():
         for M in Ms:
             for n_in in ins:
                 for n_out in outs:
-                    for r in rs:
-                        for G in Gs:
-                            print(json.dumps(bench_linear(M, n_in, n_out, r, G, 10)), flush=True)
+                    for row in bench_linear_shape(M, n_in, n_out, rs, Gs, a.iters if a.iters < 20 else 8):
+                        print(json.dumps(row), flush=True)
+                    torch.cuda.empty_cache()
     elif a.what == "epilogues":
         for row in bench_epilogues(a.M, a.n_in, 4 * a.n_in, a.iters):
             print(json.dumps(row), flush=True)
