@@ -303,6 +303,17 @@ def run_gpu(args, w):
     barrier()
     ms_e2e = e0.elapsed_time(e1)
 
+    # ---- host cost of enqueueing one round: the stream is empty when the calls start, so nothing in
+    # them waits for the device (a round is fewer launches than the launch queue holds) ----
+    enq = []
+    for s in range(3):
+        barrier()
+        t0 = time.perf_counter()
+        step_dev(s)
+        enq.append((time.perf_counter() - t0) * 1e3)
+    barrier()
+    host_enqueue_empty_ms = min(enq)
+
     # ---- per-class breakdown (outside the timed regions): events around every launch ----
     eng.profile_enable(1)
     eng.profile_report()
@@ -365,7 +376,8 @@ def run_gpu(args, w):
         par = (f"weak: {w.n_clients} clients on each of {world} GPUs, NCCL all-reduce of the server adapter gradients "
                f"and of one client's worth of aggregation sums")
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms / args.steps, "host_enqueue_ms_per_step": host_ms / args.steps, "higher_is_better": True, "scaling": args.scaling, "vs_baseline": None,
+            "ms_per_step": ms / args.steps, "host_enqueue_ms_per_step": host_ms / args.steps,
+            "host_enqueue_empty_stream_ms": host_enqueue_empty_ms, "higher_is_better": True, "scaling": args.scaling, "vs_baseline": None,
             "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": workload_description(w), "parallelism": par,
             "clocks": clocks,

@@ -168,12 +168,32 @@ def bench_split(config: int, cut: int, agg_interval: int, n_clients: int, steps:
         t, l = synth.make_tokens(w, round_index=s)
         batches.append((torch.from_numpy(t).cuda(), torch.from_numpy(l).cuda()))
     ms = _time(lambda i: eng.round(*batches[i % 2], counts, want_loss=False), steps, warmup=3)
+    # the same round as its three calls, each timed by itself: what runs on the clients and what on the server
+    S, dS = eng.new_activation_buffer(), eng.new_activation_buffer()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    t_client = t_server = 0.0
+    for i in range(steps):
+        ev[0].record(); eng.client_fwd(batches[i % 2][0], S)
+        ev[1].record(); eng.server_step(S, batches[i % 2][1], dS, want_loss=False)
+        ev[2].record(); eng.client_bwd(dS)
+        ev[3].record(); torch.cuda.synchronize()
+        t_client += ev[0].elapsed_time(ev[1]) + ev[2].elapsed_time(ev[3])
+        t_server += ev[1].elapsed_time(ev[2])
     assert eng.device_status() == 0
     M, es = w.tokens_per_round, 2 if w.dtype == "bf16" else 4
     per_client = w.cut * len(w.targets) * 2 * w.lora_r * w.d_model * 4
+    # algorithmic FLOPs per round (forward + backward without dW): a block's linear layers and its causal
+    # attention (forward 2 T d per token, backward 2.5 x that), the head on the server
+    d, F, T = w.d_model, w.d_ff, w.seq
+    mlp = (6.0 if w.arch == "llama" else 4.0) * d * F
+    block = M * (2.0 * (8.0 * d * d + mlp) + 3.5 * 2.0 * T * d)
+    head = 2.0 * 2.0 * M * d * w.vocab
     return {"op": "split_round", "config": config, "cut": cut, "n_layer": w.n_layer, "I": agg_interval,
             "K": w.n_clients, "tokens_per_round": M, "ms_per_round": round(ms, 3),
             "tokens_per_s": round(M / ms * 1e3, 1), "client_block_share": round(w.cut / w.n_layer, 4),
+            "client_flop_share": round(cut * block / (w.n_layer * block + head), 4),
+            "client_time_share": round(t_client / (t_client + t_server), 4),
+            "client_ms": round(t_client / steps, 3), "server_ms": round(t_server / steps, 3),
             "handoff_bytes_per_round": 2 * M * w.d_model * es + M * 4,
             "aggregation_bytes_per_client": 2 * per_client, "aggregations_per_round": round(1.0 / agg_interval, 3)}
 
