@@ -120,6 +120,21 @@ cudaError_t lora_grad(int dt, const void* Z, int64_t ldz, int zcol0, int C, cons
                       int wcol0, int r, int rp, int nt, int M, int rows_per_group, float scale, float* out,
                       int64_t out_group_stride, int64_t out_target_stride, int64_t out_sj, int64_t out_sc,
                       float* partial, cudaStream_t st, int* status = nullptr, bool use_tc = false);
+// One reduction of lora_grad as a record, for lora_grad_batch: several of them over the same token rows
+// (the adapter gradients of one layer) in one pair of launches.
+struct LoraGradJob {
+  const void* Z = nullptr; int64_t ldz = 0; int zcol0 = 0, C = 0;
+  const void* Wt = nullptr; int64_t ldwt = 0; int wcol0 = 0, r = 0, rp = 0, nt = 1;
+  float scale = 1.f; float* out = nullptr;
+  int64_t out_group_stride = 0, out_target_stride = 0, out_sj = 0, out_sc = 0;
+};
+// partial: scratch of partial_floats floats.  Falls back to one lora_grad per job where the batched
+// tensor-core path does not apply.
+cudaError_t lora_grad_batch(int dt, const LoraGradJob* jobs, int njobs, int M, int rows_per_group, float* partial,
+                            size_t partial_floats, cudaStream_t st, int* status, bool use_tc);
+cudaError_t lora_grad_tc_partial_batch(const LoraGradJob* jobs, int njobs, int M, int rows_per_group, float* partial,
+                                       size_t partial_floats, int* status, int* chunks_per_group, size_t* offsets,
+                                       cudaStream_t st);
 // The same reduction as a tcgen05 product with both operands MN-major (bf16, rp in {16, 32, 64},
 // ldwt a multiple of 64, the wanted weight columns inside one 64-column tile).  Writes per-chunk
 // partials [chunk][nt*r][C]; lora_grad adds them.  status: device word for an expired bounded wait.

@@ -151,6 +151,24 @@ lora_grad_reduce_lanes_kernel(const float* __restrict__ partial, int r, int R, i
   }
 }
 
+// The second kernel for a batch of jobs (blockIdx.z): one output per thread, chunks added in order.
+struct RedJob { const float* partial; float* out; int r, R; float scale; int64_t ogs, ots, osj, osc; };
+struct RedBatch { RedJob j[4]; };
+__global__ void __launch_bounds__(RED_THREADS)
+lora_grad_reduce_batch_kernel(RedBatch b, int C, int chunks_per_group) {
+  const RedJob& jb = b.j[blockIdx.z];
+  const int idx = blockIdx.x * RED_THREADS + threadIdx.x;   // over R*C
+  const int g = blockIdx.y;
+  if (idx >= jb.R * C) return;
+  const size_t rc = (size_t)jb.R * C;
+  const float* p = jb.partial + (size_t)g * chunks_per_group * rc + idx;
+  float s = 0.f;
+#pragma unroll 4
+  for (int k = 0; k < chunks_per_group; ++k) s += p[(size_t)k * rc];
+  const int j = idx / C, c = idx % C;
+  jb.out[(size_t)g * jb.ogs + (size_t)(j / jb.r) * jb.ots + (size_t)(j % jb.r) * jb.osj + (size_t)c * jb.osc] = jb.scale * s;
+}
+
 // picks the second kernel by the number of outputs (both add in a fixed order)
 void launch_reduce(const float* partial, int r, int R, int C, int cpg, int groups, float scale, float* out,
                    int64_t out_group_stride, int64_t out_target_stride, int64_t out_sj, int64_t out_sc, cudaStream_t st) {
@@ -225,6 +243,44 @@ cudaError_t lora_grad(int dt, const void* Z, int64_t ldz, int zcol0, int C, cons
   launch_reduce(partial, r, R, C, chunks_per_group, groups, scale, out, out_group_stride, out_target_stride, out_sj,
                 out_sc, st);
   return cudaGetLastError();
+}
+
+cudaError_t lora_grad_batch(int dt, const LoraGradJob* jobs, int njobs, int M, int rows_per_group, float* partial,
+                            size_t partial_floats, cudaStream_t st, int* status, bool use_tc) {
+  bool batched = use_tc && status && dt == DT_BF16 && njobs >= 1 && njobs <= 4;
+  for (int j = 0; j < njobs && batched; ++j) {
+    const LoraGradJob& jb = jobs[j];
+    batched = jb.C == jobs[0].C && (jb.rp == 16 || jb.rp == 32 || jb.rp == 64) &&
+              lora_grad_tc_supported(dt, jb.Z, jb.ldz, jb.zcol0, jb.C, jb.Wt, jb.ldwt, jb.wcol0, jb.r, jb.rp, jb.nt, M, rows_per_group);
+  }
+  if (batched) {
+    const int groups = rows_per_group > 0 && rows_per_group < M ? M / rows_per_group : 1;
+    int cpg = 0;
+    size_t offs[4];
+    cudaError_t e = lora_grad_tc_partial_batch(jobs, njobs, M, rows_per_group, partial, partial_floats, status, &cpg, offs, st);
+    if (e == cudaSuccess) {
+      RedBatch rb;
+      int maxRC = 0;
+      for (int j = 0; j < 4; ++j) {
+        const LoraGradJob& jb = jobs[j < njobs ? j : 0];
+        rb.j[j] = {partial + offs[j < njobs ? j : 0], jb.out, jb.r, jb.nt * jb.r, jb.scale, jb.out_group_stride,
+                   jb.out_target_stride, jb.out_sj, jb.out_sc};
+        if (j < njobs && jb.nt * jb.r * jb.C > maxRC) maxRC = jb.nt * jb.r * jb.C;
+      }
+      dim3 g2((maxRC + RED_THREADS - 1) / RED_THREADS, groups, njobs);
+      lora_grad_reduce_batch_kernel<<<g2, RED_THREADS, 0, st>>>(rb, jobs[0].C, cpg);
+      return cudaGetLastError();
+    }
+    if (e != cudaErrorInvalidValue) return e;      // invalid value: the scratch does not hold the batch, go one by one
+  }
+  for (int j = 0; j < njobs; ++j) {
+    const LoraGradJob& jb = jobs[j];
+    cudaError_t e = lora_grad(dt, jb.Z, jb.ldz, jb.zcol0, jb.C, jb.Wt, jb.ldwt, jb.wcol0, jb.r, jb.rp, jb.nt, M, rows_per_group,
+                              jb.scale, jb.out, jb.out_group_stride, jb.out_target_stride, jb.out_sj, jb.out_sc, partial, st,
+                              status, use_tc);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace sl

@@ -38,6 +38,17 @@ struct LgParams {
   float* partial;
   int* status;
 };
+// Up to LT_MAX_JOBS reductions over the same token rows in one launch (blockIdx.z picks the job): the
+// adapter gradients of one layer, e.g. G_A of all targets from u and G_B of each target from its slice
+// of dy.  One launch instead of one per job: the jobs are short (tens of microseconds), so their start-up,
+// tail and launch gaps weigh as much as their traffic.
+constexpr int LT_MAX_JOBS = 4;
+struct LgBatch {
+  CUtensorMap mapZ[LT_MAX_JOBS];
+  CUtensorMap mapW[LT_MAX_JOBS];
+  LgParams p[LT_MAX_JOBS];
+  int wx0[LT_MAX_JOBS];
+};
 
 // MN-major operand stored as [k rows][64 elements] boxes (128-byte rows, 128-byte swizzle): groups
 // of 8 k-rows are 1024 bytes apart; `mn_stride` is the distance between consecutive 64-element
@@ -53,7 +64,11 @@ __device__ __forceinline__ uint64_t desc_mn(uint32_t addr, uint32_t mn_stride) {
 }
 
 __global__ void __launch_bounds__(LT_THREADS, 2)
-lora_grad_tc_kernel(const __grid_constant__ CUtensorMap mapZ, const __grid_constant__ CUtensorMap mapW, LgParams p, int wx0) {
+lora_grad_tc_kernel(const __grid_constant__ LgBatch bt) {
+  const CUtensorMap& mapZ = bt.mapZ[blockIdx.z];
+  const CUtensorMap& mapW = bt.mapW[blockIdx.z];
+  const LgParams& p = bt.p[blockIdx.z];
+  const int wx0 = bt.wx0[blockIdx.z];
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -184,33 +199,64 @@ bool lora_grad_tc_supported(int dt, const void* Z, int64_t ldz, int zcol0, int C
   return true;
 }
 
-// Chunk partials go to `partial` as [chunk][R][C] (R = nt*r); returns the number of chunks per group
-// through *chunks_per_group so that the caller's second kernel can add them.
-cudaError_t lora_grad_tc_partial(const void* Z, int64_t ldz, int zcol0, int C, const void* Wt, int64_t ldwt, int wcol0,
-                                 int r, int rp, int nt, int M, int rows_per_group, float* partial, int* status,
-                                 int* chunks_per_group, cudaStream_t st) {
+// Chunks per group for a grid of `ctas_per_chunk_set` CTAs per chunk: the choice that minimises
+// (waves of 296 resident CTAs) x (rows per chunk), every chunk a whole number of 128-row blocks.
+static int pick_chunks(int ctas_per_chunk_set, int rpg) {
+  int best = 1;
+  double best_cost = 1e300;
+  for (int s = 1; s <= rpg / 128; ++s) {
+    if (rpg % (s * 128) != 0) continue;
+    const int ctas = ctas_per_chunk_set * s;
+    const double cost = (double)((ctas + 295) / 296) * ((double)rpg / s + 256.0);   // + a chunk's start-up, in rows
+    if (cost < best_cost) { best_cost = cost; best = s; }
+  }
+  return best;
+}
+
+// Chunk partials of job j go to partial + offset_j as [chunk][R_j][C] (R_j = nt*r); *chunks_per_group
+// receives the number of chunks per group (the same for every job) so that the caller's second kernel
+// can add them, offsets[j] the start of job j's partials (floats).  All jobs share M, rows_per_group and C.
+cudaError_t lora_grad_tc_partial_batch(const LoraGradJob* jobs, int njobs, int M, int rows_per_group, float* partial,
+                                       size_t partial_floats, int* status, int* chunks_per_group, size_t* offsets,
+                                       cudaStream_t st) {
+  if (njobs < 1 || njobs > LT_MAX_JOBS) return cudaErrorInvalidValue;
   if (!init_device()) return cudaErrorNotSupported;
   if (!status) status = library_status_word();
   if (!status) return cudaErrorNotSupported;
   const int rpg = rows_per_group > 0 ? rows_per_group : M;
   const int groups = M / rpg;
+  const int C = jobs[0].C;
   const int ctiles = (C + LT_C - 1) / LT_C;
-  // as many chunks per group as keep the grid within one resident wave (2 CTAs per SM on 148 SMs),
-  // every chunk a whole number of 128-row blocks
-  int s = 296 / (ctiles * groups);
-  if (s < 1) s = 1;
-  if (s > rpg / 128) s = rpg / 128;
-  while (rpg % (s * 128) != 0) --s;
-  CUtensorMap mZ, mW;
-  if (!make_map(&mZ, (const bf16*)Z + zcol0, (uint64_t)M, (uint64_t)C, (uint64_t)ldz)) return cudaErrorInvalidValue;
-  if (!make_map(&mW, Wt, (uint64_t)M, (uint64_t)ldwt, (uint64_t)ldwt)) return cudaErrorInvalidValue;
-  LgParams p;
-  p.C = C; p.rows_per_chunk = rpg / s; p.R = nt * r; p.r = r; p.rp = rp; p.wsel0 = wcol0 % LT_N;
-  p.partial = partial; p.status = status;
-  dim3 grid(ctiles, groups * s);
-  lora_grad_tc_kernel<<<grid, LT_THREADS, LT_SMEM, st>>>(mZ, mW, p, wcol0 - p.wsel0);
+  const int s = pick_chunks(ctiles * groups * njobs, rpg);
+  LgBatch bt;
+  size_t off = 0;
+  for (int j = 0; j < njobs; ++j) {
+    const LoraGradJob& jb = jobs[j];
+    if (jb.C != C) return cudaErrorInvalidValue;
+    if (!make_map(&bt.mapZ[j], (const bf16*)jb.Z + jb.zcol0, (uint64_t)M, (uint64_t)C, (uint64_t)jb.ldz)) return cudaErrorInvalidValue;
+    if (!make_map(&bt.mapW[j], jb.Wt, (uint64_t)M, (uint64_t)jb.ldwt, (uint64_t)jb.ldwt)) return cudaErrorInvalidValue;
+    LgParams& p = bt.p[j];
+    p.C = C; p.rows_per_chunk = rpg / s; p.R = jb.nt * jb.r; p.r = jb.r; p.rp = jb.rp; p.wsel0 = jb.wcol0 % LT_N;
+    p.partial = partial + off; p.status = status;
+    bt.wx0[j] = jb.wcol0 - p.wsel0;
+    offsets[j] = off;
+    off += (size_t)groups * s * p.R * C;
+  }
+  if (off > partial_floats) return cudaErrorInvalidValue;
+  for (int j = njobs; j < LT_MAX_JOBS; ++j) { bt.mapZ[j] = bt.mapZ[0]; bt.mapW[j] = bt.mapW[0]; bt.p[j] = bt.p[0]; bt.wx0[j] = bt.wx0[0]; }
+  dim3 grid(ctiles, groups * s, njobs);
+  lora_grad_tc_kernel<<<grid, LT_THREADS, LT_SMEM, st>>>(bt);
   *chunks_per_group = s;
   return cudaGetLastError();
+}
+
+cudaError_t lora_grad_tc_partial(const void* Z, int64_t ldz, int zcol0, int C, const void* Wt, int64_t ldwt, int wcol0,
+                                 int r, int rp, int nt, int M, int rows_per_group, float* partial, int* status,
+                                 int* chunks_per_group, cudaStream_t st) {
+  LoraGradJob jb;
+  jb.Z = Z; jb.ldz = ldz; jb.zcol0 = zcol0; jb.C = C; jb.Wt = Wt; jb.ldwt = ldwt; jb.wcol0 = wcol0; jb.r = r; jb.rp = rp; jb.nt = nt;
+  size_t off;
+  return lora_grad_tc_partial_batch(&jb, 1, M, rows_per_group, partial, (size_t)-1, status, chunks_per_group, &off, st);
 }
 
 }  // namespace sl

@@ -100,6 +100,7 @@ struct splitlora_ctx {
   void *emb = nullptr, *u2 = nullptr, *act = nullptr, *xf = nullptr, *logits = nullptr;
   float *meanf = nullptr, *rstdf = nullptr, *row_loss = nullptr, *rowdot = nullptr, *loss_dev = nullptr,
         *grad_scratch = nullptr;
+  size_t grad_scratch_floats = 0;
   int *n_valid = nullptr, *status = nullptr;
   void *g_a = nullptr, *g_b = nullptr, *g_dz = nullptr, *g_du2 = nullptr, *g_dxmid = nullptr, *g_do = nullptr,
        *g_dqkv = nullptr, *g_dhcat = nullptr, *g_du = nullptr, *g_dhcat_o = nullptr;
@@ -244,7 +245,8 @@ size_t plan(splitlora_ctx* c, char* ws) {
   c->xf = a.take(M * d * es); c->logits = a.take(M * (size_t)c->Vpad * es);
   c->meanf = (float*)a.take(M * 4); c->rstdf = (float*)a.take(M * 4); c->row_loss = (float*)a.take(M * 4);
   c->rowdot = (float*)a.take((size_t)c->nseq * c->cfg.n_head * c->cfg.seq * 4);
-  c->grad_scratch = (float*)a.take(lora_grad_scratch_floats(c->M, c->nq * c->r, c->d) * 4);
+  c->grad_scratch_floats = lora_grad_scratch_floats(c->M, c->nq * c->r, c->d);
+  c->grad_scratch = (float*)a.take(c->grad_scratch_floats * 4);
   if (c->has_o) c->g_dhcat_o = a.take(M * ext_o * es);
   c->g_a = a.take(M * d * es); c->g_b = a.take(M * d * es); c->g_dz = a.take(M * Fz * es);
   c->g_du2 = a.take(M * d * es); c->g_dxmid = a.take(M * d * es); c->g_do = a.take(M * d * es);
@@ -535,16 +537,22 @@ cudaError_t block_backward(splitlora_ctx* c, int l, const Span& sp, const void* 
     }
     if ((e = linear(c, "lora_down_bwd", a))) return e;
   }
-  // G_A = dh^T u, G_B = (alpha/r) dy^T h, per group (Eq. 4-7)
-  { Scope s(c, "lora_grad", 2);   // every qkv target's G_A in one pass over u
-    if ((e = lora_grad(c->dt, u, d, 0, d, c->g_dhcat, ext, 0, c->r, c->rp, c->nq, M, rpg, 1.0f, gbase,
-                       gstride, (int64_t)2 * c->r * d, d, 1, c->grad_scratch, c->st, c->status, c->tc))) return e; }
-  for (int t = 0; t < c->nq; ++t) {
-    float* gB = gbase + (size_t)t * 2 * c->r * d + (size_t)c->r * d;
+  // G_A = dh^T u (every qkv target in one pass over u) and G_B = (alpha/r) dy^T h of each target, per
+  // group (Eq. 4-7): one batch, i.e. one pair of launches where the tensor-core path applies
+  { LoraGradJob jobs[4];
+    int nj = 0;
+    LoraGradJob& ja = jobs[nj++];
+    ja.Z = u; ja.ldz = d; ja.zcol0 = 0; ja.C = d; ja.Wt = c->g_dhcat; ja.ldwt = ext; ja.wcol0 = 0; ja.r = c->r; ja.rp = c->rp;
+    ja.nt = c->nq; ja.scale = 1.0f; ja.out = gbase; ja.out_group_stride = gstride; ja.out_target_stride = (int64_t)2 * c->r * d;
+    ja.out_sj = d; ja.out_sc = 1;
+    for (int t = 0; t < c->nq; ++t) {
+      LoraGradJob& jb = jobs[nj++];
+      jb.Z = c->g_dqkv; jb.ldz = 3 * d; jb.zcol0 = c->slice_idx[t] * d; jb.C = d; jb.Wt = hcat; jb.ldwt = ext; jb.wcol0 = t * c->rp;
+      jb.r = c->r; jb.rp = c->rp; jb.nt = 1; jb.scale = c->scale; jb.out = gbase + (size_t)t * 2 * c->r * d + (size_t)c->r * d;
+      jb.out_group_stride = gstride; jb.out_target_stride = 0; jb.out_sj = 1; jb.out_sc = c->r;
+    }
     Scope s(c, "lora_grad", 2);
-    if ((e = lora_grad(c->dt, c->g_dqkv, 3 * d, c->slice_idx[t] * d, d, hcat, ext, t * c->rp, c->r, c->rp, 1, M,
-                       rpg, c->scale, gB, gstride, 0, 1, c->r, c->grad_scratch, c->st, c->status, c->tc))) return e;
-  }
+    if ((e = lora_grad_batch(c->dt, jobs, nj, M, rpg, c->grad_scratch, c->grad_scratch_floats, c->st, c->status, c->tc))) return e; }
   if (dx) {
     GemmArgs a = base_args(c, c->g_dqkv, 3 * d, f.qkvwT, 3 * d, c->g_du, d, M, d, 3 * d);
     a.rows_per_group = rpg;

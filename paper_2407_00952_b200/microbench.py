@@ -43,6 +43,27 @@ def _time(fn, iters, warmup=3):
     return e0.elapsed_time(e1) / iters
 
 
+def _time_graph(fn, iters, warmup=2):
+    """Like _time, with the `iters` calls captured in a CUDA graph and replayed: an operator call is half a
+    dozen launches from Python, which at small shapes takes the host longer to issue than the device to
+    run.  `fn` must allocate nothing."""
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(iters):
+            fn(i)
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
 def bench_linear_shape(M, n_in, n_out, rs, Gs, iters=10, backward=True, tc=True):
     """One (M, in, out) shape of the grouped LoRA linear for every rank in rs and group count in Gs.
     Forward, and the backward in its parts: the rank-r projections, dx, and dA + dB, each timed by itself
@@ -66,8 +87,8 @@ def bench_linear_shape(M, n_in, n_out, rs, Gs, iters=10, backward=True, tc=True)
             A = torch.randn(G, r, n_in, device="cuda", generator=g) * n_in ** -0.5
             Bm = torch.randn(G, n_out, r, device="cuda", generator=g) * r ** -0.5
             ws = B.lora_linear_workspace(B.DTYPE_BF16, M, n_in, n_out, r, G)
-            fwd = _time(lambda i: B.lora_linear_fwd(xs[i % nset], W, None, A, Bm, 16.0, y=ys[i % nset], workspace=ws,
-                                                    use_tensor_cores=tc), iters)
+            fwd = _time_graph(lambda i: B.lora_linear_fwd(xs[i % nset], W, None, A, Bm, 16.0, y=ys[i % nset], workspace=ws,
+                                                          use_tensor_cores=tc), iters)
             flops = 2.0 * M * n_in * n_out + 2.0 * M * r * (n_in + n_out)
             out = {"op": "lora_linear", "M": M, "n_in": n_in, "n_out": n_out, "r": r, "G": G, "buffer_sets": nset,
                    "fwd_us": round(fwd * 1e3, 1), "fwd_tflops": round(flops / fwd / 1e9, 1),
@@ -75,9 +96,9 @@ def bench_linear_shape(M, n_in, n_out, rs, Gs, iters=10, backward=True, tc=True)
             if backward:
                 dA = torch.empty(G, r, n_in, dtype=torch.float32, device="cuda")
                 dB = torch.empty(G, n_out, r, dtype=torch.float32, device="cuda")
-                run = lambda parts: _time(lambda i: B.lora_linear_bwd(xs[i % nset], Wt, dys[i % nset], A, Bm, 16.0, workspace=ws,
-                                                                      use_tensor_cores=tc, parts=parts,
-                                                                      out=(dxs[i % nset], dA, dB)), iters)
+                run = lambda parts: _time_graph(lambda i: B.lora_linear_bwd(xs[i % nset], Wt, dys[i % nset], A, Bm, 16.0,
+                                                                            workspace=ws, use_tensor_cores=tc, parts=parts,
+                                                                            out=(dxs[i % nset], dA, dB)), iters)
                 t_down = run(1)                       # h = x A^T and dh = s dy B: skinny, HBM-bound
                 t_dx = run(1 | 2) - t_down            # dx = dy W + dh A on the tensor cores
                 t_g = run(1 | 4) - t_down             # dA = dh^T x, dB = s dy^T h: skinny reductions over the tokens
