@@ -297,6 +297,14 @@ int splitlora_lora_linear_bwd(int dtype, int use_tensor_cores, const void* x, co
                               const float* A, const float* B, float alpha, int M, int n_in, int n_out,
                               int r, int G, void* dx, float* dA, float* dB,
                               void* workspace, size_t workspace_bytes, void* stream);
+/* The same forward in parts, so that they can be timed one by one: parts is a sum of 1 (the adapters'
+ * compute copies and the rank-r projection h = x A_g^T, left in the workspace) and 2 (the product with
+ * the frozen W with the rank-r term fused in; needs a preceding call with part 1 on the same workspace
+ * and operands).  parts = 3 is splitlora_lora_linear_fwd. */
+int splitlora_lora_linear_fwd_parts(int dtype, int use_tensor_cores, const void* x, const void* W, const void* bias,
+                                    const float* A, const float* B, float alpha, int M, int n_in, int n_out,
+                                    int r, int G, void* y, void* workspace, size_t workspace_bytes, void* stream,
+                                    int parts);
 /* The same backward in parts, so that they can be timed one by one: parts is a sum of 1 (the two rank-r
  * projections h = x A_g^T and dh = (alpha/r) dy B_g, which the other parts read from the workspace),
  * 2 (dx) and 4 (dA and dB).  Parts 2 and 4 need a preceding call with part 1 on the same workspace and

@@ -35,6 +35,7 @@ EXPORTS = [
     "splitlora_handoff_quantize",
     "splitlora_handoff_dequantize", "splitlora_round_compressed", "splitlora_set_client_ranks",
     "splitlora_library_status", "splitlora_set_client_cuts", "splitlora_lora_linear_bwd_parts",
+    "splitlora_lora_linear_fwd_parts",
 ]
 
 
@@ -322,7 +323,7 @@ def lora_linear_workspace(dtype: int, M, n_in, n_out, r, G) -> torch.Tensor:
     return torch.empty(n.value, dtype=torch.uint8, device="cuda")
 
 
-def lora_linear_fwd(x, W, bias, A, B, alpha, y=None, workspace=None, use_tensor_cores=True):
+def lora_linear_fwd(x, W, bias, A, B, alpha, y=None, workspace=None, use_tensor_cores=True, parts=3):
     lib = load()
     M, n_in = x.shape
     n_out = W.shape[0]
@@ -331,9 +332,9 @@ def lora_linear_fwd(x, W, bias, A, B, alpha, y=None, workspace=None, use_tensor_
         y = torch.empty(M, n_out, dtype=x.dtype, device="cuda")
     if workspace is None:
         workspace = lora_linear_workspace(_dt(x), M, n_in, n_out, r, G)
-    _rc(lib.splitlora_lora_linear_fwd(_dt(x), 1 if use_tensor_cores else 0, _ptr(x), _ptr(W), _ptr(bias), _ptr(A),
-                                      _ptr(B), C.c_float(alpha), M, n_in, n_out, r, G, _ptr(y), _ptr(workspace),
-                                      C.c_size_t(workspace.numel()), _stream_ptr()), "lora_linear_fwd")
+    _rc(lib.splitlora_lora_linear_fwd_parts(_dt(x), 1 if use_tensor_cores else 0, _ptr(x), _ptr(W), _ptr(bias), _ptr(A),
+                                            _ptr(B), C.c_float(alpha), M, n_in, n_out, r, G, _ptr(y), _ptr(workspace),
+                                            C.c_size_t(workspace.numel()), _stream_ptr(), int(parts)), "lora_linear_fwd")
     return y
 
 

@@ -1,8 +1,9 @@
 // Causal multi-head attention forward for heads of width 64 on the 5th-generation tensor cores
 // (tcgen05 + TMEM + TMA), bf16, sequence length a multiple of 128.
 //
-// Persistent CTAs, two per SM.  The work units are 128-row query tiles of (sequence, head) items, longest
-// first, dealt round-robin to the CTAs.  A query tile walks its keys in HALF-STEPS of 64 keys:
+// Persistent CTAs, two per SM.  The work units are 128-row query tiles of (sequence, head) items; the
+// tiles of one item run on neighbouring CTAs at about the same time (K and V come from memory once).
+// A query tile walks its keys in HALF-STEPS of 64 keys:
 //   S  = Q K^T      tcgen05.mma M128 N64 K16 x4 into one of two 64-column score buffers
 //   softmax         ONE thread per query row reads its 64 scores from tensor memory once, keeps them in
 //                   registers for the row maximum and the exponentials (no second read, no exchange
@@ -83,12 +84,16 @@ attn_fwd_t5_h64_kernel(const __grid_constant__ CUtensorMap mapQKV, F64Params p) 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nq = p.T / BQ;
-  // work units: (query tile, item) pairs in falling cost; this CTA takes units blockIdx.x + k * gridDim.x
-  const int n_units = p.nitems * nq;
-  const int my_tiles = (int)blockIdx.x < n_units ? (n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-  auto unit_of = [&](int tq) { return (int)blockIdx.x + tq * (int)gridDim.x; };
-  auto qt_of = [&](int tq) { return nq - 1 - unit_of(tq) / p.nitems; };
-  auto item_of = [&](int tq) { return unit_of(tq) % p.nitems; };
+  // Work units are (item, query tile) pairs.  The grid is a multiple of nq CTAs; in round t the CTAs
+  // nq*s .. nq*s + nq-1 take the nq query tiles of one item (s-th item of the round's block of items), so an
+  // item's K and V are read from memory once and found in L2 by its other tiles, which run at about the
+  // same time.  Which of the item's tiles a CTA takes rotates with the round, so that every CTA gets the
+  // same mix of long and short tiles.
+  const int ipb = (int)gridDim.x / nq;             // items per round
+  const int slot = (int)blockIdx.x / nq, pos = (int)blockIdx.x % nq;
+  const int my_tiles = (slot < ipb && slot < p.nitems) ? (p.nitems - slot + ipb - 1) / ipb : 0;
+  auto qt_of = [&](int tq) { return (pos + tq) % nq; };
+  auto item_of = [&](int tq) { return tq * ipb + slot; };
   auto head_of = [&](int tq) { return item_of(tq) % p.H; };
   auto row0_of = [&](int tq) { return (item_of(tq) / p.H) * p.T; };
 
@@ -368,8 +373,10 @@ cudaError_t attention_fwd_t5_h64(const void* qkv, int nseq, int T, int H, int d,
   F64Params p;
   p.T = T; p.H = H; p.d = d; p.scale_log2 = LOG2E / sqrtf((float)DH); p.o = (bf16*)o; p.lse = lse; p.status = status;
   p.nitems = nseq * H;
-  const int units = p.nitems * (T / BQ), cap = 2 * sms;
-  attn_fwd_t5_h64_kernel<<<units < cap ? units : cap, THREADS, SMEM, st>>>(mQKV, p);
+  const int nq = T / BQ, units = p.nitems * nq, cap = 2 * sms;
+  const int grid = ((units < cap ? units : cap) / nq) * nq;          // a multiple of nq: whole items per round
+  if (grid < nq) return cudaErrorInvalidValue;
+  attn_fwd_t5_h64_kernel<<<grid, THREADS, SMEM, st>>>(mQKV, p);
   return cudaGetLastError();
 }
 

@@ -89,8 +89,16 @@ static int make_copies(int dtype, const LinearPlan& p, const float* A, const flo
 int splitlora_lora_linear_fwd(int dtype, int use_tc, const void* x, const void* W, const void* bias, const float* A,
                               const float* B, float alpha, int M, int n_in, int n_out, int r, int G, void* y,
                               void* workspace, size_t workspace_bytes, void* stream) {
+  return splitlora_lora_linear_fwd_parts(dtype, use_tc, x, W, bias, A, B, alpha, M, n_in, n_out, r, G, y, workspace,
+                                         workspace_bytes, stream, 3);
+}
+
+int splitlora_lora_linear_fwd_parts(int dtype, int use_tc, const void* x, const void* W, const void* bias, const float* A,
+                                    const float* B, float alpha, int M, int n_in, int n_out, int r, int G, void* y,
+                                    void* workspace, size_t workspace_bytes, void* stream, int parts) {
   int rc = check_linear(dtype, M, n_in, n_out, r, G);
   if (rc) return rc;
+  if (parts < 1 || parts > 3) return SPLITLORA_ERR_ARG;
   if (!x || !W || !A || !B || !y || !workspace) return SPLITLORA_ERR_ARG;
   if (!aligned16(x) || !aligned16(W) || !aligned16(y) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return SPLITLORA_ERR_ALIGN;
   LinearPlan p = plan_linear(dtype, M, n_in, n_out, r, G);
@@ -98,13 +106,16 @@ int splitlora_lora_linear_fwd(int dtype, int use_tc, const void* x, const void* 
   cudaStream_t st = (cudaStream_t)stream;
   char* ws = (char*)workspace;
   if (gemm_tc_init() != 0) return SPLITLORA_ERR_CUDA;
-  if ((rc = make_copies(dtype, p, A, B, alpha, n_in, n_out, r, G, ws, true, st))) return rc;
   const int rpg = G > 1 ? M / G : 0;
   int* status = (int*)(ws + p.off_status);
-  GemmArgs h;
-  h.dtype = dtype; h.X = x; h.ldx = n_in; h.W = ws + p.off_acat; h.ldw = n_in; h.Y = ws + p.off_h; h.ldy = p.ext;
-  h.M = M; h.N = p.ext; h.K = n_in; h.rows_per_group = rpg; h.w_grouped = G > 1;
-  if (run_gemm(use_tc, h, status, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
+  if (parts & 1) {
+    if ((rc = make_copies(dtype, p, A, B, alpha, n_in, n_out, r, G, ws, true, st))) return rc;
+    GemmArgs h;
+    h.dtype = dtype; h.X = x; h.ldx = n_in; h.W = ws + p.off_acat; h.ldw = n_in; h.Y = ws + p.off_h; h.ldy = p.ext;
+    h.M = M; h.N = p.ext; h.K = n_in; h.rows_per_group = rpg; h.w_grouped = G > 1;
+    if (run_gemm(use_tc, h, status, st) != cudaSuccess) return SPLITLORA_ERR_CUDA;
+  }
+  if (!(parts & 2)) return SPLITLORA_OK;
   GemmArgs a;
   a.dtype = dtype; a.X = x; a.ldx = n_in; a.W = W; a.ldw = n_in; a.Y = y; a.ldy = n_out;
   a.M = M; a.N = n_out; a.K = n_in; a.bias = bias; a.rows_per_group = rpg;

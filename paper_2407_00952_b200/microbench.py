@@ -2,7 +2,8 @@
 the Eq. 8-9 aggregation and causal attention.  Prints one JSON line per case.
 
   python -m paper_2407_00952_b200.microbench linear --M 32768 --n-in 1024 --n-out 3072 --r 4 --G 8
-  python -m paper_2407_00952_b200.microbench linear-sweep [--quick]
+  python -m paper_2407_00952_b200.microbench linear-sweep [--quick] > sweep.jsonl
+  python -m paper_2407_00952_b200.microbench linear-sweep-table --file sweep.jsonl
   python -m paper_2407_00952_b200.microbench aggregate-sweep
   python -m paper_2407_00952_b200.microbench attention --nseq 64 --T 512 --heads 16
 
@@ -87,10 +88,13 @@ def bench_linear_shape(M, n_in, n_out, rs, Gs, iters=10, backward=True, tc=True)
             A = torch.randn(G, r, n_in, device="cuda", generator=g) * n_in ** -0.5
             Bm = torch.randn(G, n_out, r, device="cuda", generator=g) * r ** -0.5
             ws = B.lora_linear_workspace(B.DTYPE_BF16, M, n_in, n_out, r, G)
-            fwd = _time_graph(lambda i: B.lora_linear_fwd(xs[i % nset], W, None, A, Bm, 16.0, y=ys[i % nset], workspace=ws,
-                                                          use_tensor_cores=tc), iters)
-            flops = 2.0 * M * n_in * n_out + 2.0 * M * r * (n_in + n_out)
+            runf = lambda parts: _time_graph(lambda i: B.lora_linear_fwd(xs[i % nset], W, None, A, Bm, 16.0, y=ys[i % nset],
+                                                                         workspace=ws, use_tensor_cores=tc, parts=parts), iters)
+            f_down = runf(1)                          # compute copies of the adapters and h = x A^T: skinny, HBM-bound
+            fwd = runf(3) - f_down                    # y = x W^T + (alpha/r) h B^T on the tensor cores
+            flops = 2.0 * M * n_in * n_out + 2.0 * M * r * n_out
             out = {"op": "lora_linear", "M": M, "n_in": n_in, "n_out": n_out, "r": r, "G": G, "buffer_sets": nset,
+                   "fwd_down_us": round(f_down * 1e3, 1), "fwd_down_frac_of_hbm": round(2.0 * M * n_in / f_down / 1e6 / hbm, 3),
                    "fwd_us": round(fwd * 1e3, 1), "fwd_tflops": round(flops / fwd / 1e9, 1),
                    "fwd_frac_of_bf16_peak": round(flops / fwd / 1e9 / tflops, 3), "peak_source": src + " burst"}
             if backward:
@@ -289,10 +293,33 @@ def bench_ranks(config: int, steps: int):
     return rows
 
 
+def sweep_table(path):
+    """Markdown summary of a linear-sweep output file (one JSON line per case): per (M, in, out) shape the
+    range over ranks and group counts, and one shape in full."""
+    rows = [json.loads(l) for l in open(path) if l.strip().startswith("{")]
+    shapes = {}
+    for r in rows:
+        shapes.setdefault((r["M"], r["n_in"], r["n_out"]), []).append(r)
+    rng = lambda rs, k, f=1.0: f"{min(x[k] for x in rs) * f:.0f}-{max(x[k] for x in rs) * f:.0f}"
+    out = ["| M | in | out | fwd TF/s | fwd % of burst | dx TF/s | dx % of burst | rank-r projections % of HBM (fwd / bwd) | dA + dB % of HBM |",
+           "|---|---|---|---|---|---|---|---|---|"]
+    for (M, i, o), rs in sorted(shapes.items()):
+        out.append(f"| {M} | {i} | {o} | {rng(rs, 'fwd_tflops')} | {rng(rs, 'fwd_frac_of_bf16_peak', 100)} | "
+                   f"{rng(rs, 'dx_tflops')} | {rng(rs, 'dx_frac_of_bf16_peak', 100)} | "
+                   f"{rng(rs, 'fwd_down_frac_of_hbm', 100)} / {rng(rs, 'down_frac_of_hbm', 100)} | {rng(rs, 'dAdB_frac_of_hbm', 100)} |")
+    out += ["", "One shape in full (M 16384, 1024 -> 3072):", "",
+            "| r | G | fwd us | fwd TF/s | dx us | dx TF/s | rank-r fwd us | rank-r bwd us | dA + dB us | dA + dB GB/s |", "|---|---|---|---|---|---|---|---|---|---|"]
+    for r in sorted(shapes.get((16384, 1024, 3072), []), key=lambda x: (x["r"], x["G"])):
+        out.append(f"| {r['r']} | {r['G']} | {r['fwd_us']} | {r['fwd_tflops']} | {r['dx_us']} | {r['dx_tflops']} | {r['fwd_down_us']} | "
+                   f"{r['down_us']} | {r['dAdB_us']} | {r['dAdB_GBps']} |")
+    return "\n".join(out)
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["linear", "linear-sweep", "epilogues", "aggregate", "aggregate-sweep", "attention",
-                                     "split-sweep", "handoff", "ranks"])
+    ap.add_argument("what", choices=["linear", "linear-sweep", "linear-sweep-table", "epilogues", "aggregate", "aggregate-sweep",
+                                     "attention", "split-sweep", "handoff", "ranks"])
+    ap.add_argument("--file", default="", help="linear-sweep-table: the sweep's output file")
     ap.add_argument("--config", type=int, default=3)
     ap.add_argument("--M", type=int, default=32768)
     ap.add_argument("--n-in", type=int, default=1024)
@@ -309,6 +336,9 @@ def main():
     ap.add_argument("--no-backward", action="store_true")
     ap.add_argument("--quick", action="store_true")
     a = ap.parse_args()
+    if a.what == "linear-sweep-table":
+        print(sweep_table(a.file))
+        return
     if a.what == "linear":
         print(json.dumps(bench_linear(a.M, a.n_in, a.n_out, a.r, a.G, a.iters, not a.no_backward)))
     elif a.what == "linear-sweep":
