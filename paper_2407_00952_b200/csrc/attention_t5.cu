@@ -400,12 +400,12 @@ bool init_device() {
 }  // namespace
 
 bool attention_t5_supported(int dt, int T, int H, int d) {
-  return dt == DT_BF16 && H > 0 && d % H == 0 && d / H == 64 && T >= BQ && T % BQ == 0;
+  return dt == DT_BF16 && H > 0 && d % H == 0 && d / H == 64 && T >= BQ && T % BQ == 0 && T / BQ <= 64;
 }
 
 // The forward kernel also exists for heads of width 128 (the backward kernels do not).
 bool attention_fwd_t5_supported(int dt, int T, int H, int d) {
-  return dt == DT_BF16 && H > 0 && d % H == 0 && (d / H == 64 || d / H == 128) && T >= BQ && T % BQ == 0;
+  return dt == DT_BF16 && H > 0 && d % H == 0 && (d / H == 64 || d / H == 128) && T >= BQ && T % BQ == 0 && T / BQ <= 64;
 }
 
 cudaError_t attention_fwd_t5(const void* qkv, int nseq, int T, int H, int d, void* o, float* lse, int* status,

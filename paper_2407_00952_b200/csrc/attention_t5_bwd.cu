@@ -197,11 +197,14 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
   }
   T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, QD_EMPTY, QD_EMPTY + RINGN)
   const int nq = p.T / BT;
-  // persistent: the work units are (tile, item) pairs, item = (sequence, head), ordered by falling
-  // cost (the tile with the most steps of every item first); this CTA takes units blockIdx.x,
-  // blockIdx.x + gridDim.x, ..., so every CTA gets the same mix of long and short tiles, and every role
-  // walks its units in one flat loop, so loads for the next unit are issued while this one ends
-  const int my_tiles = (p.nitems * nq - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+  // persistent: the work units are (item, tile) pairs, item = (sequence, head).  The grid is a multiple of
+  // nq CTAs; in round t the CTAs nq*s .. nq*s + nq-1 take the nq tiles of one item (the s-th of the round's
+  // block of items), so an item's Q, K, V and dO are read from memory once and found in L2 by its other
+  // tiles, which run at about the same time; which tile a CTA takes rotates with the round, so that every
+  // CTA gets the same mix of long and short tiles.  Every role walks its units in one flat loop, so loads
+  // for the next unit are issued while this one ends.
+  const int ipb = (int)gridDim.x / nq, slot = (int)blockIdx.x / nq, pos = (int)blockIdx.x % nq;
+  const int my_tiles = (slot < ipb && slot < p.nitems) ? (p.nitems - slot + ipb - 1) / ipb : 0;
   const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDV = tmem_base + 256u, tDK = tmem_base + 256u + (uint32_t)DHT;
   // P^T, dS^T (bf16): 64 columns each after dK, or on top of S^T and dP^T
   const uint32_t tPT = ALIAS ? tS : tmem_base + 384u, tDST = ALIAS ? tDP : tmem_base + 448u;
@@ -211,7 +214,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       bool ok = true;
       int s = 0, n = 0;                            // ring stage and how often it has been used
       for (int tk = 0; tk < my_tiles && ok; ++tk) {
-        const int u = (int)blockIdx.x + tk * (int)gridDim.x, item = u % p.nitems, kt = u / p.nitems;
+        const int item = tk * ipb + slot, kt = (pos + tk) % nq;
         const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -253,7 +256,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       const uint32_t lo_kv = desc_lo(base + OFF_KV), lo_qd = desc_lo(base + OFF_QD);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int tk = 0; tk < my_tiles && ok; ++tk) {
-        const int u = (int)blockIdx.x + tk * (int)gridDim.x, item = u % p.nitems, kt = u / p.nitems;
+        const int item = tk * ipb + slot, kt = (pos + tk) % nq;
         const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -292,7 +295,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       const uint32_t lo_qd = desc_lo(base + OFF_QD);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int tk = 0; tk < my_tiles && ok; ++tk) {
-        const int u = (int)blockIdx.x + tk * (int)gridDim.x, item = u % p.nitems, kt = u / p.nitems;
+        const int item = tk * ipb + slot, kt = (pos + tk) % nq;
         const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -330,7 +333,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     bool ok = true;
     int it = 0, s = 0, n = 0;
     for (int tk = 0; tk < my_tiles; ++tk) {
-      const int u = (int)blockIdx.x + tk * (int)gridDim.x, item = u % p.nitems, kt = u / p.nitems;
+      const int item = tk * ipb + slot, kt = (pos + tk) % nq;
       const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
       const int seq_row0 = b * p.T;
       const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -406,7 +409,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     bool ok = true;
     for (int tk = 0; tk < my_tiles; ++tk) {
-      const int u = (int)blockIdx.x + tk * (int)gridDim.x, item = u % p.nitems, kt = u / p.nitems;
+      const int item = tk * ipb + slot, kt = (pos + tk) % nq;
       const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
       const int seq_row0 = b * p.T;
       const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -497,11 +500,14 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
   constexpr bool HAS_O = C::HAS_O;
   T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, KV_EMPTY, KV_EMPTY + RINGN)
   const int nq = p.T / BT;
-  // persistent: the work units are (tile, item) pairs, item = (sequence, head), ordered by falling
-  // cost (the tile with the most steps of every item first); this CTA takes units blockIdx.x,
-  // blockIdx.x + gridDim.x, ..., so every CTA gets the same mix of long and short tiles, and every role
-  // walks its units in one flat loop, so loads for the next unit are issued while this one ends
-  const int my_tiles = (p.nitems * nq - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+  // persistent: the work units are (item, tile) pairs, item = (sequence, head).  The grid is a multiple of
+  // nq CTAs; in round t the CTAs nq*s .. nq*s + nq-1 take the nq tiles of one item (the s-th of the round's
+  // block of items), so an item's Q, K, V and dO are read from memory once and found in L2 by its other
+  // tiles, which run at about the same time; which tile a CTA takes rotates with the round, so that every
+  // CTA gets the same mix of long and short tiles.  Every role walks its units in one flat loop, so loads
+  // for the next unit are issued while this one ends.
+  const int ipb = (int)gridDim.x / nq, slot = (int)blockIdx.x / nq, pos = (int)blockIdx.x % nq;
+  const int my_tiles = (slot < ipb && slot < p.nitems) ? (p.nitems - slot + ipb - 1) / ipb : 0;
   const uint32_t tS = tmem_base, tDP = tmem_base + 128u, tDQ = tmem_base + 256u;      // dQ: DHT columns
   const uint32_t tDS = tmem_base + 256u + (uint32_t)DHT;               // dS: bf16, 64 columns
 
@@ -511,7 +517,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       bool ok = true;
       int s = 0, n = 0;
       for (int tq = 0; tq < my_tiles && ok; ++tq) {
-        const int u = (int)blockIdx.x + tq * (int)gridDim.x, item = u % p.nitems, qi = u / p.nitems;
+        const int item = tq * ipb + slot, qi = (pos + tq) % nq;
         const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -547,7 +553,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       const uint32_t lo_qo = desc_lo(base + OFF_QO), lo_kv = desc_lo(base + OFF_KV);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int tq = 0; tq < my_tiles && ok; ++tq) {
-        const int u = (int)blockIdx.x + tq * (int)gridDim.x, item = u % p.nitems, qi = u / p.nitems;
+        const int item = tq * ipb + slot, qi = (pos + tq) % nq;
         const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -585,7 +591,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       const uint32_t lo_kv = desc_lo(base + OFF_KV);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int tq = 0; tq < my_tiles && ok; ++tq) {
-        const int u = (int)blockIdx.x + tq * (int)gridDim.x, item = u % p.nitems, qi = u / p.nitems;
+        const int item = tq * ipb + slot, qi = (pos + tq) % nq;
         const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
         const int seq_row0 = b * p.T;
         const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -620,7 +626,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
     bool ok = true;
     int it = 0;
     for (int tq = 0; tq < my_tiles; ++tq) {
-      const int u = (int)blockIdx.x + tq * (int)gridDim.x, item = u % p.nitems, qi = u / p.nitems;
+      const int item = tq * ipb + slot, qi = (pos + tq) % nq;
       const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
       const int seq_row0 = b * p.T;
       const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -700,7 +706,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     bool ok = true;
     for (int tq = 0; tq < my_tiles; ++tq) {
-      const int u = (int)blockIdx.x + tq * (int)gridDim.x, item = u % p.nitems, qi = u / p.nitems;
+      const int item = tq * ipb + slot, qi = (pos + tq) % nq;
       const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
       const int seq_row0 = b * p.T;
       const size_t stat0 = ((size_t)b * p.H + h) * p.T;
@@ -781,7 +787,8 @@ cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, c
   p.T = T; p.H = H; p.d = d; p.scale = 1.0f / sqrtf((float)DH); p.lse = lse; p.rowdot = rowdot; p.rowdot_out = rowdot;
   p.status = status;
   p.nitems = nseq * H;
-  dim3 grid((unsigned)(p.nitems < sms ? p.nitems : sms));     // one persistent CTA per SM
+  const int nq = T / BT, units = p.nitems * nq;
+  dim3 grid((unsigned)(((units < sms ? units : sms) / nq) * nq));   // one persistent CTA per SM, whole items per round
   // dQ first: it leaves D[row] = sum(dO * O) in `rowdot` for the dK/dV kernel
   attn_bwd_dq_t5_kernel<64><<<grid, NTHREADS, dq::Cfg<64>::SMEM, st>>>(mQKV, mDO, mO, mDQKV, p);
   attn_bwd_dkv_t5_kernel<64><<<grid, NTHREADS, dkv::Cfg<64>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
@@ -790,7 +797,7 @@ cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, c
 
 // Heads of width 128: D[row] = sum(dO * O) must already be in `rowdot` (both kernels read it).
 bool attention_bwd_t5_128_supported(int dt, int T, int H, int d) {
-  return dt == DT_BF16 && H > 0 && d % H == 0 && d / H == 128 && T >= BT && T % BT == 0;
+  return dt == DT_BF16 && H > 0 && d % H == 0 && d / H == 128 && T >= BT && T % BT == 0 && T / BT <= 64;
 }
 
 cudaError_t attention_bwd_t5_128(const void* qkv, const float* lse, const void* d_o, const float* rowdot, int nseq,
@@ -809,7 +816,8 @@ cudaError_t attention_bwd_t5_128(const void* qkv, const float* lse, const void* 
   p.T = T; p.H = H; p.d = d; p.scale = 1.0f / sqrtf(128.0f); p.lse = lse; p.rowdot = rowdot; p.rowdot_out = nullptr;
   p.status = status;
   p.nitems = nseq * H;
-  dim3 grid((unsigned)(p.nitems < sms ? p.nitems : sms));
+  const int nq = T / BT, units = p.nitems * nq;
+  dim3 grid((unsigned)(((units < sms ? units : sms) / nq) * nq));
   attn_bwd_dq_t5_kernel<128><<<grid, NTHREADS, dq::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDO /* unused */, mDQKV, p);
   attn_bwd_dkv_t5_kernel<128><<<grid, NTHREADS, dkv::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
   return cudaGetLastError();

@@ -188,6 +188,7 @@ LINEAR_CASES = [
     (2048, 1024, 1000, 8, 8),
     (1024, 512, 72, 1, 1),
     (2048, 1024, 4096, 64, 4),
+    (4096, 768, 768, 8, 16),
 ]
 
 
@@ -273,12 +274,13 @@ def test_attention_bf16(nseq, T, Hh, d, use_tc):
     assert B.library_status() == 0          # no bounded wait of the stand-alone kernels expired
 
 
-@pytest.mark.parametrize("Hh,d", [(2, 128), (2, 256)])
-def test_attention_bf16_peaked_scores(Hh, d):
+@pytest.mark.parametrize("Hh,d,T", [(2, 128, 512), (2, 256, 512), (2, 128, 1024)])
+def test_attention_bf16_peaked_scores(Hh, d, T):
     """Scores with a standard deviation of about 6 and a drift along the keys: the row maximum keeps
-    moving from key tile to key tile (the running rescale of O and of the row sum does real work),
-    most probabilities underflow, a few carry the row."""
-    nseq, T = 2, 512
+    moving from key tile to key tile (the running rescale of O and of the row sum does real work, also in
+    the kernel that rescales only when the maximum has moved by more than 2^8: with this spread it does so
+    several times per row), most probabilities underflow, a few carry the row."""
+    nseq = 2
     g = torch.Generator(device="cpu").manual_seed(d)
     dh = d // Hh
     qkv = torch.randn(nseq * T, 3 * d, generator=g)
