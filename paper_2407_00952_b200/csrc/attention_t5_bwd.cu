@@ -44,6 +44,11 @@ constexpr uint32_t IDESC_64KK = make_idesc(BT, DH);                   // [128 x 
 constexpr uint32_t IDESC_64MN = make_idesc(BT, DH) | (1u << 16);      // [128 x 64] products, right operand MN-major
 constexpr float LOG2E = 1.4426950408889634f;
 
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -330,6 +335,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     const int r = q4 * 32 + lane;                // key row inside the tile = accumulator lane
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     const float scale_log2 = p.scale * LOG2E;
+    const uint64_t sc2 = pack2(scale_log2, scale_log2), nlog2 = pack2(-LOG2E, -LOG2E), neg1 = pack2(-1.f, -1.f);
     bool ok = true;
     int it = 0, s = 0, n = 0;
     for (int tk = 0; tk < my_tiles; ++tk) {
@@ -360,6 +366,10 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
             tc_ld32(tS + lane_off + (uint32_t)c, sv);
             tc_ld32(tDP + lane_off + (uint32_t)c, dv);
             tc_wait_ld();
+            if (!ALIAS) {                              // the values are in registers: this half of S^T, dP^T
+              tc_fence_before();                       // may be overwritten by the next step's products
+              mbar_arrive(B(S_FREE + hh));
+            }
             // The causal mask goes onto the scores first (exp2(-inf) = 0), so that the element loop
             // below has no test in it: with one, every element is a basic block of its own and the
             // 32 independent chains run one after another instead of interleaved.
@@ -369,15 +379,18 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
             }
 #pragma unroll
             for (int e = 0; e < 32; e += 4) {
-              const float4 l4 = *reinterpret_cast<const float4*>(Ls + c + e);
-              const float4 d4 = *reinterpret_cast<const float4*>(Ds + c + e);
-              const float p0 = ex2(fmaf(sv[e], scale_log2, -l4.x * LOG2E));
-              const float p1 = ex2(fmaf(sv[e + 1], scale_log2, -l4.y * LOG2E));
-              const float p2 = ex2(fmaf(sv[e + 2], scale_log2, -l4.z * LOG2E));
-              const float p3 = ex2(fmaf(sv[e + 3], scale_log2, -l4.w * LOG2E));
+              // two elements per instruction: the row statistics come out of shared memory as pairs
+              const ulonglong2 l4 = *reinterpret_cast<const ulonglong2*>(Ls + c + e);
+              const ulonglong2 d4 = *reinterpret_cast<const ulonglong2*>(Ds + c + e);
+              float a0, a1, a2, a3;
+              unpack2(fma2(pack2(sv[e], sv[e + 1]), sc2, mul2(l4.x, nlog2)), a0, a1);
+              unpack2(fma2(pack2(sv[e + 2], sv[e + 3]), sc2, mul2(l4.y, nlog2)), a2, a3);
+              const float p0 = ex2(a0), p1 = ex2(a1), p2 = ex2(a2), p3 = ex2(a3);
+              float g0, g1, g2, g3;
+              unpack2(mul2(pack2(p0, p1), fma2(d4.x, neg1, pack2(dv[e], dv[e + 1]))), g0, g1);
+              unpack2(mul2(pack2(p2, p3), fma2(d4.y, neg1, pack2(dv[e + 2], dv[e + 3]))), g2, g3);
               __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
-              __nv_bfloat162 da = __floats2bfloat162_rn(p0 * (dv[e] - d4.x), p1 * (dv[e + 1] - d4.y));
-              __nv_bfloat162 db = __floats2bfloat162_rn(p2 * (dv[e + 2] - d4.z), p3 * (dv[e + 3] - d4.w));
+              __nv_bfloat162 da = __floats2bfloat162_rn(g0, g1), db = __floats2bfloat162_rn(g2, g3);
               pk[e >> 1] = *reinterpret_cast<uint32_t*>(&pa);
               pk[(e >> 1) + 1] = *reinterpret_cast<uint32_t*>(&pb);
               dk[e >> 1] = *reinterpret_cast<uint32_t*>(&da);
@@ -386,6 +399,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
           } else {
 #pragma unroll
             for (int e = 0; e < 16; ++e) { pk[e] = 0u; dk[e] = 0u; }
+            if (!ALIAS) mbar_arrive(B(S_FREE + hh));
           }
           // 32 bf16 = 16 columns: packed side by side, or over the first half of the chunk just read
           const uint32_t pcol = ALIAS ? (uint32_t)c : (uint32_t)(c >> 1);
@@ -393,7 +407,6 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
           tc_st16(tDST + lane_off + pcol, dk);
           tc_wait_st();
           tc_fence_before();
-          if (!ALIAS) mbar_arrive(B(S_FREE + hh));     // this half of S^T, dP^T may be overwritten
           mbar_arrive(B(P_READY + hh));                // this half of P^T, dS^T is complete
         }
         if (!ok) break;
@@ -623,6 +636,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
     const int r = q4 * 32 + lane;                // query row inside the tile
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     const float scale_log2 = p.scale * LOG2E;
+    const uint64_t sc2 = pack2(scale_log2, scale_log2);
     bool ok = true;
     int it = 0;
     for (int tq = 0; tq < my_tiles; ++tq) {
@@ -660,6 +674,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
           if (wsel == 0) p.rowdot_out[stat0 + (size_t)i * BT + r] = Dr;
         }
       }
+      const uint64_t nl2 = pack2(-L2, -L2), nd2 = pack2(-Dr, -Dr);
       for (int j = 0; j <= i && ok; ++j, ++it) {
         const bool diag = (j == i);
         // on the diagonal tile only keys <= this query count: chunks wholly after the warp's rows are zero
@@ -676,24 +691,29 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
             tc_ld32(tS + lane_off + (uint32_t)c, sv);
             tc_ld32(tDP + lane_off + (uint32_t)c, dv);
             tc_wait_ld();
+            tc_fence_before();                  // the values are in registers: the next step's products
+            mbar_arrive(B(S_FREE + hh));        // may overwrite this half of S and dP
             if (diag && c == c_last) {          // mask on the scores: the element loop stays free of tests
 #pragma unroll
               for (int e = 0; e < 32; ++e) sv[e] = (c + e > r) ? -INFINITY : sv[e];
             }
 #pragma unroll
             for (int e = 0; e < 32; e += 2) {
-              const float p0 = ex2(fmaf(sv[e], scale_log2, -L2)), p1 = ex2(fmaf(sv[e + 1], scale_log2, -L2));
-              __nv_bfloat162 db = __floats2bfloat162_rn(p0 * (dv[e] - Dr), p1 * (dv[e + 1] - Dr));
+              float a0, a1, g0, g1;
+              unpack2(fma2(pack2(sv[e], sv[e + 1]), sc2, nl2), a0, a1);
+              const float p0 = ex2(a0), p1 = ex2(a1);
+              unpack2(mul2(pack2(p0, p1), add2(pack2(dv[e], dv[e + 1]), nd2)), g0, g1);
+              __nv_bfloat162 db = __floats2bfloat162_rn(g0, g1);
               dk[e >> 1] = *reinterpret_cast<uint32_t*>(&db);
             }
           } else {
 #pragma unroll
             for (int e = 0; e < 16; ++e) dk[e] = 0u;
+            mbar_arrive(B(S_FREE + hh));
           }
           tc_st16(tDS + lane_off + (uint32_t)(c >> 1), dk);
           tc_wait_st();
           tc_fence_before();
-          mbar_arrive(B(S_FREE + hh));
           mbar_arrive(B(P_READY + hh));
         }
         if (!ok) break;
