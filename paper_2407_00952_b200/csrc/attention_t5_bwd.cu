@@ -34,11 +34,21 @@ using namespace tc;
 constexpr int DH = 64;
 constexpr int BT = 128;                   // rows of a query tile and of a key tile
 constexpr int TILE = BT * DH * 2;         // 16 KB: one [128 x 64] bf16 tile
-constexpr int NTHREADS = 480;             // TMA warp, two MMA-issuing warps (1 and 10), 8 element-wise warps, 4 output warps
-constexpr int OUT_WARP0 = 11;             // warps 11..14 move finished accumulators to global memory
 constexpr int OUT_THREADS = 128;
-constexpr int ACC_WARP = 10;              // issues the products that accumulate dK, dV / dQ
-constexpr int EW_THREADS = 256;           // two warps per accumulator lane quarter, 64 columns each
+// Warp roles: warp 0 TMA, warp 1 score products, then the element-wise warps (EWQ per accumulator lane
+// quarter, each computing CW of a half's 64 columns), one warp for the accumulating products, and four
+// output warps that move finished accumulators to global memory.  Head width 64 takes four
+// element-wise warps per quarter: the element-wise work is a chain of dependent instructions per element,
+// and two warps per scheduler left it waiting on its own latencies for half of the time.  Head width 128
+// keeps two (P^T and dS^T are written over the score columns there, chunk by chunk of 32).
+template <int DHT> struct Roles {
+  static constexpr int EWQ = DHT == 64 ? 4 : 2;
+  static constexpr int CW = 64 / EWQ;
+  static constexpr int EW_THREADS = 128 * EWQ;
+  static constexpr int ACC_WARP = 2 + 4 * EWQ;
+  static constexpr int OUT_WARP0 = ACC_WARP + 1;
+  static constexpr int NTHREADS = (OUT_WARP0 + 4) * 32;
+};
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t IDESC_64KK = make_idesc(BT, DH);                   // [128 x 64] products, both operands K-major
 constexpr uint32_t IDESC_64MN = make_idesc(BT, DH) | (1u << 16);      // [128 x 64] products, right operand MN-major
@@ -48,6 +58,28 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
   uint64_t d;
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
+}
+// 16 consecutive tensor-memory columns of this thread's lane
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+// 8 packed words of this thread's lane to 8 consecutive tensor-memory columns
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t* w) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+      ::"r"(taddr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
+template <int CW> __device__ __forceinline__ void tc_ld_cw(uint32_t taddr, float* v) {
+  if constexpr (CW == 32) tc_ld32(taddr, v); else tc_ld16(taddr, v);
+}
+template <int CW> __device__ __forceinline__ void tc_st_cw(uint32_t taddr, const uint32_t* w) {   // CW / 2 packed words
+  if constexpr (CW == 32) tc_st16(taddr, w); else tc_st8(taddr, w);
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -182,11 +214,13 @@ template <int DHT> struct Cfg {
 }  // namespace dkv
 
 template <int DHT>
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __launch_bounds__(Roles<DHT>::NTHREADS, 1)
 attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
                        const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dkv;
   using C = Cfg<DHT>;
+  constexpr int CW = Roles<DHT>::CW, EW_THREADS = Roles<DHT>::EW_THREADS, ACC_WARP = Roles<DHT>::ACC_WARP,
+                OUT_WARP0 = Roles<DHT>::OUT_WARP0;
   constexpr int NB = C::NB, KVB = C::KVB, RINGN = C::RINGN, OFF_KV = C::OFF_KV, OFF_QD = C::OFF_QD, OFF_OUT = C::OFF_OUT,
                 OFF_STAT = C::OFF_STAT, OFF_BAR = C::OFF_BAR;
   constexpr bool ALIAS = C::ALIAS;
@@ -331,7 +365,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
   } else if (warp < ACC_WARP) {
     // ---------------- element-wise warps 2..9 ----------------
     const int q4 = warp & 3;
-    const int wsel = (warp - 2) >> 2;            // which of the two warps of this accumulator lane quarter
+    const int wsel = (warp - 2) >> 2;            // which of the EWQ warps of this accumulator lane quarter
     const int r = q4 * 32 + lane;                // key row inside the tile = accumulator lane
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     const float scale_log2 = p.scale * LOG2E;
@@ -349,22 +383,21 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
         const float* Ds = Ls + 128;
         if (!mbar_wait(B(QD_FULL + s), done(n), abort_flag, p.status, 48)) { ok = false; break; }
         const bool diag = (i == kt);
-        // on the diagonal tile only queries >= this key count: chunks wholly before the warp's rows are zero
-        const int c_first = diag ? q4 * 32 : 0;
-        // The 128 query columns go in two halves of 64 (one 32-column chunk per warp and half): the
+        // The 128 query columns go in two halves of 64 (one CW-column chunk per warp and half): the
         // products that contract over the first half run while the second half is being computed.
 #pragma unroll 1
         for (int hh = 0; hh < 2; ++hh) {
-          const int c = hh * 64 + wsel * 32;
+          const int c = hh * 64 + wsel * CW;
           if (!mbar_wait(B(S_FULL + hh), done(it), abort_flag, p.status, 49)) { ok = false; break; }
           // (with P^T on top of S^T, S_FULL already implies that the previous step's products are done)
           if (!ALIAS && !mbar_wait(B(P_FREE + hh), freed(it), abort_flag, p.status, 50)) { ok = false; break; }
           tc_fence_after();
-          uint32_t pk[16], dk[16];
-          if (c >= c_first) {
-            float sv[32], dv[32];
-            tc_ld32(tS + lane_off + (uint32_t)c, sv);
-            tc_ld32(tDP + lane_off + (uint32_t)c, dv);
+          uint32_t pk[CW / 2], dk[CW / 2];
+          // on the diagonal tile only queries >= this key count: chunks wholly before the warp's rows are zero
+          if (!diag || c + CW > q4 * 32) {
+            float sv[CW], dv[CW];
+            tc_ld_cw<CW>(tS + lane_off + (uint32_t)c, sv);
+            tc_ld_cw<CW>(tDP + lane_off + (uint32_t)c, dv);
             tc_wait_ld();
             if (!ALIAS) {                              // the values are in registers: this half of S^T, dP^T
               tc_fence_before();                       // may be overwritten by the next step's products
@@ -372,13 +405,13 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
             }
             // The causal mask goes onto the scores first (exp2(-inf) = 0), so that the element loop
             // below has no test in it: with one, every element is a basic block of its own and the
-            // 32 independent chains run one after another instead of interleaved.
-            if (diag && c == c_first) {
+            // independent chains run one after another instead of interleaved.
+            if (diag && c < q4 * 32 + 32) {
 #pragma unroll
-              for (int e = 0; e < 32; ++e) sv[e] = (c + e < r) ? -INFINITY : sv[e];
+              for (int e = 0; e < CW; ++e) sv[e] = (c + e < r) ? -INFINITY : sv[e];
             }
 #pragma unroll
-            for (int e = 0; e < 32; e += 4) {
+            for (int e = 0; e < CW; e += 4) {
               // two elements per instruction: the row statistics come out of shared memory as pairs
               const ulonglong2 l4 = *reinterpret_cast<const ulonglong2*>(Ls + c + e);
               const ulonglong2 d4 = *reinterpret_cast<const ulonglong2*>(Ds + c + e);
@@ -398,13 +431,13 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
             }
           } else {
 #pragma unroll
-            for (int e = 0; e < 16; ++e) { pk[e] = 0u; dk[e] = 0u; }
+            for (int e = 0; e < CW / 2; ++e) { pk[e] = 0u; dk[e] = 0u; }
             if (!ALIAS) mbar_arrive(B(S_FREE + hh));
           }
-          // 32 bf16 = 16 columns: packed side by side, or over the first half of the chunk just read
+          // CW bf16 = CW / 2 columns: packed side by side, or over the first half of the chunk just read
           const uint32_t pcol = ALIAS ? (uint32_t)c : (uint32_t)(c >> 1);
-          tc_st16(tPT + lane_off + pcol, pk);
-          tc_st16(tDST + lane_off + pcol, dk);
+          tc_st_cw<CW>(tPT + lane_off + pcol, pk);
+          tc_st_cw<CW>(tDST + lane_off + pcol, dk);
           tc_wait_st();
           tc_fence_before();
           mbar_arrive(B(P_READY + hh));                // this half of P^T, dS^T is complete
@@ -503,11 +536,13 @@ template <int DHT> struct Cfg {
 }  // namespace dq
 
 template <int DHT>
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __launch_bounds__(Roles<DHT>::NTHREADS, 1)
 attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
                       const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dq;
   using C = Cfg<DHT>;
+  constexpr int CW = Roles<DHT>::CW, EW_THREADS = Roles<DHT>::EW_THREADS, ACC_WARP = Roles<DHT>::ACC_WARP,
+                OUT_WARP0 = Roles<DHT>::OUT_WARP0;
   constexpr int NB = C::NB, QOB = C::QOB, RINGN = C::RINGN, QO_TILES = C::QO_TILES, OFF_QO = C::OFF_QO, OFF_KV = C::OFF_KV,
                 OFF_OUT = C::OFF_OUT, OFF_BAR = C::OFF_BAR;
   constexpr bool HAS_O = C::HAS_O;
@@ -632,7 +667,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
   } else if (warp < ACC_WARP) {
     // ---------------- element-wise warps 2..9 ----------------
     const int q4 = warp & 3;
-    const int wsel = (warp - 2) >> 2;            // which of the two warps of this accumulator lane quarter
+    const int wsel = (warp - 2) >> 2;            // which of the EWQ warps of this accumulator lane quarter
     const int r = q4 * 32 + lane;                // query row inside the tile
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     const float scale_log2 = p.scale * LOG2E;
@@ -677,28 +712,27 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       const uint64_t nl2 = pack2(-L2, -L2), nd2 = pack2(-Dr, -Dr);
       for (int j = 0; j <= i && ok; ++j, ++it) {
         const bool diag = (j == i);
-        // on the diagonal tile only keys <= this query count: chunks wholly after the warp's rows are zero
-        const int c_last = diag ? q4 * 32 : BT - 32;
 #pragma unroll 1
         for (int hh = 0; hh < 2; ++hh) {
-          const int c = hh * 64 + wsel * 32;
+          const int c = hh * 64 + wsel * CW;
           if (!mbar_wait(B(S_FULL + hh), done(it), abort_flag, p.status, 68)) { ok = false; break; }
           if (!mbar_wait(B(P_FREE + hh), freed(it), abort_flag, p.status, 69)) { ok = false; break; }
           tc_fence_after();
-          uint32_t dk[16];
-          if (c <= c_last) {
-            float sv[32], dv[32];
-            tc_ld32(tS + lane_off + (uint32_t)c, sv);
-            tc_ld32(tDP + lane_off + (uint32_t)c, dv);
+          uint32_t dk[CW / 2];
+          // on the diagonal tile only keys <= this query count: chunks wholly after the warp's rows are zero
+          if (!diag || c < q4 * 32 + 32) {
+            float sv[CW], dv[CW];
+            tc_ld_cw<CW>(tS + lane_off + (uint32_t)c, sv);
+            tc_ld_cw<CW>(tDP + lane_off + (uint32_t)c, dv);
             tc_wait_ld();
             tc_fence_before();                  // the values are in registers: the next step's products
             mbar_arrive(B(S_FREE + hh));        // may overwrite this half of S and dP
-            if (diag && c == c_last) {          // mask on the scores: the element loop stays free of tests
+            if (diag && c + CW > q4 * 32 + 1) { // mask on the scores: the element loop stays free of tests
 #pragma unroll
-              for (int e = 0; e < 32; ++e) sv[e] = (c + e > r) ? -INFINITY : sv[e];
+              for (int e = 0; e < CW; ++e) sv[e] = (c + e > r) ? -INFINITY : sv[e];
             }
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) {
+            for (int e = 0; e < CW; e += 2) {
               float a0, a1, g0, g1;
               unpack2(fma2(pack2(sv[e], sv[e + 1]), sc2, nl2), a0, a1);
               const float p0 = ex2(a0), p1 = ex2(a1);
@@ -708,10 +742,10 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
             }
           } else {
 #pragma unroll
-            for (int e = 0; e < 16; ++e) dk[e] = 0u;
+            for (int e = 0; e < CW / 2; ++e) dk[e] = 0u;
             mbar_arrive(B(S_FREE + hh));
           }
-          tc_st16(tDS + lane_off + (uint32_t)(c >> 1), dk);
+          tc_st_cw<CW>(tDS + lane_off + (uint32_t)(c >> 1), dk);
           tc_wait_st();
           tc_fence_before();
           mbar_arrive(B(P_READY + hh));
@@ -810,8 +844,8 @@ cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, c
   const int nq = T / BT, units = p.nitems * nq;
   dim3 grid((unsigned)(((units < sms ? units : sms) / nq) * nq));   // one persistent CTA per SM, whole items per round
   // dQ first: it leaves D[row] = sum(dO * O) in `rowdot` for the dK/dV kernel
-  attn_bwd_dq_t5_kernel<64><<<grid, NTHREADS, dq::Cfg<64>::SMEM, st>>>(mQKV, mDO, mO, mDQKV, p);
-  attn_bwd_dkv_t5_kernel<64><<<grid, NTHREADS, dkv::Cfg<64>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
+  attn_bwd_dq_t5_kernel<64><<<grid, Roles<64>::NTHREADS, dq::Cfg<64>::SMEM, st>>>(mQKV, mDO, mO, mDQKV, p);
+  attn_bwd_dkv_t5_kernel<64><<<grid, Roles<64>::NTHREADS, dkv::Cfg<64>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
   return cudaGetLastError();
 }
 
@@ -838,8 +872,8 @@ cudaError_t attention_bwd_t5_128(const void* qkv, const float* lse, const void* 
   p.nitems = nseq * H;
   const int nq = T / BT, units = p.nitems * nq;
   dim3 grid((unsigned)(((units < sms ? units : sms) / nq) * nq));
-  attn_bwd_dq_t5_kernel<128><<<grid, NTHREADS, dq::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDO /* unused */, mDQKV, p);
-  attn_bwd_dkv_t5_kernel<128><<<grid, NTHREADS, dkv::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
+  attn_bwd_dq_t5_kernel<128><<<grid, Roles<128>::NTHREADS, dq::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDO /* unused */, mDQKV, p);
+  attn_bwd_dkv_t5_kernel<128><<<grid, Roles<128>::NTHREADS, dkv::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
   return cudaGetLastError();
 }
 
