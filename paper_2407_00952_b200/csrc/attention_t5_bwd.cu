@@ -47,8 +47,56 @@ template <int DHT> struct Roles {
   static constexpr int EW_THREADS = 128 * EWQ;
   static constexpr int ACC_WARP = 2 + 4 * EWQ;
   static constexpr int OUT_WARP0 = ACC_WARP + 1;
-  static constexpr int NTHREADS = (OUT_WARP0 + 4) * 32;
+  // Head width 64 folds the row statistics into the score products (see "augmented contraction" below);
+  // one more warp turns them into the operand rows that carries them.
+  static constexpr bool AUG = DHT == 64;
+  static constexpr int STAT_WARP = OUT_WARP0 + 4;               // dK/dV kernel only
+  static constexpr int NTHREADS_DQ = (OUT_WARP0 + 4) * 32;
+  static constexpr int NTHREADS_DKV = (OUT_WARP0 + 4 + (AUG ? 1 : 0)) * 32;
 };
+
+// Augmented contraction.  The element-wise threads need exp(scale * S - lse) and dP - D, where lse and D
+// belong to the query (a row of the dQ kernel's tiles, a column of the dK/dV kernel's).  Both shifts are
+// rank-one terms, so the tensor core adds them: each score product takes one more 16-deep step whose
+// operands are a constant tile of ones and a tile that holds, per query, -lse/scale and -D, each as a sum of
+// two bf16 values (hi + lo: the pair carries 16 mantissa bits, the products with 1 are exact and the
+// accumulation is fp32).  The accumulators then hold S - lse/scale and dP - D, and an element costs the
+// element-wise threads two multiplications, one exponential and the conversions.
+// These tiles are [128 rows x 16] bf16, K-major without swizzle: 8-row groups of 256 bytes, in a group the
+// 16-byte rows of columns 0..7 (128 bytes) and then those of columns 8..15.  Columns: 0, 1 = -lse/scale
+// (hi, lo), 2, 3 = -D (hi, lo), the rest zero; the constant tiles have ones in columns 0, 1 (for S) or 2, 3
+// (for dP).
+constexpr int AUG_TILE = 128 * 16 * 2;
+constexpr uint32_t DESC_HI_AUG = (uint32_t)(256 >> 4) | (1u << 14);           // 8-row groups 256 bytes apart, no swizzle
+__device__ __forceinline__ uint32_t desc_lo_aug(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | ((uint32_t)(128 >> 4) << 16); }
+__device__ __forceinline__ void tc_mma_aug(uint32_t d_tmem, uint32_t alo, uint32_t blo, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, 1, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(alo), "r"(blo), "r"(DESC_HI_AUG), "r"(idesc) : "memory");
+}
+// byte offset of row r's columns 0..7 inside such a tile
+__device__ __forceinline__ uint32_t aug_row(int r) { return (uint32_t)(r >> 3) * 256u + (uint32_t)(r & 7) * 16u; }
+// -x as hi + lo, two bf16 values in one word (hi in the low half)
+__device__ __forceinline__ uint32_t neg_split(float x) {
+  const __nv_bfloat16 hi = __float2bfloat16_rn(-x);
+  const __nv_bfloat16 lo = __float2bfloat16_rn(-x - __bfloat162float(hi));
+  return (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16);
+}
+// zeroes `bytes` of shared memory and writes the two constant tiles: ones in columns 0, 1 / in columns 2, 3
+__device__ __forceinline__ void aug_init(uint8_t* ones_s, uint8_t* ones_d, int rows, uint8_t* zero, int zero_bytes) {
+  for (int i = threadIdx.x; i < zero_bytes / 16; i += blockDim.x) reinterpret_cast<uint4*>(zero)[i] = make_uint4(0u, 0u, 0u, 0u);
+  for (int i = threadIdx.x; i < rows * 2; i += blockDim.x) {       // 16-byte pieces: row i / 2, columns 0..7 or 8..15
+    const int r = i >> 1;
+    const uint32_t off = aug_row(r) + (uint32_t)(i & 1) * 128u;
+    const uint32_t one2 = 0x3F803F80u;
+    *reinterpret_cast<uint4*>(ones_s + off) = make_uint4((i & 1) ? 0u : one2, 0u, 0u, 0u);
+    *reinterpret_cast<uint4*>(ones_d + off) = make_uint4(0u, (i & 1) ? 0u : one2, 0u, 0u);
+  }
+}
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t IDESC_64KK = make_idesc(BT, DH);                   // [128 x 64] products, both operands K-major
 constexpr uint32_t IDESC_64MN = make_idesc(BT, DH) | (1u << 16);      // [128 x 64] products, right operand MN-major
@@ -139,7 +187,7 @@ struct BwdParams {
   int* status;
 };
 
-#define T5_SETUP(NBARS, CNT128_A, CNT128_B, CNT128_C, CNT128_D, CNT_OUT, CNT2_LO, CNT2_HI)                                                     \
+#define T5_SETUP(NBARS, CNT128_A, CNT128_B, CNT128_C, CNT128_D, CNT_OUT, CNT2_LO, CNT2_HI, CNT_OUT_LO, CNT_OUT_HI)                                                     \
   extern __shared__ uint8_t smem_raw[];                                                                   \
   const uint32_t raw = smem_u32(smem_raw);                                                                \
   const uint32_t base = (raw + 1023u) & ~1023u;                                                           \
@@ -151,7 +199,7 @@ struct BwdParams {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;                                             \
   if (threadIdx.x == 0) {                                                                                 \
     for (int i = 0; i < NBARS; ++i)                                                                       \
-      mbar_init(B(i), (i == CNT128_A || i == CNT128_B || i == CNT128_C || i == CNT128_D) ? EW_THREADS : i == CNT_OUT ? OUT_THREADS \
+      mbar_init(B(i), (i == CNT128_A || i == CNT128_B || i == CNT128_C || i == CNT128_D) ? EW_THREADS : (i == CNT_OUT || (i >= CNT_OUT_LO && i < CNT_OUT_HI)) ? OUT_THREADS \
                       : (i >= CNT2_LO && i < CNT2_HI) ? 2 : 1);                                           \
     *abort_flag = 0;                                                                                      \
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");                                    \
@@ -188,7 +236,8 @@ __device__ __forceinline__ uint32_t freed(int n) { return ((uint32_t)n & 1u) ^ 1
 namespace dkv {
 enum { KV_FULL = 0 /*+buffer*/, KV_FULL1, KV_EMPTY /*+buffer*/, KV_EMPTY1, QD_FULL /*+s*/, QD_FULL1, QD_FULL2,
        QD_EMPTY /*+s*/, QD_EMPTY1, QD_EMPTY2, S_FULL /*+half*/, S_FULL1, S_FREE /*+half*/, S_FREE1,
-       P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, N_BARS };
+       P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, AUG_READY /*+s*/, AUG_READY1, AUG_READY2,
+       N_BARS };
 // Head width 64: K, V of a key tile are double buffered (the next key tile's arrive during this
 // one's last steps); Q, dO and the row statistics of a step go through a ring of three stages; P^T
 // and dS^T have tensor-memory columns of their own.
@@ -207,20 +256,22 @@ template <int DHT> struct Cfg {
   static constexpr int OFF_QD = KVB * 2 * NB * TILE;                // stage s: Q blocks at +s*2*NB*TILE, dO blocks after them
   static constexpr int OFF_OUT = OFF_QD + RINGN * 2 * NB * TILE;    // two blocks staged for the TMA stores
   static constexpr int OFF_STAT = OFF_OUT + 2 * TILE;               // stage s: lse at +s*1024, D at +512
-  static constexpr int OFF_BAR = OFF_STAT + RINGN * 1024;
+  static constexpr int OFF_AUG = OFF_STAT + RINGN * 1024;           // ones for S^T, ones for dP^T, then one tile per stage
+  static constexpr int OFF_BAR = OFF_AUG + (DHT == 64 ? (2 + RINGN) * AUG_TILE : 0);
   static constexpr int USED = OFF_BAR + 256;
   static constexpr int SMEM = DHT == 64 ? USED + 1024 : 232448;     // width 128 takes all a CTA can have
 };
 }  // namespace dkv
 
 template <int DHT>
-__global__ void __launch_bounds__(Roles<DHT>::NTHREADS, 1)
+__global__ void __launch_bounds__(Roles<DHT>::NTHREADS_DKV, 1)
 attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
                        const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dkv;
   using C = Cfg<DHT>;
   constexpr int CW = Roles<DHT>::CW, EW_THREADS = Roles<DHT>::EW_THREADS, ACC_WARP = Roles<DHT>::ACC_WARP,
-                OUT_WARP0 = Roles<DHT>::OUT_WARP0;
+                OUT_WARP0 = Roles<DHT>::OUT_WARP0, STAT_WARP = Roles<DHT>::STAT_WARP, OFF_AUG = C::OFF_AUG;
+  constexpr bool AUG = Roles<DHT>::AUG;
   constexpr int NB = C::NB, KVB = C::KVB, RINGN = C::RINGN, OFF_KV = C::OFF_KV, OFF_QD = C::OFF_QD, OFF_OUT = C::OFF_OUT,
                 OFF_STAT = C::OFF_STAT, OFF_BAR = C::OFF_BAR;
   constexpr bool ALIAS = C::ALIAS;
@@ -234,7 +285,12 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       return;
     }
   }
-  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, QD_EMPTY, QD_EMPTY + RINGN)
+  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, QD_EMPTY, QD_EMPTY + RINGN, 0, 0)
+  if (AUG) {
+    aug_init(base_ptr + OFF_AUG, base_ptr + OFF_AUG + AUG_TILE, BT, base_ptr + OFF_AUG + 2 * AUG_TILE, RINGN * AUG_TILE);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+  }
   const int nq = p.T / BT;
   // persistent: the work units are (item, tile) pairs, item = (sequence, head).  The grid is a multiple of
   // nq CTAs; in round t the CTAs nq*s .. nq*s + nq-1 take the nq tiles of one item (the s-th of the round's
@@ -292,7 +348,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     if (lane == 0) {
       bool ok = true;
       int it = 0, s = 0, n = 0;
-      const uint32_t lo_kv = desc_lo(base + OFF_KV), lo_qd = desc_lo(base + OFF_QD);
+      const uint32_t lo_kv = desc_lo(base + OFF_KV), lo_qd = desc_lo(base + OFF_QD), lo_aug = desc_lo_aug(base + OFF_AUG);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int tk = 0; tk < my_tiles && ok; ++tk) {
         const int item = tk * ipb + slot, kt = (pos + tk) % nq;
@@ -306,6 +362,8 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
         for (int i = kt; i < nq && ok; ++i, ++it) {
           const uint32_t lo_q = lo_qd + (uint32_t)(s * 2 * NB) * TILE16, lo_do = lo_q + (uint32_t)NB * TILE16;
           if (!mbar_wait(B(QD_FULL + s), done(n), abort_flag, p.status, 43)) { ok = false; break; }
+          if (AUG && !mbar_wait(B(AUG_READY + s), done(n), abort_flag, p.status, 52)) { ok = false; break; }
+          const uint32_t lo_aq = lo_aug + (uint32_t)((2 + s) * AUG_TILE >> 4);      // this stage's -lse/scale, -D rows
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             // the half's columns are free once read (own P^T columns) or, where P^T and dS^T lie on
@@ -315,9 +373,12 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb)           // contraction over the head's features, 64 per block
               mma_score_half(tS + 64u * hh, lo_k + (uint32_t)nb * TILE16, lo_q + (uint32_t)nb * TILE16, hh, nb == 0);
+            // one more step: ones x (-lse/scale) of the half's 64 queries (8 row groups = 2048 bytes per half)
+            if (AUG) tc_mma_aug(tS + 64u * hh, lo_aug, lo_aq + (uint32_t)(128 * hh), IDESC_64KK);
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb)
               mma_score_half(tDP + 64u * hh, lo_v + (uint32_t)nb * TILE16, lo_do + (uint32_t)nb * TILE16, hh, nb == 0);
+            if (AUG) tc_mma_aug(tDP + 64u * hh, lo_aug + (uint32_t)(AUG_TILE >> 4), lo_aq + (uint32_t)(128 * hh), IDESC_64KK);
             tc_commit(B(S_FULL + hh));
           }
           if (ok) tc_commit(B(QD_EMPTY + s));        // second arrival comes from the accumulating thread
@@ -381,7 +442,9 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       for (int i = kt; i < nq && ok; ++i, ++it) {
         const float* Ls = reinterpret_cast<const float*>(base_ptr + OFF_STAT + s * 1024);
         const float* Ds = Ls + 128;
-        if (!mbar_wait(B(QD_FULL + s), done(n), abort_flag, p.status, 48)) { ok = false; break; }
+        (void)Ls; (void)Ds;
+        // (with the statistics folded into the products these threads read nothing of the stage)
+        if (!AUG && !mbar_wait(B(QD_FULL + s), done(n), abort_flag, p.status, 48)) { ok = false; break; }
         const bool diag = (i == kt);
         // The 128 query columns go in two halves of 64 (one CW-column chunk per warp and half): the
         // products that contract over the first half run while the second half is being computed.
@@ -410,6 +473,19 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
 #pragma unroll
               for (int e = 0; e < CW; ++e) sv[e] = (c + e < r) ? -INFINITY : sv[e];
             }
+            if constexpr (AUG) {
+              // the accumulators hold S^T - lse/scale and dP^T - D already
+#pragma unroll
+              for (int e = 0; e < CW; e += 2) {
+                float a0, a1, g0, g1;
+                unpack2(mul2(pack2(sv[e], sv[e + 1]), sc2), a0, a1);
+                const float p0 = ex2(a0), p1 = ex2(a1);
+                unpack2(mul2(pack2(p0, p1), pack2(dv[e], dv[e + 1])), g0, g1);
+                __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), da = __floats2bfloat162_rn(g0, g1);
+                pk[e >> 1] = *reinterpret_cast<uint32_t*>(&pa);
+                dk[e >> 1] = *reinterpret_cast<uint32_t*>(&da);
+              }
+            } else {
 #pragma unroll
             for (int e = 0; e < CW; e += 4) {
               // two elements per instruction: the row statistics come out of shared memory as pairs
@@ -429,6 +505,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
               dk[e >> 1] = *reinterpret_cast<uint32_t*>(&da);
               dk[(e >> 1) + 1] = *reinterpret_cast<uint32_t*>(&db);
             }
+            }
           } else {
 #pragma unroll
             for (int e = 0; e < CW / 2; ++e) { pk[e] = 0u; dk[e] = 0u; }
@@ -446,7 +523,30 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
         if (++s == RINGN) { s = 0; ++n; }
       }
     }
-  } else if (warp >= OUT_WARP0) {
+  } else if (AUG && warp == STAT_WARP) {
+    // ---------------- the queries' -lse/scale and -D of a stage as operand rows ----------------
+    bool ok = true;
+    int s = 0, n = 0;
+    const float inv_scale = 1.0f / p.scale;
+    for (int tk = 0; tk < my_tiles && ok; ++tk) {
+      const int kt = (pos + tk) % nq;
+      for (int i = kt; i < nq; ++i) {
+        if (!mbar_wait(B(QD_FULL + s), done(n), abort_flag, p.status, 53)) { ok = false; break; }
+        const float* Ls = reinterpret_cast<const float*>(base_ptr + OFF_STAT + s * 1024);
+        const float* Ds = Ls + 128;
+        uint8_t* rows = base_ptr + OFF_AUG + (2 + s) * AUG_TILE;
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4) {
+          const int j = lane + 32 * k4;
+          *reinterpret_cast<uint2*>(rows + aug_row(j)) = make_uint2(neg_split(Ls[j] * inv_scale), neg_split(Ds[j]));
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(B(AUG_READY + s));
+        if (++s == RINGN) { s = 0; ++n; }
+      }
+    }
+  } else if (warp >= OUT_WARP0 && warp < OUT_WARP0 + 4) {
     // ---------------- output: dK (scaled) and dV of a finished key tile ----------------
     // Own warps, so that the element-wise warps go on with the next key tile while the last
     // products of this one drain: tensor memory -> bf16 -> shared memory -> TMA stores.
@@ -515,7 +615,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
 namespace dq {
 enum { QO_FULL = 0 /*+buffer*/, QO_FULL1, QO_EMPTY /*+buffer*/, QO_EMPTY1, KV_FULL /*+s*/, KV_FULL1, KV_FULL2,
        KV_EMPTY /*+s*/, KV_EMPTY1, KV_EMPTY2, S_FULL /*+half*/, S_FULL1, S_FREE /*+half*/, S_FREE1,
-       P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, N_BARS };
+       P_READY /*+half*/, P_READY1, P_FREE /*+half*/, P_FREE1, ACC_FULL, ACC_FREE, AUG_READY /*+buffer*/, AUG_READY1, N_BARS };
 // Head width 64: Q, dO and O of a query tile are double buffered (O only serves D[row] = sum(dO * O),
 // which the kernel then computes for itself and leaves in global memory for the dK/dV kernel); K, V
 // of a step go through a ring of three stages.  Head width 128: every operand is two 64-feature
@@ -530,23 +630,32 @@ template <int DHT> struct Cfg {
   static constexpr int OFF_QO = 0;
   static constexpr int OFF_KV = QOB * QO_TILES * TILE;          // stage s: K blocks at +s*2*NB*TILE, V blocks after them
   static constexpr int OFF_OUT = OFF_KV + RINGN * 2 * NB * TILE;   // dQ staged for the TMA store
-  static constexpr int OFF_BAR = OFF_OUT + NB * TILE;
+  static constexpr int OFF_AUG = OFF_OUT + NB * TILE;              // ones for S, ones for dP (64 key rows each), then one tile per Q buffer
+  static constexpr int OFF_BAR = OFF_AUG + (DHT == 64 ? AUG_TILE + QOB * AUG_TILE : 0);
   static constexpr int SMEM = OFF_BAR + 256 + 1024;
 };
 }  // namespace dq
 
 template <int DHT>
-__global__ void __launch_bounds__(Roles<DHT>::NTHREADS, 1)
+__global__ void __launch_bounds__(Roles<DHT>::NTHREADS_DQ, 1)
 attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_constant__ CUtensorMap mapDO,
                       const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapDQKV, BwdParams p) {
   using namespace dq;
   using C = Cfg<DHT>;
   constexpr int CW = Roles<DHT>::CW, EW_THREADS = Roles<DHT>::EW_THREADS, ACC_WARP = Roles<DHT>::ACC_WARP,
-                OUT_WARP0 = Roles<DHT>::OUT_WARP0;
+                OUT_WARP0 = Roles<DHT>::OUT_WARP0, OFF_AUG = C::OFF_AUG;
+  constexpr bool AUG = Roles<DHT>::AUG;
+  static_assert(!AUG || C::HAS_O, "the statistics warp computes D from the staged O tile");
   constexpr int NB = C::NB, QOB = C::QOB, RINGN = C::RINGN, QO_TILES = C::QO_TILES, OFF_QO = C::OFF_QO, OFF_KV = C::OFF_KV,
                 OFF_OUT = C::OFF_OUT, OFF_BAR = C::OFF_BAR;
   constexpr bool HAS_O = C::HAS_O;
-  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, KV_EMPTY, KV_EMPTY + RINGN)
+  T5_SETUP(N_BARS, S_FREE, S_FREE1, P_READY, P_READY1, ACC_FREE, KV_EMPTY, KV_EMPTY + RINGN, AUG_READY, AUG_READY + 2)
+  if (AUG) {
+    // the two constant tiles need 64 rows each (a half's key columns): they share one tile's room
+    aug_init(base_ptr + OFF_AUG, base_ptr + OFF_AUG + AUG_TILE / 2, 64, base_ptr + OFF_AUG + AUG_TILE, QOB * AUG_TILE);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+  }
   const int nq = p.T / BT;
   // persistent: the work units are (item, tile) pairs, item = (sequence, head).  The grid is a multiple of
   // nq CTAs; in round t the CTAs nq*s .. nq*s + nq-1 take the nq tiles of one item (the s-th of the round's
@@ -598,7 +707,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
     if (lane == 0) {
       bool ok = true;
       int it = 0, s = 0, n = 0;
-      const uint32_t lo_qo = desc_lo(base + OFF_QO), lo_kv = desc_lo(base + OFF_KV);
+      const uint32_t lo_qo = desc_lo(base + OFF_QO), lo_kv = desc_lo(base + OFF_KV), lo_aug = desc_lo_aug(base + OFF_AUG);
       constexpr uint32_t TILE16 = TILE >> 4;
       for (int tq = 0; tq < my_tiles && ok; ++tq) {
         const int item = tq * ipb + slot, qi = (pos + tq) % nq;
@@ -610,9 +719,14 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
         const int qb = tq % QOB;
         const uint32_t lo_q = lo_qo + (uint32_t)(qb * QO_TILES) * TILE16, lo_do = lo_q + (uint32_t)NB * TILE16;
         if (!mbar_wait(B(QO_FULL + qb), done(tq / QOB), abort_flag, p.status, 65)) { ok = false; break; }
+        const uint32_t lo_aq = lo_aug + (uint32_t)((1 + qb) * AUG_TILE >> 4);       // this tile's -lse/scale, -D rows
         for (int st = 0; st < steps && ok; ++st, ++it) {
           const uint32_t lo_k = lo_kv + (uint32_t)(s * 2 * NB) * TILE16;
           if (!mbar_wait(B(KV_FULL + s), done(n), abort_flag, p.status, 63)) { ok = false; break; }
+          // The rows with -lse/scale and -D are written by the statistics warp once Q, dO and O have arrived.
+          // In a tile's first step both halves' products over the features are issued before that is waited
+          // for, so the statistics are computed while the tensor pipe already works on the tile.
+          const bool late_aug = AUG && st == 0;
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             if (!mbar_wait(B(S_FREE + hh), freed(it), abort_flag, p.status, 64)) { ok = false; break; }
@@ -623,7 +737,21 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb)
               mma_score_half(tDP + 64u * hh, lo_do + (uint32_t)nb * TILE16, lo_k + (uint32_t)(NB + nb) * TILE16, hh, nb == 0);
-            tc_commit(B(S_FULL + hh));
+            if (AUG && !late_aug) {
+              // one more step: (-lse/scale of the queries) x ones, then (-D) x ones
+              tc_mma_aug(tS + 64u * hh, lo_aq, lo_aug, IDESC_64KK);
+              tc_mma_aug(tDP + 64u * hh, lo_aq, lo_aug + (uint32_t)(AUG_TILE / 2 >> 4), IDESC_64KK);
+            }
+            if (!late_aug) tc_commit(B(S_FULL + hh));
+          }
+          if (ok && late_aug) {
+            if (!mbar_wait(B(AUG_READY + qb), done(tq / QOB), abort_flag, p.status, 72)) { ok = false; break; }
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+              tc_mma_aug(tS + 64u * hh, lo_aq, lo_aug, IDESC_64KK);
+              tc_mma_aug(tDP + 64u * hh, lo_aq, lo_aug + (uint32_t)(AUG_TILE / 2 >> 4), IDESC_64KK);
+              tc_commit(B(S_FULL + hh));
+            }
           }
           if (ok) tc_commit(B(KV_EMPTY + s));        // second arrival comes from the accumulating thread
           if (++s == RINGN) { s = 0; ++n; }
@@ -681,11 +809,13 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       const size_t stat0 = ((size_t)b * p.H + h) * p.T;
       (void)seq_row0; (void)stat0;
       const int i = nq - 1 - qi;
-      const float L2 = p.lse[stat0 + (size_t)i * BT + r] * LOG2E;
+      // (with the statistics folded into the products these threads need neither lse nor D)
+      const float L2 = AUG ? 0.f : p.lse[stat0 + (size_t)i * BT + r] * LOG2E;
       // D[row] = sum(dO * O) from the staged tiles: both have the same swizzle, so 16-byte chunk j of
       // one row holds the same eight columns in both
       float Dr = 0.f;
-      if (!HAS_O) {
+      if (AUG) {
+      } else if (!HAS_O) {
         Dr = p.rowdot[stat0 + (size_t)i * BT + r];
       } else {
         const int qb = tq % QOB;
@@ -734,9 +864,17 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
 #pragma unroll
             for (int e = 0; e < CW; e += 2) {
               float a0, a1, g0, g1;
-              unpack2(fma2(pack2(sv[e], sv[e + 1]), sc2, nl2), a0, a1);
+              if constexpr (AUG) {      // the accumulators hold S - lse/scale and dP - D already
+                unpack2(mul2(pack2(sv[e], sv[e + 1]), sc2), a0, a1);
+              } else {
+                unpack2(fma2(pack2(sv[e], sv[e + 1]), sc2, nl2), a0, a1);
+              }
               const float p0 = ex2(a0), p1 = ex2(a1);
-              unpack2(mul2(pack2(p0, p1), add2(pack2(dv[e], dv[e + 1]), nd2)), g0, g1);
+              if constexpr (AUG) {
+                unpack2(mul2(pack2(p0, p1), pack2(dv[e], dv[e + 1])), g0, g1);
+              } else {
+                unpack2(mul2(pack2(p0, p1), add2(pack2(dv[e], dv[e + 1]), nd2)), g0, g1);
+              }
               __nv_bfloat162 db = __floats2bfloat162_rn(g0, g1);
               dk[e >> 1] = *reinterpret_cast<uint32_t*>(&db);
             }
@@ -753,12 +891,46 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
         if (!ok) break;
       }
     }
-  } else if (warp >= OUT_WARP0) {
+  } else if (warp >= OUT_WARP0 && warp < OUT_WARP0 + 4) {
     // ---------------- output: dQ (scaled) of a finished query tile (own warps, see the dK/dV kernel) ----------------
     const int q4 = warp & 3;
     const int r = q4 * 32 + lane;
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     bool ok = true;
+    // These warps idle while a tile's products run, so they also prepare the next tile's row statistics
+    // (one thread per query row): D[row] = sum(dO * O) from the staged tiles, left in global memory for the
+    // dK/dV kernel, and the operand row that carries -lse/scale and -D into the tile's score products.
+    const float inv_scale = 1.0f / p.scale;
+    auto statistics = [&](int t) {
+      const int item = t * ipb + slot, qi = (pos + t) % nq;
+      const int h = item % p.H, b = item / p.H;
+      const size_t row = ((size_t)b * p.H + h) * p.T + (size_t)(nq - 1 - qi) * BT + r;
+      const int qb = t % QOB;
+      const float L = p.lse[row];
+      if (!mbar_wait(B(QO_FULL + qb), done(t / QOB), abort_flag, p.status, 73)) { ok = false; return; }
+      // dO and O tiles have the same swizzle, so 16-byte chunk j of one row holds the same eight columns in both
+      const uint8_t* dorow = base_ptr + OFF_QO + qb * QO_TILES * TILE + TILE + r * 128;
+      const uint8_t* orow = dorow + TILE;
+      float Dr = 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int jj = (j ^ (r & 7)) << 4;       // lanes of a warp spread over all banks
+        const uint4 av = *reinterpret_cast<const uint4*>(dorow + jj);
+        const uint4 bv = *reinterpret_cast<const uint4*>(orow + jj);
+        const uint32_t* aw = reinterpret_cast<const uint32_t*>(&av);
+        const uint32_t* bw = reinterpret_cast<const uint32_t*>(&bv);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          Dr = fmaf(__uint_as_float(aw[e] << 16), __uint_as_float(bw[e] << 16), Dr);
+          Dr = fmaf(__uint_as_float(aw[e] & 0xffff0000u), __uint_as_float(bw[e] & 0xffff0000u), Dr);
+        }
+      }
+      p.rowdot_out[row] = Dr;
+      *reinterpret_cast<uint2*>(base_ptr + OFF_AUG + (1 + qb) * AUG_TILE + aug_row(r)) = make_uint2(neg_split(L * inv_scale), neg_split(Dr));
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(B(AUG_READY + qb));
+    };
+    if (AUG && my_tiles > 0) statistics(0);
     for (int tq = 0; tq < my_tiles; ++tq) {
       const int item = tq * ipb + slot, qi = (pos + tq) % nq;
       const int h = item % p.H, b = item / p.H;      // this CTA walks several (sequence, head) items
@@ -766,6 +938,9 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       const size_t stat0 = ((size_t)b * p.H + h) * p.T;
       (void)seq_row0; (void)stat0;
       const int i = nq - 1 - qi;
+      // (the next tile's Q, dO and O were requested when the tile before this one had been read: they arrive
+      // long before this tile's accumulator is complete)
+      if (AUG && ok && tq + 1 < my_tiles) statistics(tq + 1);
       if (ok && !mbar_wait(B(ACC_FULL), done(tq), abort_flag, p.status, 70)) ok = false;
       if (ok) {
         tc_fence_after();
@@ -844,8 +1019,8 @@ cudaError_t attention_bwd_t5(const void* qkv, const void* o, const float* lse, c
   const int nq = T / BT, units = p.nitems * nq;
   dim3 grid((unsigned)(((units < sms ? units : sms) / nq) * nq));   // one persistent CTA per SM, whole items per round
   // dQ first: it leaves D[row] = sum(dO * O) in `rowdot` for the dK/dV kernel
-  attn_bwd_dq_t5_kernel<64><<<grid, Roles<64>::NTHREADS, dq::Cfg<64>::SMEM, st>>>(mQKV, mDO, mO, mDQKV, p);
-  attn_bwd_dkv_t5_kernel<64><<<grid, Roles<64>::NTHREADS, dkv::Cfg<64>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
+  attn_bwd_dq_t5_kernel<64><<<grid, Roles<64>::NTHREADS_DQ, dq::Cfg<64>::SMEM, st>>>(mQKV, mDO, mO, mDQKV, p);
+  attn_bwd_dkv_t5_kernel<64><<<grid, Roles<64>::NTHREADS_DKV, dkv::Cfg<64>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
   return cudaGetLastError();
 }
 
@@ -872,8 +1047,8 @@ cudaError_t attention_bwd_t5_128(const void* qkv, const float* lse, const void* 
   p.nitems = nseq * H;
   const int nq = T / BT, units = p.nitems * nq;
   dim3 grid((unsigned)(((units < sms ? units : sms) / nq) * nq));
-  attn_bwd_dq_t5_kernel<128><<<grid, Roles<128>::NTHREADS, dq::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDO /* unused */, mDQKV, p);
-  attn_bwd_dkv_t5_kernel<128><<<grid, Roles<128>::NTHREADS, dkv::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
+  attn_bwd_dq_t5_kernel<128><<<grid, Roles<128>::NTHREADS_DQ, dq::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDO /* unused */, mDQKV, p);
+  attn_bwd_dkv_t5_kernel<128><<<grid, Roles<128>::NTHREADS_DKV, dkv::Cfg<128>::SMEM, st>>>(mQKV, mDO, mDQKV, p);
   return cudaGetLastError();
 }
 
