@@ -18,10 +18,13 @@
 //
 // D[row] = sum(dO * O) is computed by the dQ kernel from its staged dO and O tiles and left in global
 // memory for the dK/dV kernel, which runs second (head width 128: shared memory has no room for O,
-// both kernels read D from global memory, where a small kernel has put it beforehand).  Warp roles (480 threads): warp 0 TMA producer,
-// warp 1 tensor-memory owner + issuer of the score products, warp 10 issuer of the accumulating
-// products, warps 2..9 element-wise work (thread = accumulator lane, two warps per lane quarter),
-// warps 11..14 output of the finished accumulators.
+// both kernels read D from global memory, where a small kernel has put it beforehand).
+// Warp roles (struct Roles below): warp 0 TMA producer, warp 1 tensor-memory owner + issuer of the score
+// products, then the element-wise warps (thread = accumulator lane; four warps per lane quarter at head
+// width 64, two at 128), one warp that issues the accumulating products, four warps that move finished
+// accumulators to global memory, and in the dK/dV kernel at head width 64 one warp that prepares the row
+// statistics of each stage.  At head width 64 the statistics enter the score products as one more
+// contraction step ("augmented contraction" below), so the element-wise threads never read them.
 // All mbarrier waits are bounded (tc_common.cuh); on expiry a code is left in `status`.
 #include "host_common.h"
 #include "tc_common.cuh"
