@@ -133,19 +133,20 @@ class ClockSampler:
                 "power_w_max": max(float(r[3]) for r in mine), "reasons": sorted(reasons)}
 
 
-def oracle_sample_workload(w):
-    """The bounded sample the CPU oracle is timed on: same model, 2 clients x 1 sequence.  A model whose
+def oracle_sample_workload(w, rounds=1):
+    """The bounded sample the CPU oracle is timed on: same model, 2 clients x 1 sequence (1 client when more
+    than six rounds are asked for, so that the whole run still ends within a few minutes).  A model whose
     fp64 round would take many minutes even so (width 4096) is cut to one client block and one server
     block on one sequence; time_oracle_rounds scales the time back up to the full depth."""
     if w.d_model >= 2048:
         return synth.scaled(w, n_layer=2, cut=1, n_clients=1, batch_per_client=1, counts=None)
-    return synth.scaled(w, n_clients=min(2, w.n_clients), batch_per_client=1, counts=None)
+    return synth.scaled(w, n_clients=min(2 if rounds <= 6 else 1, w.n_clients), batch_per_client=1, counts=None)
 
 
 def time_oracle_rounds(w, steps, warmup):
     """Times oracle rounds (as the oracle stands) on the host cores."""
     from oracle import splitlora_oracle as O
-    ws = oracle_sample_workload(w)
+    ws = oracle_sample_workload(w, steps + warmup)
     frozen = synth.make_frozen(ws)          # fp32 arrays holding bf16-exact values; widened on use
     cads = [synth.make_adapters(ws, range(ws.cut)) for _ in range(ws.n_clients)]
     sads = synth.make_adapters(ws, range(ws.cut, ws.n_layer))
