@@ -347,7 +347,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
     // of that half done.  The halves are separate products so that the next step's first half is
     // computed while the element-wise warps still work on this step's second.  The accumulating
     // products are issued by another thread (warp ACC_WARP): one thread cannot issue 32 products of
-    // 48 cycles each per step next to eight busy element-wise warps.
+    // 48 cycles each per step next to the busy element-wise warps.
     if (lane == 0) {
       bool ok = true;
       int it = 0, s = 0, n = 0;
@@ -427,7 +427,7 @@ attn_bwd_dkv_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_
       }
     }
   } else if (warp < ACC_WARP) {
-    // ---------------- element-wise warps 2..9 ----------------
+    // ---------------- element-wise warps (2 .. ACC_WARP - 1) ----------------
     const int q4 = warp & 3;
     const int wsel = (warp - 2) >> 2;            // which of the EWQ warps of this accumulator lane quarter
     const int r = q4 * 32 + lane;                // key row inside the tile = accumulator lane
@@ -796,7 +796,7 @@ attn_bwd_dq_t5_kernel(const __grid_constant__ CUtensorMap mapQKV, const __grid_c
       }
     }
   } else if (warp < ACC_WARP) {
-    // ---------------- element-wise warps 2..9 ----------------
+    // ---------------- element-wise warps (2 .. ACC_WARP - 1) ----------------
     const int q4 = warp & 3;
     const int wsel = (warp - 2) >> 2;            // which of the EWQ warps of this accumulator lane quarter
     const int r = q4 * 32 + lane;                // query row inside the tile
